@@ -1,0 +1,260 @@
+/*
+ * AdaS-Attn oracle: a plain, slow, fp64 CPU statement of Adaptive Cube-Selective Attention.
+ *
+ * TEST INFRASTRUCTURE ONLY.  Nothing in the product path may call this file; it shares no
+ * code with the CUDA implementation.  It follows the paper's definitions step by step, with
+ * no blocking, fusion or reordering:
+ *
+ *   O1  cube partition / cube-major order        Sec. 3.1; Algorithm 1 ("Reshape K,V into Cubes")
+ *   O2  mean key per cube and KV head            Sec. 3.2, text under Eq. 1
+ *   O3  selection scores + softmax over cubes    Eq. 1
+ *   O4  nucleus (Top-p) cube selection           Eq. 2
+ *   O5  attention over selected cubes + own-cube Eq. 3 and the text-token rule that follows it
+ *       prefix (video) or text prefix (text)
+ *   O6  decode = a text-rule row appended after the cached sequence (same code as O5)
+ *
+ * Readings taken where the paper is silent (each also listed in the design notes):
+ *   - a query attends itself (standard causal "<="), otherwise p = 1 would not be dense
+ *     causal attention;
+ *   - cubes are numbered row-major over (time block, row block, column block), tokens inside
+ *     a cube row-major over (t, y, x); "preceding" refers to this cube-major order;
+ *   - Top-p = the shortest prefix of the cubes sorted by (probability descending, index
+ *     ascending) whose cumulative probability is >= p; p >= 1 selects every candidate;
+ *   - the own cube is never a candidate; text queries see every video cube as a candidate;
+ *   - with grouped-query attention the mean keys are per KV head, the selection per query
+ *     head (kv head = query head / group size).
+ *
+ * Pins (tests/test_oracle_*.py): closed-form permutation examples, numpy reshape-mean,
+ * brute force over all cube subsets, p -> 0 argmax, p = 1 equals an independently written
+ * dense causal attention, first-cube special case, equal-keys error bound, V-linearity,
+ * logit-shift invariance.  The paper prints no worked numeric example, so absolute output
+ * values are pinned only through those identities.
+ *
+ * All tensors are raster order, row-major:  Q [B,S,Hq,D], K,V [B,S,Hkv,D] as float (the
+ * bf16-rounded inputs widened exactly), S = T*H*W + n_text, text after video.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+typedef struct {
+    int32_t B, T, H, W;      /* batch, frames, patch rows, patch columns              */
+    int32_t ct, ch, cw;      /* cube window                                           */
+    int32_t n_text;          /* text tokens after the video                           */
+    int32_t Hq, Hkv, D;      /* query heads, KV heads, head dim                       */
+    double top_p;            /* nucleus mass p                                        */
+    double scale;            /* logit scale, 1/sqrt(D) in the paper                   */
+} adas_shape;
+
+static int64_t n_cubes(const adas_shape *s) {
+    return (int64_t)(s->T / s->ct) * (s->H / s->ch) * (s->W / s->cw);
+}
+static int64_t cube_tokens(const adas_shape *s) { return (int64_t)s->ct * s->ch * s->cw; }
+static int64_t video_tokens(const adas_shape *s) { return (int64_t)s->T * s->H * s->W; }
+static int64_t seq_len(const adas_shape *s) { return video_tokens(s) + s->n_text; }
+
+int64_t adas_oracle_num_cubes(const adas_shape *s) { return n_cubes(s); }
+
+/* O1 (Sec. 3.1): raster index n = (t*H + y)*W + x of a video token -> cube-major position
+ * c*C + r; a text token u keeps position S_v + u. */
+int64_t adas_oracle_position(const adas_shape *s, int64_t n) {
+    int64_t Sv = video_tokens(s);
+    if (n >= Sv) return n;
+    int64_t x = n % s->W, y = (n / s->W) % s->H, t = n / ((int64_t)s->W * s->H);
+    int64_t cube = ((t / s->ct) * (s->H / s->ch) + y / s->ch) * (s->W / s->cw) + x / s->cw;
+    int64_t rank = ((t % s->ct) * s->ch + y % s->ch) * s->cw + x % s->cw;
+    return cube * cube_tokens(s) + rank;
+}
+
+/* pos_of_raster[n] and its inverse raster_of_pos[pos], both length S. */
+void adas_oracle_positions(const adas_shape *s, int64_t *pos_of_raster, int64_t *raster_of_pos) {
+    int64_t S = seq_len(s);
+    for (int64_t n = 0; n < S; ++n) {
+        int64_t pos = adas_oracle_position(s, n);
+        pos_of_raster[n] = pos;
+        raster_of_pos[pos] = n;
+    }
+}
+
+/* O2: kbar[b][g][c][:] = (1/C) * sum of the C keys of cube c (KV head g).  kbar: [B,Hkv,N,D]. */
+void adas_oracle_mean_keys(const adas_shape *s, const float *K, double *kbar) {
+    int64_t S = seq_len(s), Sv = video_tokens(s), N = n_cubes(s), C = cube_tokens(s);
+    int64_t D = s->D, Hkv = s->Hkv;
+    memset(kbar, 0, sizeof(double) * (size_t)(s->B * Hkv * N * D));
+    for (int64_t b = 0; b < s->B; ++b)
+        for (int64_t n = 0; n < Sv; ++n) {
+            int64_t c = adas_oracle_position(s, n) / C;
+            for (int64_t g = 0; g < Hkv; ++g) {
+                const float *k = K + ((b * S + n) * Hkv + g) * D;
+                double *m = kbar + ((b * Hkv + g) * N + c) * D;
+                for (int64_t d = 0; d < D; ++d) m[d] += (double)k[d];
+            }
+        }
+    for (int64_t i = 0; i < s->B * Hkv * N * D; ++i) kbar[i] /= (double)C;
+}
+
+typedef struct { double p; int64_t j; } prob_idx;
+
+static int by_prob_desc_then_index(const void *a, const void *b) {
+    const prob_idx *x = (const prob_idx *)a, *y = (const prob_idx *)b;
+    if (x->p > y->p) return -1;
+    if (x->p < y->p) return 1;
+    return (x->j > y->j) - (x->j < y->j);
+}
+
+/* O3 + O4 for one query row.
+ *   q       [D] query (float), kbar_g [N][D] mean keys of its KV head
+ *   n_cand  number of candidate cubes J = {0..n_cand-1}
+ * Outputs: sel[j] in {0,1} for j < n_cand (caller zeroes beyond), returns |S|.
+ *   probs   (nullable) [n_cand] the softmax P
+ *   margin  (nullable) tie margin of the row: min(|c_k* - p|, |c_(k*-1) - p|,
+ *           p_(k*) - p_(k*+1)); +inf when nothing can tie (no candidates, or p >= 1). */
+int64_t adas_oracle_select_row(const float *q, const double *kbar_g, int64_t n_cand, int64_t D,
+                               double scale, double top_p, uint8_t *sel, double *probs,
+                               double *margin) {
+    if (margin) *margin = INFINITY;
+    if (n_cand <= 0) return 0;
+    double *logit = (double *)malloc(sizeof(double) * (size_t)n_cand);
+    prob_idx *order = (prob_idx *)malloc(sizeof(prob_idx) * (size_t)n_cand);
+    /* Eq. 1: s_j = <q, kbar_j> / sqrt(d_k), P = softmax(s) */
+    double mx = -INFINITY;
+    for (int64_t j = 0; j < n_cand; ++j) {
+        double acc = 0.0;
+        for (int64_t d = 0; d < D; ++d) acc += (double)q[d] * kbar_g[j * D + d];
+        logit[j] = acc * scale;
+        if (logit[j] > mx) mx = logit[j];
+    }
+    double Z = 0.0;
+    for (int64_t j = 0; j < n_cand; ++j) Z += exp(logit[j] - mx);
+    for (int64_t j = 0; j < n_cand; ++j) {
+        order[j].p = exp(logit[j] - mx) / Z;
+        order[j].j = j;
+        if (probs) probs[j] = order[j].p;
+    }
+    /* Eq. 2: nucleus = shortest sorted prefix with cumulative mass >= p */
+    qsort(order, (size_t)n_cand, sizeof(prob_idx), by_prob_desc_then_index);
+    int64_t kstar = n_cand;
+    double cum = 0.0, cum_before = 0.0;
+    if (top_p < 1.0) {
+        for (int64_t k = 0; k < n_cand; ++k) {
+            double before = cum;
+            cum += order[k].p;
+            if (cum >= top_p) {
+                kstar = k + 1;
+                cum_before = before;
+                break;
+            }
+        }
+        if (margin && kstar <= n_cand && cum >= top_p) {
+            double m = fabs(cum - top_p);
+            if (fabs(cum_before - top_p) < m) m = fabs(cum_before - top_p);
+            if (kstar < n_cand) {
+                double gap = order[kstar - 1].p - order[kstar].p;
+                if (gap < m) m = gap;
+            }
+            *margin = m;
+        }
+    }
+    for (int64_t j = 0; j < n_cand; ++j) sel[j] = 0;
+    for (int64_t k = 0; k < kstar; ++k) sel[order[k].j] = 1;
+    free(logit);
+    free(order);
+    return kstar;
+}
+
+/* O5 for one row whose selection is known.  Key set A = all tokens of every selected cube,
+ * plus (video) the own-cube tokens at cube-major positions <= the query's, or (text) the
+ * text tokens <= the query's.  One softmax over A (Eq. 3), output [D] in fp64. */
+static void attend_row(const adas_shape *s, const float *Q, const float *K, const float *V,
+                       const int64_t *raster_of_pos, int64_t b, int64_t h, int64_t n_raster,
+                       int64_t pos, const uint8_t *sel, int64_t n_cand, double *out) {
+    int64_t S = seq_len(s), Sv = video_tokens(s), C = cube_tokens(s), D = s->D;
+    int64_t g = h / (s->Hq / s->Hkv);
+    const float *q = Q + ((b * S + n_raster) * s->Hq + h) * D;
+    /* gather the cube-major positions of A */
+    int64_t cap = n_cand * C + (pos < Sv ? C : s->n_text) + 1, na = 0;
+    int64_t *att = (int64_t *)malloc(sizeof(int64_t) * (size_t)cap);
+    for (int64_t j = 0; j < n_cand; ++j)
+        if (sel[j])
+            for (int64_t r = 0; r < C; ++r) att[na++] = j * C + r;
+    if (pos < Sv) {
+        for (int64_t pp = (pos / C) * C; pp <= pos; ++pp) att[na++] = pp;
+    } else {
+        for (int64_t pp = Sv; pp <= pos; ++pp) att[na++] = pp;
+    }
+    double *w = (double *)malloc(sizeof(double) * (size_t)na);
+    double mx = -INFINITY;
+    for (int64_t a = 0; a < na; ++a) {
+        const float *k = K + ((b * S + raster_of_pos[att[a]]) * s->Hkv + g) * D;
+        double acc = 0.0;
+        for (int64_t d = 0; d < D; ++d) acc += (double)q[d] * (double)k[d];
+        w[a] = acc * s->scale;
+        if (w[a] > mx) mx = w[a];
+    }
+    double Z = 0.0;
+    for (int64_t a = 0; a < na; ++a) { w[a] = exp(w[a] - mx); Z += w[a]; }
+    for (int64_t d = 0; d < D; ++d) out[d] = 0.0;
+    for (int64_t a = 0; a < na; ++a) {
+        const float *v = V + ((b * S + raster_of_pos[att[a]]) * s->Hkv + g) * D;
+        double wa = w[a] / Z;
+        for (int64_t d = 0; d < D; ++d) out[d] += wa * (double)v[d];
+    }
+    free(w);
+    free(att);
+}
+
+/* Evaluate a list of rows.  rows[3*i + {0,1,2}] = (batch b, query head h, raster token n).
+ *   kbar        [B,Hkv,N,D] from adas_oracle_mean_keys
+ *   out         (nullable) [nrows, D] fp64 attention output; NULL = selection only
+ *   sel         [nrows, N] 0/1 flags (zero beyond the row's candidates)
+ *   count       [nrows] |S_i|
+ *   margin      (nullable) [nrows] tie margin (see adas_oracle_select_row)
+ *   n_attended  (nullable) [nrows] |A|, the number of key tokens the row attends
+ * Rows are independent; OpenMP splits them over the host cores. */
+void adas_oracle_rows(const adas_shape *s, const float *Q, const float *K, const float *V,
+                      const double *kbar, int64_t nrows, const int64_t *rows, double *out,
+                      uint8_t *sel, int32_t *count, double *margin, int64_t *n_attended) {
+    int64_t S = seq_len(s), Sv = video_tokens(s), N = n_cubes(s), C = cube_tokens(s), D = s->D;
+    int64_t *pos_of_raster = (int64_t *)malloc(sizeof(int64_t) * (size_t)S);
+    int64_t *raster_of_pos = (int64_t *)malloc(sizeof(int64_t) * (size_t)S);
+    adas_oracle_positions(s, pos_of_raster, raster_of_pos);
+    int64_t G = s->Hq / s->Hkv;
+#pragma omp parallel for schedule(dynamic, 16)
+    for (int64_t i = 0; i < nrows; ++i) {
+        int64_t b = rows[3 * i], h = rows[3 * i + 1], n = rows[3 * i + 2];
+        int64_t pos = pos_of_raster[n];
+        int64_t n_cand = pos < Sv ? pos / C : N;   /* preceding cubes; text sees all cubes */
+        const float *q = Q + ((b * S + n) * s->Hq + h) * D;
+        const double *kbar_g = kbar + ((b * s->Hkv + h / G) * N) * D;
+        uint8_t *sel_i = sel + i * N;
+        memset(sel_i, 0, (size_t)N);
+        int64_t cnt = adas_oracle_select_row(q, kbar_g, n_cand, D, s->scale, s->top_p, sel_i,
+                                             NULL, margin ? margin + i : NULL);
+        count[i] = (int32_t)cnt;
+        if (n_attended)
+            n_attended[i] = cnt * C + (pos < Sv ? pos - (pos / C) * C + 1 : pos - Sv + 1);
+        if (out) attend_row(s, Q, K, V, raster_of_pos, b, h, n, pos, sel_i, n_cand, out + i * D);
+    }
+    free(pos_of_raster);
+    free(raster_of_pos);
+}
+
+/* Same as adas_oracle_rows' attention step but with the selection supplied by the caller
+ * (used by tests that plant a selection, e.g. "all cubes" for the dense identity). */
+void adas_oracle_attend_given(const adas_shape *s, const float *Q, const float *K, const float *V,
+                              int64_t nrows, const int64_t *rows, const uint8_t *sel, double *out) {
+    int64_t S = seq_len(s), Sv = video_tokens(s), N = n_cubes(s), C = cube_tokens(s), D = s->D;
+    int64_t *pos_of_raster = (int64_t *)malloc(sizeof(int64_t) * (size_t)S);
+    int64_t *raster_of_pos = (int64_t *)malloc(sizeof(int64_t) * (size_t)S);
+    adas_oracle_positions(s, pos_of_raster, raster_of_pos);
+#pragma omp parallel for schedule(dynamic, 16)
+    for (int64_t i = 0; i < nrows; ++i) {
+        int64_t b = rows[3 * i], h = rows[3 * i + 1], n = rows[3 * i + 2];
+        int64_t pos = pos_of_raster[n];
+        int64_t n_cand = pos < Sv ? pos / C : N;
+        attend_row(s, Q, K, V, raster_of_pos, b, h, n, pos, sel + i * N, n_cand, out + i * D);
+    }
+    free(pos_of_raster);
+    free(raster_of_pos);
+}
