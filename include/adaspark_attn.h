@@ -1,0 +1,153 @@
+/*
+ * adaspark_attn.h - C ABI of the B200 (sm_100a) implementation of Adaptive Cube-Selective
+ * Attention (AdaS-Attn; Sec. 3.1-3.2 and Algorithm 1 of the AdaSpark paper).
+ *
+ * The library computes, for a sequence laid out as [video tokens (T x H x W raster)][text tokens]:
+ *   1. the cube partition of the video tokens by a (cube_t, cube_h, cube_w) window and the
+ *      cube-major re-layout of K and V                       (Sec. 3.1; Algorithm 1, "Reshape K,V");
+ *   2. one mean key per cube and KV head                      (Sec. 3.2, definition under Eq. 1);
+ *   3. for every query row the softmax over the scaled scores against the mean keys of its
+ *      candidate cubes (the preceding cubes for a video query, all cubes for a text query)
+ *                                                             (Eq. 1; text rule after Eq. 3);
+ *   4. the nucleus (Top-p) cube set: the shortest prefix of the cubes sorted by probability
+ *      (descending; equal probabilities by lower cube index) whose mass reaches top_p (Eq. 2);
+ *   5. one softmax attention over the tokens of the selected cubes plus the causal prefix of
+ *      the query's own cube (video) or of the text (text), written back in raster order
+ *                                                             (Eq. 3; Algorithm 1, "Restore").
+ * A decode step evaluates one new text token per sequence against caches built by the prefill.
+ *
+ * Conventions
+ *   - All tensor pointers are DEVICE pointers owned by the caller; the library never allocates
+ *     device memory in _forward / _decode and never synchronises the host with the device.
+ *     Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = default stream).
+ *   - Tensors are bf16, row-major, raster order: q/out [B,S,Hq,D], k/v [B,S,Hkv,D] with
+ *     S = T*H*W + n_text and video token (t,y,x) at s = (t*H + y)*W + x.  Q and K are post-RoPE.
+ *   - Query head h uses KV head h / (Hq/Hkv).  Mean keys are per KV head, selection per query head.
+ *   - Errors are return codes; argument errors are found on the host before any launch.
+ *     adaspark_attn_last_error() returns a message for the most recent failure on a handle.
+ *   - No CPU fallback exists: without a CUDA device every compute entry point fails.
+ */
+#ifndef ADASPARK_ATTN_H_
+#define ADASPARK_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct adaspark_attn adaspark_attn_t; /* opaque, library-owned */
+
+typedef enum {
+    ADASPARK_OK = 0,
+    ADASPARK_ERR_INVALID_ARG = 1,
+    ADASPARK_ERR_UNSUPPORTED = 2,
+    ADASPARK_ERR_NOT_PARTITIONED = 3,
+    ADASPARK_ERR_WORKSPACE_TOO_SMALL = 4,
+    ADASPARK_ERR_CUDA = 5,
+    ADASPARK_ERR_TIMEOUT = 6
+} adaspark_status_t;
+
+/* Problem statement of Algorithm 1: cube window, heads, head_dim, nucleus mass p. */
+typedef struct {
+    int32_t cube_t, cube_h, cube_w; /* cube window in frames / patch rows / patch columns     */
+    int32_t n_q_heads, n_kv_heads;  /* n_kv_heads must divide n_q_heads (GQA group size <= 16) */
+    int32_t head_dim;               /* 64 or 128                                               */
+    float top_p;                    /* in (0, 1]; >= 1 selects every candidate cube (dense)    */
+    float softmax_scale;            /* 0 => 1/sqrt(head_dim) (Eqs. 1, 3); used for both        */
+    int32_t device;                 /* CUDA ordinal                                            */
+} adaspark_attn_config_t;
+
+/* Sizes fixed by _partition.  "pos" below is the cube-major position of a token:
+ * pos = cube * cube_tokens + rank for video tokens, s_video + u for text token u. */
+typedef struct {
+    int64_t n_cubes;         /* N                                                              */
+    int64_t cube_tokens;     /* C = cube_t*cube_h*cube_w                                       */
+    int64_t s_video;         /* T*H*W                                                          */
+    int64_t s_cap;           /* cache rows per (batch, kv head): s_video + n_text_max + 1
+                                rounded up to a multiple of 128                                */
+    int64_t bitmap_words;    /* ceil(N/32): uint32 words per selection bitmap row              */
+    int64_t k_cube_bytes;    /* bf16 [B, Hkv, s_cap, D]: keys at cube-major positions          */
+    int64_t v_cube_bytes;    /* bf16 [B, Hkv, s_cap/64, D, 64]: per 64-position block, V^T     */
+    int64_t cube_keys_bytes; /* fp32 [B, Hkv, N, D]: mean keys                                 */
+    int64_t forward_workspace_bytes;
+    int64_t decode_workspace_bytes;
+} adaspark_attn_layout_t;
+
+/* Create a handle for one configuration.  Host only.  Fails with ERR_UNSUPPORTED for a
+ * head_dim other than 64/128, a cube window whose token count C is not one of
+ * {16, 32, 64, 128, 256, 512}, or a GQA group size above 16; with ERR_INVALID_ARG for
+ * non-positive sizes, top_p <= 0, or a NULL pointer. */
+adaspark_status_t adaspark_attn_create(const adaspark_attn_config_t *config,
+                                       adaspark_attn_t **out_handle);
+
+/* Sec. 3.1: fix the video grid and derive the cube partition (N cubes of C tokens) and every
+ * buffer size.  `batch`, `frames`, `grid_h`, `grid_w` describe the video token grid;
+ * `n_text_max` is the largest number of text tokens any later _forward/_decode will hold.
+ * `*workspace_bytes` (nullable) receives max(forward, decode) workspace size.  Host only.
+ * ERR_UNSUPPORTED if the grid is not divisible by the cube window or N > 4096. */
+adaspark_status_t adaspark_attn_partition(adaspark_attn_t *handle, int32_t batch, int32_t frames,
+                                          int32_t grid_h, int32_t grid_w, int32_t n_text_max,
+                                          size_t *workspace_bytes);
+
+/* Sizes derived by the last _partition.  ERR_NOT_PARTITIONED before it. */
+adaspark_status_t adaspark_attn_get_layout(const adaspark_attn_t *handle,
+                                           adaspark_attn_layout_t *out_layout);
+
+/* Prefill (Algorithm 1, the AdaS-Attn lines; Eqs. 1-3).
+ *   q, k, v      in : bf16 [B, S, H*, D] raster, S = s_video + n_text, 0 <= n_text <= n_text_max.
+ *                     q and out may both be NULL: then only the caches are built.
+ *   out          out: bf16 [B, S, Hq, D] raster.
+ *   k_cube, v_cube, cube_keys
+ *                out: the caches described in adaspark_attn_layout_t (caller-allocated, written
+ *                     in full; rows beyond S are zero-filled).
+ *   sel_bitmap   out, nullable: uint32 [B, Hq, S, bitmap_words], bit j of a row (raster token
+ *                     order) is set iff cube j is in the row's nucleus S_i.
+ *   sel_count    out, nullable: int32 [B, Hq, S] = |S_i|.
+ *   workspace    device scratch of at least forward_workspace_bytes, 256-byte aligned.
+ * Enqueues kernels on the stream and returns; no host synchronisation. */
+adaspark_status_t adaspark_attn_forward(adaspark_attn_t *handle, const void *q, const void *k,
+                                        const void *v, int32_t n_text, void *out, void *k_cube,
+                                        void *v_cube, float *cube_keys, uint32_t *sel_bitmap,
+                                        int32_t *sel_count, void *workspace,
+                                        size_t workspace_bytes, void *cuda_stream);
+
+/* Decode: one new text token per sequence (the text-token rule after Eq. 3 applied to a row
+ * appended after the cached sequence; the new token attends itself).
+ *   q_new        in : bf16 [B, 1, Hq, D].
+ *   k_new, v_new in : bf16 [B, 1, Hkv, D]; appended to the caches at text slot text_len[b]
+ *                     (both NULL: the caller already appended them and text_len[b] counts them
+ *                     out, i.e. the row attends text slots 0..text_len[b]-1... see below).
+ *   k_cube, v_cube  in/out, cube_keys in: caches written by _forward.
+ *   text_len     in : device int32 [B], text tokens already cached (before this step);
+ *                     text_len[b] + 1 <= n_text_max + 1.  With k_new/v_new NULL the row attends
+ *                     text slots 0..text_len[b] and slot text_len[b] must already hold the
+ *                     new token's K/V.
+ *   out          out: bf16 [B, 1, Hq, D].
+ *   sel_bitmap   out, nullable: uint32 [B, Hq, bitmap_words].
+ *   workspace    device scratch of at least decode_workspace_bytes, 256-byte aligned. */
+adaspark_status_t adaspark_attn_decode(adaspark_attn_t *handle, const void *q_new,
+                                       const void *k_new, const void *v_new, void *k_cube,
+                                       void *v_cube, const float *cube_keys,
+                                       const int32_t *text_len, void *out, uint32_t *sel_bitmap,
+                                       void *workspace, size_t workspace_bytes,
+                                       void *cuda_stream);
+
+/* Release the handle (host memory only). NULL is accepted. */
+adaspark_status_t adaspark_attn_destroy(adaspark_attn_t *handle);
+
+/* Message of the most recent error on this handle ("" if none). Never NULL. */
+const char *adaspark_attn_last_error(const adaspark_attn_t *handle);
+
+/* Number of kernel launches the most recent _forward / _decode enqueued (host counter). */
+int64_t adaspark_attn_last_launch_count(const adaspark_attn_t *handle);
+
+/* Selects the prefill attention kernel: 0 = mma.sync (legacy tensor path), 1 = tcgen05/TMEM
+ * with TMA-staged tiles.  Default 1 when built in. ERR_UNSUPPORTED for an unknown value. */
+adaspark_status_t adaspark_attn_set_prefill_kernel(adaspark_attn_t *handle, int32_t which);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ADASPARK_ATTN_H_ */

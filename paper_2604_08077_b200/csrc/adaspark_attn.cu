@@ -1,0 +1,351 @@
+// C-ABI entry points of libadaspark_attn: host-side validation, workspace carving and kernel
+// launches.  All arithmetic lives in the kernels included below; see include/adaspark_attn.h for
+// the contract of every call.
+#include "../../include/adaspark_attn.h"
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+#include "relayout_pool.cuh"
+#include "score_select.cuh"
+#include "attn_prefill_mma.cuh"
+#include "decode.cuh"
+#ifdef ADASPARK_WITH_TCGEN05
+#include "attn_prefill_tc.cuh"
+#endif
+
+using namespace adaspark;
+
+struct adaspark_attn {
+    adaspark_attn_config_t cfg;
+    bool partitioned;
+    int B, T, H, W, n_text_max;
+    int C, N, S_v, S_cap;
+    adaspark_attn_layout_t layout;
+    // workspace carving (byte offsets)
+    size_t fw_status_off, fw_mask_off, fw_logits_off, fw_qcube_off, fw_total;
+    int fw_chunk_tiles;
+    size_t dc_status_off, dc_bitmap_off, dc_items_off, dc_nitems_off, dc_partial_off, dc_total;
+    int dc_splits;
+    int prefill_kernel;
+    int sm_count;
+    int64_t launches;
+    char err[256];
+};
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr size_t kLogitsBudget = 64ull << 20;   // score scratch stays well inside the 126 MB L2
+size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
+
+adaspark_status_t fail(adaspark_attn* h, adaspark_status_t st, const char* fmt, ...) {
+    if (h) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(h->err, sizeof(h->err), fmt, ap);
+        va_end(ap);
+    }
+    return st;
+}
+
+Geom make_geom(const adaspark_attn* h, int n_text) {
+    Geom g;
+    g.B = h->B; g.T = h->T; g.H = h->H; g.W = h->W;
+    g.ct = h->cfg.cube_t; g.ch = h->cfg.cube_h; g.cw = h->cfg.cube_w;
+    g.nH = h->H / g.ch; g.nW = h->W / g.cw;
+    g.C = h->C; g.N = h->N;
+    g.S_v = h->S_v; g.n_text = n_text; g.S = h->S_v + n_text;
+    g.S_cap = h->S_cap;
+    g.n_words = (h->N + 31) / 32;
+    g.n_tiles = (g.S + kTileRows - 1) / kTileRows;
+    g.n_tiles_cap = h->S_cap / kTileRows;
+    g.n_kv_blocks_cap = h->S_cap / kBlockTok;
+    g.Hq = h->cfg.n_q_heads; g.Hkv = h->cfg.n_kv_heads; g.G = g.Hq / g.Hkv; g.D = h->cfg.head_dim;
+    g.N_ld = (h->N + 63) / 64 * 64;
+    double scale = h->cfg.softmax_scale > 0.f ? (double)h->cfg.softmax_scale : 1.0 / std::sqrt((double)g.D);
+    g.scale_d = scale;
+    g.scale = (float)scale;
+    g.scale_log2 = (float)(scale * 1.4426950408889634);
+    g.top_p = (double)h->cfg.top_p;
+    return g;
+}
+
+bool launch_ok(adaspark_attn* h, const char* what) {
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        fail(h, ADASPARK_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+        return false;
+    }
+    h->launches++;
+    return true;
+}
+
+template <typename K>
+bool set_smem(adaspark_attn* h, K kernel, size_t bytes, const char* what) {
+    if (bytes <= 48 * 1024) return true;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e != cudaSuccess) {
+        fail(h, ADASPARK_ERR_CUDA, "%s: cudaFuncSetAttribute(%zu): %s", what, bytes, cudaGetErrorString(e));
+        return false;
+    }
+    return true;
+}
+
+}  // namespace
+
+extern "C" {
+
+adaspark_status_t adaspark_attn_create(const adaspark_attn_config_t* config, adaspark_attn_t** out_handle) {
+    if (!config || !out_handle) return ADASPARK_ERR_INVALID_ARG;
+    *out_handle = nullptr;
+    if (config->cube_t <= 0 || config->cube_h <= 0 || config->cube_w <= 0 || config->n_q_heads <= 0 ||
+        config->n_kv_heads <= 0 || config->head_dim <= 0 || !(config->top_p > 0.f) ||
+        config->softmax_scale < 0.f || config->device < 0)
+        return ADASPARK_ERR_INVALID_ARG;
+    if (config->n_q_heads % config->n_kv_heads != 0) return ADASPARK_ERR_INVALID_ARG;
+    if (config->head_dim != 64 && config->head_dim != 128) return ADASPARK_ERR_UNSUPPORTED;
+    if (config->n_q_heads / config->n_kv_heads > 16) return ADASPARK_ERR_UNSUPPORTED;
+    long long C = (long long)config->cube_t * config->cube_h * config->cube_w;
+    if (C != 16 && C != 32 && C != 64 && C != 128 && C != 256 && C != 512) return ADASPARK_ERR_UNSUPPORTED;
+    adaspark_attn* h = new (std::nothrow) adaspark_attn();
+    if (!h) return ADASPARK_ERR_INVALID_ARG;
+    std::memset(h, 0, sizeof(*h));
+    h->cfg = *config;
+    h->C = (int)C;
+#ifdef ADASPARK_WITH_TCGEN05
+    h->prefill_kernel = 1;
+#else
+    h->prefill_kernel = 0;
+#endif
+    *out_handle = h;
+    return ADASPARK_OK;
+}
+
+adaspark_status_t adaspark_attn_partition(adaspark_attn_t* h, int32_t batch, int32_t frames, int32_t grid_h,
+                                          int32_t grid_w, int32_t n_text_max, size_t* workspace_bytes) {
+    if (!h) return ADASPARK_ERR_INVALID_ARG;
+    if (batch <= 0 || frames <= 0 || grid_h <= 0 || grid_w <= 0 || n_text_max < 0)
+        return fail(h, ADASPARK_ERR_INVALID_ARG, "partition: non-positive size");
+    const adaspark_attn_config_t& c = h->cfg;
+    if (frames % c.cube_t || grid_h % c.cube_h || grid_w % c.cube_w)
+        return fail(h, ADASPARK_ERR_UNSUPPORTED, "partition: grid %dx%dx%d not divisible by cube %dx%dx%d",
+                    frames, grid_h, grid_w, c.cube_t, c.cube_h, c.cube_w);
+    long long N = (long long)(frames / c.cube_t) * (grid_h / c.cube_h) * (grid_w / c.cube_w);
+    if (N > 4096) return fail(h, ADASPARK_ERR_UNSUPPORTED, "partition: %lld cubes > 4096", N);
+    long long S_v = (long long)frames * grid_h * grid_w;
+    long long S_cap = (S_v + n_text_max + 1 + 127) / 128 * 128;
+    if ((long long)batch * S_cap * c.n_q_heads * c.head_dim >= (1ll << 40) || S_cap >= (1ll << 30))
+        return fail(h, ADASPARK_ERR_UNSUPPORTED, "partition: problem too large");
+    h->B = batch; h->T = frames; h->H = grid_h; h->W = grid_w; h->n_text_max = n_text_max;
+    h->N = (int)N; h->S_v = (int)S_v; h->S_cap = (int)S_cap;
+
+    const int D = c.head_dim, Hq = c.n_q_heads, Hkv = c.n_kv_heads;
+    const size_t n_words = (size_t)(N + 31) / 32, N_ld = (size_t)(N + 63) / 64 * 64;
+    const size_t n_tiles_cap = (size_t)S_cap / kTileRows;
+    adaspark_attn_layout_t& L = h->layout;
+    L.n_cubes = N; L.cube_tokens = h->C; L.s_video = S_v; L.s_cap = S_cap; L.bitmap_words = (int64_t)n_words;
+    L.k_cube_bytes = (int64_t)((size_t)batch * Hkv * S_cap * D * 2);
+    L.v_cube_bytes = L.k_cube_bytes;
+    L.cube_keys_bytes = (int64_t)((size_t)batch * Hkv * N * D * 4);
+
+    // forward workspace: status | per-tile mask matrix | score scratch | cube-major Q (tcgen05 path)
+    size_t off = 0;
+    h->fw_status_off = off; off = align_up(off + 256);
+    h->fw_mask_off = off; off = align_up(off + (size_t)batch * Hq * n_tiles_cap * n_words * kTileRows * 4);
+    size_t total_tiles = (size_t)batch * Hq * n_tiles_cap;
+    size_t tile_bytes = (size_t)kTileRows * N_ld * 8;
+    size_t chunk = kLogitsBudget / tile_bytes;
+    if (chunk < 1) chunk = 1;
+    if (chunk > total_tiles) chunk = total_tiles;
+    h->fw_chunk_tiles = (int)chunk;
+    h->fw_logits_off = off; off = align_up(off + chunk * tile_bytes);
+    h->fw_qcube_off = off; off = align_up(off + (size_t)batch * Hq * S_cap * D * 2);
+    h->fw_total = off;
+    L.forward_workspace_bytes = (int64_t)off;
+
+    // decode workspace: status | bitmaps | block lists | counts | split partials
+    int splits = (int)((4 * 148 + (size_t)batch * Hkv - 1) / ((size_t)batch * Hkv));
+    if (splits < 1) splits = 1;
+    if (splits > 64) splits = 64;
+    h->dc_splits = splits;
+    off = 0;
+    h->dc_status_off = off; off = align_up(off + 256);
+    h->dc_bitmap_off = off; off = align_up(off + (size_t)batch * Hq * n_words * 4);
+    h->dc_items_off = off; off = align_up(off + (size_t)batch * Hkv * (S_cap / kBlockTok) * 4);
+    h->dc_nitems_off = off; off = align_up(off + (size_t)batch * Hkv * 4);
+    h->dc_partial_off = off; off = align_up(off + (size_t)batch * Hkv * splits * 16 * (D + 2) * 4);
+    h->dc_total = off;
+    L.decode_workspace_bytes = (int64_t)off;
+
+    h->partitioned = true;
+    h->err[0] = 0;
+    if (workspace_bytes) *workspace_bytes = h->fw_total > h->dc_total ? h->fw_total : h->dc_total;
+    return ADASPARK_OK;
+}
+
+adaspark_status_t adaspark_attn_get_layout(const adaspark_attn_t* h, adaspark_attn_layout_t* out_layout) {
+    if (!h || !out_layout) return ADASPARK_ERR_INVALID_ARG;
+    if (!h->partitioned) return ADASPARK_ERR_NOT_PARTITIONED;
+    *out_layout = h->layout;
+    return ADASPARK_OK;
+}
+
+adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const void* k, const void* v,
+                                        int32_t n_text, void* out, void* k_cube, void* v_cube, float* cube_keys,
+                                        uint32_t* sel_bitmap, int32_t* sel_count, void* workspace,
+                                        size_t workspace_bytes, void* cuda_stream) {
+    if (!h) return ADASPARK_ERR_INVALID_ARG;
+    if (!h->partitioned) return fail(h, ADASPARK_ERR_NOT_PARTITIONED, "forward: call adaspark_attn_partition first");
+    if (!k || !v || !k_cube || !v_cube || !cube_keys) return fail(h, ADASPARK_ERR_INVALID_ARG, "forward: NULL k/v/cache pointer");
+    if ((q == nullptr) != (out == nullptr)) return fail(h, ADASPARK_ERR_INVALID_ARG, "forward: q and out must both be given or both be NULL");
+    if (n_text < 0 || n_text > h->n_text_max) return fail(h, ADASPARK_ERR_INVALID_ARG, "forward: n_text %d outside [0, %d]", n_text, h->n_text_max);
+    const bool cache_only = (q == nullptr);
+    if (!cache_only) {
+        if (!workspace) return fail(h, ADASPARK_ERR_INVALID_ARG, "forward: NULL workspace");
+        if (workspace_bytes < h->fw_total) return fail(h, ADASPARK_ERR_WORKSPACE_TOO_SMALL, "forward: workspace %zu < %zu bytes", workspace_bytes, h->fw_total);
+        if ((uintptr_t)workspace % kAlign) return fail(h, ADASPARK_ERR_INVALID_ARG, "forward: workspace not 256-byte aligned");
+    }
+    cudaError_t ce = cudaSetDevice(h->cfg.device);
+    if (ce != cudaSuccess) return fail(h, ADASPARK_ERR_CUDA, "forward: cudaSetDevice(%d): %s", h->cfg.device, cudaGetErrorString(ce));
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    h->launches = 0;
+    const Geom g = make_geom(h, n_text);
+    const int D = g.D;
+    auto* kb = (const __nv_bfloat16*)k;
+    auto* vb = (const __nv_bfloat16*)v;
+    auto* kc = (__nv_bfloat16*)k_cube;
+    auto* vc = (__nv_bfloat16*)v_cube;
+
+    // K1: re-layout + pooling
+    {
+        dim3 grid(g.n_kv_blocks_cap, g.Hkv, g.B);
+        if (D == 128) relayout_pool_kernel<128><<<grid, 256, 0, st>>>(g, kb, vb, kc, vc, cube_keys);
+        else relayout_pool_kernel<64><<<grid, 256, 0, st>>>(g, kb, vb, kc, vc, cube_keys);
+        if (!launch_ok(h, "relayout_pool_kernel")) return ADASPARK_ERR_CUDA;
+        if (g.C > kBlockTok) {
+            pool_large_cubes_kernel<<<dim3(g.N, g.Hkv, g.B), D, 0, st>>>(g, kc, cube_keys);
+            if (!launch_ok(h, "pool_large_cubes_kernel")) return ADASPARK_ERR_CUDA;
+        }
+    }
+    if (cache_only) return ADASPARK_OK;
+
+    char* ws = (char*)workspace;
+    uint32_t* tile_mask = (uint32_t*)(ws + h->fw_mask_off);
+    double* logits = (double*)(ws + h->fw_logits_off);
+    auto* qb = (const __nv_bfloat16*)q;
+
+    // K3: scoring + selection, chunk by chunk
+    {
+        const int total_gt = g.B * g.Hq * g.n_tiles;
+        const size_t sel_smem = (size_t)4 * g.N_ld * sizeof(double);
+        if (!set_smem(h, select_kernel, sel_smem, "select_kernel")) return ADASPARK_ERR_CUDA;
+        for (int gt0 = 0; gt0 < total_gt; gt0 += h->fw_chunk_tiles) {
+            int n_gt = total_gt - gt0 < h->fw_chunk_tiles ? total_gt - gt0 : h->fw_chunk_tiles;
+            dim3 sgrid(n_gt, g.N_ld / kScoreCols);
+            if (D == 128) score_kernel<128><<<sgrid, 256, 0, st>>>(g, gt0, qb, cube_keys, logits);
+            else score_kernel<64><<<sgrid, 256, 0, st>>>(g, gt0, qb, cube_keys, logits);
+            if (!launch_ok(h, "score_kernel")) return ADASPARK_ERR_CUDA;
+            select_kernel<<<n_gt * kTileRows / 4, 128, sel_smem, st>>>(g, gt0, n_gt, logits, tile_mask, sel_bitmap, sel_count);
+            if (!launch_ok(h, "select_kernel")) return ADASPARK_ERR_CUDA;
+        }
+    }
+
+    // K4: gathered attention
+    {
+        dim3 grid(g.n_tiles, g.Hq, g.B);
+        if (D == 128) {
+            size_t smem = sizeof(MmaAttnSmem<128>);
+            if (!set_smem(h, attn_prefill_mma_kernel<128>, smem, "attn_prefill_mma_kernel")) return ADASPARK_ERR_CUDA;
+            attn_prefill_mma_kernel<128><<<grid, 256, smem, st>>>(g, qb, kc, vc, tile_mask, (__nv_bfloat16*)out);
+        } else {
+            size_t smem = sizeof(MmaAttnSmem<64>);
+            if (!set_smem(h, attn_prefill_mma_kernel<64>, smem, "attn_prefill_mma_kernel")) return ADASPARK_ERR_CUDA;
+            attn_prefill_mma_kernel<64><<<grid, 256, smem, st>>>(g, qb, kc, vc, tile_mask, (__nv_bfloat16*)out);
+        }
+        if (!launch_ok(h, "attn_prefill_mma_kernel")) return ADASPARK_ERR_CUDA;
+    }
+    return ADASPARK_OK;
+}
+
+adaspark_status_t adaspark_attn_decode(adaspark_attn_t* h, const void* q_new, const void* k_new, const void* v_new,
+                                       void* k_cube, void* v_cube, const float* cube_keys, const int32_t* text_len,
+                                       void* out, uint32_t* sel_bitmap, void* workspace, size_t workspace_bytes,
+                                       void* cuda_stream) {
+    if (!h) return ADASPARK_ERR_INVALID_ARG;
+    if (!h->partitioned) return fail(h, ADASPARK_ERR_NOT_PARTITIONED, "decode: call adaspark_attn_partition first");
+    if (!q_new || !k_cube || !v_cube || !cube_keys || !text_len || !out || !workspace)
+        return fail(h, ADASPARK_ERR_INVALID_ARG, "decode: NULL pointer");
+    if ((k_new == nullptr) != (v_new == nullptr)) return fail(h, ADASPARK_ERR_INVALID_ARG, "decode: k_new and v_new must both be given or both be NULL");
+    if (workspace_bytes < h->dc_total) return fail(h, ADASPARK_ERR_WORKSPACE_TOO_SMALL, "decode: workspace %zu < %zu bytes", workspace_bytes, h->dc_total);
+    if ((uintptr_t)workspace % kAlign) return fail(h, ADASPARK_ERR_INVALID_ARG, "decode: workspace not 256-byte aligned");
+    cudaError_t ce = cudaSetDevice(h->cfg.device);
+    if (ce != cudaSuccess) return fail(h, ADASPARK_ERR_CUDA, "decode: cudaSetDevice(%d): %s", h->cfg.device, cudaGetErrorString(ce));
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    h->launches = 0;
+    const Geom g = make_geom(h, h->n_text_max);
+    const int D = g.D;
+    char* ws = (char*)workspace;
+    int32_t* status = (int32_t*)(ws + h->dc_status_off);
+    uint32_t* dec_bitmap = (uint32_t*)(ws + h->dc_bitmap_off);
+    int32_t* items = (int32_t*)(ws + h->dc_items_off);
+    int32_t* n_items = (int32_t*)(ws + h->dc_nitems_off);
+    float* partial = (float*)(ws + h->dc_partial_off);
+    auto* kc = (__nv_bfloat16*)k_cube;
+    auto* vc = (__nv_bfloat16*)v_cube;
+    auto* qn = (const __nv_bfloat16*)q_new;
+
+    if (k_new) {
+        decode_append_kernel<<<g.B, 256, 0, st>>>(g, (const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new, kc, vc, text_len, status);
+        if (!launch_ok(h, "decode_append_kernel")) return ADASPARK_ERR_CUDA;
+    }
+    {
+        size_t smem = (size_t)g.N_ld * sizeof(double);
+        decode_score_select_kernel<<<dim3(g.Hq, g.B), 256, smem, st>>>(g, qn, cube_keys, dec_bitmap, sel_bitmap);
+        if (!launch_ok(h, "decode_score_select_kernel")) return ADASPARK_ERR_CUDA;
+    }
+    decode_plan_kernel<<<dim3(g.Hkv, g.B), 32, 0, st>>>(g, dec_bitmap, text_len, items, n_items);
+    if (!launch_ok(h, "decode_plan_kernel")) return ADASPARK_ERR_CUDA;
+    {
+        dim3 grid(h->dc_splits, g.Hkv, g.B);
+        if (D == 128) {
+            size_t smem = sizeof(DecodeSmem<128>);
+            if (!set_smem(h, decode_splitkv_kernel<128>, smem, "decode_splitkv_kernel")) return ADASPARK_ERR_CUDA;
+            decode_splitkv_kernel<128><<<grid, kDecodeThreads, smem, st>>>(g, h->dc_splits, qn, kc, vc, dec_bitmap, text_len, items, n_items, partial);
+        } else {
+            size_t smem = sizeof(DecodeSmem<64>);
+            if (!set_smem(h, decode_splitkv_kernel<64>, smem, "decode_splitkv_kernel")) return ADASPARK_ERR_CUDA;
+            decode_splitkv_kernel<64><<<grid, kDecodeThreads, smem, st>>>(g, h->dc_splits, qn, kc, vc, dec_bitmap, text_len, items, n_items, partial);
+        }
+        if (!launch_ok(h, "decode_splitkv_kernel")) return ADASPARK_ERR_CUDA;
+    }
+    decode_combine_kernel<<<dim3(g.Hq, g.B), D, 0, st>>>(g, h->dc_splits, partial, (__nv_bfloat16*)out);
+    if (!launch_ok(h, "decode_combine_kernel")) return ADASPARK_ERR_CUDA;
+    return ADASPARK_OK;
+}
+
+adaspark_status_t adaspark_attn_destroy(adaspark_attn_t* h) {
+    delete h;
+    return ADASPARK_OK;
+}
+
+const char* adaspark_attn_last_error(const adaspark_attn_t* h) { return h ? h->err : ""; }
+
+int64_t adaspark_attn_last_launch_count(const adaspark_attn_t* h) { return h ? h->launches : 0; }
+
+adaspark_status_t adaspark_attn_set_prefill_kernel(adaspark_attn_t* h, int32_t which) {
+    if (!h) return ADASPARK_ERR_INVALID_ARG;
+#ifdef ADASPARK_WITH_TCGEN05
+    if (which != 0 && which != 1) return fail(h, ADASPARK_ERR_UNSUPPORTED, "set_prefill_kernel: unknown kernel %d", which);
+#else
+    if (which != 0) return fail(h, ADASPARK_ERR_UNSUPPORTED, "set_prefill_kernel: kernel %d not built", which);
+#endif
+    h->prefill_kernel = which;
+    return ADASPARK_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,116 @@
+// Shared device-side definitions for the AdaS-Attn kernels (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace adaspark {
+
+constexpr int kTileRows = 128;  // query rows per tile (cube-major positions)
+constexpr int kBlockTok = 64;   // key/value tokens per block (cube-major positions)
+
+// Geometry of one partitioned problem (Sec. 3.1).  "pos" is the cube-major position of a token:
+// video token of cube c with intra-cube rank r sits at pos = c*C + r, text token u at S_v + u.
+struct Geom {
+    int B, T, H, W;      // batch, frames, patch rows, patch columns
+    int ct, ch, cw;      // cube window
+    int nH, nW;          // cube grid: H/ch, W/cw
+    int C, N;            // tokens per cube, cubes
+    int S_v, n_text, S;  // video tokens, text tokens of this call, total
+    int S_cap;           // cache rows per (b, kv head), multiple of 128
+    int n_words;         // ceil(N/32)
+    int n_tiles;         // ceil(S/128) query tiles of this call
+    int n_tiles_cap;     // S_cap/128 (stride of per-tile buffers)
+    int n_kv_blocks_cap; // S_cap/64
+    int Hq, Hkv, G, D;
+    int N_ld;            // leading dimension of the logits scratch (N rounded up to 64)
+    float scale;         // logit scale as float (attention softmax)
+    float scale_log2;    // scale * log2(e)
+    double scale_d;      // logit scale in double (selection scores)
+    double top_p;
+};
+
+// O1 inverse: cube-major position -> raster token index.
+__device__ __forceinline__ int pos_to_raster(const Geom& g, int pos) {
+    if (pos >= g.S_v) return pos;
+    int c = pos / g.C, r = pos - c * g.C;
+    int cx = c % g.nW;
+    int cy = (c / g.nW) % g.nH;
+    int cb = c / (g.nW * g.nH);
+    int rx = r % g.cw;
+    int ry = (r / g.cw) % g.ch;
+    int rt = r / (g.cw * g.ch);
+    return ((cb * g.ct + rt) * g.H + (cy * g.ch + ry)) * g.W + (cx * g.cw + rx);
+}
+
+// Number of candidate cubes of the row at `pos`: preceding cubes for video, all cubes for text.
+__device__ __forceinline__ int n_candidates(const Geom& g, int pos) {
+    return pos < g.S_v ? pos / g.C : g.N;
+}
+
+// Per-tile selection mask matrix: word w of row r of global tile gt at
+// mask[(gt * n_words + w) * 128 + r]; gt = (b*Hq + h) * n_tiles_cap + tile.
+__device__ __forceinline__ size_t mask_index(const Geom& g, int b, int h, int tile, int w, int r) {
+    return ((size_t)((b * g.Hq + h) * g.n_tiles_cap + tile) * g.n_words + w) * kTileRows + r;
+}
+
+// Key visibility (Eq. 3 + text rule): may the row at cube-major position pr attend the key at pk?
+// `word` is the row's selection word that covers cube pk/C (bits of cubes that are not
+// candidates of the row are never set by the selection kernel).
+__device__ __forceinline__ bool key_allowed(const Geom& g, int pr, int pk, uint32_t word) {
+    if (pk <= pr && (pk >= g.S_v || pk / g.C == pr / g.C)) return true;  // own cube / text prefix
+    if (pk < g.S_v) return (word >> ((pk / g.C) & 31)) & 1u;              // selected cube
+    return false;
+}
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(smem_u32(smem_dst)),
+                 "l"(gmem_src));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;\n" ::"n"(N));
+}
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3,
+                                            const void* smem_ptr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(smem_u32(smem_ptr)));
+}
+
+// D = A(16x16, row) * B(16x8, col) + D, bf16 inputs, fp32 accumulate.
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0,
+                                               uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, "
+        "{%8,%9}, {%0,%1,%2,%3};\n"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// D = A(8x4, row) * B(4x8, col) + D in fp64.
+__device__ __forceinline__ void mma_f64_884(double (&d)[2], double a, double b) {
+    asm volatile(
+        "mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};\n"
+        : "+d"(d[0]), "+d"(d[1])
+        : "d"(a), "d"(b));
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm volatile("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+    return y;
+}
+
+}  // namespace adaspark

@@ -1,0 +1,84 @@
+// K1: cube-major re-layout of K and V (Algorithm 1, "Reshape K,V into Cubes") fused with the
+// per-cube mean key (Sec. 3.2, definition under Eq. 1).  HBM-bound: every K/V element is read
+// once and written once.
+//
+// One CTA handles one block of 64 consecutive cube-major positions of one (batch, kv head):
+//   k_cube [B,Hkv,S_cap,D]        row pos            <- K[b, raster(pos), g, :]
+//   v_cube [B,Hkv,S_cap/64,D,64]  block blk, V^T     <- V[b, raster(blk*64 + tok), g, d]
+//   cube_keys [B,Hkv,N,D] fp32    mean over the C keys of each cube inside the block (C <= 64);
+//                                 cubes larger than a block are pooled by pool_large_cubes_kernel.
+// Positions >= S are zero-filled so that later tensor-core reads never meet non-finite data.
+#pragma once
+#include "common.cuh"
+
+namespace adaspark {
+
+template <int D>
+__global__ void __launch_bounds__(256) relayout_pool_kernel(Geom g, const __nv_bfloat16* __restrict__ k,
+                                                            const __nv_bfloat16* __restrict__ v,
+                                                            __nv_bfloat16* __restrict__ k_cube,
+                                                            __nv_bfloat16* __restrict__ v_cube,
+                                                            float* __restrict__ cube_keys) {
+    constexpr int kChunks = D / 8;    // 16-byte chunks per row
+    constexpr int kVPitch = D + 2;    // padded pitch (elements) of the V staging tile
+    __shared__ __align__(16) __nv_bfloat16 Ks[kBlockTok][D];
+    __shared__ __align__(16) __nv_bfloat16 Vs[kBlockTok][kVPitch];
+
+    const int blk = blockIdx.x, gk = blockIdx.y, b = blockIdx.z;
+    const int pos0 = blk * kBlockTok;
+    const int tid = threadIdx.x;
+
+    for (int idx = tid; idx < kBlockTok * kChunks; idx += 256) {
+        int row = idx / kChunks, c = idx - row * kChunks;
+        int pos = pos0 + row;
+        uint4 kv4 = make_uint4(0, 0, 0, 0), vv4 = make_uint4(0, 0, 0, 0);
+        if (pos < g.S) {
+            size_t src = ((size_t)(b * g.S + pos_to_raster(g, pos)) * g.Hkv + gk) * D + c * 8;
+            kv4 = *reinterpret_cast<const uint4*>(k + src);
+            vv4 = *reinterpret_cast<const uint4*>(v + src);
+        }
+        *reinterpret_cast<uint4*>(&Ks[row][c * 8]) = kv4;
+        *reinterpret_cast<uint4*>(k_cube + ((size_t)(b * g.Hkv + gk) * g.S_cap + pos) * D + c * 8) = kv4;
+        uint32_t* vdst = reinterpret_cast<uint32_t*>(&Vs[row][c * 8]);
+        vdst[0] = vv4.x; vdst[1] = vv4.y; vdst[2] = vv4.z; vdst[3] = vv4.w;
+    }
+    __syncthreads();
+
+    // V^T: 8 consecutive threads write one 128-byte row (64 tokens of one d).
+    __nv_bfloat16* vt = v_cube + ((size_t)(b * g.Hkv + gk) * g.n_kv_blocks_cap + blk) * D * kBlockTok;
+    for (int idx = tid; idx < D * 8; idx += 256) {
+        int d = idx >> 3, tc = idx & 7;
+        __align__(16) __nv_bfloat16 tmp[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) tmp[i] = Vs[tc * 8 + i][d];
+        *reinterpret_cast<uint4*>(vt + d * kBlockTok + tc * 8) = *reinterpret_cast<uint4*>(tmp);
+    }
+
+    // Mean keys of the cubes that lie inside this block (exact fp64 sum, one rounding to fp32).
+    if (g.C <= kBlockTok && pos0 < g.S_v) {
+        int cubes_here = kBlockTok / g.C;
+        for (int idx = tid; idx < cubes_here * D; idx += 256) {
+            int cb = idx / D, d = idx - cb * D;
+            int cube = pos0 / g.C + cb;
+            if (cube < g.N) {
+                double acc = 0.0;
+                for (int r = 0; r < g.C; ++r) acc += (double)__bfloat162float(Ks[cb * g.C + r][d]);
+                cube_keys[((size_t)(b * g.Hkv + gk) * g.N + cube) * D + d] = (float)(acc / (double)g.C);
+            }
+        }
+    }
+}
+
+// Mean keys for cubes of more than 64 tokens: one CTA per (cube, kv head, batch), D threads,
+// reading the cube-major keys just written by relayout_pool_kernel.
+__global__ void pool_large_cubes_kernel(Geom g, const __nv_bfloat16* __restrict__ k_cube,
+                                        float* __restrict__ cube_keys) {
+    const int cube = blockIdx.x, gk = blockIdx.y, b = blockIdx.z, d = threadIdx.x;
+    if (d >= g.D) return;
+    const __nv_bfloat16* src = k_cube + ((size_t)(b * g.Hkv + gk) * g.S_cap + (size_t)cube * g.C) * g.D + d;
+    double acc = 0.0;
+    for (int r = 0; r < g.C; ++r) acc += (double)__bfloat162float(src[(size_t)r * g.D]);
+    cube_keys[((size_t)(b * g.Hkv + gk) * g.N + cube) * g.D + d] = (float)(acc / (double)g.C);
+}
+
+}  // namespace adaspark

@@ -1,0 +1,103 @@
+"""GPU parity of the decode step (append, score+select, split-KV attention, combine) against the
+CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2604_08077_b200 import inputs
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+def run_decode(wl, text_len, *, top_p=None, n_text_max=None, append=True):
+    eng = pu.make_engine(wl, n_text_max=n_text_max, top_p=top_p)
+    k, v = wl.k.cuda(), wl.v.cuda()
+    eng.forward(None, k, v, wl.n_text)                    # build the caches only
+    tl = torch.tensor(text_len, dtype=torch.int32, device="cuda")
+    if append:
+        out, bitmap = eng.decode(wl.q_new.cuda(), wl.k_new.cuda(), wl.v_new.cuda(), tl,
+                                 want_selection=True)
+    else:
+        out, bitmap = eng.decode(wl.q_new.cuda(), None, None, tl, want_selection=True)
+    torch.cuda.synchronize()
+    return eng, out, bitmap
+
+
+def compare_decode(wl, text_len, out, bitmap, *, top_p=None, batch_index=None, label=""):
+    sh = pu.oracle_shape(wl, top_p)
+    res = oracle.decode(sh, wl.k, wl.v, text_len, wl.q_new, wl.k_new, wl.v_new,
+                        batch_index=batch_index)
+    idx = list(range(wl.B)) if batch_index is None else list(batch_index)
+    got_sel = pu.unpack_bitmap(bitmap, sh.N)[idx]
+    same = (got_sel == res["sel"]).all(axis=-1)
+    bad = ~same & (res["margin"] >= pu.TIE_MARGIN)
+    assert not bad.any(), f"{label}: selection differs on rows {np.argwhere(bad)[:5].tolist()}"
+    got = out[idx, 0].float().cpu().numpy()
+    ref = res["out"]
+    max_abs = float(np.abs(got[same] - ref[same]).max())
+    mean_rel = float(np.abs(got[same] - ref[same]).mean() / np.abs(ref[same]).mean())
+    assert max_abs <= pu.MAX_ABS_TOL and mean_rel <= pu.MEAN_REL_TOL, (label, max_abs, mean_rel)
+    return {"rows": int(same.size), "tie_exempt": int((~same).sum()), "max_abs": max_abs,
+            "mean_rel": mean_rel, "mean_selected": float(res["count"].mean())}
+
+
+@pytest.mark.parametrize("case", ["d128_c64", "d64_c32", "c256", "c16_straddle"])
+def test_small_decode(case):
+    kw = {"d128_c64": dict(),
+          "d64_c32": dict(T=8, H=8, W=8, cube=(2, 4, 4), n_text=64, Hq=4, Hkv=4, D=64, top_p=0.7),
+          "c256": dict(T=8, H=16, W=16, cube=(4, 8, 8), n_text=10, Hq=16, Hkv=1, D=128),
+          "c16_straddle": dict(T=2, H=4, W=12, cube=(1, 4, 4), n_text=70, Hq=6, Hkv=2, D=64)}[case]
+    wl = inputs.small_decode(seed=40, **kw)
+    text_len = [wl.n_text - 3 * b for b in range(wl.B)]      # different lengths per sequence
+    eng, out, bitmap = run_decode(wl, text_len)
+    print(case, compare_decode(wl, text_len, out, bitmap, label=case))
+    # the appended token landed in the caches
+    for b in range(wl.B):
+        pos = wl.S_v + text_len[b]
+        assert torch.equal(eng.k_cube[b, :, pos].cpu(), wl.k_new[b, 0])
+        assert torch.equal(eng.v_cube[b, :, pos // 64, :, pos % 64].cpu(), wl.v_new[b, 0])
+
+
+def test_decode_without_append_uses_the_cached_token():
+    wl = inputs.small_decode(seed=41)
+    text_len = [wl.n_text, wl.n_text - 1]
+    eng, out1, bm1 = run_decode(wl, text_len, n_text_max=wl.n_text + 4)
+    tl = torch.tensor(text_len, dtype=torch.int32, device="cuda")
+    out2, bm2 = eng.decode(wl.q_new.cuda(), None, None, tl, want_selection=True)
+    torch.cuda.synchronize()
+    assert torch.equal(out1, out2) and torch.equal(bm1, bm2)
+
+
+def test_decode_zero_text_and_dense_p():
+    wl = inputs.small_decode(seed=42, n_text=0)
+    eng, out, bitmap = run_decode(wl, [0, 0], top_p=1.0, n_text_max=8)
+    rep = compare_decode(wl, [0, 0], out, bitmap, top_p=1.0, label="p=1")
+    assert pu.unpack_bitmap(bitmap, wl.N).all()
+    print(rep)
+
+
+def test_decode_matches_prefill_last_row():
+    """A decode step equals the last text row of a prefill over the appended sequence."""
+    wl = inputs.small_decode(seed=43, B=1, n_text=21)
+    eng, out, bitmap = run_decode(wl, [wl.n_text])
+    full = inputs.Workload(name="appended", B=1, T=wl.T, H=wl.H, W=wl.W, cube=wl.cube,
+                           n_text=wl.n_text + 1, Hq=wl.Hq, Hkv=wl.Hkv, D=wl.D, top_p=wl.top_p,
+                           q=torch.cat([torch.zeros(1, wl.S, wl.Hq, wl.D, dtype=torch.bfloat16), wl.q_new], 1),
+                           k=torch.cat([wl.k, wl.k_new], 1), v=torch.cat([wl.v, wl.v_new], 1))
+    _, out_p, bitmap_p, _ = pu.run_forward(full)
+    assert torch.equal(bitmap_p[0, :, -1], bitmap[0])
+    np.testing.assert_allclose(out[0, 0].float().cpu().numpy(), out_p[0, -1].float().cpu().numpy(),
+                               atol=1e-2)
+
+
+def test_config5_shape_reduced_batch():
+    """Config-5 geometry (131072-token video cache, 2048 cubes, 512 text) at batch 2; the oracle
+    evaluates every (sequence, head) row."""
+    wl = inputs.config5(B=2)
+    text_len = [512, 300]
+    eng, out, bitmap = run_decode(wl, text_len)
+    rep = compare_decode(wl, text_len, out, bitmap, label="cfg5")
+    print("cfg5", rep)

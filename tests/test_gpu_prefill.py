@@ -1,0 +1,117 @@
+"""GPU parity of the prefill path (re-layout, pooling, scoring, selection, attention) against
+the CPU oracle, through the C ABI, on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2604_08077_b200 import inputs
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+def check_caches(wl, eng):
+    """k_cube / v_cube / cube_keys against the oracle's permutation and mean keys (bit-exact)."""
+    sh = oracle.shape_of(wl)
+    _, inv = oracle.positions(sh)
+    inv_t = torch.from_numpy(inv)
+    S, s_cap = wl.S, eng.layout.s_cap
+    k_ref = wl.k[:, inv_t].permute(0, 2, 1, 3)                         # [B,Hkv,S,D]
+    v_ref = wl.v[:, inv_t].permute(0, 2, 1, 3)
+    k_got = eng.k_cube.cpu()
+    assert torch.equal(k_got[:, :, :S], k_ref)
+    assert (k_got[:, :, S:] == 0).all()
+    v_got = eng.v_cube.cpu().permute(0, 1, 2, 4, 3).reshape(wl.B, wl.Hkv, s_cap, wl.D)
+    assert torch.equal(v_got[:, :, :S], v_ref)
+    assert (v_got[:, :, S:] == 0).all()
+    kbar = oracle.mean_keys(sh, wl.k).astype(np.float32)                # one rounding to fp32
+    assert np.array_equal(eng.cube_keys.cpu().numpy(), kbar)
+
+
+SMALL_CASES = {
+    "cfg1": lambda: inputs.config1(),
+    "d128_c64_ragged_text": lambda: inputs.small_prefill(seed=7),
+    "d64_c32_no_text": lambda: inputs.small_prefill(seed=8, T=4, H=8, W=8, cube=(2, 4, 4), n_text=0,
+                                                    Hq=2, Hkv=2, D=64, top_p=0.7),
+    "c256_gqa4": lambda: inputs.small_prefill(seed=9, T=8, H=16, W=8, cube=(4, 8, 8), n_text=5,
+                                              Hq=4, Hkv=1, D=128, top_p=0.8),
+    "c16_batch2_odd_cubes": lambda: inputs.small_prefill(seed=10, B=2, T=3, H=4, W=12, cube=(1, 4, 4),
+                                                         n_text=130, Hq=2, Hkv=1, D=64, top_p=0.9),
+    "single_cube": lambda: inputs.small_prefill(seed=11, T=4, H=4, W=4, cube=(4, 4, 4), n_text=3,
+                                                Hq=1, Hkv=1, D=128, top_p=0.9),
+    "sharp_scores": lambda: inputs.small_prefill(seed=12, T=16, H=8, W=8, n_text=17, top_p=0.5,
+                                                 offset_std=3.0),
+}
+
+
+@pytest.mark.parametrize("case", sorted(SMALL_CASES))
+@pytest.mark.parametrize("kernel", [0])
+def test_small_prefill_every_row(case, kernel):
+    """Element-by-element parity on every row: caches, selection bitmaps, counts, outputs."""
+    wl = SMALL_CASES[case]()
+    eng, out, bitmap, count = pu.run_forward(wl, prefill_kernel=kernel)
+    check_caches(wl, eng)
+    rep = pu.compare_rows(wl, oracle.all_rows(oracle.shape_of(wl)), out, bitmap, count, label=case)
+    assert rep["rows"] == wl.B * wl.Hq * wl.S
+    print(case, rep)
+
+
+@pytest.mark.parametrize("p", [1.0, 1e-6])
+def test_degenerate_p(p):
+    """p = 1 is dense causal attention over the cube-major order; p -> 0 keeps the argmax cube."""
+    wl = inputs.small_prefill(seed=21, T=8, H=8, W=8, n_text=20)
+    eng, out, bitmap, count = pu.run_forward(wl, top_p=p)
+    rep = pu.compare_rows(wl, oracle.all_rows(oracle.shape_of(wl)), out, bitmap, count, top_p=p,
+                          label=f"p={p}")
+    sel = pu.unpack_bitmap(bitmap, wl.N)
+    sh = oracle.shape_of(wl)
+    pos, _ = oracle.positions(sh)
+    n_cand = np.where(np.arange(wl.S) < wl.S_v, pos // wl.C, wl.N)
+    if p >= 1.0:
+        assert np.array_equal(sel.sum(-1), np.broadcast_to(n_cand, sel.shape[:-1]))
+    else:
+        assert np.array_equal(sel.sum(-1), np.broadcast_to(np.minimum(n_cand, 1), sel.shape[:-1]))
+    print(rep)
+
+
+def test_cache_only_forward_builds_the_caches():
+    wl = inputs.small_prefill(seed=31)
+    eng = pu.make_engine(wl)
+    eng.forward(None, wl.k.cuda(), wl.v.cuda(), wl.n_text)
+    torch.cuda.synchronize()
+    check_caches(wl, eng)
+
+
+def test_selection_only_outputs_are_optional_and_repeatable():
+    wl = inputs.small_prefill(seed=32)
+    eng, out1, bitmap, count = pu.run_forward(wl)
+    out2, b2, c2 = eng.forward(wl.q.cuda(), wl.k.cuda(), wl.v.cuda(), wl.n_text, want_selection=False)
+    torch.cuda.synchronize()
+    assert b2 is None and c2 is None
+    assert torch.equal(out1, out2)
+    assert eng.launches() >= 4
+
+
+def test_config2_full_size_sampled_rows():
+    """Config 2 at full size (the bench workload): selection on a large row sample, outputs on
+    a sample that includes whole query tiles (first, middle, text)."""
+    wl = inputs.config2()
+    eng, out, bitmap, count = pu.run_forward(wl)
+    rows = pu.sample_rows(wl, 1500, seed=2, whole_tiles=[(0, 0, 0), (0, 13, 64), (0, 27, 128)])
+    rep = pu.compare_rows(wl, rows, out, bitmap, count, label="cfg2")
+    print("cfg2", rep)
+    # selection only, many more rows
+    sh = pu.oracle_shape(wl)
+    rng = np.random.default_rng(5)
+    rows = np.stack([np.zeros(40000, np.int64), rng.integers(0, wl.Hq, 40000),
+                     rng.integers(0, wl.S, 40000)], axis=1)
+    res = oracle.rows(sh, wl.q, wl.k, wl.v, rows, attend=False)
+    dev = bitmap.device
+    got = pu.unpack_bitmap(bitmap[0, torch.from_numpy(rows[:, 1]).to(dev),
+                                  torch.from_numpy(rows[:, 2]).to(dev)], wl.N)
+    diff = (got != res["sel"]).any(axis=1)
+    assert not (diff & (res["margin"] >= pu.TIE_MARGIN)).any()
+    print("cfg2 selection rows", len(rows), "tie-exempt", int(diff.sum()),
+          "near-tie", int((res["margin"] < pu.TIE_MARGIN).sum()))
