@@ -75,6 +75,16 @@ typedef struct {
     int64_t decode_workspace_bytes;
 } adaspark_attn_layout_t;
 
+/* Header the library keeps in the first bytes of the workspace of _forward / _decode.  It is
+ * reset at the start of every call; the caller may copy it to the host after synchronising. */
+typedef struct {
+    int32_t status;               /* 0 = ok; 1 = text_len out of range (decode)              */
+    int32_t reserved;
+    uint64_t executed_kv_blocks;  /* prefill: (query tile, 64-key block) pairs the attention
+                                     kernel computed; executed FLOPs = this * 128*64*D*4    */
+    uint64_t decode_kv_blocks;    /* decode: 64-key blocks gathered, summed over (b, kv head) */
+} adaspark_attn_workspace_header_t;
+
 /* Create a handle for one configuration.  Host only.  Fails with ERR_UNSUPPORTED for a
  * head_dim other than 64/128, a cube window whose token count C is not one of
  * {16, 32, 64, 128, 256, 512}, or a GQA group size above 16; with ERR_INVALID_ARG for
@@ -116,14 +126,14 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t *handle, const void *q, 
 /* Decode: one new text token per sequence (the text-token rule after Eq. 3 applied to a row
  * appended after the cached sequence; the new token attends itself).
  *   q_new        in : bf16 [B, 1, Hq, D].
- *   k_new, v_new in : bf16 [B, 1, Hkv, D]; appended to the caches at text slot text_len[b]
- *                     (both NULL: the caller already appended them and text_len[b] counts them
- *                     out, i.e. the row attends text slots 0..text_len[b]-1... see below).
+ *   k_new, v_new in : bf16 [B, 1, Hkv, D]; written into the caches at text slot text_len[b].
+ *                     Both may be NULL when the caller has already stored the new token's K/V
+ *                     in slot text_len[b] of the caches.
  *   k_cube, v_cube  in/out, cube_keys in: caches written by _forward.
- *   text_len     in : device int32 [B], text tokens already cached (before this step);
- *                     text_len[b] + 1 <= n_text_max + 1.  With k_new/v_new NULL the row attends
- *                     text slots 0..text_len[b] and slot text_len[b] must already hold the
- *                     new token's K/V.
+ *   text_len     in : device int32 [B], text tokens cached before this step, 0 <= text_len[b]
+ *                     <= n_text_max.  The row attends text slots 0..text_len[b] (itself included).
+ *                     A value outside that range sets `status` in the workspace header to 1 and
+ *                     yields a zero output row for that sequence.
  *   out          out: bf16 [B, 1, Hq, D].
  *   sel_bitmap   out, nullable: uint32 [B, Hq, bitmap_words].
  *   workspace    device scratch of at least decode_workspace_bytes, 256-byte aligned. */
@@ -142,6 +152,14 @@ const char *adaspark_attn_last_error(const adaspark_attn_t *handle);
 
 /* Number of kernel launches the most recent _forward / _decode enqueued (host counter). */
 int64_t adaspark_attn_last_launch_count(const adaspark_attn_t *handle);
+
+/* Stage timing for measurement: when enabled, _forward / _decode record CUDA events on the
+ * caller's stream around their stages.  adaspark_attn_get_stage_times waits for the last
+ * recorded event (the only host synchronisation in the library, and only in this call) and
+ * returns milliseconds: prefill {re-layout+pooling, scoring+selection, attention, 0};
+ * decode {append, scoring+selection+plan, split-KV attention, combine}. */
+adaspark_status_t adaspark_attn_enable_stage_timing(adaspark_attn_t *handle, int32_t enable);
+adaspark_status_t adaspark_attn_get_stage_times(adaspark_attn_t *handle, float *ms_out /* host [4] */);
 
 /* Selects the prefill attention kernel: 0 = mma.sync (legacy tensor path), 1 = tcgen05/TMEM
  * with TMA-staged tiles.  Default 1 when built in. ERR_UNSUPPORTED for an unknown value. */

@@ -45,7 +45,8 @@ _lib: Optional[ctypes.CDLL] = None
 EXPORTS = ["adaspark_attn_create", "adaspark_attn_partition", "adaspark_attn_get_layout",
            "adaspark_attn_forward", "adaspark_attn_decode", "adaspark_attn_destroy",
            "adaspark_attn_last_error", "adaspark_attn_last_launch_count",
-           "adaspark_attn_set_prefill_kernel"]
+           "adaspark_attn_set_prefill_kernel", "adaspark_attn_enable_stage_timing",
+           "adaspark_attn_get_stage_times"]
 
 
 def load() -> ctypes.CDLL:
@@ -69,6 +70,8 @@ def load() -> ctypes.CDLL:
     lib.adaspark_attn_last_launch_count.argtypes = [vp]
     lib.adaspark_attn_last_launch_count.restype = ctypes.c_int64
     lib.adaspark_attn_set_prefill_kernel.argtypes = [vp, i32]
+    lib.adaspark_attn_enable_stage_timing.argtypes = [vp, i32]
+    lib.adaspark_attn_get_stage_times.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     for name in EXPORTS:
         if name not in ("adaspark_attn_last_error", "adaspark_attn_last_launch_count"):
             getattr(lib, name).restype = ctypes.c_int
@@ -150,6 +153,22 @@ def adaspark_attn_set_prefill_kernel(handle: int, which: int):
     _check(handle, load().adaspark_attn_set_prefill_kernel(handle, which))
 
 
+def adaspark_attn_enable_stage_timing(handle: int, enable: bool):
+    _check(handle, load().adaspark_attn_enable_stage_timing(handle, int(enable)))
+
+
+def adaspark_attn_get_stage_times(handle: int):
+    """Milliseconds of the four stages of the last timed call (waits for its last event)."""
+    ms = (ctypes.c_float * 4)()
+    _check(handle, load().adaspark_attn_get_stage_times(handle, ms))
+    return [float(x) for x in ms]
+
+
+class WorkspaceHeader(ctypes.Structure):
+    _fields_ = [("status", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("executed_kv_blocks", ctypes.c_uint64), ("decode_kv_blocks", ctypes.c_uint64)]
+
+
 # ---- a small convenience owner of the handle and of the caller-side buffers --------------------
 
 class AdaSAttn:
@@ -204,6 +223,11 @@ class AdaSAttn:
                              self.cube_keys, text_len, out, bitmap, self.workspace, self.ws_bytes,
                              stream)
         return out, bitmap
+
+    def header(self) -> WorkspaceHeader:
+        """Copy of the workspace header of the last call (synchronises the device)."""
+        raw = self.workspace[:ctypes.sizeof(WorkspaceHeader)].cpu().numpy().tobytes()
+        return WorkspaceHeader.from_buffer_copy(raw)
 
     def launches(self) -> int:
         return adaspark_attn_last_launch_count(self.handle)

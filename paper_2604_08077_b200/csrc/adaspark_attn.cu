@@ -34,6 +34,9 @@ struct adaspark_attn {
     int prefill_kernel;
     int sm_count;
     int64_t launches;
+    bool timing;
+    cudaEvent_t ev[5];
+    bool ev_recorded;
     char err[256];
 };
 
@@ -73,6 +76,13 @@ Geom make_geom(const adaspark_attn* h, int n_text) {
     g.scale_log2 = (float)(scale * 1.4426950408889634);
     g.top_p = (double)h->cfg.top_p;
     return g;
+}
+
+void mark(adaspark_attn* h, int i, cudaStream_t st) {
+    if (h->timing) {
+        cudaEventRecord(h->ev[i], st);
+        h->ev_recorded = true;
+    }
 }
 
 bool launch_ok(adaspark_attn* h, const char* what) {
@@ -221,6 +231,8 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
     auto* kc = (__nv_bfloat16*)k_cube;
     auto* vc = (__nv_bfloat16*)v_cube;
 
+    if (!cache_only) cudaMemsetAsync((char*)workspace + h->fw_status_off, 0, 256, st);
+    mark(h, 0, st);
     // K1: re-layout + pooling
     {
         dim3 grid(g.n_kv_blocks_cap, g.Hkv, g.B);
@@ -232,9 +244,11 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
             if (!launch_ok(h, "pool_large_cubes_kernel")) return ADASPARK_ERR_CUDA;
         }
     }
+    mark(h, 1, st);
     if (cache_only) return ADASPARK_OK;
 
     char* ws = (char*)workspace;
+    auto* hdr = (adaspark_attn_workspace_header_t*)(ws + h->fw_status_off);
     uint32_t* tile_mask = (uint32_t*)(ws + h->fw_mask_off);
     double* logits = (double*)(ws + h->fw_logits_off);
     auto* qb = (const __nv_bfloat16*)q;
@@ -255,20 +269,23 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
         }
     }
 
+    mark(h, 2, st);
     // K4: gathered attention
     {
         dim3 grid(g.n_tiles, g.Hq, g.B);
         if (D == 128) {
             size_t smem = sizeof(MmaAttnSmem<128>);
             if (!set_smem(h, attn_prefill_mma_kernel<128>, smem, "attn_prefill_mma_kernel")) return ADASPARK_ERR_CUDA;
-            attn_prefill_mma_kernel<128><<<grid, 256, smem, st>>>(g, qb, kc, vc, tile_mask, (__nv_bfloat16*)out);
+            attn_prefill_mma_kernel<128><<<grid, 256, smem, st>>>(g, qb, kc, vc, tile_mask, (__nv_bfloat16*)out, (unsigned long long*)&hdr->executed_kv_blocks);
         } else {
             size_t smem = sizeof(MmaAttnSmem<64>);
             if (!set_smem(h, attn_prefill_mma_kernel<64>, smem, "attn_prefill_mma_kernel")) return ADASPARK_ERR_CUDA;
-            attn_prefill_mma_kernel<64><<<grid, 256, smem, st>>>(g, qb, kc, vc, tile_mask, (__nv_bfloat16*)out);
+            attn_prefill_mma_kernel<64><<<grid, 256, smem, st>>>(g, qb, kc, vc, tile_mask, (__nv_bfloat16*)out, (unsigned long long*)&hdr->executed_kv_blocks);
         }
         if (!launch_ok(h, "attn_prefill_mma_kernel")) return ADASPARK_ERR_CUDA;
     }
+    mark(h, 3, st);
+    mark(h, 4, st);
     return ADASPARK_OK;
 }
 
@@ -290,7 +307,10 @@ adaspark_status_t adaspark_attn_decode(adaspark_attn_t* h, const void* q_new, co
     const Geom g = make_geom(h, h->n_text_max);
     const int D = g.D;
     char* ws = (char*)workspace;
-    int32_t* status = (int32_t*)(ws + h->dc_status_off);
+    auto* hdr = (adaspark_attn_workspace_header_t*)(ws + h->dc_status_off);
+    int32_t* status = &hdr->status;
+    cudaMemsetAsync(hdr, 0, 256, st);
+    mark(h, 0, st);
     uint32_t* dec_bitmap = (uint32_t*)(ws + h->dc_bitmap_off);
     int32_t* items = (int32_t*)(ws + h->dc_items_off);
     int32_t* n_items = (int32_t*)(ws + h->dc_nitems_off);
@@ -303,13 +323,15 @@ adaspark_status_t adaspark_attn_decode(adaspark_attn_t* h, const void* q_new, co
         decode_append_kernel<<<g.B, 256, 0, st>>>(g, (const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new, kc, vc, text_len, status);
         if (!launch_ok(h, "decode_append_kernel")) return ADASPARK_ERR_CUDA;
     }
+    mark(h, 1, st);
     {
         size_t smem = (size_t)g.N_ld * sizeof(double);
         decode_score_select_kernel<<<dim3(g.Hq, g.B), 256, smem, st>>>(g, qn, cube_keys, dec_bitmap, sel_bitmap);
         if (!launch_ok(h, "decode_score_select_kernel")) return ADASPARK_ERR_CUDA;
     }
-    decode_plan_kernel<<<dim3(g.Hkv, g.B), 32, 0, st>>>(g, dec_bitmap, text_len, items, n_items);
+    decode_plan_kernel<<<dim3(g.Hkv, g.B), 32, 0, st>>>(g, dec_bitmap, text_len, items, n_items, (unsigned long long*)&hdr->decode_kv_blocks);
     if (!launch_ok(h, "decode_plan_kernel")) return ADASPARK_ERR_CUDA;
+    mark(h, 2, st);
     {
         dim3 grid(h->dc_splits, g.Hkv, g.B);
         if (D == 128) {
@@ -323,13 +345,41 @@ adaspark_status_t adaspark_attn_decode(adaspark_attn_t* h, const void* q_new, co
         }
         if (!launch_ok(h, "decode_splitkv_kernel")) return ADASPARK_ERR_CUDA;
     }
+    mark(h, 3, st);
     decode_combine_kernel<<<dim3(g.Hq, g.B), D, 0, st>>>(g, h->dc_splits, partial, (__nv_bfloat16*)out);
     if (!launch_ok(h, "decode_combine_kernel")) return ADASPARK_ERR_CUDA;
+    mark(h, 4, st);
     return ADASPARK_OK;
 }
 
 adaspark_status_t adaspark_attn_destroy(adaspark_attn_t* h) {
+    if (h && h->timing)
+        for (int i = 0; i < 5; ++i) cudaEventDestroy(h->ev[i]);
     delete h;
+    return ADASPARK_OK;
+}
+
+adaspark_status_t adaspark_attn_enable_stage_timing(adaspark_attn_t* h, int32_t enable) {
+    if (!h) return ADASPARK_ERR_INVALID_ARG;
+    if (enable && !h->timing) {
+        cudaError_t ce = cudaSetDevice(h->cfg.device);
+        for (int i = 0; i < 5 && ce == cudaSuccess; ++i) ce = cudaEventCreate(&h->ev[i]);
+        if (ce != cudaSuccess) return fail(h, ADASPARK_ERR_CUDA, "enable_stage_timing: %s", cudaGetErrorString(ce));
+        h->timing = true;
+        h->ev_recorded = false;
+    } else if (!enable && h->timing) {
+        for (int i = 0; i < 5; ++i) cudaEventDestroy(h->ev[i]);
+        h->timing = false;
+    }
+    return ADASPARK_OK;
+}
+
+adaspark_status_t adaspark_attn_get_stage_times(adaspark_attn_t* h, float* ms_out) {
+    if (!h || !ms_out) return ADASPARK_ERR_INVALID_ARG;
+    if (!h->timing || !h->ev_recorded) return fail(h, ADASPARK_ERR_INVALID_ARG, "get_stage_times: no timed call recorded");
+    cudaError_t ce = cudaEventSynchronize(h->ev[4]);
+    for (int i = 0; i < 4 && ce == cudaSuccess; ++i) ce = cudaEventElapsedTime(&ms_out[i], h->ev[i], h->ev[i + 1]);
+    if (ce != cudaSuccess) return fail(h, ADASPARK_ERR_CUDA, "get_stage_times: %s", cudaGetErrorString(ce));
     return ADASPARK_OK;
 }
 

@@ -28,7 +28,8 @@ __global__ void __launch_bounds__(256) attn_prefill_mma_kernel(Geom g, const __n
                                                                const __nv_bfloat16* __restrict__ k_cube,
                                                                const __nv_bfloat16* __restrict__ v_cube,
                                                                const uint32_t* __restrict__ tile_mask,
-                                                               __nv_bfloat16* __restrict__ out) {
+                                                               __nv_bfloat16* __restrict__ out,
+                                                               unsigned long long* __restrict__ executed_blocks) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     MmaAttnSmem<D>& sm = *reinterpret_cast<MmaAttnSmem<D>*>(smem_raw);
     constexpr int kQChunks = D / 8;   // 16-byte chunks per K/Q row
@@ -114,8 +115,9 @@ __global__ void __launch_bounds__(256) attn_prefill_mma_kernel(Geom g, const __n
     int kb = next_block(0);
     if (kb < n_blk) load_block(kb, 0);
     cp_async_commit();
-    int stage = 0;
+    int stage = 0, visited = 0;
     while (kb < n_blk) {
+        ++visited;
         int kb_next = next_block(kb + 1);
         if (kb_next < n_blk) load_block(kb_next, stage ^ 1);
         cp_async_commit();
@@ -210,6 +212,7 @@ __global__ void __launch_bounds__(256) attn_prefill_mma_kernel(Geom g, const __n
         kb = kb_next;
     }
     cp_async_wait<0>();
+    if (tid == 0) atomicAdd(executed_blocks, (unsigned long long)visited);
 
     // ---- normalise and store at the raster position
     lA += __shfl_xor_sync(0xffffffffu, lA, 1);

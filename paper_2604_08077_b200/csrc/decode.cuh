@@ -92,7 +92,7 @@ __global__ void __launch_bounds__(256) decode_score_select_kernel(Geom g, const 
 // grid (Hkv, B), 32 threads.  items[(b*Hkv+gk) * n_kv_blocks_cap + i] = block index.
 __global__ void decode_plan_kernel(Geom g, const uint32_t* __restrict__ dec_bitmap,
                                    const int32_t* __restrict__ text_len, int32_t* __restrict__ items,
-                                   int32_t* __restrict__ n_items) {
+                                   int32_t* __restrict__ n_items, unsigned long long* __restrict__ total_blocks) {
     const int gk = blockIdx.x, b = blockIdx.y, lane = threadIdx.x;
     const int tl = text_len[b];
     const int last_pos = g.S_v + tl;                     // position of the new token
@@ -120,7 +120,10 @@ __global__ void decode_plan_kernel(Geom g, const uint32_t* __restrict__ dec_bitm
         if (need) dst[count + __popc(ball & ((1u << lane) - 1u))] = kb;
         count += __popc(ball);
     }
-    if (lane == 0) n_items[b * g.Hkv + gk] = count;
+    if (lane == 0) {
+        n_items[b * g.Hkv + gk] = count;
+        atomicAdd(total_blocks, (unsigned long long)count);
+    }
 }
 
 template <int D>

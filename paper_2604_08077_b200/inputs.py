@@ -65,14 +65,16 @@ class Workload:
         return (self.T // ct) * (self.H // ch) * (self.W // cw)
 
 
-def _gen(seed: int) -> torch.Generator:
-    g = torch.Generator(device="cpu")
+def _gen(seed: int, device: str = "cpu") -> torch.Generator:
+    """Seeded generator.  Tests draw on the CPU (the oracle reads the same bytes); the bench may
+    draw the largest workloads directly on the GPU (same recipe, a different stream of draws)."""
+    g = torch.Generator(device=device)
     g.manual_seed(int(seed))
     return g
 
 
 def _randn(g: torch.Generator, *shape: int, std: float = 1.0) -> torch.Tensor:
-    x = torch.randn(*shape, generator=g, dtype=torch.float32)
+    x = torch.randn(*shape, generator=g, dtype=torch.float32, device=g.device)
     if std != 1.0:
         x.mul_(std)
     return x
@@ -93,9 +95,10 @@ def _add_cube_offsets(k_video: torch.Tensor, g: torch.Generator, T: int, H: int,
 
 def make_prefill(name: str, *, seed: int, B: int, T: int, H: int, W: int,
                  cube: Tuple[int, int, int], n_text: int, Hq: int, Hkv: int, D: int,
-                 top_p: float, offset_std: float, with_q: bool = True) -> Workload:
+                 top_p: float, offset_std: float, with_q: bool = True,
+                 device: str = "cpu") -> Workload:
     """i.i.d. N(0,1) Q/K/V; video K gets a per-cube shared offset of std ``offset_std``."""
-    g = _gen(seed)
+    g = _gen(seed, device)
     S_v = T * H * W
     S = S_v + n_text
     k = _randn(g, B, S, Hkv, D)
@@ -139,9 +142,10 @@ def _static_dynamic_kv(g: torch.Generator, B: int, T: int, H: int, W: int,
 def make_heterogeneous(name: str, *, seed: int, B: int, T: int, H: int, W: int,
                        cube: Tuple[int, int, int], n_text: int, Hq: int, Hkv: int, D: int,
                        top_p: float, offset_std: float = 1.5, noise_std: float = 0.05,
-                       with_q: bool = True, with_decode_token: bool = False) -> Workload:
+                       with_q: bool = True, with_decode_token: bool = False,
+                       device: str = "cpu") -> Workload:
     """Half-static / half-dynamic video (load-imbalance stress), optional text and decode token."""
-    g = _gen(seed)
+    g = _gen(seed, device)
     assert T % 2 == 0 and (T // 2) % cube[0] == 0
     k, v = _static_dynamic_kv(g, B, T, H, W, cube, Hkv, D, offset_std, noise_std)
     if n_text > 0:
@@ -168,32 +172,33 @@ def config1(variant: int = 0) -> Workload:
                         n_text=32, Hq=4, Hkv=4, D=64, top_p=0.9, offset_std=2.0)
 
 
-def config2(variant: int = 0, top_p: float = 0.9) -> Workload:
+def config2(variant: int = 0, top_p: float = 0.9, device: str = "cpu") -> Workload:
     """Qwen2-7B-shaped layer: 64x16x16 video, cube 4x4x4, 128 text, 28/4 heads, D=128."""
     return make_prefill("cfg2_qwen7b_16k", seed=2000 + variant, B=1, T=64, H=16, W=16,
                         cube=(4, 4, 4), n_text=128, Hq=28, Hkv=4, D=128, top_p=top_p,
-                        offset_std=1.5)
+                        offset_std=1.5, device=device)
 
 
-def config3(sigma: float = 1.5, top_p: float = 0.9) -> Workload:
+def config3(sigma: float = 1.5, top_p: float = 0.9, device: str = "cpu") -> Workload:
     """Sweep: 256x16x16 video (1024 cubes), 256 text; sigma in {0.5,1.5,3.0}; p in {.5,.7,.9,.95,1}."""
     variant = {0.5: 0, 1.5: 1, 3.0: 2}[float(sigma)]
     return make_prefill(f"cfg3_sweep_s{sigma}_p{top_p}", seed=3000 + variant, B=1, T=256, H=16,
                         W=16, cube=(4, 4, 4), n_text=256, Hq=28, Hkv=4, D=128, top_p=top_p,
-                        offset_std=float(sigma))
+                        offset_std=float(sigma), device=device)
 
 
-def config4(variant: int = 0) -> Workload:
+def config4(variant: int = 0, device: str = "cpu") -> Workload:
     """Heterogeneous complexity: 512x16x16 video (2048 cubes), first half static, no text."""
     return make_heterogeneous("cfg4_hetero_128k", seed=4000 + variant, B=1, T=512, H=16, W=16,
-                              cube=(4, 4, 4), n_text=0, Hq=28, Hkv=4, D=128, top_p=0.9)
+                              cube=(4, 4, 4), n_text=0, Hq=28, Hkv=4, D=128, top_p=0.9,
+                              device=device)
 
 
-def config5(variant: int = 0, B: int = 16) -> Workload:
+def config5(variant: int = 0, B: int = 16, device: str = "cpu") -> Workload:
     """Decode: B sequences, 131072-token video cache (cfg-4 distribution) + 512 text + 1 new token."""
     return make_heterogeneous("cfg5_decode_128k", seed=5000 + variant, B=B, T=512, H=16, W=16,
                               cube=(4, 4, 4), n_text=512, Hq=28, Hkv=4, D=128, top_p=0.9,
-                              with_q=False, with_decode_token=True)
+                              with_q=False, with_decode_token=True, device=device)
 
 
 def small_prefill(seed: int = 7, *, B: int = 1, T: int = 8, H: int = 8, W: int = 8,
