@@ -144,6 +144,37 @@ adaspark_status_t adaspark_attn_decode(adaspark_attn_t *handle, const void *q_ne
                                        void *workspace, size_t workspace_bytes,
                                        void *cuda_stream);
 
+/* Bytes of decode scratch built into the library image (see adaspark_attn_decode_static). */
+#define ADASPARK_ATTN_STATIC_SCRATCH_BYTES (8u << 20)
+
+/* adaspark_attn_decode without a workspace argument.  (The paper has no counterpart: this entry
+ * point exists only for the convenience of some callers.)
+ *
+ * It is meant for callers that have no way to allocate device memory at the moment they decode:
+ * a serving process that has handed all of the GPU's memory to its own pool and cannot carve a
+ * workspace out of it for a foreign library, or a latency-critical decode loop in which a
+ * cudaMalloc (which may block on all outstanding work of the device) is not acceptable.  Such a
+ * caller passes only the inputs, caches and the output; the split-KV partials, block lists and
+ * bitmaps go to a fixed array of ADASPARK_ATTN_STATIC_SCRATCH_BYTES (8 MiB) that is part of the
+ * library itself.  Every GPU on which the library is loaded holds that array until the process
+ * exits, whether or not this call is ever used.
+ *
+ * Arguments, results and errors are those of adaspark_attn_decode.  In addition:
+ *   - ERR_WORKSPACE_TOO_SMALL if the partition's decode_workspace_bytes exceeds the 8 MiB
+ *     (config 5, batch 16, needs about 6 MiB); use adaspark_attn_decode then.
+ *   - The first call on each device looks up the array's device address (a one-time host-side
+ *     set-up with that device current); make that first call before any stream capture begins.
+ *   - The call performs no cudaMalloc / cudaFree and uses no allocating library routine.
+ *   - All calls on a device share the one array, which keeps whatever the previous call left in
+ *     it; the header that must start at zero is cleared by every call.  Two calls whose kernels
+ *     may overlap on the GPU (different streams, or different handles on the same device) race
+ *     on the array: serialise them. */
+adaspark_status_t adaspark_attn_decode_static(adaspark_attn_t *handle, const void *q_new,
+                                              const void *k_new, const void *v_new, void *k_cube,
+                                              void *v_cube, const float *cube_keys,
+                                              const int32_t *text_len, void *out,
+                                              uint32_t *sel_bitmap, void *cuda_stream);
+
 /* Release the handle (host memory only). NULL is accepted. */
 adaspark_status_t adaspark_attn_destroy(adaspark_attn_t *handle);
 

@@ -46,7 +46,7 @@ EXPORTS = ["adaspark_attn_create", "adaspark_attn_partition", "adaspark_attn_get
            "adaspark_attn_forward", "adaspark_attn_decode", "adaspark_attn_destroy",
            "adaspark_attn_last_error", "adaspark_attn_last_launch_count",
            "adaspark_attn_set_prefill_kernel", "adaspark_attn_enable_stage_timing",
-           "adaspark_attn_get_stage_times"]
+           "adaspark_attn_get_stage_times", "adaspark_attn_decode_static"]
 
 
 def load() -> ctypes.CDLL:
@@ -64,6 +64,7 @@ def load() -> ctypes.CDLL:
     lib.adaspark_attn_get_layout.argtypes = [vp, ctypes.POINTER(Layout)]
     lib.adaspark_attn_forward.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.adaspark_attn_decode.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.adaspark_attn_decode_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.adaspark_attn_destroy.argtypes = [vp]
     lib.adaspark_attn_last_error.argtypes = [vp]
     lib.adaspark_attn_last_error.restype = ctypes.c_char_p
@@ -139,6 +140,19 @@ def adaspark_attn_decode(handle: int, q_new, k_new, v_new, k_cube, v_cube, cube_
         handle, _ptr(q_new), _ptr(k_new), _ptr(v_new), _ptr(k_cube), _ptr(v_cube), _ptr(cube_keys),
         _ptr(text_len), _ptr(out), _ptr(sel_bitmap), _ptr(workspace), workspace_bytes,
         _stream_ptr(stream)))
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def adaspark_attn_decode_static(handle: int, q_new, k_new, v_new, k_cube, v_cube, cube_keys, text_len,
+                                out, sel_bitmap, stream=None):
+    """Decode step that takes no workspace: for callers that cannot allocate device memory when
+    they decode (all memory already owned by their own pool, or no cudaMalloc allowed inside the
+    serving loop).  Scratch is the library's built-in 8 MiB array, shared by all calls on a device."""
+    _check(handle, load().adaspark_attn_decode_static(
+        handle, _ptr(q_new), _ptr(k_new), _ptr(v_new), _ptr(k_cube), _ptr(v_cube), _ptr(cube_keys),
+        _ptr(text_len), _ptr(out), _ptr(sel_bitmap), _stream_ptr(stream)))
 
 
 def adaspark_attn_destroy(handle: int):

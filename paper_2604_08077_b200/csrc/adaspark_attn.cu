@@ -399,3 +399,50 @@ adaspark_status_t adaspark_attn_set_prefill_kernel(adaspark_attn_t* h, int32_t w
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// Decode for callers that cannot hand over a workspace (see adaspark_attn_decode_static in the
+// header).  The scratch lives in this library image: one fixed array per GPU that loads it.
+// In host code `g_decode_scratch` is only a stand-in for the symbol, not a device address, so
+// the address is looked up once per device with cudaGetSymbolAddress and cached.
+// ---------------------------------------------------------------------------------------------
+#include <mutex>
+
+static __device__ __align__(256) unsigned char g_decode_scratch[ADASPARK_ATTN_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void* g_scratch_addr[kMaxDevices] = {nullptr};
+}  // namespace
+
+extern "C" adaspark_status_t adaspark_attn_decode_static(adaspark_attn_t* h, const void* q_new, const void* k_new,
+                                                         const void* v_new, void* k_cube, void* v_cube,
+                                                         const float* cube_keys, const int32_t* text_len, void* out,
+                                                         uint32_t* sel_bitmap, void* cuda_stream) {
+    if (!h) return ADASPARK_ERR_INVALID_ARG;
+    if (!h->partitioned) return fail(h, ADASPARK_ERR_NOT_PARTITIONED, "decode_static: call adaspark_attn_partition first");
+    if (h->dc_total > (size_t)ADASPARK_ATTN_STATIC_SCRATCH_BYTES)
+        return fail(h, ADASPARK_ERR_WORKSPACE_TOO_SMALL,
+                    "decode_static: this partition needs %zu bytes of decode scratch but the built-in scratch holds "
+                    "only %zu; use adaspark_attn_decode with a caller workspace",
+                    h->dc_total, (size_t)ADASPARK_ATTN_STATIC_SCRATCH_BYTES);
+    const int dev = h->cfg.device;
+    if (dev < 0 || dev >= kMaxDevices) return fail(h, ADASPARK_ERR_UNSUPPORTED, "decode_static: device ordinal %d", dev);
+    cudaError_t ce = cudaSetDevice(dev);
+    if (ce != cudaSuccess) return fail(h, ADASPARK_ERR_CUDA, "decode_static: cudaSetDevice(%d): %s", dev, cudaGetErrorString(ce));
+    void* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_scratch_mutex);
+        if (!g_scratch_addr[dev]) {   // first call on this device: resolve the symbol's device address
+            void* p = nullptr;
+            ce = cudaGetSymbolAddress(&p, g_decode_scratch);
+            if (ce != cudaSuccess || !p)
+                return fail(h, ADASPARK_ERR_CUDA, "decode_static: cudaGetSymbolAddress: %s", cudaGetErrorString(ce));
+            g_scratch_addr[dev] = p;
+        }
+        scratch = g_scratch_addr[dev];
+    }
+    return adaspark_attn_decode(h, q_new, k_new, v_new, k_cube, v_cube, cube_keys, text_len, out, sel_bitmap, scratch,
+                                (size_t)ADASPARK_ATTN_STATIC_SCRATCH_BYTES, cuda_stream);
+}
