@@ -1,0 +1,29 @@
+/*
+ * adaspark_attn_debug.h - diagnostic entry points of libadaspark_attn (not part of the AdaS-Attn
+ * path; the paper has no counterpart).  They exercise hardware building blocks in isolation so
+ * that a failure of the attention kernel can be told apart from a failure of its primitives.
+ */
+#ifndef ADASPARK_ATTN_DEBUG_H_
+#define ADASPARK_ATTN_DEBUG_H_
+
+#include <stdint.h>
+
+#include "adaspark_attn.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* One 128x128x128 problem through the tcgen05 path on the current device:
+ *   d_out = A * B^T (fp32 [128,128]),  e_out = bf16(d_out / 64) * C^T (fp32 [128,128]),
+ * with A, B, C bf16 row-major [128,128] device buffers (16-byte aligned).  `status` is a device
+ * int32 the kernel sets to ADASPARK_ERR_TIMEOUT if a bounded wait expired (caller zeroes it).
+ * Returns ERR_CUDA if the tensor maps cannot be encoded or the launch fails. */
+adaspark_status_t adaspark_attn_debug_umma_selftest(const void *a, const void *b, const void *c,
+                                                    float *d_out, float *e_out, int32_t *status,
+                                                    void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ADASPARK_ATTN_DEBUG_H_ */

@@ -46,7 +46,8 @@ EXPORTS = ["adaspark_attn_create", "adaspark_attn_partition", "adaspark_attn_get
            "adaspark_attn_forward", "adaspark_attn_decode", "adaspark_attn_destroy",
            "adaspark_attn_last_error", "adaspark_attn_last_launch_count",
            "adaspark_attn_set_prefill_kernel", "adaspark_attn_enable_stage_timing",
-           "adaspark_attn_get_stage_times", "adaspark_attn_decode_static"]
+           "adaspark_attn_get_stage_times", "adaspark_attn_decode_static",
+           "adaspark_attn_debug_umma_selftest"]
 
 
 def load() -> ctypes.CDLL:
@@ -65,6 +66,7 @@ def load() -> ctypes.CDLL:
     lib.adaspark_attn_forward.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.adaspark_attn_decode.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.adaspark_attn_decode_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.adaspark_attn_debug_umma_selftest.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     lib.adaspark_attn_destroy.argtypes = [vp]
     lib.adaspark_attn_last_error.argtypes = [vp]
     lib.adaspark_attn_last_error.restype = ctypes.c_char_p
@@ -153,6 +155,12 @@ def adaspark_attn_decode_static(handle: int, q_new, k_new, v_new, k_cube, v_cube
     _check(handle, load().adaspark_attn_decode_static(
         handle, _ptr(q_new), _ptr(k_new), _ptr(v_new), _ptr(k_cube), _ptr(v_cube), _ptr(cube_keys),
         _ptr(text_len), _ptr(out), _ptr(sel_bitmap), _stream_ptr(stream)))
+
+
+def adaspark_attn_debug_umma_selftest(a, b, c, d_out, e_out, status, stream=None) -> int:
+    """128x128x128 tcgen05 self-test (see include/adaspark_attn_debug.h); returns the status code."""
+    return int(load().adaspark_attn_debug_umma_selftest(_ptr(a), _ptr(b), _ptr(c), _ptr(d_out),
+                                                       _ptr(e_out), _ptr(status), _stream_ptr(stream)))
 
 
 def adaspark_attn_destroy(handle: int):

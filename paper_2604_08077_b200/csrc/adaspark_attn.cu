@@ -446,3 +446,23 @@ extern "C" adaspark_status_t adaspark_attn_decode_static(adaspark_attn_t* h, con
     return adaspark_attn_decode(h, q_new, k_new, v_new, k_cube, v_cube, cube_keys, text_len, out, sel_bitmap, scratch,
                                 (size_t)ADASPARK_ATTN_STATIC_SCRATCH_BYTES, cuda_stream);
 }
+
+// ---------------------------------------------------------------------------------------------
+// Diagnostics (include/adaspark_attn_debug.h)
+// ---------------------------------------------------------------------------------------------
+#include "../../include/adaspark_attn_debug.h"
+#include "umma_selftest.cuh"
+
+extern "C" adaspark_status_t adaspark_attn_debug_umma_selftest(const void* a, const void* b, const void* c, float* d_out,
+                                                               float* e_out, int32_t* status, void* cuda_stream) {
+    if (!a || !b || !c || !d_out || !e_out || !status) return ADASPARK_ERR_INVALID_ARG;
+    CUtensorMap tmA, tmB, tmC;
+    if (!encode_bf16_2d(&tmA, a, 128, 128, 64, 128) || !encode_bf16_2d(&tmB, b, 128, 128, 64, 128) ||
+        !encode_bf16_2d(&tmC, c, 128, 128, 64, 128))
+        return ADASPARK_ERR_CUDA;
+    const size_t smem = sizeof(SelftestSmem) + 1024;
+    if (cudaFuncSetAttribute(umma_selftest_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return ADASPARK_ERR_CUDA;
+    umma_selftest_kernel<<<1, 128, smem, (cudaStream_t)cuda_stream>>>(tmA, tmB, tmC, d_out, e_out, status);
+    return cudaGetLastError() == cudaSuccess ? ADASPARK_OK : ADASPARK_ERR_CUDA;
+}

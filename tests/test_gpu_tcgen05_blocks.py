@@ -1,0 +1,23 @@
+"""tcgen05 / TMA / TMEM building blocks checked in isolation on one 128x128x128 product."""
+import pytest
+import torch
+
+from paper_2604_08077_b200 import binding
+
+pytestmark = pytest.mark.gpu
+
+
+def test_umma_selftest_matches_matmul():
+    g = torch.Generator(device="cpu").manual_seed(3)
+    a, b, c = (torch.randn(128, 128, generator=g).to(torch.bfloat16).cuda() for _ in range(3))
+    d = torch.full((128, 128), float("nan"), device="cuda")
+    e = torch.full((128, 128), float("nan"), device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    rc = binding.adaspark_attn_debug_umma_selftest(a, b, c, d, e, status)
+    torch.cuda.synchronize()
+    assert rc == binding.OK and int(status.item()) == 0
+    d_ref = a.double() @ b.double().T
+    assert torch.allclose(d.double(), d_ref, atol=1e-3, rtol=1e-4), (d.double() - d_ref).abs().max()
+    p = (d / 64).to(torch.bfloat16)
+    e_ref = p.double() @ c.double().T
+    assert torch.allclose(e.double(), e_ref, atol=1e-3, rtol=1e-4), (e.double() - e_ref).abs().max()
