@@ -62,6 +62,8 @@ Geom make_geom(const adaspark_attn* h, int n_text) {
     g.ct = h->cfg.cube_t; g.ch = h->cfg.cube_h; g.cw = h->cfg.cube_w;
     g.nH = h->H / g.ch; g.nW = h->W / g.cw;
     g.C = h->C; g.N = h->N;
+    g.c_shift = 0;
+    while ((1 << g.c_shift) < g.C) ++g.c_shift;
     g.S_v = h->S_v; g.n_text = n_text; g.S = h->S_v + n_text;
     g.S_cap = h->S_cap;
     g.n_words = (h->N + 31) / 32;
@@ -271,6 +273,33 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
 
     mark(h, 2, st);
     // K4: gathered attention
+#ifdef ADASPARK_WITH_TCGEN05
+    if (h->prefill_kernel == 1) {
+        __nv_bfloat16* q_cube = (__nv_bfloat16*)(ws + h->fw_qcube_off);
+        dim3 rgrid((g.S + 31) / 32, g.B);
+        if (D == 128) relayout_q_kernel<128><<<rgrid, 256, 0, st>>>(g, qb, q_cube);
+        else relayout_q_kernel<64><<<rgrid, 256, 0, st>>>(g, qb, q_cube);
+        if (!launch_ok(h, "relayout_q_kernel")) return ADASPARK_ERR_CUDA;
+        CUtensorMap tmQ, tmK, tmV;
+        if (!encode_bf16_2d(&tmQ, q_cube, (uint64_t)g.B * g.Hq * g.S_cap, D, 64, 128) ||
+            !encode_bf16_2d(&tmK, kc, (uint64_t)g.B * g.Hkv * g.S_cap, D, 64, 64) ||
+            !encode_bf16_2d(&tmV, vc, (uint64_t)g.B * g.Hkv * g.n_kv_blocks_cap * D, 64, 64, D))
+            return fail(h, ADASPARK_ERR_CUDA, "forward: cuTensorMapEncodeTiled failed");
+        dim3 grid((g.S + kPairRows - 1) / kPairRows, g.Hq, g.B);
+        if (D == 128) {
+            size_t smem = sizeof(TcAttnSmem<128>) + 1024;
+            if (!set_smem(h, attn_prefill_tc_kernel<128>, smem, "attn_prefill_tc_kernel")) return ADASPARK_ERR_CUDA;
+            attn_prefill_tc_kernel<128><<<grid, kTcThreads, smem, st>>>(g, tmQ, tmK, tmV, tile_mask, (__nv_bfloat16*)out,
+                                                                        (unsigned long long*)&hdr->executed_kv_blocks, &hdr->status);
+        } else {
+            size_t smem = sizeof(TcAttnSmem<64>) + 1024;
+            if (!set_smem(h, attn_prefill_tc_kernel<64>, smem, "attn_prefill_tc_kernel")) return ADASPARK_ERR_CUDA;
+            attn_prefill_tc_kernel<64><<<grid, kTcThreads, smem, st>>>(g, tmQ, tmK, tmV, tile_mask, (__nv_bfloat16*)out,
+                                                                       (unsigned long long*)&hdr->executed_kv_blocks, &hdr->status);
+        }
+        if (!launch_ok(h, "attn_prefill_tc_kernel")) return ADASPARK_ERR_CUDA;
+    } else
+#endif
     {
         dim3 grid(g.n_tiles, g.Hq, g.B);
         if (D == 128) {

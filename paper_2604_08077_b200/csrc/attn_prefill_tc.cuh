@@ -1,0 +1,409 @@
+// K4: gathered flash-style attention on the 5th-generation tensor cores (Eq. 3; un-permute of
+// Algorithm 1 fused into the epilogue).
+//
+// One CTA = one "pair tile": 256 consecutive cube-major query rows of one query head, handled as
+// two 128-row MMA tiles that ping-pong on the tensor core.  Roles (320 threads):
+//   warps 0-3   softmax of tile 0 (thread = query row = TMEM lane)
+//   warps 4-7   softmax of tile 1
+//   warp  8     TMA producer: Q tiles once, then K / V^T tiles of the needed key blocks
+//   warp  9     MMA issuer: S_t = Q_t K^T (operands in shared memory), O_t += P_t V (P in TMEM)
+// Key blocks (64 cube-major positions) are visited in pairs (128 keys per step).  A block is
+// needed if any row of the pair tile selected a cube inside it or if it overlaps the tile's local
+// range (own cubes / text prefix).  Each softmax thread masks its own row: one selection bit per
+// (row, cube) for blocks before the local range, the exact per-key rule inside it.
+//
+// TMEM (512 columns): tile t owns [256t, 256t+128) for S_t (fp32) -- P_t (bf16 pairs) overwrites
+// its first 64 columns -- and [256t+128, 256t+128+D) for O_t.  The issue order
+//   S0(0) S1(0) | PV0(j) S0(j+1) PV1(j) S1(j+1) ...
+// lets the softmax of one tile overlap the MMAs of the other, and makes "S_t(j+1) ready" imply
+// "PV_t(j) finished", so the lazy rescale of O_t needs no extra barrier.
+#pragma once
+#include "tc_common.cuh"
+
+namespace adaspark {
+
+constexpr int kTcThreads = 320;
+constexpr int kPairRows = 256;
+constexpr int kMaxBlockWords = 1024;   // up to 32768 key blocks (2M positions) per sequence
+
+template <int D>
+struct TcAttnSmem {
+    __nv_bfloat16 q[2][D / 64][128][64];      // [tile][d panel][row][64 d]
+    __nv_bfloat16 k[2][D / 64][128][64];      // [stage][d panel][key (2 blocks)][64 d]
+    __nv_bfloat16 v[2][2][D][64];             // [stage][block][d][64 keys]  (V^T)
+    uint32_t blk_words[kMaxBlockWords];       // bit kb set <=> key block kb is visited
+    uint32_t union_words[128];                // OR of the 256 rows' selection words
+    uint64_t q_full, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], p_ready[2], o_final;
+    uint32_t tmem_base;
+    int abort_flag;
+    int n_needed;                             // number of visited key blocks
+};
+
+// Iterates the set bits of blk_words in ascending order.
+struct BlockIter {
+    const uint32_t* words;
+    int wi;
+    uint32_t cur;
+    __device__ __forceinline__ BlockIter(const uint32_t* w) : words(w), wi(0), cur(w[0]) {}
+    __device__ __forceinline__ int next() {   // caller guarantees a set bit remains
+        while (cur == 0) cur = words[++wi];
+        int b = __ffs(cur) - 1;
+        cur &= cur - 1;
+        return wi * 32 + b;
+    }
+};
+
+template <int D>
+__global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
+    Geom g, const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+    const __grid_constant__ CUtensorMap tmV, const uint32_t* __restrict__ tile_mask, __nv_bfloat16* __restrict__ out,
+    unsigned long long* __restrict__ executed_blocks, int32_t* __restrict__ status) {
+    extern __shared__ unsigned char tc_smem_raw[];
+    TcAttnSmem<D>& sm = *reinterpret_cast<TcAttnSmem<D>*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~(uintptr_t)1023);
+    constexpr int kPanels = D / 64;
+    constexpr int kQKSteps = D / 16;                            // k-steps of S = Q K^T
+    constexpr uint32_t kIdescS = tc::make_idesc_bf16(128, 128);  // S tile: 128 rows x 128 keys
+    constexpr uint32_t kIdescO = tc::make_idesc_bf16(128, D);    // O tile: 128 rows x D
+    constexpr uint32_t kQBytes = 2 * 128 * D * 2, kKBytes = 128 * D * 2, kVBytes = 2 * D * 64 * 2;
+
+    const int n_pairs = (g.S + kPairRows - 1) / kPairRows;
+    const int pair = n_pairs - 1 - blockIdx.x;                  // long (late) tiles first
+    const int h = blockIdx.y, b = blockIdx.z, gk = h / g.G;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int pair_pos0 = pair * kPairRows;
+    const int pair_end = min(pair_pos0 + kPairRows, g.S);       // exclusive
+    const int n_blk = (pair_end + kBlockTok - 1) / kBlockTok;   // key blocks that can matter
+    const int local_start = pair_pos0 < g.S_v ? ((pair_pos0 >> g.c_shift) << g.c_shift) : g.S_v;
+    const int first_local_blk = local_start / kBlockTok;
+
+    // ---------------------------------------------------------------- set-up
+    if (tid == 0) {
+        tc::mbar_init(&sm.q_full, 1);
+        for (int i = 0; i < 2; ++i) {
+            tc::mbar_init(&sm.k_full[i], 1);
+            tc::mbar_init(&sm.k_empty[i], 1);
+            tc::mbar_init(&sm.v_full[i], 1);
+            tc::mbar_init(&sm.v_empty[i], 1);
+            tc::mbar_init(&sm.s_full[i], 1);
+            tc::mbar_init(&sm.p_ready[i], 128);
+        }
+        tc::mbar_init(&sm.o_final, 1);
+        sm.abort_flag = 0;
+        tc::fence_barrier_init();
+    }
+    if (warp == 8) {
+        tc::tmem_alloc<512>(&sm.tmem_base);
+        if (lane == 0) {
+            tc::prefetch_tensormap(&tmQ);
+            tc::prefetch_tensormap(&tmK);
+            tc::prefetch_tensormap(&tmV);
+        }
+    }
+    // union of the selection words of the 256 rows (two 128-row tiles of the mask matrix)
+    for (int w = warp; w < g.n_words; w += kTcThreads / 32) {
+        uint32_t u = 0;
+        for (int r = lane; r < kPairRows; r += 32) {
+            int tile = pair * 2 + (r >> 7);
+            if (tile < g.n_tiles) u |= tile_mask[mask_index(g, b, h, tile, w, r & 127)];
+        }
+        u = __reduce_or_sync(0xffffffffu, u);
+        if (lane == 0) sm.union_words[w] = u;
+    }
+    tc::tc_fence_before_sync();
+    __syncthreads();
+    tc::tc_fence_after_sync();
+    // block bitmap: one thread per word of 32 key blocks
+    const int n_blk_words = (n_blk + 31) / 32;
+    for (int wi = tid; wi < n_blk_words; wi += kTcThreads) {
+        uint32_t bits = 0;
+        for (int i = 0; i < 32; ++i) {
+            int kb = wi * 32 + i;
+            if (kb >= n_blk) break;
+            bool need = kb >= first_local_blk;
+            if (!need) {
+                int c_lo = (kb * kBlockTok) >> g.c_shift, c_hi = (kb * kBlockTok + kBlockTok - 1) >> g.c_shift;
+                uint32_t span = c_hi - c_lo + 1;   // <= 4 cubes, aligned: never crosses a word
+                uint32_t m = (span >= 32 ? 0xffffffffu : ((1u << span) - 1u)) << (c_lo & 31);
+                need = (sm.union_words[c_lo >> 5] & m) != 0;
+            }
+            if (need) bits |= 1u << i;
+        }
+        sm.blk_words[wi] = bits;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        int cnt = 0;
+        for (int wi = lane; wi < n_blk_words; wi += 32) cnt += __popc(sm.blk_words[wi]);
+        cnt = __reduce_add_sync(0xffffffffu, cnt);
+        if (lane == 0) sm.n_needed = cnt;
+    }
+    __syncthreads();
+    const int n_needed = sm.n_needed;
+    const int n_steps = (n_needed + 1) / 2;                      // >= 1: the local range is never empty
+    const uint32_t tbase = sm.tmem_base;
+    volatile int* abort_flag = &sm.abort_flag;
+
+    if (warp == 8) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            const int q_row0 = (b * g.Hq + h) * g.S_cap + pair_pos0;
+            const int kv_row0 = (b * g.Hkv + gk) * g.S_cap;
+            const int v_row0 = (b * g.Hkv + gk) * g.n_kv_blocks_cap * D;
+            tc::mbar_arrive_expect_tx(&sm.q_full, kQBytes);
+            for (int t = 0; t < 2; ++t)
+                for (int p = 0; p < kPanels; ++p) tc::tma_load_2d(&sm.q[t][p][0][0], &tmQ, p * 64, q_row0 + t * 128, &sm.q_full);
+            BlockIter it(sm.blk_words);
+            for (int j = 0; j < n_steps; ++j) {
+                const int st = j & 1, u = j >> 1;
+                const int kb_a = it.next();
+                const int kb_b = (2 * j + 1 < n_needed) ? it.next() : kb_a;   // odd count: repeat, masked later
+                if (!tc::mbar_wait(&sm.k_empty[st], (u & 1) ^ 1, abort_flag)) break;
+                tc::mbar_arrive_expect_tx(&sm.k_full[st], kKBytes);
+                for (int p = 0; p < kPanels; ++p) {
+                    tc::tma_load_2d(&sm.k[st][p][0][0], &tmK, p * 64, kv_row0 + kb_a * kBlockTok, &sm.k_full[st]);
+                    tc::tma_load_2d(&sm.k[st][p][64][0], &tmK, p * 64, kv_row0 + kb_b * kBlockTok, &sm.k_full[st]);
+                }
+                if (!tc::mbar_wait(&sm.v_empty[st], (u & 1) ^ 1, abort_flag)) break;
+                tc::mbar_arrive_expect_tx(&sm.v_full[st], kVBytes);
+                tc::tma_load_2d(&sm.v[st][0][0][0], &tmV, 0, v_row0 + kb_a * D, &sm.v_full[st]);
+                tc::tma_load_2d(&sm.v[st][1][0][0], &tmV, 0, v_row0 + kb_b * D, &sm.v_full[st]);
+            }
+        }
+    } else if (warp == 9) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            auto issue_s = [&](int t, int st) {   // S_t = Q_t K(st)^T
+#pragma unroll
+                for (int ks = 0; ks < kQKSteps; ++ks) {
+                    uint64_t da = tc::make_smem_desc_sw128(smem_u32(&sm.q[t][ks >> 2][0][0]) + (ks & 3) * 32);
+                    uint64_t db = tc::make_smem_desc_sw128(smem_u32(&sm.k[st][ks >> 2][0][0]) + (ks & 3) * 32);
+                    tc::umma_ss(tbase + t * 256, da, db, kIdescS, ks > 0);
+                }
+            };
+            auto issue_pv = [&](int t, int st, bool first) {   // O_t (+)= P_t V(st)
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    uint64_t db = tc::make_smem_desc_sw128(smem_u32(&sm.v[st][ks >> 2][0][0]) + (ks & 3) * 32);
+                    tc::umma_ts(tbase + t * 256 + 128, tbase + t * 256 + ks * 8, db, kIdescO, !(first && ks == 0));
+                }
+            };
+            bool ok = tc::mbar_wait(&sm.q_full, 0, abort_flag) && tc::mbar_wait(&sm.k_full[0], 0, abort_flag);
+            if (ok) {
+                tc::tc_fence_after_sync();
+                issue_s(0, 0);
+                tc::umma_commit(&sm.s_full[0]);
+                issue_s(1, 0);
+                tc::umma_commit(&sm.s_full[1]);
+                tc::umma_commit(&sm.k_empty[0]);
+            }
+            for (int j = 0; ok && j < n_steps; ++j) {
+                const int st = j & 1, u = j >> 1;
+                const bool more = j + 1 < n_steps;
+                const int st1 = (j + 1) & 1, u1 = (j + 1) >> 1;
+                if (!(ok = tc::mbar_wait(&sm.v_full[st], u & 1, abort_flag))) break;
+                if (!(ok = tc::mbar_wait(&sm.p_ready[0], j & 1, abort_flag))) break;
+                tc::tc_fence_after_sync();
+                issue_pv(0, st, j == 0);
+                if (more) {
+                    if (!(ok = tc::mbar_wait(&sm.k_full[st1], u1 & 1, abort_flag))) break;
+                    tc::tc_fence_after_sync();
+                    issue_s(0, st1);
+                    tc::umma_commit(&sm.s_full[0]);
+                }
+                if (!(ok = tc::mbar_wait(&sm.p_ready[1], j & 1, abort_flag))) break;
+                tc::tc_fence_after_sync();
+                issue_pv(1, st, j == 0);
+                tc::umma_commit(&sm.v_empty[st]);
+                if (more) {
+                    issue_s(1, st1);
+                    tc::umma_commit(&sm.s_full[1]);
+                    tc::umma_commit(&sm.k_empty[st1]);
+                }
+            }
+            if (ok) tc::umma_commit(&sm.o_final);
+        }
+    } else {
+        // ------------------------------------------------------------ softmax warps
+        const int t = warp >> 2;                                  // tile of this warpgroup
+        const int row = (warp & 3) * 32 + lane;                   // row inside the tile = TMEM lane
+        const int tile = pair * 2 + t;
+        const int pr = pair_pos0 + t * 128 + row;                 // cube-major position of the row
+        const uint32_t lane_addr = tbase + ((uint32_t)((warp & 3) * 32) << 16) + t * 256;
+        const bool tile_live = tile < g.n_tiles;
+        const uint32_t* my_mask = tile_mask + mask_index(g, b, h, tile_live ? tile : 0, 0, row);
+        int cached_w = -1;
+        uint32_t cached_word = 0;
+        auto get_word = [&](int w) -> uint32_t {
+            if (w != cached_w) {
+                cached_w = w;
+                cached_word = tile_live ? my_mask[(size_t)w * kTileRows] : 0u;
+            }
+            return cached_word;
+        };
+        float m_ref = -INFINITY, l_sum = 0.f;
+        BlockIter it(sm.blk_words);
+        bool ok = true;
+        for (int j = 0; j < n_steps; ++j) {
+            const int kb_a = it.next();
+            const bool has_b = 2 * j + 1 < n_needed;
+            const int kb_b = has_b ? it.next() : kb_a;
+            // ---- visibility of the 128 keys of this step for this row: one bit per key
+            uint32_t amask[4];
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+                const int kb = hf ? kb_b : kb_a;
+                const int pk0 = kb * kBlockTok;
+                uint32_t m0 = 0, m1 = 0;
+                if (hf == 1 && !has_b) {
+                    // repeated block of an odd count: nothing visible
+                } else if (kb < first_local_blk) {
+                    const int cube0 = pk0 >> g.c_shift;
+                    const uint32_t wbits = get_word(cube0 >> 5) >> (cube0 & 31);
+                    if (g.c_shift >= 6) {
+                        m0 = m1 = (wbits & 1u) ? 0xffffffffu : 0u;
+                    } else if (g.c_shift == 5) {
+                        m0 = (wbits & 1u) ? 0xffffffffu : 0u;
+                        m1 = (wbits & 2u) ? 0xffffffffu : 0u;
+                    } else {
+                        m0 = ((wbits & 1u) ? 0x0000ffffu : 0u) | ((wbits & 2u) ? 0xffff0000u : 0u);
+                        m1 = ((wbits & 4u) ? 0x0000ffffu : 0u) | ((wbits & 8u) ? 0xffff0000u : 0u);
+                    }
+                } else {
+                    const uint32_t word = pk0 < g.S_v ? get_word((pk0 >> g.c_shift) >> 5) : 0u;
+                    for (int i = 0; i < 32; ++i) {
+                        if (key_allowed(g, pr, pk0 + i, word)) m0 |= 1u << i;
+                        if (key_allowed(g, pr, pk0 + 32 + i, word)) m1 |= 1u << i;
+                    }
+                }
+                amask[hf * 2] = m0;
+                amask[hf * 2 + 1] = m1;
+            }
+            if (!(ok = tc::mbar_wait(&sm.s_full[t], j & 1, abort_flag))) break;
+            tc::tc_fence_after_sync();
+            uint32_t s[4][32];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tc::tmem_ld_32x32(lane_addr + c * 32, s[c]);
+            tc::tmem_wait_ld();
+            // ---- row maximum over the visible keys
+            float mx = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const uint32_t am = amask[c];
+                if (am == 0xffffffffu) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(s[c][i]));
+                } else if (am != 0u) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if ((am >> i) & 1u) mx = fmaxf(mx, __uint_as_float(s[c][i]));
+                }
+            }
+            const float mx_x = mx * g.scale_log2;                 // scale > 0: max commutes with it
+            // ---- lazy rescale: move the reference only when it grows by more than 2^8
+            const bool need = mx_x > m_ref + 8.f;                  // also true on the first visible key
+            if (__any_sync(0xffffffffu, need)) {
+                const float factor = need ? exp2f(m_ref - mx_x) : 1.f;   // 0 when nothing was visible before
+                if (j > 0) {
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t o[32];
+                        tc::tmem_ld_32x32(lane_addr + 128 + c * 32, o);
+                        tc::tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
+                        tc::tmem_st_32x32(lane_addr + 128 + c * 32, o);
+                    }
+                }
+                l_sum *= factor;
+                if (need) m_ref = mx_x;
+            }
+            // ---- P = 2^(s*scale - m_ref) on visible keys, 0 elsewhere; bf16 pairs into TMEM
+            const float neg_ref = -m_ref;                          // finite whenever a key is visible
+            float psum = 0.f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const uint32_t am = amask[c];
+                uint32_t pk[16];
+                if (am == 0xffffffffu) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        float p0 = fast_exp2(fmaf(__uint_as_float(s[c][2 * i]), g.scale_log2, neg_ref));
+                        float p1 = fast_exp2(fmaf(__uint_as_float(s[c][2 * i + 1]), g.scale_log2, neg_ref));
+                        psum += p0 + p1;
+                        pk[i] = pack_bf16x2(p0, p1);
+                    }
+                } else if (am != 0u) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        float p0 = ((am >> (2 * i)) & 1u) ? fast_exp2(fmaf(__uint_as_float(s[c][2 * i]), g.scale_log2, neg_ref)) : 0.f;
+                        float p1 = ((am >> (2 * i + 1)) & 1u) ? fast_exp2(fmaf(__uint_as_float(s[c][2 * i + 1]), g.scale_log2, neg_ref)) : 0.f;
+                        psum += p0 + p1;
+                        pk[i] = pack_bf16x2(p0, p1);
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) pk[i] = 0u;
+                }
+                tc::tmem_st_32x16(lane_addr + c * 16, pk);
+            }
+            l_sum += psum;
+            tc::tmem_wait_st();
+            tc::tc_fence_before_sync();
+            tc::mbar_arrive(&sm.p_ready[t]);
+        }
+        // ---- epilogue: O / l -> bf16 at the raster position of the row
+        if (ok) ok = tc::mbar_wait(&sm.o_final, 0, abort_flag);
+        if (ok) {
+            tc::tc_fence_after_sync();
+            const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
+            const bool live = pr < g.S;
+            __nv_bfloat16* dst = out + ((size_t)(b * g.S + (live ? pos_to_raster(g, pr) : 0)) * g.Hq + h) * D;
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t o[32];
+                tc::tmem_ld_32x32(lane_addr + 128 + c * 32, o);
+                tc::tmem_wait_ld();
+                if (live) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        uint4 val;
+                        val.x = pack_bf16x2(__uint_as_float(o[8 * i + 0]) * inv, __uint_as_float(o[8 * i + 1]) * inv);
+                        val.y = pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv, __uint_as_float(o[8 * i + 3]) * inv);
+                        val.z = pack_bf16x2(__uint_as_float(o[8 * i + 4]) * inv, __uint_as_float(o[8 * i + 5]) * inv);
+                        val.w = pack_bf16x2(__uint_as_float(o[8 * i + 6]) * inv, __uint_as_float(o[8 * i + 7]) * inv);
+                        *reinterpret_cast<uint4*>(dst + c * 32 + i * 8) = val;
+                    }
+                }
+            }
+        }
+    }
+    // ---------------------------------------------------------------- teardown
+    tc::tc_fence_before_sync();
+    __syncthreads();
+    if (tid == 0) {
+        if (sm.abort_flag) atomicExch(status, 6);   // a bounded wait expired
+        else atomicAdd(executed_blocks, (unsigned long long)(2 * n_needed));
+    }
+    if (warp == 8) tc::tmem_dealloc<512>(tbase);
+}
+
+// cube-major staging of Q for the TMA loads of the attention kernel:
+// q_cube[(b*Hq + h) * S_cap + pos][:] = q[b, raster(pos), h, :]
+template <int D>
+__global__ void __launch_bounds__(256) relayout_q_kernel(Geom g, const __nv_bfloat16* __restrict__ q,
+                                                         __nv_bfloat16* __restrict__ q_cube) {
+    constexpr int kChunks = D / 8;
+    const int pos0 = blockIdx.x * 32;                   // 32 positions x all heads per CTA
+    const int b = blockIdx.y;
+    const int per_pos = g.Hq * kChunks;
+    for (int idx = threadIdx.x; idx < 32 * per_pos; idx += 256) {
+        int p = idx / per_pos, rem = idx - p * per_pos;
+        int h = rem / kChunks, c = rem - h * kChunks;
+        int pos = pos0 + p;
+        if (pos >= g.S) break;
+        uint4 val = *reinterpret_cast<const uint4*>(q + ((size_t)(b * g.S + pos_to_raster(g, pos)) * g.Hq + h) * D + c * 8);
+        *reinterpret_cast<uint4*>(q_cube + ((size_t)(b * g.Hq + h) * g.S_cap + pos) * D + c * 8) = val;
+    }
+}
+
+}  // namespace adaspark

@@ -15,7 +15,8 @@ struct Geom {
     int B, T, H, W;      // batch, frames, patch rows, patch columns
     int ct, ch, cw;      // cube window
     int nH, nW;          // cube grid: H/ch, W/cw
-    int C, N;            // tokens per cube, cubes
+    int C, N;            // tokens per cube (a power of two), cubes
+    int c_shift;         // log2(C)
     int S_v, n_text, S;  // video tokens, text tokens of this call, total
     int S_cap;           // cache rows per (b, kv head), multiple of 128
     int n_words;         // ceil(N/32)
@@ -45,7 +46,7 @@ __device__ __forceinline__ int pos_to_raster(const Geom& g, int pos) {
 
 // Number of candidate cubes of the row at `pos`: preceding cubes for video, all cubes for text.
 __device__ __forceinline__ int n_candidates(const Geom& g, int pos) {
-    return pos < g.S_v ? pos / g.C : g.N;
+    return pos < g.S_v ? (pos >> g.c_shift) : g.N;
 }
 
 // Per-tile selection mask matrix: word w of row r of global tile gt at
@@ -58,8 +59,8 @@ __device__ __forceinline__ size_t mask_index(const Geom& g, int b, int h, int ti
 // `word` is the row's selection word that covers cube pk/C (bits of cubes that are not
 // candidates of the row are never set by the selection kernel).
 __device__ __forceinline__ bool key_allowed(const Geom& g, int pr, int pk, uint32_t word) {
-    if (pk <= pr && (pk >= g.S_v || pk / g.C == pr / g.C)) return true;  // own cube / text prefix
-    if (pk < g.S_v) return (word >> ((pk / g.C) & 31)) & 1u;              // selected cube
+    if (pk <= pr && (pk >= g.S_v || (pk >> g.c_shift) == (pr >> g.c_shift))) return true;  // own cube / text prefix
+    if (pk < g.S_v) return (word >> ((pk >> g.c_shift) & 31)) & 1u;                        // selected cube
     return false;
 }
 

@@ -47,7 +47,7 @@ SMALL_CASES = {
 
 
 @pytest.mark.parametrize("case", sorted(SMALL_CASES))
-@pytest.mark.parametrize("kernel", [0])
+@pytest.mark.parametrize("kernel", [0, 1])
 def test_small_prefill_every_row(case, kernel):
     """Element-by-element parity on every row: caches, selection bitmaps, counts, outputs."""
     wl = SMALL_CASES[case]()
