@@ -2,11 +2,13 @@
 // Algorithm 1 fused into the epilogue).
 //
 // One CTA = one "pair tile": 256 consecutive cube-major query rows of one query head, handled as
-// two 128-row MMA tiles that ping-pong on the tensor core.  Roles (320 threads):
+// two 128-row MMA tiles that ping-pong on the tensor core.  Roles (384 threads):
 //   warps 0-3   softmax of tile 0 (thread = query row = TMEM lane)
 //   warps 4-7   softmax of tile 1
 //   warp  8     TMA producer: Q tiles once, then K / V^T tiles of the needed key blocks
 //   warp  9     MMA issuer: S_t = Q_t K^T (operands in shared memory), O_t += P_t V (P in TMEM)
+//   warps 10-11 idle; they complete the third warpgroup so that it can hand registers to the
+//               softmax warpgroups (setmaxnreg), which hold a whole 128-column score row each
 // Key blocks (64 cube-major positions) are visited in pairs (128 keys per step).  A block is
 // needed if any row of the pair tile selected a cube inside it or if it overlaps the tile's local
 // range (own cubes / text prefix).  Each softmax thread masks its own row: one selection bit per
@@ -22,7 +24,9 @@
 
 namespace adaspark {
 
-constexpr int kTcThreads = 320;
+constexpr int kTcThreads = 384;
+constexpr int kSoftmaxRegs = 216;   // per-thread registers of the softmax warpgroups after setmaxnreg
+constexpr int kHelperRegs = 72;     // ... of the producer / MMA warpgroup
 constexpr int kPairRows = 256;
 constexpr int kMaxBlockWords = 1024;   // up to 32768 key blocks (2M positions) per sequence
 
@@ -143,6 +147,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     const uint32_t tbase = sm.tmem_base;
     volatile int* abort_flag = &sm.abort_flag;
 
+    if (warp >= 8) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kHelperRegs));
     if (warp == 8) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -222,8 +227,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
             }
             if (ok) tc::umma_commit(&sm.o_final);
         }
-    } else {
+    } else if (warp < 8) {
         // ------------------------------------------------------------ softmax warps
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kSoftmaxRegs));
         const int t = warp >> 2;                                  // tile of this warpgroup
         const int row = (warp & 3) * 32 + lane;                   // row inside the tile = TMEM lane
         const int tile = pair * 2 + t;
@@ -231,6 +237,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
         const uint32_t lane_addr = tbase + ((uint32_t)((warp & 3) * 32) << 16) + t * 256;
         const bool tile_live = tile < g.n_tiles;
         const uint32_t* my_mask = tile_mask + mask_index(g, b, h, tile_live ? tile : 0, 0, row);
+        const float scale_log2 = g.scale_log2;
         int cached_w = -1;
         uint32_t cached_word = 0;
         auto get_word = [&](int w) -> uint32_t {
@@ -278,27 +285,43 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
                 amask[hf * 2] = m0;
                 amask[hf * 2 + 1] = m1;
             }
+            // every 32-key chunk of every row of the warp fully visible or fully hidden?
+            const bool uniform = __all_sync(0xffffffffu, (amask[0] + 1u <= 1u) && (amask[1] + 1u <= 1u) &&
+                                                             (amask[2] + 1u <= 1u) && (amask[3] + 1u <= 1u));
             if (!(ok = tc::mbar_wait(&sm.s_full[t], j & 1, abort_flag))) break;
             tc::tc_fence_after_sync();
             uint32_t s[4][32];
 #pragma unroll
             for (int c = 0; c < 4; ++c) tc::tmem_ld_32x32(lane_addr + c * 32, s[c]);
             tc::tmem_wait_ld();
-            // ---- row maximum over the visible keys
+            // ---- row maximum over the visible keys (four independent chains per chunk)
             float mx = -INFINITY;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 const uint32_t am = amask[c];
-                if (am == 0xffffffffu) {
+                float a0 = -INFINITY, a1 = -INFINITY, a2 = -INFINITY, a3 = -INFINITY;
+                if (uniform) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(s[c][i]));
-                } else if (am != 0u) {
+                    for (int i = 0; i < 8; ++i) {
+                        a0 = fmaxf(a0, __uint_as_float(s[c][4 * i]));
+                        a1 = fmaxf(a1, __uint_as_float(s[c][4 * i + 1]));
+                        a2 = fmaxf(a2, __uint_as_float(s[c][4 * i + 2]));
+                        a3 = fmaxf(a3, __uint_as_float(s[c][4 * i + 3]));
+                    }
+                    const float cm = fmaxf(fmaxf(a0, a1), fmaxf(a2, a3));
+                    mx = am ? fmaxf(mx, cm) : mx;
+                } else {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if ((am >> i) & 1u) mx = fmaxf(mx, __uint_as_float(s[c][i]));
+                    for (int i = 0; i < 8; ++i) {
+                        a0 = fmaxf(a0, ((am >> (4 * i)) & 1u) ? __uint_as_float(s[c][4 * i]) : -INFINITY);
+                        a1 = fmaxf(a1, ((am >> (4 * i + 1)) & 1u) ? __uint_as_float(s[c][4 * i + 1]) : -INFINITY);
+                        a2 = fmaxf(a2, ((am >> (4 * i + 2)) & 1u) ? __uint_as_float(s[c][4 * i + 2]) : -INFINITY);
+                        a3 = fmaxf(a3, ((am >> (4 * i + 3)) & 1u) ? __uint_as_float(s[c][4 * i + 3]) : -INFINITY);
+                    }
+                    mx = fmaxf(mx, fmaxf(fmaxf(a0, a1), fmaxf(a2, a3)));
                 }
             }
-            const float mx_x = mx * g.scale_log2;                 // scale > 0: max commutes with it
+            const float mx_x = mx * scale_log2;                   // scale > 0: max commutes with it
             // ---- lazy rescale: move the reference only when it grows by more than 2^8
             const bool need = mx_x > m_ref + 8.f;                  // also true on the first visible key
             if (__any_sync(0xffffffffu, need)) {
@@ -319,34 +342,38 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
             }
             // ---- P = 2^(s*scale - m_ref) on visible keys, 0 elsewhere; bf16 pairs into TMEM
             const float neg_ref = -m_ref;                          // finite whenever a key is visible
-            float psum = 0.f;
+            float ps0 = 0.f, ps1 = 0.f, ps2 = 0.f, ps3 = 0.f;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 const uint32_t am = amask[c];
                 uint32_t pk[16];
-                if (am == 0xffffffffu) {
+                if (uniform) {
+                    const float addend = am ? neg_ref : -INFINITY;   // 2^(-inf) = 0 hides the chunk
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        float p0 = fast_exp2(fmaf(__uint_as_float(s[c][2 * i]), g.scale_log2, neg_ref));
-                        float p1 = fast_exp2(fmaf(__uint_as_float(s[c][2 * i + 1]), g.scale_log2, neg_ref));
-                        psum += p0 + p1;
-                        pk[i] = pack_bf16x2(p0, p1);
-                    }
-                } else if (am != 0u) {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        float p0 = ((am >> (2 * i)) & 1u) ? fast_exp2(fmaf(__uint_as_float(s[c][2 * i]), g.scale_log2, neg_ref)) : 0.f;
-                        float p1 = ((am >> (2 * i + 1)) & 1u) ? fast_exp2(fmaf(__uint_as_float(s[c][2 * i + 1]), g.scale_log2, neg_ref)) : 0.f;
-                        psum += p0 + p1;
-                        pk[i] = pack_bf16x2(p0, p1);
+                    for (int i = 0; i < 8; ++i) {
+                        float p0 = fast_exp2(fmaf(__uint_as_float(s[c][4 * i]), scale_log2, addend));
+                        float p1 = fast_exp2(fmaf(__uint_as_float(s[c][4 * i + 1]), scale_log2, addend));
+                        float p2 = fast_exp2(fmaf(__uint_as_float(s[c][4 * i + 2]), scale_log2, addend));
+                        float p3 = fast_exp2(fmaf(__uint_as_float(s[c][4 * i + 3]), scale_log2, addend));
+                        ps0 += p0; ps1 += p1; ps2 += p2; ps3 += p3;
+                        pk[2 * i] = pack_bf16x2(p0, p1);
+                        pk[2 * i + 1] = pack_bf16x2(p2, p3);
                     }
                 } else {
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) pk[i] = 0u;
+                    for (int i = 0; i < 8; ++i) {
+                        float p0 = fast_exp2(fmaf(__uint_as_float(s[c][4 * i]), scale_log2, ((am >> (4 * i)) & 1u) ? neg_ref : -INFINITY));
+                        float p1 = fast_exp2(fmaf(__uint_as_float(s[c][4 * i + 1]), scale_log2, ((am >> (4 * i + 1)) & 1u) ? neg_ref : -INFINITY));
+                        float p2 = fast_exp2(fmaf(__uint_as_float(s[c][4 * i + 2]), scale_log2, ((am >> (4 * i + 2)) & 1u) ? neg_ref : -INFINITY));
+                        float p3 = fast_exp2(fmaf(__uint_as_float(s[c][4 * i + 3]), scale_log2, ((am >> (4 * i + 3)) & 1u) ? neg_ref : -INFINITY));
+                        ps0 += p0; ps1 += p1; ps2 += p2; ps3 += p3;
+                        pk[2 * i] = pack_bf16x2(p0, p1);
+                        pk[2 * i + 1] = pack_bf16x2(p2, p3);
+                    }
                 }
                 tc::tmem_st_32x16(lane_addr + c * 16, pk);
             }
-            l_sum += psum;
+            l_sum += (ps0 + ps1) + (ps2 + ps3);
             tc::tmem_wait_st();
             tc::tc_fence_before_sync();
             tc::mbar_arrive(&sm.p_ready[t]);
