@@ -59,28 +59,30 @@ __global__ void __launch_bounds__(256) decode_score_select_kernel(Geom g, const 
     }
     __syncthreads();
     if (warp != 0) return;
-    double* e = dsel_smem;
+    unsigned long long* keys = reinterpret_cast<unsigned long long*>(dsel_smem);
     const int n = g.N;
-    OrderKey bd{0ull, 0x7fffffff};
+    unsigned long long bd = 0ull;
     if (g.top_p < 1.0) {
         double mx = -INFINITY;
-        for (int j = lane; j < n; j += 32) mx = fmax(mx, e[j]);
+        for (int j = lane; j < n; j += 32) mx = fmax(mx, dsel_smem[j]);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) mx = fmax(mx, __shfl_xor_sync(0xffffffffu, mx, o));
         double z = 0.0;
         for (int j = lane; j < n; j += 32) {
-            double ej = exp(e[j] - mx);
-            e[j] = ej;
+            double ej = exp(dsel_smem[j] - mx);
+            keys[j] = order_key(ej, j);
             z += ej;
         }
         z = warp_sum(z);
         __syncwarp();
-        bd = nucleus_boundary(e, n, g.top_p * z, lane);
+        bd = nucleus_boundary(keys, n, g.top_p * z, lane);
+    } else {
+        for (int j = lane; j < n; j += 32) keys[j] = order_key(1.0, j);
+        __syncwarp();
     }
-    const unsigned long long* ek = reinterpret_cast<const unsigned long long*>(e);
     for (int w = 0; w < g.n_words; ++w) {
         int j = w * 32 + lane;
-        bool on = (j < n) && !precedes(bd.key, bd.idx, ek[j < n ? j : 0], j);
+        bool on = j < n && keys[j] >= bd;
         uint32_t word = __ballot_sync(0xffffffffu, on);
         if (lane == 0) {
             dec_bitmap[((size_t)b * g.Hq + h) * g.n_words + w] = word;

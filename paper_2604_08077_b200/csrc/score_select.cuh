@@ -103,21 +103,27 @@ __global__ void __launch_bounds__(256) score_kernel(Geom g, int gt0,
 
 // ---------------------------------------------------------------------------------------------
 // Nucleus boundary of one row, executed by one full warp.
-//   e[0..n)   unnormalised probabilities exp(s_j - max) as doubles in shared memory (all >= 0)
-//   target    top_p * sum(e)
-// Cubes are ordered by (e descending, index ascending); the nucleus is the shortest prefix of
-// that order whose mass reaches target.  Returns the boundary element (key bits, index): cube j
-// is selected iff it precedes or equals the boundary.  The search narrows an open interval
-// (lo, hi) of the order around the boundary: each pass takes one pivot from the interval, sums
-// the interval's mass that precedes the pivot, and keeps the side holding the crossing.
-// Non-negative doubles order like their bit patterns, so all comparisons are on integers.
+//
+// Cubes are ordered by (probability descending, index ascending); the nucleus is the shortest
+// prefix of that order whose mass reaches the target.  Each candidate j is represented by one
+// 64-bit ORDER KEY: the bit pattern of e_j = exp(s_j - max) >= 0 (non-negative doubles order like
+// their bit patterns) with its 13 lowest mantissa bits replaced by (4096 - j).  A larger key comes
+// earlier in the order; equal probabilities are ordered by lower index.  Replacing the low
+// mantissa bits changes a value by less than 2^-39 relative, far below the 1e-6 tie margin that
+// bounds which rows may legitimately differ from an exact evaluation.  Keys are never zero.
+//
+// The search narrows an open interval (hi_key < key < lo_key) around the boundary: each pass picks
+// one interval element as pivot, sums the interval's mass above the pivot (warp reduction) and
+// keeps the side that holds the crossing.  Returns the boundary key: cube j is selected iff
+// key_j >= boundary (0 selects everything).
 // ---------------------------------------------------------------------------------------------
-struct OrderKey {
-    unsigned long long key;
-    int idx;
-};
-__device__ __forceinline__ bool precedes(unsigned long long ka, int ia, unsigned long long kb, int ib) {
-    return ka > kb || (ka == kb && ia < ib);
+constexpr unsigned long long kIdxMask = 0x1FFFull;
+
+__device__ __forceinline__ unsigned long long order_key(double e, int j) {
+    return ((unsigned long long)__double_as_longlong(e) & ~kIdxMask) | (unsigned long long)(4096 - j);
+}
+__device__ __forceinline__ double key_mass(unsigned long long key) {
+    return __longlong_as_double((long long)(key & ~kIdxMask));
 }
 
 __device__ __forceinline__ double warp_sum(double x) {
@@ -126,84 +132,55 @@ __device__ __forceinline__ double warp_sum(double x) {
     return x;
 }
 
-// Sort 32 (key, idx) pairs, one per lane, into the selection order (bitonic network via shuffles).
-__device__ __forceinline__ void warp_sort_order(unsigned long long& key, int& idx, int lane) {
-#pragma unroll
-    for (int k = 2; k <= 32; k <<= 1) {
-#pragma unroll
-        for (int j = k >> 1; j > 0; j >>= 1) {
-            unsigned long long ok = __shfl_xor_sync(0xffffffffu, key, j);
-            int oi = __shfl_xor_sync(0xffffffffu, idx, j);
-            bool up = ((lane & k) == 0);          // ascending segment (in selection order)
-            bool lower = ((lane & j) == 0);       // this lane keeps the earlier element
-            bool other_first = precedes(ok, oi, key, idx);
-            bool take = (lower == up) ? other_first : !other_first;
-            if (take) { key = ok; idx = oi; }
-        }
-    }
-}
-
-__device__ OrderKey nucleus_boundary(const double* e, int n, double target, int lane) {
-    const unsigned long long* ek = reinterpret_cast<const unsigned long long*>(e);
-    // open interval (lo, hi): lo precedes every element, hi follows every element
-    unsigned long long lo_k = ~0ull, hi_k = 0ull;
-    int lo_i = -1, hi_i = 0x7fffffff;
-    double base = 0.0;  // mass of everything that precedes or equals lo
-    // first pivot candidates: each lane offers its first element
-    unsigned long long cand_k = 0ull;
-    int cand_i = 0x7fffffff;
-    if (lane < n) { cand_k = ek[lane]; cand_i = lane; }
-    int n_cand = min(n, 32);
-
+__device__ unsigned long long nucleus_boundary(const unsigned long long* keys, int n, double target, int lane) {
+    unsigned long long lo = ~0ull, hi = 0ull;   // interval: hi < key < lo
+    double base = 0.0;                          // mass of every key >= lo
+    unsigned long long cand = lane < n ? keys[lane] : 0ull;   // each lane offers one interval element
     for (int iter = 0; iter < n + 2; ++iter) {
-        if (n_cand == 0) break;
-        // pivot = median of the offered candidates (absent lanes sort last)
-        unsigned long long sk = cand_k;
-        int si = cand_i;
-        warp_sort_order(sk, si, lane);
-        unsigned long long pv_k = __shfl_sync(0xffffffffu, sk, n_cand >> 1);
-        int pv_i = __shfl_sync(0xffffffffu, si, n_cand >> 1);
-
-        double mass_before = 0.0;
-        unsigned long long ca_k = 0ull, cb_k = 0ull;
-        int ca_i = 0x7fffffff, cb_i = 0x7fffffff;   // first element of each side seen by this lane
+        const uint32_t have = __ballot_sync(0xffffffffu, cand != 0ull);
+        if (have == 0u) break;
+        // pivot: the offer of one offering lane, rotating the starting lane every pass (offers are
+        // in index order, i.e. unordered in value)
+        const int rot = (iter * 11) & 31;
+        const int src = (__ffs(__funnelshift_r(have, have, rot)) - 1 + rot) & 31;
+        const unsigned long long pv = __shfl_sync(0xffffffffu, cand, src);
+        double mass_above = 0.0;
+        unsigned long long cand_above = 0ull, cand_below = 0ull;
         for (int j = lane; j < n; j += 32) {
-            unsigned long long kj = ek[j];
-            if (!precedes(lo_k, lo_i, kj, j) || !precedes(kj, j, hi_k, hi_i)) continue;
-            if (precedes(kj, j, pv_k, pv_i)) {
-                mass_before += __longlong_as_double((long long)kj);
-                if (ca_i == 0x7fffffff) { ca_k = kj; ca_i = j; }
-            } else if (precedes(pv_k, pv_i, kj, j)) {
-                if (cb_i == 0x7fffffff) { cb_k = kj; cb_i = j; }
+            const unsigned long long kj = keys[j];
+            if (kj >= lo || kj <= hi) continue;
+            if (kj > pv) {
+                mass_above += key_mass(kj);
+                if (cand_above == 0ull) cand_above = kj;
+            } else if (kj < pv) {
+                if (cand_below == 0ull) cand_below = kj;
             }
         }
-        mass_before = warp_sum(mass_before);
-        double pv_e = __longlong_as_double((long long)pv_k);
-        if (base + mass_before >= target) {          // crossing strictly before the pivot
-            hi_k = pv_k; hi_i = pv_i;
-            cand_k = ca_k; cand_i = ca_i;
-        } else if (base + mass_before + pv_e >= target) {
-            return OrderKey{pv_k, pv_i};              // the pivot is the crossing element
+        mass_above = warp_sum(mass_above);
+        const double pv_mass = key_mass(pv);
+        if (base + mass_above >= target) {              // crossing strictly above the pivot
+            hi = pv;
+            cand = cand_above;
+        } else if (base + mass_above + pv_mass >= target) {
+            return pv;                                   // the pivot is the crossing element
         } else {
-            base += mass_before + pv_e;
-            lo_k = pv_k; lo_i = pv_i;
-            cand_k = cb_k; cand_i = cb_i;
+            base += mass_above + pv_mass;
+            lo = pv;
+            cand = cand_below;
         }
-        n_cand = __popc(__ballot_sync(0xffffffffu, cand_i != 0x7fffffff));
     }
-    // Interval exhausted without reaching the target (rounding of partial sums): keep all up to hi.
-    if (hi_i == 0x7fffffff) return OrderKey{0ull, 0x7fffffff};
-    return OrderKey{lo_k, lo_i};
+    // Interval exhausted without reaching the target (rounding of partial sums): keep all above hi.
+    return hi == 0ull ? 0ull : lo;
 }
 
 // One warp per query row of the chunk.  Writes the per-tile mask matrix (always) and the
-// optional raster-ordered bitmap / count outputs.  dynamic smem: warps_per_cta * N_ld doubles.
+// optional raster-ordered bitmap / count outputs.  dynamic smem: warps_per_cta * N_ld keys.
 __global__ void __launch_bounds__(128) select_kernel(Geom g, int gt0, int n_gt,
                                                      const double* __restrict__ logits,
                                                      uint32_t* __restrict__ tile_mask,
                                                      uint32_t* __restrict__ sel_bitmap,
                                                      int32_t* __restrict__ sel_count) {
-    extern __shared__ double sel_smem[];
+    extern __shared__ unsigned long long sel_smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int row_id = blockIdx.x * 4 + warp;        // row within the chunk
     if (row_id >= n_gt * kTileRows) return;
@@ -211,11 +188,11 @@ __global__ void __launch_bounds__(128) select_kernel(Geom g, int gt0, int n_gt,
     const int tile = gt % g.n_tiles, bh = gt / g.n_tiles;
     const int h = bh % g.Hq, b = bh / g.Hq;
     const int pos = tile * kTileRows + r;
-    double* e = sel_smem + (size_t)warp * g.N_ld;
+    unsigned long long* keys = sel_smem + (size_t)warp * g.N_ld;
     const double* s = logits + (size_t)row_id * g.N_ld;
 
     const int n = pos < g.S ? n_candidates(g, pos) : 0;
-    OrderKey bd{0ull, 0x7fffffff};                  // default: everything precedes the boundary
+    unsigned long long bd = 0ull;                    // default: every candidate is selected
     if (n > 0 && g.top_p < 1.0) {
         double mx = -INFINITY;
         for (int j = lane; j < n; j += 32) mx = fmax(mx, s[j]);
@@ -224,27 +201,22 @@ __global__ void __launch_bounds__(128) select_kernel(Geom g, int gt0, int n_gt,
         double z = 0.0;
         for (int j = lane; j < n; j += 32) {
             double ej = exp(s[j] - mx);
-            e[j] = ej;
+            keys[j] = order_key(ej, j);
             z += ej;
         }
         z = warp_sum(z);
         __syncwarp();
-        bd = nucleus_boundary(e, n, g.top_p * z, lane);
+        bd = nucleus_boundary(keys, n, g.top_p * z, lane);
     } else {
-        for (int j = lane; j < n; j += 32) e[j] = 1.0;
+        for (int j = lane; j < n; j += 32) keys[j] = order_key(1.0, j);
         __syncwarp();
     }
 
-    const unsigned long long* ek = reinterpret_cast<const unsigned long long*>(e);
     const int raster = pos < g.S ? pos_to_raster(g, pos) : 0;
     int count = 0;
     for (int w = 0; w < g.n_words; ++w) {
         int j = w * 32 + lane;
-        bool on = false;
-        if (j < n) {
-            unsigned long long kj = ek[j];
-            on = !precedes(bd.key, bd.idx, kj, j);   // j precedes or equals the boundary
-        }
+        bool on = j < n && keys[j] >= bd;
         uint32_t word = __ballot_sync(0xffffffffu, on);
         count += __popc(word);
         if (lane == 0) {
