@@ -13,7 +13,9 @@
 #include "relayout_pool.cuh"
 #include "score_select.cuh"
 #include "attn_prefill_mma.cuh"
+#include "tc_common.cuh"
 #include "decode.cuh"
+#include "decode_splitkv.cuh"
 #ifdef ADASPARK_WITH_TCGEN05
 #include "attn_prefill_tc.cuh"
 #endif
@@ -181,16 +183,26 @@ adaspark_status_t adaspark_attn_partition(adaspark_attn_t* h, int32_t batch, int
     L.forward_workspace_bytes = (int64_t)off;
 
     // decode workspace: status | bitmaps | block lists | counts | split partials
-    int splits = (int)((4 * 148 + (size_t)batch * Hkv - 1) / ((size_t)batch * Hkv));
-    if (splits < 1) splits = 1;
-    if (splits > 64) splits = 64;
+    // split count: at least ~2 waves of CTAs over the 148 SMs, and among those the count that
+    // leaves the last wave fullest (one CTA per SM is resident)
+    int splits = 1;
+    {
+        const long long base = (long long)batch * Hkv;
+        double best = -1.0;
+        for (int s = 1; s <= 64; ++s) {
+            long long ctas = base * s;
+            double eff = (double)ctas / (double)((ctas + 147) / 148 * 148);
+            if (ctas < 2 * 148 && s < 64) continue;
+            if (eff > best + 1e-9) { best = eff; splits = s; }
+        }
+    }
     h->dc_splits = splits;
     off = 0;
     h->dc_status_off = off; off = align_up(off + 256);
     h->dc_bitmap_off = off; off = align_up(off + (size_t)batch * Hq * n_words * 4);
     h->dc_items_off = off; off = align_up(off + (size_t)batch * Hkv * (S_cap / kBlockTok) * 4);
     h->dc_nitems_off = off; off = align_up(off + (size_t)batch * Hkv * 4);
-    h->dc_partial_off = off; off = align_up(off + (size_t)batch * Hkv * splits * 16 * (D + 2) * 4);
+    h->dc_partial_off = off; off = align_up(off + (size_t)batch * Hkv * splits * (Hq / Hkv) * (D + 2) * 4);
     h->dc_total = off;
     L.decode_workspace_bytes = (int64_t)off;
 
@@ -246,6 +258,15 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
             if (!launch_ok(h, "pool_large_cubes_kernel")) return ADASPARK_ERR_CUDA;
         }
     }
+#ifdef ADASPARK_WITH_TCGEN05
+    if (!cache_only && h->prefill_kernel == 1) {   // cube-major staging of Q for the TMA loads of K4
+        dim3 rgrid((g.S + 31) / 32, g.B);
+        __nv_bfloat16* q_cube = (__nv_bfloat16*)((char*)workspace + h->fw_qcube_off);
+        if (D == 128) relayout_q_kernel<128><<<rgrid, 256, 0, st>>>(g, (const __nv_bfloat16*)q, q_cube);
+        else relayout_q_kernel<64><<<rgrid, 256, 0, st>>>(g, (const __nv_bfloat16*)q, q_cube);
+        if (!launch_ok(h, "relayout_q_kernel")) return ADASPARK_ERR_CUDA;
+    }
+#endif
     mark(h, 1, st);
     if (cache_only) return ADASPARK_OK;
 
@@ -276,10 +297,6 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
 #ifdef ADASPARK_WITH_TCGEN05
     if (h->prefill_kernel == 1) {
         __nv_bfloat16* q_cube = (__nv_bfloat16*)(ws + h->fw_qcube_off);
-        dim3 rgrid((g.S + 31) / 32, g.B);
-        if (D == 128) relayout_q_kernel<128><<<rgrid, 256, 0, st>>>(g, qb, q_cube);
-        else relayout_q_kernel<64><<<rgrid, 256, 0, st>>>(g, qb, q_cube);
-        if (!launch_ok(h, "relayout_q_kernel")) return ADASPARK_ERR_CUDA;
         CUtensorMap tmQ, tmK, tmV;
         if (!encode_bf16_2d(&tmQ, q_cube, (uint64_t)g.B * g.Hq * g.S_cap, D, 64, 128) ||
             !encode_bf16_2d(&tmK, kc, (uint64_t)g.B * g.Hkv * g.S_cap, D, 64, 64) ||
@@ -354,23 +371,32 @@ adaspark_status_t adaspark_attn_decode(adaspark_attn_t* h, const void* q_new, co
     }
     mark(h, 1, st);
     {
-        size_t smem = (size_t)g.N_ld * sizeof(double);
-        decode_score_select_kernel<<<dim3(g.Hq, g.B), 256, smem, st>>>(g, qn, cube_keys, dec_bitmap, sel_bitmap);
-        if (!launch_ok(h, "decode_score_select_kernel")) return ADASPARK_ERR_CUDA;
+        size_t smem = (size_t)decode_rows_per_pass(g.N_ld) * g.N_ld * sizeof(double) + (size_t)g.G * g.n_words * 4;
+        auto* blocks = (unsigned long long*)&hdr->decode_kv_blocks;
+        if (D == 128) {
+            if (!set_smem(h, decode_select_plan_kernel<128>, smem, "decode_select_plan_kernel")) return ADASPARK_ERR_CUDA;
+            decode_select_plan_kernel<128><<<dim3(g.Hkv, g.B), 256, smem, st>>>(g, qn, cube_keys, text_len, dec_bitmap, sel_bitmap, items, n_items, blocks);
+        } else {
+            if (!set_smem(h, decode_select_plan_kernel<64>, smem, "decode_select_plan_kernel")) return ADASPARK_ERR_CUDA;
+            decode_select_plan_kernel<64><<<dim3(g.Hkv, g.B), 256, smem, st>>>(g, qn, cube_keys, text_len, dec_bitmap, sel_bitmap, items, n_items, blocks);
+        }
+        if (!launch_ok(h, "decode_select_plan_kernel")) return ADASPARK_ERR_CUDA;
     }
-    decode_plan_kernel<<<dim3(g.Hkv, g.B), 32, 0, st>>>(g, dec_bitmap, text_len, items, n_items, (unsigned long long*)&hdr->decode_kv_blocks);
-    if (!launch_ok(h, "decode_plan_kernel")) return ADASPARK_ERR_CUDA;
     mark(h, 2, st);
     {
+        CUtensorMap tmK, tmV;
+        if (!encode_bf16_2d(&tmK, kc, (uint64_t)g.B * g.Hkv * g.S_cap, D, 64, 64) ||
+            !encode_bf16_2d(&tmV, vc, (uint64_t)g.B * g.Hkv * g.n_kv_blocks_cap * D, 64, 64, D))
+            return fail(h, ADASPARK_ERR_CUDA, "decode: cuTensorMapEncodeTiled failed");
         dim3 grid(h->dc_splits, g.Hkv, g.B);
         if (D == 128) {
-            size_t smem = sizeof(DecodeSmem<128>);
+            size_t smem = sizeof(DecodeSmem<128>) + 1024;
             if (!set_smem(h, decode_splitkv_kernel<128>, smem, "decode_splitkv_kernel")) return ADASPARK_ERR_CUDA;
-            decode_splitkv_kernel<128><<<grid, kDecodeThreads, smem, st>>>(g, h->dc_splits, qn, kc, vc, dec_bitmap, text_len, items, n_items, partial);
+            decode_splitkv_kernel<128><<<grid, kDecodeThreads, smem, st>>>(g, h->dc_splits, tmK, tmV, qn, dec_bitmap, text_len, items, n_items, partial, status);
         } else {
-            size_t smem = sizeof(DecodeSmem<64>);
+            size_t smem = sizeof(DecodeSmem<64>) + 1024;
             if (!set_smem(h, decode_splitkv_kernel<64>, smem, "decode_splitkv_kernel")) return ADASPARK_ERR_CUDA;
-            decode_splitkv_kernel<64><<<grid, kDecodeThreads, smem, st>>>(g, h->dc_splits, qn, kc, vc, dec_bitmap, text_len, items, n_items, partial);
+            decode_splitkv_kernel<64><<<grid, kDecodeThreads, smem, st>>>(g, h->dc_splits, tmK, tmV, qn, dec_bitmap, text_len, items, n_items, partial, status);
         }
         if (!launch_ok(h, "decode_splitkv_kernel")) return ADASPARK_ERR_CUDA;
     }
