@@ -279,7 +279,7 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
     // K3: scoring + selection, chunk by chunk
     {
         const int total_gt = g.B * g.Hq * g.n_tiles;
-        const size_t sel_smem = (size_t)4 * g.N_ld * sizeof(double);
+        const size_t sel_smem = select_smem_bytes(g.N_ld);
         if (!set_smem(h, select_kernel, sel_smem, "select_kernel")) return ADASPARK_ERR_CUDA;
         for (int gt0 = 0; gt0 < total_gt; gt0 += h->fw_chunk_tiles) {
             int n_gt = total_gt - gt0 < h->fw_chunk_tiles ? total_gt - gt0 : h->fw_chunk_tiles;
@@ -287,7 +287,7 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
             if (D == 128) score_kernel<128><<<sgrid, 256, 0, st>>>(g, gt0, qb, cube_keys, logits);
             else score_kernel<64><<<sgrid, 256, 0, st>>>(g, gt0, qb, cube_keys, logits);
             if (!launch_ok(h, "score_kernel")) return ADASPARK_ERR_CUDA;
-            select_kernel<<<n_gt * kTileRows / 4, 128, sel_smem, st>>>(g, gt0, n_gt, logits, tile_mask, sel_bitmap, sel_count);
+            select_kernel<<<n_gt * kTileRows / kSelectWarps, kSelectWarps * 32, sel_smem, st>>>(g, gt0, n_gt, logits, tile_mask, sel_bitmap, sel_count);
             if (!launch_ok(h, "select_kernel")) return ADASPARK_ERR_CUDA;
         }
     }

@@ -43,6 +43,11 @@ SMALL_CASES = {
                                                 Hq=1, Hkv=1, D=128, top_p=0.9),
     "sharp_scores": lambda: inputs.small_prefill(seed=12, T=16, H=8, W=8, n_text=17, top_p=0.5,
                                                  offset_std=3.0),
+    # nucleus boundaries far down the tail of a sharp distribution (many octaves below the maximum)
+    "deep_tail": lambda: inputs.small_prefill(seed=13, T=32, H=8, W=8, n_text=9, Hq=2, Hkv=1,
+                                              top_p=0.999999, offset_std=4.0),
+    "flat_scores": lambda: inputs.small_prefill(seed=14, T=32, H=8, W=8, n_text=9, Hq=2, Hkv=1,
+                                                top_p=0.6, offset_std=0.0),
 }
 
 
