@@ -23,6 +23,10 @@ adaspark_status_t adaspark_attn_debug_umma_selftest(const void *a, const void *b
                                                     float *d_out, float *e_out, int32_t *status,
                                                     void *cuda_stream);
 
+/* Host only: n / d computed by the multiply-shift routine the kernels use for their index
+ * arithmetic (0 <= n < 2^31, 1 <= d < 2^31); -1 for arguments outside that range. */
+int32_t adaspark_attn_debug_fastdiv(int32_t n, int32_t d);
+
 #ifdef __cplusplus
 }
 #endif

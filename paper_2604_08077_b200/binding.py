@@ -47,7 +47,7 @@ EXPORTS = ["adaspark_attn_create", "adaspark_attn_partition", "adaspark_attn_get
            "adaspark_attn_last_error", "adaspark_attn_last_launch_count",
            "adaspark_attn_set_prefill_kernel", "adaspark_attn_enable_stage_timing",
            "adaspark_attn_get_stage_times", "adaspark_attn_decode_static",
-           "adaspark_attn_debug_umma_selftest"]
+           "adaspark_attn_debug_umma_selftest", "adaspark_attn_debug_fastdiv"]
 
 
 def load() -> ctypes.CDLL:
@@ -67,6 +67,8 @@ def load() -> ctypes.CDLL:
     lib.adaspark_attn_decode.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.adaspark_attn_decode_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.adaspark_attn_debug_umma_selftest.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    lib.adaspark_attn_debug_fastdiv.argtypes = [ctypes.c_int32, ctypes.c_int32]
+    lib.adaspark_attn_debug_fastdiv.restype = ctypes.c_int32
     lib.adaspark_attn_destroy.argtypes = [vp]
     lib.adaspark_attn_last_error.argtypes = [vp]
     lib.adaspark_attn_last_error.restype = ctypes.c_char_p
@@ -161,6 +163,11 @@ def adaspark_attn_debug_umma_selftest(a, b, c, d_out, e_out, status, stream=None
     """128x128x128 tcgen05 self-test (see include/adaspark_attn_debug.h); returns the status code."""
     return int(load().adaspark_attn_debug_umma_selftest(_ptr(a), _ptr(b), _ptr(c), _ptr(d_out),
                                                        _ptr(e_out), _ptr(status), _stream_ptr(stream)))
+
+
+def adaspark_attn_debug_fastdiv(n: int, d: int) -> int:
+    """n // d by the kernels' multiply-shift index arithmetic (host only)."""
+    return int(load().adaspark_attn_debug_fastdiv(n, d))
 
 
 def adaspark_attn_destroy(handle: int):

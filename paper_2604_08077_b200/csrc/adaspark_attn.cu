@@ -66,13 +66,21 @@ Geom make_geom(const adaspark_attn* h, int n_text) {
     g.C = h->C; g.N = h->N;
     g.c_shift = 0;
     while ((1 << g.c_shift) < g.C) ++g.c_shift;
+    g.cw_shift = 0;
+    while ((1 << g.cw_shift) < g.cw) ++g.cw_shift;
+    g.ch_shift = 0;
+    while ((1 << g.ch_shift) < g.ch) ++g.ch_shift;
     g.S_v = h->S_v; g.n_text = n_text; g.S = h->S_v + n_text;
     g.S_cap = h->S_cap;
     g.n_words = (h->N + 31) / 32;
     g.n_tiles = (g.S + kTileRows - 1) / kTileRows;
     g.n_tiles_cap = h->S_cap / kTileRows;
+    g.div_nW.init(g.nW);
+    g.div_nH.init(g.nH);
+    g.div_n_tiles.init(g.n_tiles);
     g.n_kv_blocks_cap = h->S_cap / kBlockTok;
     g.Hq = h->cfg.n_q_heads; g.Hkv = h->cfg.n_kv_heads; g.G = g.Hq / g.Hkv; g.D = h->cfg.head_dim;
+    g.div_Hq.init(g.Hq);
     g.N_ld = (h->N + 63) / 64 * 64;
     double scale = h->cfg.softmax_scale > 0.f ? (double)h->cfg.softmax_scale : 1.0 / std::sqrt((double)g.D);
     g.scale_d = scale;
@@ -507,6 +515,13 @@ extern "C" adaspark_status_t adaspark_attn_decode_static(adaspark_attn_t* h, con
 // ---------------------------------------------------------------------------------------------
 #include "../../include/adaspark_attn_debug.h"
 #include "umma_selftest.cuh"
+
+extern "C" int32_t adaspark_attn_debug_fastdiv(int32_t n, int32_t d) {
+    if (n < 0 || d <= 0) return -1;
+    FastDiv f;
+    f.init(d);
+    return f.div(n);
+}
 
 extern "C" adaspark_status_t adaspark_attn_debug_umma_selftest(const void* a, const void* b, const void* c, float* d_out,
                                                                float* e_out, int32_t* status, void* cuda_stream) {

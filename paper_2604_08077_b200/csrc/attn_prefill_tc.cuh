@@ -294,31 +294,30 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
 #pragma unroll
             for (int c = 0; c < 4; ++c) tc::tmem_ld_32x32(lane_addr + c * 32, s[c]);
             tc::tmem_wait_ld();
-            // ---- row maximum over the visible keys (four independent chains per chunk)
+            // ---- row maximum over the visible keys
             float mx = -INFINITY;
+            if (uniform) {
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const uint32_t am = amask[c];
-                float a0 = -INFINITY, a1 = -INFINITY, a2 = -INFINITY, a3 = -INFINITY;
-                if (uniform) {
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        a0 = fmaxf(a0, __uint_as_float(s[c][4 * i]));
-                        a1 = fmaxf(a1, __uint_as_float(s[c][4 * i + 1]));
-                        a2 = fmaxf(a2, __uint_as_float(s[c][4 * i + 2]));
-                        a3 = fmaxf(a3, __uint_as_float(s[c][4 * i + 3]));
-                    }
-                    const float cm = fmaxf(fmaxf(a0, a1), fmaxf(a2, a3));
-                    mx = am ? fmaxf(mx, cm) : mx;
-                } else {
+                for (int c = 0; c < 4; ++c) {
+                    float a0 = -INFINITY, a1 = -INFINITY;
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
-                        a0 = fmaxf(a0, ((am >> (4 * i)) & 1u) ? __uint_as_float(s[c][4 * i]) : -INFINITY);
-                        a1 = fmaxf(a1, ((am >> (4 * i + 1)) & 1u) ? __uint_as_float(s[c][4 * i + 1]) : -INFINITY);
-                        a2 = fmaxf(a2, ((am >> (4 * i + 2)) & 1u) ? __uint_as_float(s[c][4 * i + 2]) : -INFINITY);
-                        a3 = fmaxf(a3, ((am >> (4 * i + 3)) & 1u) ? __uint_as_float(s[c][4 * i + 3]) : -INFINITY);
+                        a0 = fmax3(a0, __uint_as_float(s[c][4 * i]), __uint_as_float(s[c][4 * i + 1]));
+                        a1 = fmax3(a1, __uint_as_float(s[c][4 * i + 2]), __uint_as_float(s[c][4 * i + 3]));
                     }
-                    mx = fmaxf(mx, fmaxf(fmaxf(a0, a1), fmaxf(a2, a3)));
+                    mx = fmax3(mx, amask[c] ? a0 : -INFINITY, amask[c] ? a1 : -INFINITY);
+                }
+            } else {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const uint32_t am = amask[c];
+                    float a0 = -INFINITY, a1 = -INFINITY;
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        a0 = fmaxf(a0, ((am >> (2 * i)) & 1u) ? __uint_as_float(s[c][2 * i]) : -INFINITY);
+                        a1 = fmaxf(a1, ((am >> (2 * i + 1)) & 1u) ? __uint_as_float(s[c][2 * i + 1]) : -INFINITY);
+                    }
+                    mx = fmax3(mx, a0, a1);
                 }
             }
             const float mx_x = mx * scale_log2;                   // scale > 0: max commutes with it
@@ -342,38 +341,49 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
             }
             // ---- P = 2^(s*scale - m_ref) on visible keys, 0 elsewhere; bf16 pairs into TMEM
             const float neg_ref = -m_ref;                          // finite whenever a key is visible
-            float ps0 = 0.f, ps1 = 0.f, ps2 = 0.f, ps3 = 0.f;
+            if (uniform) {
+                const unsigned long long scale2 = pack_f32x2(scale_log2, scale_log2);
+                unsigned long long acc2[4];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const uint32_t am = amask[c];
-                uint32_t pk[16];
-                if (uniform) {
-                    const float addend = am ? neg_ref : -INFINITY;   // 2^(-inf) = 0 hides the chunk
+                for (int c = 0; c < 4; ++c) {
+                    const float addend = amask[c] ? neg_ref : -INFINITY;   // 2^(-inf) = 0 hides the chunk
+                    const unsigned long long addend2 = pack_f32x2(addend, addend);
+                    uint32_t pk[16];
+                    unsigned long long a = 0ull, b = 0ull;                  // two (lo, hi) partial sums
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
-                        float p0 = fast_exp2(fmaf(__uint_as_float(s[c][4 * i]), scale_log2, addend));
-                        float p1 = fast_exp2(fmaf(__uint_as_float(s[c][4 * i + 1]), scale_log2, addend));
-                        float p2 = fast_exp2(fmaf(__uint_as_float(s[c][4 * i + 2]), scale_log2, addend));
-                        float p3 = fast_exp2(fmaf(__uint_as_float(s[c][4 * i + 3]), scale_log2, addend));
-                        ps0 += p0; ps1 += p1; ps2 += p2; ps3 += p3;
+                        float x0, x1, x2, x3;
+                        unpack_f32x2(ffma2(pack_u32x2(s[c][4 * i], s[c][4 * i + 1]), scale2, addend2), x0, x1);
+                        unpack_f32x2(ffma2(pack_u32x2(s[c][4 * i + 2], s[c][4 * i + 3]), scale2, addend2), x2, x3);
+                        const float p0 = fast_exp2(x0), p1 = fast_exp2(x1), p2 = fast_exp2(x2), p3 = fast_exp2(x3);
+                        a = fadd2(a, pack_f32x2(p0, p1));
+                        b = fadd2(b, pack_f32x2(p2, p3));
                         pk[2 * i] = pack_bf16x2(p0, p1);
                         pk[2 * i + 1] = pack_bf16x2(p2, p3);
                     }
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        float p0 = fast_exp2(fmaf(__uint_as_float(s[c][4 * i]), scale_log2, ((am >> (4 * i)) & 1u) ? neg_ref : -INFINITY));
-                        float p1 = fast_exp2(fmaf(__uint_as_float(s[c][4 * i + 1]), scale_log2, ((am >> (4 * i + 1)) & 1u) ? neg_ref : -INFINITY));
-                        float p2 = fast_exp2(fmaf(__uint_as_float(s[c][4 * i + 2]), scale_log2, ((am >> (4 * i + 2)) & 1u) ? neg_ref : -INFINITY));
-                        float p3 = fast_exp2(fmaf(__uint_as_float(s[c][4 * i + 3]), scale_log2, ((am >> (4 * i + 3)) & 1u) ? neg_ref : -INFINITY));
-                        ps0 += p0; ps1 += p1; ps2 += p2; ps3 += p3;
-                        pk[2 * i] = pack_bf16x2(p0, p1);
-                        pk[2 * i + 1] = pack_bf16x2(p2, p3);
-                    }
+                    tc::tmem_st_32x16(lane_addr + c * 16, pk);
+                    acc2[c] = fadd2(a, b);
                 }
-                tc::tmem_st_32x16(lane_addr + c * 16, pk);
+                float l0, l1;
+                unpack_f32x2(fadd2(fadd2(acc2[0], acc2[1]), fadd2(acc2[2], acc2[3])), l0, l1);
+                l_sum += l0 + l1;
+            } else {
+                float ps0 = 0.f, ps1 = 0.f;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const uint32_t am = amask[c];
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        float p0 = fast_exp2(fmaf(__uint_as_float(s[c][2 * i]), scale_log2, ((am >> (2 * i)) & 1u) ? neg_ref : -INFINITY));
+                        float p1 = fast_exp2(fmaf(__uint_as_float(s[c][2 * i + 1]), scale_log2, ((am >> (2 * i + 1)) & 1u) ? neg_ref : -INFINITY));
+                        ps0 += p0; ps1 += p1;
+                        pk[i] = pack_bf16x2(p0, p1);
+                    }
+                    tc::tmem_st_32x16(lane_addr + c * 16, pk);
+                }
+                l_sum += ps0 + ps1;
             }
-            l_sum += (ps0 + ps1) + (ps2 + ps3);
             tc::tmem_wait_st();
             tc::tc_fence_before_sync();
             tc::mbar_arrive(&sm.p_ready[t]);

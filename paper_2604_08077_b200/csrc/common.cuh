@@ -9,6 +9,30 @@ namespace adaspark {
 constexpr int kTileRows = 128;  // query rows per tile (cube-major positions)
 constexpr int kBlockTok = 64;   // key/value tokens per block (cube-major positions)
 
+// Division of a non-negative int (< 2^31) by a runtime constant without a divide instruction:
+// with s = ceil(log2 d) and mul = floor(2^32 * (2^s - d) / d) + 1, n / d = (hi32(n * mul) + n) >> s.
+struct FastDiv {
+    uint32_t mul, shift;
+    int d;
+    __host__ void init(int divisor) {
+        d = divisor;
+        shift = 0;
+        while ((1ll << shift) < (long long)divisor) ++shift;
+        mul = (uint32_t)((((1ull << shift) - (unsigned long long)divisor) << 32) / (unsigned long long)divisor + 1ull);
+    }
+    __host__ __device__ __forceinline__ int div(int n) const {
+#ifdef __CUDA_ARCH__
+        return (int)((__umulhi((uint32_t)n, mul) + (uint32_t)n) >> shift);
+#else
+        return (int)(((uint32_t)(((unsigned long long)(uint32_t)n * mul) >> 32) + (uint32_t)n) >> shift);
+#endif
+    }
+    __host__ __device__ __forceinline__ void divmod(int n, int& q, int& r) const {
+        q = div(n);
+        r = n - q * d;
+    }
+};
+
 // Geometry of one partitioned problem (Sec. 3.1).  "pos" is the cube-major position of a token:
 // video token of cube c with intra-cube rank r sits at pos = c*C + r, text token u at S_v + u.
 struct Geom {
@@ -17,6 +41,8 @@ struct Geom {
     int nH, nW;          // cube grid: H/ch, W/cw
     int C, N;            // tokens per cube (a power of two), cubes
     int c_shift;         // log2(C)
+    int cw_shift, ch_shift;   // log2(cw), log2(ch): C is a power of two, so every window side is one
+    FastDiv div_nW, div_nH, div_n_tiles, div_Hq;
     int S_v, n_text, S;  // video tokens, text tokens of this call, total
     int S_cap;           // cache rows per (b, kv head), multiple of 128
     int n_words;         // ceil(N/32)
@@ -34,13 +60,13 @@ struct Geom {
 // O1 inverse: cube-major position -> raster token index.
 __device__ __forceinline__ int pos_to_raster(const Geom& g, int pos) {
     if (pos >= g.S_v) return pos;
-    int c = pos / g.C, r = pos - c * g.C;
-    int cx = c % g.nW;
-    int cy = (c / g.nW) % g.nH;
-    int cb = c / (g.nW * g.nH);
-    int rx = r % g.cw;
-    int ry = (r / g.cw) % g.ch;
-    int rt = r / (g.cw * g.ch);
+    const int c = pos >> g.c_shift, r = pos & (g.C - 1);
+    int cx, cy, cb, t;
+    g.div_nW.divmod(c, t, cx);
+    g.div_nH.divmod(t, cb, cy);
+    const int rx = r & (g.cw - 1);
+    const int ry = (r >> g.cw_shift) & (g.ch - 1);
+    const int rt = r >> (g.cw_shift + g.ch_shift);
     return ((cb * g.ct + rt) * g.H + (cy * g.ch + ry)) * g.W + (cx * g.cw + rx);
 }
 
@@ -112,6 +138,37 @@ __device__ __forceinline__ float fast_exp2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
     return y;
+}
+
+// ---- sm_100 packed / three-input float operations ------------------------------------------
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ unsigned long long pack_u32x2(uint32_t lo, uint32_t hi) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(unsigned long long v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+// (a.lo*b.lo + c.lo, a.hi*b.hi + c.hi) in one instruction
+__device__ __forceinline__ unsigned long long ffma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ unsigned long long fadd2(unsigned long long a, unsigned long long b) {
+    unsigned long long d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
 }
 
 }  // namespace adaspark

@@ -30,8 +30,9 @@ __global__ void __launch_bounds__(256) score_kernel(Geom g, int gt0,
     __shared__ double Ks[kScoreCols][kScorePitch];
 
     const int gt = gt0 + blockIdx.x;
-    const int tile = gt % g.n_tiles, bh = gt / g.n_tiles;
-    const int h = bh % g.Hq, b = bh / g.Hq;
+    int tile, bh, h, b;
+    g.div_n_tiles.divmod(gt, bh, tile);
+    g.div_Hq.divmod(bh, b, h);
     const int gk = h / g.G;
     const int col0 = blockIdx.y * kScoreCols;
     // candidates of the last valid row bound the columns this tile needs
@@ -380,8 +381,9 @@ __global__ void __launch_bounds__(kSelectWarps * 32) select_kernel(Geom g, int g
     const int row_id = blockIdx.x * kSelectWarps + warp;        // row within the chunk
     if (row_id >= n_gt * kTileRows) return;
     const int gt = gt0 + row_id / kTileRows, r = row_id % kTileRows;
-    const int tile = gt % g.n_tiles, bh = gt / g.n_tiles;
-    const int h = bh % g.Hq, b = bh / g.Hq;
+    int tile, bh, h, b;
+    g.div_n_tiles.divmod(gt, bh, tile);
+    g.div_Hq.divmod(bh, b, h);
     const int pos = tile * kTileRows + r;
     unsigned long long* scratch = sel_smem + (size_t)warp * kSelWarpScratch;
     unsigned long long* keys = sel_smem + (size_t)kSelectWarps * kSelWarpScratch + (size_t)warp * g.N_ld;
@@ -392,7 +394,8 @@ __global__ void __launch_bounds__(kSelectWarps * 32) select_kernel(Geom g, int g
     const bool all = !(g.top_p < 1.0);
     if (n > 0 && !all) bd = nucleus_boundary_radix(s, n, g.top_p, keys, scratch, lane);
 
-    const int raster = pos < g.S ? pos_to_raster(g, pos) : 0;
+    const bool extra = (sel_bitmap != nullptr || sel_count != nullptr) && pos < g.S;
+    const int raster = extra ? pos_to_raster(g, pos) : 0;
     int count = 0;
     for (int w = 0; w < g.n_words; ++w) {
         int j = w * 32 + lane;
@@ -401,11 +404,11 @@ __global__ void __launch_bounds__(kSelectWarps * 32) select_kernel(Geom g, int g
         count += __popc(word);
         if (lane == 0) {
             tile_mask[mask_index(g, b, h, tile, w, r)] = word;
-            if (sel_bitmap && pos < g.S)
+            if (sel_bitmap && extra)
                 sel_bitmap[((size_t)(b * g.Hq + h) * g.S + raster) * g.n_words + w] = word;
         }
     }
-    if (sel_count && lane == 0 && pos < g.S) sel_count[(size_t)(b * g.Hq + h) * g.S + raster] = count;
+    if (sel_count && lane == 0 && extra) sel_count[(size_t)(b * g.Hq + h) * g.S + raster] = count;
 }
 
 }  // namespace adaspark

@@ -145,3 +145,20 @@ def test_missing_library_raises(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
         binding.load()
+
+
+def test_index_division_matches_integer_division(lib):
+    """The multiply-shift division behind the kernels' index arithmetic equals n // d on every
+    divisor a partition can produce (small ones exhaustively, large ones sampled)."""
+    import numpy as np
+    rng = np.random.default_rng(0)
+    divisors = list(range(1, 300)) + [511, 512, 513, 1023, 1025, 4095, 4096, 4097, 65535, 65536,
+                                      1048575, 1048577, (1 << 30) - 1, (1 << 30) + 1, (1 << 31) - 1]
+    for d in divisors:
+        edge = [0, 1, d - 1, d, d + 1, 2 * d - 1, 2 * d, (1 << 31) - 1,
+                ((1 << 31) - 1) // d * d, max(((1 << 31) - 1) // d * d - 1, 0)]
+        ns = [int(x) for x in edge if 0 <= x < (1 << 31)] + [int(x) for x in rng.integers(0, 1 << 31, 40)]
+        for n in ns:
+            assert binding.adaspark_attn_debug_fastdiv(n, d) == n // d, (n, d)
+    assert binding.adaspark_attn_debug_fastdiv(-1, 3) == -1
+    assert binding.adaspark_attn_debug_fastdiv(5, 0) == -1
