@@ -310,7 +310,7 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
             !encode_bf16_2d(&tmK, kc, (uint64_t)g.B * g.Hkv * g.S_cap, D, 64, 64) ||
             !encode_bf16_2d(&tmV, vc, (uint64_t)g.B * g.Hkv * g.n_kv_blocks_cap * D, 64, 64, D))
             return fail(h, ADASPARK_ERR_CUDA, "forward: cuTensorMapEncodeTiled failed");
-        dim3 grid((g.S + kPairRows - 1) / kPairRows, g.Hq, g.B);
+        dim3 grid(((g.S + kPairRows - 1) / kPairRows) * g.Hq * g.B);
         if (D == 128) {
             size_t smem = sizeof(TcAttnSmem<128>) + 1024;
             if (!set_smem(h, attn_prefill_tc_kernel<128>, smem, "attn_prefill_tc_kernel")) return ADASPARK_ERR_CUDA;

@@ -71,8 +71,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     constexpr uint32_t kQBytes = 2 * 128 * D * 2, kKBytes = 128 * D * 2, kVBytes = 2 * D * 64 * 2;
 
     const int n_pairs = (g.S + kPairRows - 1) / kPairRows;
-    const int pair = n_pairs - 1 - blockIdx.x;                  // long (late) tiles first
-    const int h = blockIdx.y, b = blockIdx.z, gk = h / g.G;
+    // 1-D grid, pair-major: the late (long) pair tiles of every head and batch entry start first
+    const int n_hb = g.Hq * g.B;
+    const int pair = n_pairs - 1 - (int)blockIdx.x / n_hb;
+    const int hb = (int)blockIdx.x - (n_pairs - 1 - pair) * n_hb;
+    const int b = hb / g.Hq, h = hb - b * g.Hq, gk = h / g.G;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int pair_pos0 = pair * kPairRows;
     const int pair_end = min(pair_pos0 + kPairRows, g.S);       // exclusive
@@ -177,19 +180,33 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     } else if (warp == 9) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
+            // descriptor low halves of the tile bases; a k-step of 16 elements advances 32 bytes
+            // inside a 64-element panel (128-byte rows), panels / key blocks are 128 rows apart
+            constexpr uint32_t kPanelStep = (128 * 64 * 2) >> 4, kKStep = 32 >> 4;
+            constexpr uint32_t kVBlockStep = (D * 64 * 2) >> 4;
+            constexpr uint32_t kQTileStep = (uint32_t)sizeof(sm.q[0]) >> 4, kKStageStep = (uint32_t)sizeof(sm.k[0]) >> 4;
+            constexpr uint32_t kVStageStep = (uint32_t)sizeof(sm.v[0]) >> 4;
+            const uint32_t q_lo0 = tc::smem_desc_lo_sw128(smem_u32(&sm.q[0][0][0][0]));
+            const uint32_t k_lo0 = tc::smem_desc_lo_sw128(smem_u32(&sm.k[0][0][0][0]));
+            const uint32_t v_lo0 = tc::smem_desc_lo_sw128(smem_u32(&sm.v[0][0][0][0]));
             auto issue_s = [&](int t, int st) {   // S_t = Q_t K(st)^T
+                const uint32_t qa = q_lo0 + t * kQTileStep, kb = k_lo0 + st * kKStageStep, dst = tbase + t * 256;
+                tc::umma_ss_c<false>(dst, tc::smem_desc_from_halves(qa, tc::kSmemDescHiSw128),
+                                     tc::smem_desc_from_halves(kb, tc::kSmemDescHiSw128), kIdescS);
 #pragma unroll
-                for (int ks = 0; ks < kQKSteps; ++ks) {
-                    uint64_t da = tc::make_smem_desc_sw128(smem_u32(&sm.q[t][ks >> 2][0][0]) + (ks & 3) * 32);
-                    uint64_t db = tc::make_smem_desc_sw128(smem_u32(&sm.k[st][ks >> 2][0][0]) + (ks & 3) * 32);
-                    tc::umma_ss(tbase + t * 256, da, db, kIdescS, ks > 0);
+                for (int ks = 1; ks < kQKSteps; ++ks) {
+                    const uint32_t off = (ks >> 2) * kPanelStep + (ks & 3) * kKStep;
+                    tc::umma_ss_c<true>(dst, tc::smem_desc_from_halves(qa + off, tc::kSmemDescHiSw128),
+                                        tc::smem_desc_from_halves(kb + off, tc::kSmemDescHiSw128), kIdescS);
                 }
             };
             auto issue_pv = [&](int t, int st, bool first) {   // O_t (+)= P_t V(st)
+                const uint32_t vb = v_lo0 + st * kVStageStep, dst = tbase + t * 256 + 128, src = tbase + t * 256;
+                tc::umma_ts(dst, src, tc::smem_desc_from_halves(vb, tc::kSmemDescHiSw128), kIdescO, !first);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    uint64_t db = tc::make_smem_desc_sw128(smem_u32(&sm.v[st][ks >> 2][0][0]) + (ks & 3) * 32);
-                    tc::umma_ts(tbase + t * 256 + 128, tbase + t * 256 + ks * 8, db, kIdescO, !(first && ks == 0));
+                for (int ks = 1; ks < 8; ++ks) {
+                    const uint32_t off = (ks >> 2) * kVBlockStep + (ks & 3) * kKStep;
+                    tc::umma_ts_c<true>(dst, src + ks * 8, tc::smem_desc_from_halves(vb + off, tc::kSmemDescHiSw128), kIdescO);
                 }
             };
             bool ok = tc::mbar_wait(&sm.q_full, 0, abort_flag) && tc::mbar_wait(&sm.k_full[0], 0, abort_flag);
@@ -276,11 +293,22 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
                         m1 = ((wbits & 4u) ? 0x0000ffffu : 0u) | ((wbits & 8u) ? 0xffff0000u : 0u);
                     }
                 } else {
+                    // local range: every aligned group of 16 keys lies in one cube or in the text
+                    // (C >= 16 and S_v is a multiple of C), so the rule of Eq. 3 is closed-form per group
                     const uint32_t word = pk0 < g.S_v ? get_word((pk0 >> g.c_shift) >> 5) : 0u;
-                    for (int i = 0; i < 32; ++i) {
-                        if (key_allowed(g, pr, pk0 + i, word)) m0 |= 1u << i;
-                        if (key_allowed(g, pr, pk0 + 32 + i, word)) m1 |= 1u << i;
+                    uint32_t gm[4];
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        const int pg = pk0 + q4 * 16;
+                        const int n_causal = min(max(pr - pg + 1, 0), 16);           // keys pg..pr
+                        const uint32_t causal = (1u << n_causal) - 1u;
+                        const int ck = pg >> g.c_shift;
+                        const bool own = pg >= g.S_v || (pr < g.S_v && ck == (pr >> g.c_shift));
+                        const uint32_t picked = (pg < g.S_v && ((word >> (ck & 31)) & 1u)) ? 0xffffu : 0u;
+                        gm[q4] = own ? causal : picked;
                     }
+                    m0 = gm[0] | (gm[1] << 16);
+                    m1 = gm[2] | (gm[3] << 16);
                 }
                 amask[hf * 2] = m0;
                 amask[hf * 2 + 1] = m1;
