@@ -37,7 +37,7 @@ struct TcAttnSmem {
     __nv_bfloat16 v[2][2][D][64];             // [stage][block][d][64 keys]  (V^T)
     uint32_t blk_words[kMaxBlockWords];       // bit kb set <=> key block kb is visited
     uint32_t union_words[128];                // OR of the 256 rows' selection words
-    uint64_t q_full, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], p_ready[2], o_final;
+    uint64_t q_full, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], p_half[2][2], o_final;
     uint32_t tmem_base;
     int abort_flag;
     int n_needed;                             // number of visited key blocks
@@ -92,7 +92,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
             tc::mbar_init(&sm.v_full[i], 1);
             tc::mbar_init(&sm.v_empty[i], 1);
             tc::mbar_init(&sm.s_full[i], 1);
-            tc::mbar_init(&sm.p_ready[i], 128);
+            tc::mbar_init(&sm.p_half[i][0], 128);
+            tc::mbar_init(&sm.p_half[i][1], 128);
         }
         tc::mbar_init(&sm.o_final, 1);
         sm.abort_flag = 0;
@@ -200,14 +201,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
                                         tc::smem_desc_from_halves(kb + off, tc::kSmemDescHiSw128), kIdescS);
                 }
             };
-            auto issue_pv = [&](int t, int st, bool first) {   // O_t (+)= P_t V(st)
-                const uint32_t vb = v_lo0 + st * kVStageStep, dst = tbase + t * 256 + 128, src = tbase + t * 256;
+            // O_t (+)= P_t V(st), keys [64 half, 64 half + 64): the two halves are issued separately so
+            // that the first can start while the softmax warps still produce the second
+            auto issue_pv = [&](int t, int st, int half, bool first) {
+                const uint32_t vb = v_lo0 + st * kVStageStep + half * kVBlockStep, dst = tbase + t * 256 + 128;
+                const uint32_t src = tbase + t * 256 + half * 32;
                 tc::umma_ts(dst, src, tc::smem_desc_from_halves(vb, tc::kSmemDescHiSw128), kIdescO, !first);
 #pragma unroll
-                for (int ks = 1; ks < 8; ++ks) {
-                    const uint32_t off = (ks >> 2) * kVBlockStep + (ks & 3) * kKStep;
-                    tc::umma_ts_c<true>(dst, src + ks * 8, tc::smem_desc_from_halves(vb + off, tc::kSmemDescHiSw128), kIdescO);
-                }
+                for (int ks = 1; ks < 4; ++ks)
+                    tc::umma_ts_c<true>(dst, src + ks * 8, tc::smem_desc_from_halves(vb + ks * kKStep, tc::kSmemDescHiSw128), kIdescO);
             };
             bool ok = tc::mbar_wait(&sm.q_full, 0, abort_flag) && tc::mbar_wait(&sm.k_full[0], 0, abort_flag);
             if (ok) {
@@ -223,18 +225,24 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
                 const bool more = j + 1 < n_steps;
                 const int st1 = (j + 1) & 1, u1 = (j + 1) >> 1;
                 if (!(ok = tc::mbar_wait(&sm.v_full[st], u & 1, abort_flag))) break;
-                if (!(ok = tc::mbar_wait(&sm.p_ready[0], j & 1, abort_flag))) break;
+                if (!(ok = tc::mbar_wait(&sm.p_half[0][0], j & 1, abort_flag))) break;
                 tc::tc_fence_after_sync();
-                issue_pv(0, st, j == 0);
+                issue_pv(0, st, 0, j == 0);
+                if (!(ok = tc::mbar_wait(&sm.p_half[0][1], j & 1, abort_flag))) break;
+                tc::tc_fence_after_sync();
+                issue_pv(0, st, 1, false);
                 if (more) {
                     if (!(ok = tc::mbar_wait(&sm.k_full[st1], u1 & 1, abort_flag))) break;
                     tc::tc_fence_after_sync();
                     issue_s(0, st1);
                     tc::umma_commit(&sm.s_full[0]);
                 }
-                if (!(ok = tc::mbar_wait(&sm.p_ready[1], j & 1, abort_flag))) break;
+                if (!(ok = tc::mbar_wait(&sm.p_half[1][0], j & 1, abort_flag))) break;
                 tc::tc_fence_after_sync();
-                issue_pv(1, st, j == 0);
+                issue_pv(1, st, 0, j == 0);
+                if (!(ok = tc::mbar_wait(&sm.p_half[1][1], j & 1, abort_flag))) break;
+                tc::tc_fence_after_sync();
+                issue_pv(1, st, 1, false);
                 tc::umma_commit(&sm.v_empty[st]);
                 if (more) {
                     issue_s(1, st1);
@@ -325,16 +333,19 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
             // ---- row maximum over the visible keys
             float mx = -INFINITY;
             if (uniform) {
+                float a[4][2];
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    float a0 = -INFINITY, a1 = -INFINITY;
+                for (int c = 0; c < 4; ++c) a[c][0] = a[c][1] = -INFINITY;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        a0 = fmax3(a0, __uint_as_float(s[c][4 * i]), __uint_as_float(s[c][4 * i + 1]));
-                        a1 = fmax3(a1, __uint_as_float(s[c][4 * i + 2]), __uint_as_float(s[c][4 * i + 3]));
+                for (int i = 0; i < 8; ++i)          // eight independent chains
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        a[c][0] = fmax3(a[c][0], __uint_as_float(s[c][4 * i]), __uint_as_float(s[c][4 * i + 1]));
+                        a[c][1] = fmax3(a[c][1], __uint_as_float(s[c][4 * i + 2]), __uint_as_float(s[c][4 * i + 3]));
                     }
-                    mx = fmax3(mx, amask[c] ? a0 : -INFINITY, amask[c] ? a1 : -INFINITY);
-                }
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    mx = fmax3(mx, amask[c] ? a[c][0] : -INFINITY, amask[c] ? a[c][1] : -INFINITY);
             } else {
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
@@ -370,31 +381,29 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
             // ---- P = 2^(s*scale - m_ref) on visible keys, 0 elsewhere; bf16 pairs into TMEM
             const float neg_ref = -m_ref;                          // finite whenever a key is visible
             if (uniform) {
-                const unsigned long long scale2 = pack_f32x2(scale_log2, scale_log2);
-                unsigned long long acc2[4];
+                float ps0 = 0.f, ps1 = 0.f, ps2 = 0.f, ps3 = 0.f;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     const float addend = amask[c] ? neg_ref : -INFINITY;   // 2^(-inf) = 0 hides the chunk
-                    const unsigned long long addend2 = pack_f32x2(addend, addend);
                     uint32_t pk[16];
-                    unsigned long long a = 0ull, b = 0ull;                  // two (lo, hi) partial sums
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
-                        float x0, x1, x2, x3;
-                        unpack_f32x2(ffma2(pack_u32x2(s[c][4 * i], s[c][4 * i + 1]), scale2, addend2), x0, x1);
-                        unpack_f32x2(ffma2(pack_u32x2(s[c][4 * i + 2], s[c][4 * i + 3]), scale2, addend2), x2, x3);
-                        const float p0 = fast_exp2(x0), p1 = fast_exp2(x1), p2 = fast_exp2(x2), p3 = fast_exp2(x3);
-                        a = fadd2(a, pack_f32x2(p0, p1));
-                        b = fadd2(b, pack_f32x2(p2, p3));
+                        const float p0 = fast_exp2(fmaf(__uint_as_float(s[c][4 * i]), scale_log2, addend));
+                        const float p1 = fast_exp2(fmaf(__uint_as_float(s[c][4 * i + 1]), scale_log2, addend));
+                        const float p2 = fast_exp2(fmaf(__uint_as_float(s[c][4 * i + 2]), scale_log2, addend));
+                        const float p3 = fast_exp2(fmaf(__uint_as_float(s[c][4 * i + 3]), scale_log2, addend));
+                        ps0 += p0; ps1 += p1; ps2 += p2; ps3 += p3;
                         pk[2 * i] = pack_bf16x2(p0, p1);
                         pk[2 * i + 1] = pack_bf16x2(p2, p3);
                     }
                     tc::tmem_st_32x16(lane_addr + c * 16, pk);
-                    acc2[c] = fadd2(a, b);
+                    if (c == 1) {                                   // first 64 keys of P are in place
+                        tc::tmem_wait_st();
+                        tc::tc_fence_before_sync();
+                        tc::mbar_arrive(&sm.p_half[t][0]);
+                    }
                 }
-                float l0, l1;
-                unpack_f32x2(fadd2(fadd2(acc2[0], acc2[1]), fadd2(acc2[2], acc2[3])), l0, l1);
-                l_sum += l0 + l1;
+                l_sum += (ps0 + ps1) + (ps2 + ps3);
             } else {
                 float ps0 = 0.f, ps1 = 0.f;
 #pragma unroll
@@ -409,12 +418,17 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
                         pk[i] = pack_bf16x2(p0, p1);
                     }
                     tc::tmem_st_32x16(lane_addr + c * 16, pk);
+                    if (c == 1) {
+                        tc::tmem_wait_st();
+                        tc::tc_fence_before_sync();
+                        tc::mbar_arrive(&sm.p_half[t][0]);
+                    }
                 }
                 l_sum += ps0 + ps1;
             }
             tc::tmem_wait_st();
             tc::tc_fence_before_sync();
-            tc::mbar_arrive(&sm.p_ready[t]);
+            tc::mbar_arrive(&sm.p_half[t][1]);
         }
         // ---- epilogue: O / l -> bf16 at the raster position of the row
         if (ok) ok = tc::mbar_wait(&sm.o_final, 0, abort_flag);
