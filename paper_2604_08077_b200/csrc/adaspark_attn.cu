@@ -288,14 +288,17 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
     {
         const int total_gt = g.B * g.Hq * g.n_tiles;
         const size_t sel_smem = select_smem_bytes(g.N_ld);
-        if (!set_smem(h, select_kernel, sel_smem, "select_kernel")) return ADASPARK_ERR_CUDA;
+        const int lanes = select_lanes_per_row(g.N_ld);
+        auto* sel_fn = lanes == 8 ? select_kernel<8> : (lanes == 16 ? select_kernel<16> : select_kernel<32>);
+        if (!set_smem(h, sel_fn, sel_smem, "select_kernel")) return ADASPARK_ERR_CUDA;
+        const int rows_per_cta = kSelectWarps * (32 / lanes);
         for (int gt0 = 0; gt0 < total_gt; gt0 += h->fw_chunk_tiles) {
             int n_gt = total_gt - gt0 < h->fw_chunk_tiles ? total_gt - gt0 : h->fw_chunk_tiles;
             dim3 sgrid(n_gt, g.N_ld / kScoreCols);
             if (D == 128) score_kernel<128><<<sgrid, 256, 0, st>>>(g, gt0, qb, cube_keys, logits);
             else score_kernel<64><<<sgrid, 256, 0, st>>>(g, gt0, qb, cube_keys, logits);
             if (!launch_ok(h, "score_kernel")) return ADASPARK_ERR_CUDA;
-            select_kernel<<<n_gt * kTileRows / kSelectWarps, kSelectWarps * 32, sel_smem, st>>>(g, gt0, n_gt, logits, tile_mask, sel_bitmap, sel_count);
+            sel_fn<<<n_gt * kTileRows / rows_per_cta, kSelectWarps * 32, sel_smem, st>>>(g, gt0, n_gt, logits, tile_mask, sel_bitmap, sel_count);
             if (!launch_ok(h, "select_kernel")) return ADASPARK_ERR_CUDA;
         }
     }
@@ -379,7 +382,7 @@ adaspark_status_t adaspark_attn_decode(adaspark_attn_t* h, const void* q_new, co
     }
     mark(h, 1, st);
     {
-        size_t smem = (size_t)decode_rows_per_pass(g.N_ld) * g.N_ld * sizeof(double) + (size_t)g.G * g.n_words * 4;
+        size_t smem = decode_select_smem_bytes(g.N_ld, g.G, g.n_words);
         auto* blocks = (unsigned long long*)&hdr->decode_kv_blocks;
         if (D == 128) {
             if (!set_smem(h, decode_select_plan_kernel<128>, smem, "decode_select_plan_kernel")) return ADASPARK_ERR_CUDA;

@@ -9,7 +9,7 @@
 // The split-KV attention kernel itself is in decode_splitkv.cuh.
 #pragma once
 #include "common.cuh"
-#include "score_select.cuh"
+#include "select_radix.cuh"
 
 namespace adaspark {
 
@@ -34,9 +34,15 @@ __global__ void decode_append_kernel(Geom g, const __nv_bfloat16* __restrict__ k
 
 // Rows (heads) scored per pass: as many as fit next to each other in shared memory, at most 8
 // (the M of mma.m8n8k4).
+constexpr int kDecodeCandCap = 256;
 __host__ __device__ inline int decode_rows_per_pass(int N_ld) {
-    int r = (176 * 1024) / (N_ld * 8);
+    int r = (200 * 1024) / (N_ld * 8 + (kSelHistWords + kDecodeCandCap) * 8);
     return r > 8 ? 8 : (r < 1 ? 1 : r);
+}
+// dynamic smem of decode_select_plan_kernel: rows_per_pass * (N_ld scores + histogram + candidates)
+// words of 8 bytes + G * n_words bitmap words of 4 bytes
+__host__ __device__ inline size_t decode_select_smem_bytes(int N_ld, int G, int n_words) {
+    return (size_t)decode_rows_per_pass(N_ld) * ((size_t)N_ld + kSelHistWords + kDecodeCandCap) * 8 + (size_t)G * n_words * 4;
 }
 
 // grid (Hkv, B), 256 threads.  dynamic smem: rows_per_pass * N_ld doubles + G * n_words words.
@@ -51,7 +57,8 @@ __global__ void __launch_bounds__(256) decode_select_plan_kernel(
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int rpp = decode_rows_per_pass(g.N_ld);
     double* logit = dsp_smem;                                              // [rpp][N_ld]
-    uint32_t* bm = reinterpret_cast<uint32_t*>(dsp_smem + (size_t)rpp * g.N_ld);   // [G][n_words]
+    unsigned long long* sel_scratch = reinterpret_cast<unsigned long long*>(dsp_smem + (size_t)rpp * g.N_ld);   // [rpp][hist + cand]
+    uint32_t* bm = reinterpret_cast<uint32_t*>(sel_scratch + (size_t)rpp * (kSelHistWords + kDecodeCandCap));   // [G][n_words]
     const float* kbase = cube_keys + (size_t)(b * g.Hkv + gk) * g.N * D;
     const int rq = lane >> 2, kq = lane & 3;
 
@@ -95,27 +102,14 @@ __global__ void __launch_bounds__(256) decode_select_plan_kernel(
             unsigned long long* keys = reinterpret_cast<unsigned long long*>(row);
             const int n = g.N;
             unsigned long long bd = 0ull;
-            if (g.top_p < 1.0) {
-                double mx = -INFINITY;
-                for (int j = lane; j < n; j += 32) mx = fmax(mx, row[j]);
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) mx = fmax(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-                double z = 0.0;
-                for (int j = lane; j < n; j += 32) {
-                    double ej = exp(row[j] - mx);
-                    keys[j] = order_key(ej, j);
-                    z += ej;
-                }
-                z = warp_sum(z);
-                __syncwarp();
-                bd = nucleus_boundary(keys, n, g.top_p * z, lane);
-            } else {
-                for (int j = lane; j < n; j += 32) keys[j] = order_key(1.0, j);
-                __syncwarp();
+            const bool all = !(g.top_p < 1.0);
+            if (!all) {
+                unsigned long long* hist = sel_scratch + (size_t)warp * (kSelHistWords + kDecodeCandCap);
+                bd = nucleus_boundary_radix<32>(row, n, g.top_p, keys, hist, hist + kSelHistWords, kDecodeCandCap, lane);
             }
             for (int w = 0; w < g.n_words; ++w) {
                 int j = w * 32 + lane;
-                bool on = j < n && keys[j] >= bd;
+                bool on = j < n && (all || keys[j] >= bd);
                 uint32_t word = __ballot_sync(0xffffffffu, on);
                 if (lane == 0) {
                     bm[hr * g.n_words + w] = word;
