@@ -116,7 +116,12 @@ adaspark_status_t adaspark_attn_get_layout(const adaspark_attn_t *handle,
  *                     order) is set iff cube j is in the row's nucleus S_i.
  *   sel_count    out, nullable: int32 [B, Hq, S] = |S_i|.
  *   workspace    device scratch of at least forward_workspace_bytes, 256-byte aligned.
- * Enqueues kernels on the stream and returns; no host synchronisation. */
+ * Enqueues kernels and returns; no host synchronisation.  The scoring of one chunk of query tiles
+ * runs concurrently with the selection of the previous chunk: the selection kernels are enqueued
+ * on a stream private to the handle, ordered against `cuda_stream` with events in both directions,
+ * so that everything the call enqueued is complete, from the point of view of `cuda_stream`, before
+ * any later work on it.  The first _forward of a handle creates that stream and its events (make
+ * that first call before any stream capture). */
 adaspark_status_t adaspark_attn_forward(adaspark_attn_t *handle, const void *q, const void *k,
                                         const void *v, int32_t n_text, void *out, void *k_cube,
                                         void *v_cube, float *cube_keys, uint32_t *sel_bitmap,
@@ -175,7 +180,8 @@ adaspark_status_t adaspark_attn_decode_static(adaspark_attn_t *handle, const voi
                                               const int32_t *text_len, void *out,
                                               uint32_t *sel_bitmap, void *cuda_stream);
 
-/* Release the handle (host memory only). NULL is accepted. */
+/* Release the handle: host memory, and the private stream / events of a handle that ran _forward
+ * (waits for that stream to drain).  NULL is accepted. */
 adaspark_status_t adaspark_attn_destroy(adaspark_attn_t *handle);
 
 /* Message of the most recent error on this handle ("" if none). Never NULL. */

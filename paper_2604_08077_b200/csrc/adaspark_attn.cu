@@ -39,13 +39,18 @@ struct adaspark_attn {
     bool timing;
     cudaEvent_t ev[5];
     bool ev_recorded;
+    // scoring of one chunk of query tiles overlaps the selection of the previous chunk: the
+    // selection kernels run on this handle-private stream, ordered against the caller's by events
+    cudaStream_t side;
+    cudaEvent_t ev_fork, ev_score[2], ev_select[2];
+    bool side_ready;
     char err[256];
 };
 
 namespace {
 
 constexpr size_t kAlign = 256;
-constexpr size_t kLogitsBudget = 64ull << 20;   // score scratch stays well inside the 126 MB L2
+constexpr size_t kLogitsBudget = 40ull << 20;   // per buffer; two buffers stay inside the 126 MB L2
 size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 
 adaspark_status_t fail(adaspark_attn* h, adaspark_status_t st, const char* fmt, ...) {
@@ -185,7 +190,7 @@ adaspark_status_t adaspark_attn_partition(adaspark_attn_t* h, int32_t batch, int
     if (chunk < 1) chunk = 1;
     if (chunk > total_tiles) chunk = total_tiles;
     h->fw_chunk_tiles = (int)chunk;
-    h->fw_logits_off = off; off = align_up(off + chunk * tile_bytes);
+    h->fw_logits_off = off; off = align_up(off + 2 * chunk * tile_bytes);   // double-buffered
     h->fw_qcube_off = off; off = align_up(off + (size_t)batch * Hq * S_cap * D * 2);
     h->fw_total = off;
     L.forward_workspace_bytes = (int64_t)off;
@@ -292,15 +297,38 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
         auto* sel_fn = lanes == 8 ? select_kernel<8> : (lanes == 16 ? select_kernel<16> : select_kernel<32>);
         if (!set_smem(h, sel_fn, sel_smem, "select_kernel")) return ADASPARK_ERR_CUDA;
         const int rows_per_cta = kSelectWarps * (32 / lanes);
-        for (int gt0 = 0; gt0 < total_gt; gt0 += h->fw_chunk_tiles) {
-            int n_gt = total_gt - gt0 < h->fw_chunk_tiles ? total_gt - gt0 : h->fw_chunk_tiles;
-            dim3 sgrid(n_gt, g.N_ld / kScoreCols);
-            if (D == 128) score_kernel<128><<<sgrid, 256, 0, st>>>(g, gt0, qb, cube_keys, logits);
-            else score_kernel<64><<<sgrid, 256, 0, st>>>(g, gt0, qb, cube_keys, logits);
-            if (!launch_ok(h, "score_kernel")) return ADASPARK_ERR_CUDA;
-            sel_fn<<<n_gt * kTileRows / rows_per_cta, kSelectWarps * 32, sel_smem, st>>>(g, gt0, n_gt, logits, tile_mask, sel_bitmap, sel_count);
-            if (!launch_ok(h, "select_kernel")) return ADASPARK_ERR_CUDA;
+        if (!h->side_ready) {   // first forward of this handle: create the side stream and its events
+            cudaError_t e = cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming);
+            for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+                e = cudaEventCreateWithFlags(&h->ev_score[i], cudaEventDisableTiming);
+                if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_select[i], cudaEventDisableTiming);
+            }
+            if (e != cudaSuccess) return fail(h, ADASPARK_ERR_CUDA, "forward: side stream set-up: %s", cudaGetErrorString(e));
+            h->side_ready = true;
         }
+        const size_t buf_elems = (size_t)h->fw_chunk_tiles * kTileRows * g.N_ld;
+        cudaEventRecord(h->ev_fork, st);                       // the side stream starts after the re-layout
+        cudaStreamWaitEvent(h->side, h->ev_fork, 0);
+        int chunk_idx = 0;
+        for (int gt0 = 0; gt0 < total_gt; gt0 += h->fw_chunk_tiles, ++chunk_idx) {
+            int n_gt = total_gt - gt0 < h->fw_chunk_tiles ? total_gt - gt0 : h->fw_chunk_tiles;
+            const int buf = chunk_idx & 1;
+            double* chunk_logits = logits + (size_t)buf * buf_elems;
+            if (chunk_idx >= 2) cudaStreamWaitEvent(st, h->ev_select[buf], 0);   // the buffer has been consumed
+            dim3 sgrid(n_gt, g.N_ld / kScoreCols);
+            if (D == 128) score_kernel<128><<<sgrid, 256, 0, st>>>(g, gt0, qb, cube_keys, chunk_logits);
+            else score_kernel<64><<<sgrid, 256, 0, st>>>(g, gt0, qb, cube_keys, chunk_logits);
+            if (!launch_ok(h, "score_kernel")) return ADASPARK_ERR_CUDA;
+            cudaEventRecord(h->ev_score[buf], st);
+            cudaStreamWaitEvent(h->side, h->ev_score[buf], 0);
+            sel_fn<<<n_gt * kTileRows / rows_per_cta, kSelectWarps * 32, sel_smem, h->side>>>(g, gt0, n_gt, chunk_logits, tile_mask, sel_bitmap, sel_count);
+            if (!launch_ok(h, "select_kernel")) return ADASPARK_ERR_CUDA;
+            cudaEventRecord(h->ev_select[buf], h->side);
+        }
+        // join: the attention kernel needs every selection
+        cudaStreamWaitEvent(st, h->ev_select[0], 0);
+        if (chunk_idx >= 2) cudaStreamWaitEvent(st, h->ev_select[1], 0);
     }
 
     mark(h, 2, st);
@@ -421,6 +449,15 @@ adaspark_status_t adaspark_attn_decode(adaspark_attn_t* h, const void* q_new, co
 adaspark_status_t adaspark_attn_destroy(adaspark_attn_t* h) {
     if (h && h->timing)
         for (int i = 0; i < 5; ++i) cudaEventDestroy(h->ev[i]);
+    if (h && h->side_ready) {
+        cudaStreamSynchronize(h->side);
+        cudaEventDestroy(h->ev_fork);
+        for (int i = 0; i < 2; ++i) {
+            cudaEventDestroy(h->ev_score[i]);
+            cudaEventDestroy(h->ev_select[i]);
+        }
+        cudaStreamDestroy(h->side);
+    }
     delete h;
     return ADASPARK_OK;
 }

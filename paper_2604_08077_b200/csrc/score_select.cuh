@@ -108,7 +108,7 @@ __global__ void __launch_bounds__(256) score_kernel(Geom g, int gt0,
 // dynamic smem per warp: kSelHistWords + (32/G) * (N_ld keys + cand_cap candidates) words of 8 bytes.
 constexpr int kSelectWarps = 4;
 __host__ __device__ inline int select_lanes_per_row(int N_ld) { return N_ld <= 128 ? 8 : (N_ld <= 512 ? 16 : 32); }
-__host__ __device__ inline int select_cand_cap(int N_ld) { return N_ld < 256 ? N_ld : 256; }
+__host__ __device__ inline int select_cand_cap(int N_ld) { return N_ld <= 256 ? 64 : (N_ld <= 1024 ? 128 : 256); }
 __host__ __device__ inline size_t select_smem_bytes(int N_ld) {
     const int rows = 32 / select_lanes_per_row(N_ld);
     return (size_t)kSelectWarps * ((size_t)kSelHistWords + (size_t)rows * (N_ld + select_cand_cap(N_ld))) * 8;
