@@ -37,6 +37,12 @@ WORKLOAD = ("config2: AdaS-Attn prefill, batch 1, 64x16x16 video tokens (cube 4x
             "+ 128 text, 28/4 heads, head_dim 128, p=0.9")
 
 
+# DRAM bytes (read + write) of one launch of the prefill attention kernel on this workload, from the
+# ncu capture summarised in profiles/attn_prefill_tc_kernel_config2.md.  Set to None whenever that
+# kernel changes until the counters are taken again.
+ATTN_DRAM_TRAFFIC_BYTES = 255.0e6
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -308,7 +314,8 @@ def main():
         "gpu_launches": launches_per_step * args.steps,
         "roofline": {"kernel": "prefill attention", "bound": "tensor", "achieved": achieved_tflops,
                      "peak": peak_tflops, "unit": "TFLOP/s", "frac": achieved_tflops / peak_tflops,
-                     "traffic": None,
+                     "traffic": ATTN_DRAM_TRAFFIC_BYTES,
+                     "traffic_unit": "bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum)",
                      "peak_source": f"{peaks['source']} bf16 burst (kernel of ~ms inside a ~ms step)"},
         "stages_ms": {"relayout_pool": float(st_mean[0]), "score_select": float(st_mean[1]),
                       "attention": attn_ms},
