@@ -166,7 +166,8 @@ adaspark_status_t adaspark_attn_decode(adaspark_attn_t *handle, const void *q_ne
  *
  * Arguments, results and errors are those of adaspark_attn_decode.  In addition:
  *   - ERR_WORKSPACE_TOO_SMALL if the partition's decode_workspace_bytes exceeds the 8 MiB
- *     (config 5 fits up to batch 8; at batch 16 it needs about 10 MiB); use adaspark_attn_decode then.
+ *     (a 131072-token video cache in 2048 cubes with 28/4 heads of 128 fits up to batch 8; at batch 16
+ *     it needs about 10 MiB); use adaspark_attn_decode then.
  *   - The first call on each device looks up the array's device address (a one-time host-side
  *     set-up with that device current); make that first call before any stream capture begins.
  *   - The call performs no cudaMalloc / cudaFree and uses no allocating library routine.
