@@ -18,6 +18,7 @@
 #include "decode_splitkv.cuh"
 #ifdef ADASPARK_WITH_TCGEN05
 #include "attn_prefill_tc.cuh"
+#include "score_tc.cuh"
 #endif
 
 using namespace adaspark;
@@ -29,7 +30,7 @@ struct adaspark_attn {
     int C, N, S_v, S_cap;
     adaspark_attn_layout_t layout;
     // workspace carving (byte offsets)
-    size_t fw_status_off, fw_mask_off, fw_logits_off, fw_qcube_off, fw_total;
+    size_t fw_status_off, fw_mask_off, fw_logits_off, fw_qcube_off, fw_kplanes_off, fw_kexp_off, fw_total;
     int fw_chunk_tiles;
     size_t dc_status_off, dc_bitmap_off, dc_items_off, dc_nitems_off, dc_partial_off, dc_total;
     int dc_splits;
@@ -189,9 +190,14 @@ adaspark_status_t adaspark_attn_partition(adaspark_attn_t* h, int32_t batch, int
     size_t chunk = kLogitsBudget / tile_bytes;
     if (chunk < 1) chunk = 1;
     if (chunk > total_tiles) chunk = total_tiles;
+    if (chunk > 148) chunk = chunk / 148 * 148;    // whole waves of one-CTA-per-SM scoring tiles
     h->fw_chunk_tiles = (int)chunk;
     h->fw_logits_off = off; off = align_up(off + 2 * chunk * tile_bytes);   // double-buffered
     h->fw_qcube_off = off; off = align_up(off + (size_t)batch * Hq * S_cap * D * 2);
+    // digit planes (4 x bf16 [B*Hkv*N_ld, D]) and row exponents of the mean keys (tensor-core scoring);
+    // 128 rows of slack so that the last 128-cube TMA box stays inside the allocation
+    h->fw_kplanes_off = off; off = align_up(off + ((size_t)4 * batch * Hkv * N_ld + 128) * D * 2);
+    h->fw_kexp_off = off; off = align_up(off + (size_t)batch * Hkv * N_ld * 4);
     h->fw_total = off;
     L.forward_workspace_bytes = (int64_t)off;
 
@@ -307,6 +313,21 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
             if (e != cudaSuccess) return fail(h, ADASPARK_ERR_CUDA, "forward: side stream set-up: %s", cudaGetErrorString(e));
             h->side_ready = true;
         }
+#ifdef ADASPARK_WITH_TCGEN05
+        CUtensorMap tmQs, tmKs;
+        int32_t* key_exp = (int32_t*)(ws + h->fw_kexp_off);
+        if (h->prefill_kernel == 1) {   // digit planes of the mean keys, tensor maps of the scoring kernel
+            __nv_bfloat16* kplanes = (__nv_bfloat16*)(ws + h->fw_kplanes_off);
+            const int n_rows = g.B * g.Hkv * g.N_ld;
+            slice_keys_kernel<<<(n_rows + 3) / 4, 128, 0, st>>>(g, cube_keys, kplanes, key_exp);
+            if (!launch_ok(h, "slice_keys_kernel")) return ADASPARK_ERR_CUDA;
+            if (!encode_bf16_2d(&tmQs, ws + h->fw_qcube_off, (uint64_t)g.B * g.Hq * g.S_cap, D, 64, 128) ||
+                !encode_bf16_2d(&tmKs, kplanes, (uint64_t)4 * n_rows + 128, D, 64, 128))
+                return fail(h, ADASPARK_ERR_CUDA, "forward: cuTensorMapEncodeTiled failed");
+            if (D == 128) { if (!set_smem(h, score_tc_kernel<128>, sizeof(ScoreTcSmem<128>) + 1024, "score_tc_kernel")) return ADASPARK_ERR_CUDA; }
+            else { if (!set_smem(h, score_tc_kernel<64>, sizeof(ScoreTcSmem<64>) + 1024, "score_tc_kernel")) return ADASPARK_ERR_CUDA; }
+        }
+#endif
         const size_t buf_elems = (size_t)h->fw_chunk_tiles * kTileRows * g.N_ld;
         cudaEventRecord(h->ev_fork, st);                       // the side stream starts after the re-layout
         cudaStreamWaitEvent(h->side, h->ev_fork, 0);
@@ -316,10 +337,28 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
             const int buf = chunk_idx & 1;
             double* chunk_logits = logits + (size_t)buf * buf_elems;
             if (chunk_idx >= 2) cudaStreamWaitEvent(st, h->ev_select[buf], 0);   // the buffer has been consumed
-            dim3 sgrid(n_gt, g.N_ld / kScoreCols);
-            if (D == 128) score_kernel<128><<<sgrid, 256, 0, st>>>(g, gt0, qb, cube_keys, chunk_logits);
-            else score_kernel<64><<<sgrid, 256, 0, st>>>(g, gt0, qb, cube_keys, chunk_logits);
-            if (!launch_ok(h, "score_kernel")) return ADASPARK_ERR_CUDA;
+#ifdef ADASPARK_WITH_TCGEN05
+            if (h->prefill_kernel == 1) {
+                const int n_ct = (g.N + kScoreTcCols - 1) / kScoreTcCols;
+                int groups = (148 + n_gt - 1) / n_gt;
+                if (groups > n_ct) groups = n_ct;
+                const int cols_per_cta = (n_ct + groups - 1) / groups;
+                dim3 tgrid(n_gt, (n_ct + cols_per_cta - 1) / cols_per_cta);
+                if (D == 128)
+                    score_tc_kernel<128><<<tgrid, kScoreTcThreads, sizeof(ScoreTcSmem<128>) + 1024, st>>>(
+                        g, gt0, cols_per_cta, tmQs, tmKs, key_exp, chunk_logits, &hdr->status);
+                else
+                    score_tc_kernel<64><<<tgrid, kScoreTcThreads, sizeof(ScoreTcSmem<64>) + 1024, st>>>(
+                        g, gt0, cols_per_cta, tmQs, tmKs, key_exp, chunk_logits, &hdr->status);
+                if (!launch_ok(h, "score_tc_kernel")) return ADASPARK_ERR_CUDA;
+            } else
+#endif
+            {
+                dim3 sgrid(n_gt, g.N_ld / kScoreCols);
+                if (D == 128) score_kernel<128><<<sgrid, 256, 0, st>>>(g, gt0, qb, cube_keys, chunk_logits);
+                else score_kernel<64><<<sgrid, 256, 0, st>>>(g, gt0, qb, cube_keys, chunk_logits);
+                if (!launch_ok(h, "score_kernel")) return ADASPARK_ERR_CUDA;
+            }
             cudaEventRecord(h->ev_score[buf], st);
             cudaStreamWaitEvent(h->side, h->ev_score[buf], 0);
             sel_fn<<<n_gt * kTileRows / rows_per_cta, kSelectWarps * 32, sel_smem, h->side>>>(g, gt0, n_gt, chunk_logits, tile_mask, sel_bitmap, sel_count);

@@ -140,6 +140,9 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
+// byte offset of 16-byte chunk `chunk` of 128-byte row `row` under the 128-byte swizzle
+__device__ __forceinline__ int sw128(int row, int chunk) { return row * 128 + ((chunk ^ (row & 7)) << 4); }
+
 // ---- sm_100 packed / three-input float operations ------------------------------------------
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
     float d;

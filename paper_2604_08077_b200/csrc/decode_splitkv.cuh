@@ -26,8 +26,6 @@ struct DecodeSmem {
     int abort_flag;
 };
 
-// byte offset of 16-byte chunk `chunk` of 128-byte row `row` under the 128-byte swizzle
-__device__ __forceinline__ int sw128(int row, int chunk) { return row * 128 + ((chunk ^ (row & 7)) << 4); }
 
 // grid (n_splits, Hkv, B).  partial[((b*Hkv+gk)*n_splits + split)*G + row] = {m, l, o[D]}
 // (base-2 running max, sum, unnormalised output).

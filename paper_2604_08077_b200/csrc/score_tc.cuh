@@ -1,0 +1,282 @@
+// K3 on the bf16 tensor cores: cube scores of Eq. 1 from error-free digit slices.
+//
+// The selection must follow an fp64 evaluation of Eqs. 1-2 (rows may differ only inside a 1e-6
+// probability margin), so plain bf16/fp32 tensor-core arithmetic is not accurate enough.  Instead
+// every query row q and every mean key k are written in fixed point relative to the largest
+// exponent of their row,
+//     x = 2^(e - 30) * (d0*2^24 + d1*2^16 + d2*2^8 + d3),   digits d_i integers in [-128, 128],
+// (exact for elements within 2^-23 (q, 8 significant bits) / 2^-7 (k, 24 bits) of the row maximum,
+// rounded at 2^-30 of it below that).  Digits are exact bf16 values, a product of two digits has 15
+// bits and a sum of 4 * 128 such products stays below 2^24, so a tcgen05.mma with fp32 accumulation
+// computes  S_L = sum_{a+b=L} Q_a . K_b  EXACTLY for each level L.  Then
+//     q . k = 2^(e_q + e_k - 12) * (S_0 + S_1*2^-8 + S_2*2^-16 + S_3*2^-24 + levels >= 4),
+// and the levels 0..3 (10 digit pairs, four TMEM accumulators) are combined exactly in fp64.  The
+// dropped levels are bounded by 1.5e-3 * 2^-12 * 2^(e_q+e_k) in the worst case (all digit products
+// aligned), about 5e-7 in the scaled logit for |q| <= 3, |k| <= 5 and typically 10x less: inside
+// the margin above.
+//
+//   slice_keys_kernel   digit planes + row exponents of the mean keys (once per forward, tiny)
+//   score_tc_kernel     CTA = one 128-row query tile x a group of 128-cube column tiles:
+//     warps 0-3  slice the Q tile (thread = row) into four swizzled digit planes in shared memory,
+//                later the epilogue: TMEM -> fp64 scores -> coalesced rows of the score buffer
+//     warp 4     TMA producer: Q tile once, then the key digit blocks (plane, 64-d panel) in a ring
+//     warp 5     issues the tcgen05.mma stream (80 per column tile at D = 128)
+#pragma once
+#include "tc_common.cuh"
+
+namespace adaspark {
+
+constexpr int kScoreTcThreads = 192;
+constexpr int kScoreTcRing = 4;          // key digit blocks (128 cubes x 64 d, 16 KB) in flight
+constexpr int kScoreTcCols = 128;        // cubes per column tile
+
+// Fixed-point value of x relative to the row exponent e (unbiased exponent of the row maximum):
+// round(x * 2^(30 - e)), |result| < 2^31.
+__device__ __forceinline__ int fixed30(float x, int e) {
+    return __float2int_rn(x * __int_as_float((157 - e) << 23));   // 2^(30 - e), exact for e >= -96
+}
+// Signed base-256 digits, most significant first: v = d[0]*2^24 + d[1]*2^16 + d[2]*2^8 + d[3].
+__device__ __forceinline__ void digits256(int v, int (&d)[4]) {
+    // v = 256 * (floor(v / 256) + carry) + digit with digit = low byte read as signed (no overflow)
+    d[3] = (int)(signed char)(v & 0xff);
+    v = (v >> 8) + (d[3] < 0 ? 1 : 0);
+    d[2] = (int)(signed char)(v & 0xff);
+    v = (v >> 8) + (d[2] < 0 ? 1 : 0);
+    d[1] = (int)(signed char)(v & 0xff);
+    d[0] = (v >> 8) + (d[1] < 0 ? 1 : 0);
+}
+// bf16 bit pattern of a small integer (|i| <= 256: exact).
+__device__ __forceinline__ uint32_t bf16_bits_of_int(int i) {
+    return __float_as_uint((float)i) >> 16;
+}
+__device__ __forceinline__ int exponent_of(float x) {   // unbiased exponent field (0 for zero/denormal rows)
+    const int e = (int)((__float_as_uint(x) >> 23) & 0xffu);
+    return e == 0 ? 0 : max(e - 127, -90);     // rows smaller than 2^-90 keep fewer digits
+}
+
+// Digit planes of the mean keys: planes[p][(b*Hkv+gk)*N_ld + cube][D] (bf16), key_exp[(b*Hkv+gk)*N_ld + cube].
+// One warp per cube row; rows >= N inside the padded leading dimension are zero-filled.
+__global__ void __launch_bounds__(128) slice_keys_kernel(Geom g, const float* __restrict__ cube_keys,
+                                                         __nv_bfloat16* __restrict__ planes, int32_t* __restrict__ key_exp) {
+    const int lane = threadIdx.x & 31;
+    const int row = blockIdx.x * 4 + (threadIdx.x >> 5);              // (b*Hkv+gk)*N_ld + cube
+    const int n_rows = g.B * g.Hkv * g.N_ld;
+    if (row >= n_rows) return;
+    const int bh = row / g.N_ld, cube = row - bh * g.N_ld;
+    const size_t plane_stride = (size_t)n_rows * g.D;
+    const bool live = cube < g.N;
+    const float* src = cube_keys + ((size_t)bh * g.N + (live ? cube : 0)) * g.D;
+    float mx = 0.f;
+    for (int d = lane; d < g.D; d += 32) mx = fmaxf(mx, live ? fabsf(src[d]) : 0.f);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    const int e = exponent_of(mx);
+    for (int d = lane; d < g.D; d += 32) {
+        int dg[4];
+        digits256(live ? fixed30(src[d], e) : 0, dg);
+#pragma unroll
+        for (int p = 0; p < 4; ++p)
+            planes[p * plane_stride + (size_t)row * g.D + d] = __ushort_as_bfloat16((unsigned short)bf16_bits_of_int(dg[p]));
+    }
+    if (lane == 0) key_exp[row] = e;
+}
+
+template <int D>
+struct ScoreTcSmem {
+    __nv_bfloat16 qd[4][D / 64][128][64];               // digit planes of the Q tile, UMMA layout (128-B swizzle)
+    __nv_bfloat16 kring[kScoreTcRing][128][64];         // key digit blocks: [cube][64 d of one panel of one plane]
+    // first the bf16 Q tile as TMA delivers it ([D/64 panels][128 rows][64 d]), later the epilogue
+    // staging double[128 rows][32 columns] with the column index ^ (row & 31)
+    unsigned char qraw_or_stage[128 * D * 2 > 128 * 32 * 8 ? 128 * D * 2 : 128 * 32 * 8];
+    uint64_t q_full, q_sliced, k_full[kScoreTcRing], k_empty[kScoreTcRing], acc_full, acc_free;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+// grid (query tiles of the chunk, column-tile groups).  logits: the chunk's score buffer,
+// logits[(tile_in_chunk*128 + r) * N_ld + j] = scale * <q_row, kbar_j>.
+template <int D>
+__global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
+    Geom g, int gt0, int cols_per_cta, const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+    const int32_t* __restrict__ key_exp, double* __restrict__ logits, int32_t* __restrict__ status) {
+    extern __shared__ unsigned char score_tc_raw[];
+    ScoreTcSmem<D>& sm = *reinterpret_cast<ScoreTcSmem<D>*>((reinterpret_cast<uintptr_t>(score_tc_raw) + 1023) & ~(uintptr_t)1023);
+    constexpr int kPanels = D / 64;
+    constexpr int kBlocks = 4 * kPanels;                          // key digit blocks per column tile
+    constexpr uint32_t kIdesc = tc::make_idesc_bf16(128, 128);
+    constexpr uint32_t kBlockBytes = 128 * 64 * 2;
+
+    const int gt = gt0 + blockIdx.x;
+    int tile, bh, h, b;
+    g.div_n_tiles.divmod(gt, bh, tile);
+    g.div_Hq.divmod(bh, b, h);
+    const int gk = h / g.G;
+    const int last_pos = min(tile * kTileRows + kTileRows, g.S) - 1;
+    const int n_ct = (n_candidates(g, last_pos) + kScoreTcCols - 1) / kScoreTcCols;
+    const int ct0 = blockIdx.y * cols_per_cta, ct1 = min(ct0 + cols_per_cta, n_ct);
+    if (ct0 >= ct1) return;                                       // no candidate cube in this column group
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) {
+        tc::mbar_init(&sm.q_full, 1);
+        tc::mbar_init(&sm.q_sliced, 128);
+        for (int i = 0; i < kScoreTcRing; ++i) {
+            tc::mbar_init(&sm.k_full[i], 1);
+            tc::mbar_init(&sm.k_empty[i], 1);
+        }
+        tc::mbar_init(&sm.acc_full, 1);
+        tc::mbar_init(&sm.acc_free, 128);
+        sm.abort_flag = 0;
+        tc::fence_barrier_init();
+    }
+    if (warp == 4) {
+        tc::tmem_alloc<512>(&sm.tmem_base);
+        if (lane == 0) {
+            tc::prefetch_tensormap(&tmQ);
+            tc::prefetch_tensormap(&tmK);
+        }
+    }
+    tc::tc_fence_before_sync();
+    __syncthreads();
+    tc::tc_fence_after_sync();
+    const uint32_t tbase = sm.tmem_base;
+    volatile int* abort_flag = &sm.abort_flag;
+
+    if (warp == 4) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            const int q_row0 = (b * g.Hq + h) * g.S_cap + tile * kTileRows;
+            tc::mbar_arrive_expect_tx(&sm.q_full, 128 * D * 2);
+            for (int p = 0; p < kPanels; ++p) tc::tma_load_2d(sm.qraw_or_stage + p * (128 * 128), &tmQ, p * 64, q_row0, &sm.q_full);
+            const int n_rows = g.B * g.Hkv * g.N_ld;
+            const int k_row0 = (b * g.Hkv + gk) * g.N_ld;
+            int i = 0;
+            for (int ct = ct0; ct < ct1; ++ct) {
+                for (int blk = 0; blk < kBlocks; ++blk, ++i) {
+                    const int p = blk >> 2, plane = blk & 3, s = i % kScoreTcRing, u = i / kScoreTcRing;
+                    if (!tc::mbar_wait(&sm.k_empty[s], (u & 1) ^ 1, abort_flag)) { ct = ct1; break; }
+                    tc::mbar_arrive_expect_tx(&sm.k_full[s], kBlockBytes);
+                    tc::tma_load_2d(&sm.kring[s][0][0], &tmK, p * 64, plane * n_rows + k_row0 + ct * kScoreTcCols, &sm.k_full[s]);
+                }
+            }
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t kPlaneStep = (uint32_t)sizeof(sm.qd[0]) >> 4, kPanelStep = (128 * 64 * 2) >> 4;
+            constexpr uint32_t kRingStep = (uint32_t)sizeof(sm.kring[0]) >> 4, kKStep = 32 >> 4;
+            const uint32_t q_lo0 = tc::smem_desc_lo_sw128(smem_u32(&sm.qd[0][0][0][0]));
+            const uint32_t k_lo0 = tc::smem_desc_lo_sw128(smem_u32(&sm.kring[0][0][0]));
+            bool ok = tc::mbar_wait(&sm.q_sliced, 0, abort_flag);
+            int i = 0;
+            for (int ct = ct0, t = 0; ok && ct < ct1; ++ct, ++t) {
+                if (t > 0 && !(ok = tc::mbar_wait(&sm.acc_free, (t - 1) & 1, abort_flag))) break;
+                tc::tc_fence_after_sync();
+                for (int blk = 0; blk < kBlocks; ++blk, ++i) {
+                    const int p = blk >> 2, plane = blk & 3, s = i % kScoreTcRing, u = i / kScoreTcRing;
+                    if (!(ok = tc::mbar_wait(&sm.k_full[s], u & 1, abort_flag))) break;
+                    tc::tc_fence_after_sync();
+                    const uint32_t kb = k_lo0 + s * kRingStep;
+                    for (int a = 0; a + plane <= 3; ++a) {        // level a + plane
+                        const uint32_t qa = q_lo0 + a * kPlaneStep + p * kPanelStep;
+                        const uint32_t dst = tbase + (a + plane) * 128;
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks)
+                            tc::umma_ss(dst, tc::smem_desc_from_halves(qa + ks * kKStep, tc::kSmemDescHiSw128),
+                                        tc::smem_desc_from_halves(kb + ks * kKStep, tc::kSmemDescHiSw128), kIdesc,
+                                        !(blk == 0 && ks == 0));
+                    }
+                    tc::umma_commit(&sm.k_empty[s]);
+                }
+                if (ok) tc::umma_commit(&sm.acc_full);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ slicing, then epilogue (thread = row)
+        const int r = tid;                                        // row of the tile = TMEM lane
+        bool ok = tc::mbar_wait(&sm.q_full, 0, abort_flag);
+        int e_q = 0;
+        if (ok) {
+            const unsigned char* raw = sm.qraw_or_stage;
+            uint32_t mxbits = 0;
+#pragma unroll
+            for (int c = 0; c < D / 8; ++c) {
+                const uint4 v = *reinterpret_cast<const uint4*>(raw + (c >> 3) * (128 * 128) + sw128(r, c & 7));
+                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) mxbits = max(mxbits, max(w[i] & 0x7fffu, (w[i] >> 16) & 0x7fffu));
+            }
+            const int ef = (int)(mxbits >> 7);
+            e_q = ef == 0 ? 0 : max(ef - 127, -90);
+            unsigned char* dst = reinterpret_cast<unsigned char*>(&sm.qd[0][0][0][0]);
+#pragma unroll 2
+            for (int c = 0; c < D / 8; ++c) {
+                const int off = (c >> 3) * (128 * 128) + sw128(r, c & 7);
+                const uint4 v = *reinterpret_cast<const uint4*>(raw + off);
+                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+                uint32_t out[4][4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    int lo[4], hi[4];
+                    digits256(fixed30(__uint_as_float(w[i] << 16), e_q), lo);
+                    digits256(fixed30(__uint_as_float(w[i] & 0xffff0000u), e_q), hi);
+#pragma unroll
+                    for (int pl = 0; pl < 4; ++pl) out[pl][i] = bf16_bits_of_int(lo[pl]) | (bf16_bits_of_int(hi[pl]) << 16);
+                }
+#pragma unroll
+                for (int pl = 0; pl < 4; ++pl)
+                    *reinterpret_cast<uint4*>(dst + (size_t)pl * sizeof(sm.qd[0]) + off) = make_uint4(out[pl][0], out[pl][1], out[pl][2], out[pl][3]);
+            }
+            asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");   // digit planes visible to the tensor core
+            tc::mbar_arrive(&sm.q_sliced);
+        }
+        const double rowf = __hiloint2double((1023 + e_q) << 20, 0);          // 2^e_q
+        double (*stage)[32] = reinterpret_cast<double (*)[32]>(sm.qraw_or_stage);
+        const int32_t* kexp = key_exp + (size_t)(b * g.Hkv + gk) * g.N_ld;
+        const uint32_t lane_addr = tbase + ((uint32_t)(warp * 32) << 16);
+        double* out_rows = logits + (size_t)blockIdx.x * kTileRows * g.N_ld;
+        for (int ct = ct0, t = 0; ok && ct < ct1; ++ct, ++t) {
+            if (!(ok = tc::mbar_wait(&sm.acc_full, t & 1, abort_flag))) break;
+            tc::tc_fence_after_sync();
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+                const int col0 = ct * kScoreTcCols + c * 32;
+                uint32_t lv[4][32];
+#pragma unroll
+                for (int L = 0; L < 4; ++L) tc::tmem_ld_32x32(lane_addr + L * 128 + c * 32, lv[L]);
+                tc::tmem_wait_ld();
+                if (c == 3) {                                     // last read of the accumulators: release them
+                    tc::tc_fence_before_sync();
+                    tc::mbar_arrive(&sm.acc_free);
+                }
+                // column factor 2^(e_k - 36) * scale, held by the lane that owns the column
+                const int jc = col0 + lane;
+                const int ek = jc < g.N_ld ? kexp[jc] : 0;
+                const double colf = __hiloint2double((1023 + ek - 36) << 20, 0) * g.scale_d;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const double v = fma((double)__uint_as_float(lv[0][i]), 16777216.0,
+                                         fma((double)__uint_as_float(lv[1][i]), 65536.0,
+                                             fma((double)__uint_as_float(lv[2][i]), 256.0, (double)__uint_as_float(lv[3][i]))));
+                    const double cf = __shfl_sync(0xffffffffu, colf, i);
+                    stage[r][i ^ (r & 31)] = (v * rowf) * cf;
+                }
+                __syncwarp();
+                if (col0 + lane < g.N_ld) {
+                    for (int rr = 0; rr < 32; ++rr) {
+                        const int row = warp * 32 + rr;
+                        out_rows[(size_t)row * g.N_ld + col0 + lane] = stage[row][lane ^ (row & 31)];
+                    }
+                }
+                __syncwarp();
+            }
+        }
+    }
+    // ---------------------------------------------------------------- teardown
+    tc::tc_fence_before_sync();
+    __syncthreads();
+    if (tid == 0 && sm.abort_flag) atomicExch(status, 6);
+    if (warp == 4) tc::tmem_dealloc<512>(tbase);
+}
+
+}  // namespace adaspark
