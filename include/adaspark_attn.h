@@ -199,8 +199,10 @@ int64_t adaspark_attn_last_launch_count(const adaspark_attn_t *handle);
 adaspark_status_t adaspark_attn_enable_stage_timing(adaspark_attn_t *handle, int32_t enable);
 adaspark_status_t adaspark_attn_get_stage_times(adaspark_attn_t *handle, float *ms_out /* host [4] */);
 
-/* Selects the prefill attention kernel: 0 = mma.sync (legacy tensor path), 1 = tcgen05/TMEM
- * with TMA-staged tiles.  Default 1 when built in. ERR_UNSUPPORTED for an unknown value. */
+/* Selects the prefill kernels: 0 = mma.sync attention + fp64 (mma.m8n8k4.f64) scoring, the legacy
+ * tensor path kept as a cross-check; 1 = tcgen05/TMEM attention with TMA-staged tiles + tcgen05
+ * scoring from error-free digit slices (default when built in); 2 = tcgen05 attention + fp64
+ * scoring.  ERR_UNSUPPORTED for an unknown value. */
 adaspark_status_t adaspark_attn_set_prefill_kernel(adaspark_attn_t *handle, int32_t which);
 
 #ifdef __cplusplus

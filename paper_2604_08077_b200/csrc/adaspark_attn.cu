@@ -6,6 +6,7 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -51,7 +52,10 @@ struct adaspark_attn {
 namespace {
 
 constexpr size_t kAlign = 256;
-constexpr size_t kLogitsBudget = 40ull << 20;   // per buffer; two buffers stay inside the 126 MB L2
+// Per score buffer (there are two).  Large buffers mean few, many-wave launches of the scoring and
+// selection kernels: measured faster than L2-sized chunks whose launches are latency-bound, although
+// the scores then travel through HBM (config 4: 117 ms at 40 MB, 78 ms at 640 MB).
+constexpr size_t kLogitsBudget = 512ull << 20;
 size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 
 adaspark_status_t fail(adaspark_attn* h, adaspark_status_t st, const char* fmt, ...) {
@@ -187,7 +191,12 @@ adaspark_status_t adaspark_attn_partition(adaspark_attn_t* h, int32_t batch, int
     h->fw_mask_off = off; off = align_up(off + (size_t)batch * Hq * n_tiles_cap * n_words * kTileRows * 4);
     size_t total_tiles = (size_t)batch * Hq * n_tiles_cap;
     size_t tile_bytes = (size_t)kTileRows * N_ld * 8;
-    size_t chunk = kLogitsBudget / tile_bytes;
+    size_t budget = kLogitsBudget;
+    if (const char* env = std::getenv("ADASPARK_SCORE_BUFFER_MB")) {   // tuning knob: size of each of the two score buffers
+        long mb = std::atol(env);
+        if (mb >= 1 && mb <= 65536) budget = (size_t)mb << 20;
+    }
+    size_t chunk = budget / tile_bytes;
     if (chunk < 1) chunk = 1;
     if (chunk > total_tiles) chunk = total_tiles;
     if (chunk > 148) chunk = chunk / 148 * 148;    // whole waves of one-CTA-per-SM scoring tiles
@@ -278,7 +287,7 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
         }
     }
 #ifdef ADASPARK_WITH_TCGEN05
-    if (!cache_only && h->prefill_kernel == 1) {   // cube-major staging of Q for the TMA loads of K4
+    if (!cache_only && h->prefill_kernel != 0) {   // cube-major staging of Q for the TMA loads of K3 / K4
         dim3 rgrid((g.S + 31) / 32, g.B);
         __nv_bfloat16* q_cube = (__nv_bfloat16*)((char*)workspace + h->fw_qcube_off);
         if (D == 128) relayout_q_kernel<128><<<rgrid, 256, 0, st>>>(g, (const __nv_bfloat16*)q, q_cube);
@@ -373,7 +382,7 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
     mark(h, 2, st);
     // K4: gathered attention
 #ifdef ADASPARK_WITH_TCGEN05
-    if (h->prefill_kernel == 1) {
+    if (h->prefill_kernel != 0) {
         __nv_bfloat16* q_cube = (__nv_bfloat16*)(ws + h->fw_qcube_off);
         CUtensorMap tmQ, tmK, tmV;
         if (!encode_bf16_2d(&tmQ, q_cube, (uint64_t)g.B * g.Hq * g.S_cap, D, 64, 128) ||
@@ -532,7 +541,7 @@ int64_t adaspark_attn_last_launch_count(const adaspark_attn_t* h) { return h ? h
 adaspark_status_t adaspark_attn_set_prefill_kernel(adaspark_attn_t* h, int32_t which) {
     if (!h) return ADASPARK_ERR_INVALID_ARG;
 #ifdef ADASPARK_WITH_TCGEN05
-    if (which != 0 && which != 1) return fail(h, ADASPARK_ERR_UNSUPPORTED, "set_prefill_kernel: unknown kernel %d", which);
+    if (which < 0 || which > 2) return fail(h, ADASPARK_ERR_UNSUPPORTED, "set_prefill_kernel: unknown kernel %d", which);
 #else
     if (which != 0) return fail(h, ADASPARK_ERR_UNSUPPORTED, "set_prefill_kernel: kernel %d not built", which);
 #endif

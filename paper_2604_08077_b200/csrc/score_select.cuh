@@ -104,19 +104,22 @@ __global__ void __launch_bounds__(256) score_kernel(Geom g, int gt0,
 }
 
 // G lanes per query row of the chunk, 32/G rows per warp.  Writes the per-tile mask matrix (always)
-// and the optional raster-ordered bitmap / count outputs.
-// dynamic smem per warp: kSelHistWords + (32/G) * (N_ld keys + cand_cap candidates) words of 8 bytes.
+// and the optional raster-ordered bitmap / count outputs.  Short rows (G < 32) keep their order keys
+// in shared memory; long rows (G = 32) overwrite their scores in the L2-resident score buffer with
+// the keys, so that shared memory per warp stays small and many warps hide the latency of the passes.
+// dynamic smem per warp: kSelHistWords + (32/G) * (keys in smem ? N_ld : 0 + cand_cap) words of 8 bytes.
 constexpr int kSelectWarps = 4;
 __host__ __device__ inline int select_lanes_per_row(int N_ld) { return N_ld <= 128 ? 8 : (N_ld <= 512 ? 16 : 32); }
-__host__ __device__ inline int select_cand_cap(int N_ld) { return N_ld <= 256 ? 64 : (N_ld <= 1024 ? 128 : 256); }
+__host__ __device__ inline int select_cand_cap(int N_ld) { return N_ld <= 256 ? 64 : (N_ld <= 512 ? 128 : (N_ld <= 1024 ? 256 : 512)); }
 __host__ __device__ inline size_t select_smem_bytes(int N_ld) {
     const int rows = 32 / select_lanes_per_row(N_ld);
-    return (size_t)kSelectWarps * ((size_t)kSelHistWords + (size_t)rows * (N_ld + select_cand_cap(N_ld))) * 8;
+    const int lanes = select_lanes_per_row(N_ld);
+    return (size_t)kSelectWarps * ((size_t)kSelHistWords + (size_t)rows * ((lanes < 32 ? N_ld : 0) + select_cand_cap(N_ld))) * 8;
 }
 
 template <int G>
 __global__ void __launch_bounds__(kSelectWarps * 32) select_kernel(Geom g, int gt0, int n_gt,
-                                                                   const double* __restrict__ logits,
+                                                                   double* logits,
                                                                    uint32_t* __restrict__ tile_mask,
                                                                    uint32_t* __restrict__ sel_bitmap,
                                                                    int32_t* __restrict__ sel_count) {
@@ -127,10 +130,11 @@ __global__ void __launch_bounds__(kSelectWarps * 32) select_kernel(Geom g, int g
     const int row0 = (blockIdx.x * kSelectWarps + warp) * kRows;      // first row of the warp within the chunk
     if (row0 >= n_gt * kTileRows) return;
     const int cand_cap = select_cand_cap(g.N_ld);
-    const size_t per_warp = (size_t)kSelHistWords + (size_t)kRows * (g.N_ld + cand_cap);
+    constexpr bool kInPlace = (G == 32);
+    const int key_words = kInPlace ? 0 : g.N_ld;
+    const size_t per_warp = (size_t)kSelHistWords + (size_t)kRows * (key_words + cand_cap);
     unsigned long long* hist = sel_smem + (size_t)warp * per_warp;
-    unsigned long long* keys = hist + kSelHistWords + (size_t)gi * g.N_ld;
-    unsigned long long* cand = hist + kSelHistWords + (size_t)kRows * g.N_ld + (size_t)gi * cand_cap;
+    unsigned long long* cand = hist + kSelHistWords + (size_t)kRows * key_words + (size_t)gi * cand_cap;
 
     // the rows of a warp lie in one query tile (kRows divides 128)
     const int gt = gt0 + row0 / kTileRows, r = row0 % kTileRows + gi;
@@ -138,12 +142,13 @@ __global__ void __launch_bounds__(kSelectWarps * 32) select_kernel(Geom g, int g
     g.div_n_tiles.divmod(gt, bh, tile);
     g.div_Hq.divmod(bh, b, h);
     const int pos = tile * kTileRows + r;
-    const double* s = logits + (size_t)(row0 + gi) * g.N_ld;
+    double* s = logits + (size_t)(row0 + gi) * g.N_ld;
+    unsigned long long* keys = kInPlace ? reinterpret_cast<unsigned long long*>(s) : hist + kSelHistWords + (size_t)gi * g.N_ld;
 
     const int n = pos < g.S ? n_candidates(g, pos) : 0;
     const bool all = !(g.top_p < 1.0);
     unsigned long long bd = 0ull;                    // 0: every candidate is selected
-    if (!all) bd = nucleus_boundary_radix<G>(s, n, g.top_p, keys, hist, cand, cand_cap, lane);
+    if (!all) bd = nucleus_boundary_radix<G, kInPlace>(s, n, g.top_p, keys, hist, cand, cand_cap, lane);
 
     const bool extra = (sel_bitmap != nullptr || sel_count != nullptr) && pos < g.S;
     const int raster = extra ? pos_to_raster(g, pos) : 0;

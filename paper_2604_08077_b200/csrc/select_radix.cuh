@@ -233,30 +233,58 @@ __device__ unsigned long long radix_boundary(const unsigned long long* keys, int
 // first-level histogram and returns the boundary key: cube j is selected iff keys[j] >= boundary.
 // A group with n = 0 (no candidates, or nothing to search) returns 0.  Requires p < 1.
 // hist: kSelHistWords entries shared by the warp (zeroed here); keys / cand: the group's own.
-template <int G>
+// keys may be the score row itself (kInPlace: every score is replaced by its key, e.g. a row of the
+// L2-resident score buffer) or separate storage (shared memory for short rows).
+template <int G, bool kInPlace>
 __device__ unsigned long long nucleus_boundary_radix(const double* s, int n, double top_p,
                                                      unsigned long long* keys, unsigned long long* hist,
                                                      unsigned long long* cand, int cand_cap, int lane) {
     const int gl = lane & (G - 1);
     zero_hist(hist, lane);
     double* sd = reinterpret_cast<double*>(keys);
-    double mx = -INFINITY;
-    for (int j = gl; j < n; j += G) {
-        const double v = s[j];
-        sd[j] = v;
-        mx = fmax(mx, v);
+    double mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+    int j = gl;
+    for (; j + 3 * G < n; j += 4 * G) {                 // four independent loads in flight per lane
+        const double v0 = s[j], v1 = s[j + G], v2 = s[j + 2 * G], v3 = s[j + 3 * G];
+        if (!kInPlace) { sd[j] = v0; sd[j + G] = v1; sd[j + 2 * G] = v2; sd[j + 3 * G] = v3; }
+        mx0 = fmax(mx0, v0); mx1 = fmax(mx1, v1); mx2 = fmax(mx2, v2); mx3 = fmax(mx3, v3);
     }
+    for (; j < n; j += G) {
+        const double v = s[j];
+        if (!kInPlace) sd[j] = v;
+        mx0 = fmax(mx0, v);
+    }
+    double mx = fmax(fmax(mx0, mx1), fmax(mx2, mx3));
 #pragma unroll
     for (int o = G / 2; o > 0; o >>= 1) mx = fmax(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     unsigned long long z = 0ull;
-    for (int j = gl; j < n; j += G) {
-        const double e = exp(sd[j] - mx);
+    // mass, order key and first-level bucket of one candidate
+    auto make_key = [&](double v, int jj, unsigned long long& m, int& b) -> unsigned long long {
+        const double e = exp(v - mx);
         const double r = fma(e, 0x1p50, 0x1p52);                       // integer part of e * 2^50, rounded to nearest
-        const unsigned long long m = (unsigned long long)__double_as_longlong(r) & 0xFFFFFFFFFFFFFull;
+        m = (unsigned long long)__double_as_longlong(r) & 0xFFFFFFFFFFFFFull;
         const int top_bits = __double2hiint(r - 0x1p52) >> 19;        // (exponent << 1) | top mantissa bit of (double)m
-        int b = 2147 - top_bits;                                      // m = 2^50 -> 1, each half octave below -> +1
+        b = 2147 - top_bits;                                          // m = 2^50 -> 1, each half octave below -> +1
         b = b > 31 ? 31 : b;
-        keys[j] = (m << 13) | (unsigned long long)(4096 - j);
+        return (m << 13) | (unsigned long long)(4096 - jj);
+    };
+    j = gl;
+    for (; j + 3 * G < n; j += 4 * G) {                 // four exponentials interleaved, then the four updates
+        unsigned long long m[4], k[4];
+        int b[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) k[u] = make_key(sd[j + u * G], j + u * G, m[u], b[u]);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            keys[j + u * G] = k[u];
+            hist[hist_index<G>(b[u], lane)] += m[u];
+            z += m[u];
+        }
+    }
+    for (; j < n; j += G) {
+        unsigned long long m;
+        int b;
+        keys[j] = make_key(sd[j], j, m, b);
         hist[hist_index<G>(b, lane)] += m;
         z += m;
     }
