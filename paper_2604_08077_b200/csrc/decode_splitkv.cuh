@@ -3,7 +3,7 @@
 // HBM-bound: every listed block (K 64xD + V^T Dx64, bf16, 32 KB at D=128) is read once for all
 // heads of the GQA group.  One CTA = one split of one (batch, kv head):
 //   warp 4      TMA producer: per block two K panels + one V^T tile (128-byte swizzle) into a
-//               4-stage shared-memory ring, completion on mbarriers
+//               3-stage shared-memory ring, completion on mbarriers
 //   warps 0-3   each owns 16 of the 64 keys of every block: S = Q K^T and O += P V with
 //               mma.sync m16n8k16 (the 16 rows are the group's heads, at most 16), its own
 //               online softmax state; the four states are merged once at the end.
@@ -16,7 +16,9 @@
 namespace adaspark {
 
 constexpr int kDecodeThreads = 160;
-constexpr int kDecodeStages = 4;
+// 3 stages of 32 KB (D = 128): two CTAs fit one SM and overlap each other's set-up and merge phases;
+// measured 6.85 TB/s against 5.1 TB/s with 4 stages and one CTA per SM.
+constexpr int kDecodeStages = 3;
 
 template <int D>
 struct DecodeSmem {
@@ -187,6 +189,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_splitkv_kernel(
     __syncthreads();   // every stage consumed (or the waits gave up): the ring can be reused
 
     // ---- merge the four warps' (m, l, o) through shared memory, then write the CTA partial
+    static_assert(sizeof(sm.k) >= 4 * 16 * kRowF * sizeof(float), "merge buffer must fit the K ring");
     float* red = reinterpret_cast<float*>(&sm.k[0][0][0][0]);   // [4 warps][16 rows][kRowF]
     if (warp < 4) {
         lA += __shfl_xor_sync(0xffffffffu, lA, 1);
