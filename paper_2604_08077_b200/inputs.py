@@ -82,9 +82,9 @@ def _randn(g: torch.Generator, *shape: int, std: float = 1.0) -> torch.Tensor:
 
 def _add_cube_offsets(k_video: torch.Tensor, g: torch.Generator, T: int, H: int, W: int,
                       cube: Tuple[int, int, int], std: float) -> None:
-    """In place: add one N(0, std^2 I) vector per (cube window, kv head) to the video keys.
+    """In place: add one N(0, std^2 I) vector per (cube window, head) to video keys or queries.
 
-    ``k_video`` is ``[B, T*H*W, Hkv, D]`` in raster order.
+    ``k_video`` is ``[B, T*H*W, heads, D]`` in raster order.
     """
     ct, ch, cw = cube
     B, _, Hkv, D = k_video.shape
@@ -96,8 +96,13 @@ def _add_cube_offsets(k_video: torch.Tensor, g: torch.Generator, T: int, H: int,
 def make_prefill(name: str, *, seed: int, B: int, T: int, H: int, W: int,
                  cube: Tuple[int, int, int], n_text: int, Hq: int, Hkv: int, D: int,
                  top_p: float, offset_std: float, with_q: bool = True,
-                 device: str = "cpu") -> Workload:
-    """i.i.d. N(0,1) Q/K/V; video K gets a per-cube shared offset of std ``offset_std``."""
+                 device: str = "cpu", q_offset_std: float = 0.0, q_noise_std: float = 1.0) -> Workload:
+    """i.i.d. N(0,1) Q/K/V; video K gets a per-cube shared offset of std ``offset_std``.
+
+    ``q_offset_std`` > 0 additionally gives the video queries of one cube a shared offset (per query
+    head) on top of their own N(0, q_noise_std^2) part: queries of a cube then score the cubes alike
+    and select overlapping sets, the cohesion inside a spatio-temporal cube that the paper's
+    partition assumes (Sec. 3.1).  Text queries stay N(0,1)."""
     g = _gen(seed, device)
     S_v = T * H * W
     S = S_v + n_text
@@ -105,10 +110,17 @@ def make_prefill(name: str, *, seed: int, B: int, T: int, H: int, W: int,
     v = _randn(g, B, S, Hkv, D)
     if offset_std > 0:
         _add_cube_offsets(k[:, :S_v], g, T, H, W, cube, offset_std)
-    q = _randn(g, B, S, Hq, D).to(torch.bfloat16) if with_q else None
+    q = None
+    if with_q:
+        q = _randn(g, B, S, Hq, D)
+        if q_offset_std > 0:
+            if q_noise_std != 1.0:
+                q[:, :S_v].mul_(q_noise_std)
+            _add_cube_offsets(q[:, :S_v], g, T, H, W, cube, q_offset_std)
+        q = q.to(torch.bfloat16)
     return Workload(name=name, B=B, T=T, H=H, W=W, cube=cube, n_text=n_text, Hq=Hq, Hkv=Hkv,
                     D=D, top_p=top_p, q=q, k=k.to(torch.bfloat16), v=v.to(torch.bfloat16),
-                    meta={"seed": seed, "offset_std": offset_std})
+                    meta={"seed": seed, "offset_std": offset_std, "q_offset_std": q_offset_std})
 
 
 def _static_dynamic_kv(g: torch.Generator, B: int, T: int, H: int, W: int,
@@ -177,6 +189,19 @@ def config2(variant: int = 0, top_p: float = 0.9, device: str = "cpu") -> Worklo
     return make_prefill("cfg2_qwen7b_16k", seed=2000 + variant, B=1, T=64, H=16, W=16,
                         cube=(4, 4, 4), n_text=128, Hq=28, Hkv=4, D=128, top_p=top_p,
                         offset_std=1.5, device=device)
+
+
+def config2_cohesive(variant: int = 0, top_p: float = 0.9, q_offset_std: float = 1.0,
+                     q_noise_std: float = 0.25, cube: Tuple[int, int, int] = (4, 4, 4),
+                     device: str = "cpu") -> Workload:
+    """Config-2 shapes with cohesive queries: the video queries of a cube share an offset of std
+    ``q_offset_std`` per query head and an own part of std ``q_noise_std``, so the rows of a query
+    tile select overlapping cube sets and the tile's union of selected blocks is far smaller than the
+    whole prefix."""
+    return make_prefill("cfg2_cohesive_q", seed=2500 + variant, B=1, T=64, H=16, W=16,
+                        cube=cube, n_text=128, Hq=28, Hkv=4, D=128, top_p=top_p,
+                        offset_std=1.5, device=device, q_offset_std=q_offset_std,
+                        q_noise_std=q_noise_std)
 
 
 def config3(sigma: float = 1.5, top_p: float = 0.9, device: str = "cpu") -> Workload:

@@ -57,6 +57,23 @@ def test_config3_full_size_sampled_rows(sigma, p):
     _free()
 
 
+def test_cohesive_queries_256_token_cubes():
+    """Config-2 shapes with the paper's default cube size (4x8x8 = 256 tokens), p = 0.7 and queries
+    that share an offset inside a cube: the attention kernel then skips most key blocks (the union
+    of a tile's selections is sparse), which the dense-union benchmark configs never exercise."""
+    wl = inputs.config2_cohesive(top_p=0.7, cube=(4, 8, 8))
+    eng, out, bitmap, count = pu.run_forward(wl)
+    n_tiles = (wl.S + 127) // 128
+    rows = pu.sample_rows(wl, 1500, seed=6, whole_tiles=[(0, 3, 1), (0, 17, n_tiles // 2), (0, 27, n_tiles - 1)])
+    rep = pu.compare_rows(wl, rows, out, bitmap, count, label="cohesive")
+    hdr = eng.header()
+    dense_blocks = sum(2 * ((min(p * 256 + 256, wl.S) + 63) // 64) for p in range((wl.S + 255) // 256)) * wl.Hq
+    print("cohesive", rep, "executed/dense blocks", hdr.executed_kv_blocks / dense_blocks)
+    assert hdr.status == 0 and hdr.executed_kv_blocks < 0.8 * dense_blocks
+    del eng, out, bitmap, count
+    _free()
+
+
 def test_config4_full_size_sampled_rows():
     """Config 4 (131072 video tokens in 2048 cubes, half of the frames static, no text)."""
     wl = inputs.config4()
