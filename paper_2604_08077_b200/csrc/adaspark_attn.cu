@@ -320,18 +320,20 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
                 if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_select[i], cudaEventDisableTiming);
             }
             if (e != cudaSuccess) return fail(h, ADASPARK_ERR_CUDA, "forward: side stream set-up: %s", cudaGetErrorString(e));
+            int sms = 0;
+            if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->cfg.device) != cudaSuccess || sms <= 0) sms = 148;
+            h->sm_count = sms;
             h->side_ready = true;
         }
 #ifdef ADASPARK_WITH_TCGEN05
-        CUtensorMap tmQs, tmKs;
+        CUtensorMap tmKs;
         int32_t* key_exp = (int32_t*)(ws + h->fw_kexp_off);
         if (h->prefill_kernel == 1) {   // digit planes of the mean keys, tensor maps of the scoring kernel
             __nv_bfloat16* kplanes = (__nv_bfloat16*)(ws + h->fw_kplanes_off);
             const int n_rows = g.B * g.Hkv * g.N_ld;
             slice_keys_kernel<<<(n_rows + 3) / 4, 128, 0, st>>>(g, cube_keys, kplanes, key_exp);
             if (!launch_ok(h, "slice_keys_kernel")) return ADASPARK_ERR_CUDA;
-            if (!encode_bf16_2d(&tmQs, ws + h->fw_qcube_off, (uint64_t)g.B * g.Hq * g.S_cap, D, 64, 128) ||
-                !encode_bf16_2d(&tmKs, kplanes, (uint64_t)4 * n_rows + 128, D, 64, 128))
+            if (!encode_bf16_2d(&tmKs, kplanes, (uint64_t)4 * n_rows + 128, D, 64, 128))
                 return fail(h, ADASPARK_ERR_CUDA, "forward: cuTensorMapEncodeTiled failed");
             if (D == 128) { if (!set_smem(h, score_tc_kernel<128>, sizeof(ScoreTcSmem<128>) + 1024, "score_tc_kernel")) return ADASPARK_ERR_CUDA; }
             else { if (!set_smem(h, score_tc_kernel<64>, sizeof(ScoreTcSmem<64>) + 1024, "score_tc_kernel")) return ADASPARK_ERR_CUDA; }
@@ -349,16 +351,19 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
 #ifdef ADASPARK_WITH_TCGEN05
             if (h->prefill_kernel == 1) {
                 const int n_ct = (g.N + kScoreTcCols - 1) / kScoreTcCols;
-                int groups = (148 + n_gt - 1) / n_gt;
+                int groups = (h->sm_count + n_gt - 1) / n_gt;      // split the columns when tiles alone cannot fill the SMs
                 if (groups > n_ct) groups = n_ct;
                 const int cols_per_cta = (n_ct + groups - 1) / groups;
-                dim3 tgrid(n_gt, (n_ct + cols_per_cta - 1) / cols_per_cta);
+                groups = (n_ct + cols_per_cta - 1) / cols_per_cta;
+                const int n_items = n_gt * groups;
+                const int tgrid = n_items < h->sm_count ? n_items : h->sm_count;
+                const __nv_bfloat16* q_cube_c = (const __nv_bfloat16*)(ws + h->fw_qcube_off);
                 if (D == 128)
                     score_tc_kernel<128><<<tgrid, kScoreTcThreads, sizeof(ScoreTcSmem<128>) + 1024, st>>>(
-                        g, gt0, cols_per_cta, tmQs, tmKs, key_exp, chunk_logits, &hdr->status);
+                        g, gt0, n_items, groups, cols_per_cta, q_cube_c, tmKs, key_exp, chunk_logits, &hdr->status);
                 else
                     score_tc_kernel<64><<<tgrid, kScoreTcThreads, sizeof(ScoreTcSmem<64>) + 1024, st>>>(
-                        g, gt0, cols_per_cta, tmQs, tmKs, key_exp, chunk_logits, &hdr->status);
+                        g, gt0, n_items, groups, cols_per_cta, q_cube_c, tmKs, key_exp, chunk_logits, &hdr->status);
                 if (!launch_ok(h, "score_tc_kernel")) return ADASPARK_ERR_CUDA;
             } else
 #endif

@@ -16,17 +16,20 @@
 // the margin above.
 //
 //   slice_keys_kernel   digit planes + row exponents of the mean keys (once per forward, tiny)
-//   score_tc_kernel     CTA = one 128-row query tile x a group of 128-cube column tiles:
-//     warps 0-3  slice the Q tile (thread = row) into four swizzled digit planes in shared memory,
-//                later the epilogue: TMEM -> fp64 scores -> coalesced rows of the score buffer
-//     warp 4     TMA producer: Q tile once, then the key digit blocks (plane, 64-d panel) in a ring
-//     warp 5     issues the tcgen05.mma stream (80 per column tile at D = 128)
+//   score_tc_kernel     persistent CTAs, one per SM; work item = one 128-row query tile x a group of
+//                       128-cube column tiles.  Roles (320 threads), pipelined across items:
+//     warps 0-3  epilogue (thread = row = TMEM lane): TMEM -> fp64 scores -> coalesced rows of the
+//                score buffer; overlaps the slicing and the first loads of the next item
+//     warps 4-7  slicers (thread = row): read the bf16 query row, write the four swizzled digit
+//                planes of the tile into shared memory
+//     warp 8     TMA producer: key digit blocks (plane, 64-d panel) in a ring
+//     warp 9     issues the tcgen05.mma stream (80 per column tile at D = 128)
 #pragma once
 #include "tc_common.cuh"
 
 namespace adaspark {
 
-constexpr int kScoreTcThreads = 192;
+constexpr int kScoreTcThreads = 320;
 constexpr int kScoreTcRing = 4;          // key digit blocks (128 cubes x 64 d, 16 KB) in flight
 constexpr int kScoreTcCols = 128;        // cubes per column tile
 
@@ -85,20 +88,40 @@ template <int D>
 struct ScoreTcSmem {
     __nv_bfloat16 qd[4][D / 64][128][64];               // digit planes of the Q tile, UMMA layout (128-B swizzle)
     __nv_bfloat16 kring[kScoreTcRing][128][64];         // key digit blocks: [cube][64 d of one panel of one plane]
-    // first the bf16 Q tile as TMA delivers it ([D/64 panels][128 rows][64 d]), later the epilogue
-    // staging double[128 rows][32 columns] with the column index ^ (row & 31)
-    unsigned char qraw_or_stage[128 * D * 2 > 128 * 32 * 8 ? 128 * D * 2 : 128 * 32 * 8];
-    uint64_t q_full, q_sliced, k_full[kScoreTcRing], k_empty[kScoreTcRing], acc_full, acc_free;
+    double stage[128][32];                              // epilogue: scores of 32 columns, column index ^ (row & 31)
+    int row_exp[2][128];                                // row exponents of the item being sliced / being finished
+    uint64_t q_sliced, qd_free, k_full[kScoreTcRing], k_empty[kScoreTcRing], acc_full, acc_free;
     uint32_t tmem_base;
     int abort_flag;
 };
 
-// grid (query tiles of the chunk, column-tile groups).  logits: the chunk's score buffer,
-// logits[(tile_in_chunk*128 + r) * N_ld + j] = scale * <q_row, kbar_j>.
+// Work item `it` of the launch: query tile gt0 + it / groups, column tiles [ct0, ct1).
+struct ScoreItem {
+    int b, h, gk, tile, ct0, ct1, tile_in_chunk;
+};
+__device__ __forceinline__ ScoreItem score_item(const Geom& g, int gt0, int groups, int cols_per_cta, int it) {
+    ScoreItem w;
+    w.tile_in_chunk = it / groups;
+    const int grp = it - w.tile_in_chunk * groups;
+    int bh;
+    g.div_n_tiles.divmod(gt0 + w.tile_in_chunk, bh, w.tile);
+    g.div_Hq.divmod(bh, w.b, w.h);
+    w.gk = w.h / g.G;
+    const int last_pos = min(w.tile * kTileRows + kTileRows, g.S) - 1;
+    const int n_ct = (n_candidates(g, last_pos) + kScoreTcCols - 1) / kScoreTcCols;
+    w.ct0 = grp * cols_per_cta;
+    w.ct1 = min(w.ct0 + cols_per_cta, n_ct);          // ct0 >= ct1: nothing to do for this item
+    return w;
+}
+
+// grid = min(items, SMs) persistent CTAs.  logits: the chunk's score buffer,
+// logits[(tile_in_chunk*128 + r) * N_ld + j] = scale * <q_row, kbar_j>.  q_cube: cube-major bf16 queries
+// [B*Hq, S_cap, D].
 template <int D>
 __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
-    Geom g, int gt0, int cols_per_cta, const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-    const int32_t* __restrict__ key_exp, double* __restrict__ logits, int32_t* __restrict__ status) {
+    Geom g, int gt0, int n_items, int groups, int cols_per_cta, const __nv_bfloat16* __restrict__ q_cube,
+    const __grid_constant__ CUtensorMap tmK, const int32_t* __restrict__ key_exp, double* __restrict__ logits,
+    int32_t* __restrict__ status) {
     extern __shared__ unsigned char score_tc_raw[];
     ScoreTcSmem<D>& sm = *reinterpret_cast<ScoreTcSmem<D>*>((reinterpret_cast<uintptr_t>(score_tc_raw) + 1023) & ~(uintptr_t)1023);
     constexpr int kPanels = D / 64;
@@ -106,20 +129,10 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
     constexpr uint32_t kIdesc = tc::make_idesc_bf16(128, 128);
     constexpr uint32_t kBlockBytes = 128 * 64 * 2;
 
-    const int gt = gt0 + blockIdx.x;
-    int tile, bh, h, b;
-    g.div_n_tiles.divmod(gt, bh, tile);
-    g.div_Hq.divmod(bh, b, h);
-    const int gk = h / g.G;
-    const int last_pos = min(tile * kTileRows + kTileRows, g.S) - 1;
-    const int n_ct = (n_candidates(g, last_pos) + kScoreTcCols - 1) / kScoreTcCols;
-    const int ct0 = blockIdx.y * cols_per_cta, ct1 = min(ct0 + cols_per_cta, n_ct);
-    if (ct0 >= ct1) return;                                       // no candidate cube in this column group
-
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid == 0) {
-        tc::mbar_init(&sm.q_full, 1);
         tc::mbar_init(&sm.q_sliced, 128);
+        tc::mbar_init(&sm.qd_free, 1);
         for (int i = 0; i < kScoreTcRing; ++i) {
             tc::mbar_init(&sm.k_full[i], 1);
             tc::mbar_init(&sm.k_empty[i], 1);
@@ -129,12 +142,9 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
         sm.abort_flag = 0;
         tc::fence_barrier_init();
     }
-    if (warp == 4) {
+    if (warp == 8) {
         tc::tmem_alloc<512>(&sm.tmem_base);
-        if (lane == 0) {
-            tc::prefetch_tensormap(&tmQ);
-            tc::prefetch_tensormap(&tmK);
-        }
+        if (lane == 0) tc::prefetch_tensormap(&tmK);
     }
     tc::tc_fence_before_sync();
     __syncthreads();
@@ -142,84 +152,98 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
     const uint32_t tbase = sm.tmem_base;
     volatile int* abort_flag = &sm.abort_flag;
 
-    if (warp == 4) {
+    if (warp == 8) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            const int q_row0 = (b * g.Hq + h) * g.S_cap + tile * kTileRows;
-            tc::mbar_arrive_expect_tx(&sm.q_full, 128 * D * 2);
-            for (int p = 0; p < kPanels; ++p) tc::tma_load_2d(sm.qraw_or_stage + p * (128 * 128), &tmQ, p * 64, q_row0, &sm.q_full);
             const int n_rows = g.B * g.Hkv * g.N_ld;
-            const int k_row0 = (b * g.Hkv + gk) * g.N_ld;
-            int i = 0;
-            for (int ct = ct0; ct < ct1; ++ct) {
-                for (int blk = 0; blk < kBlocks; ++blk, ++i) {
-                    const int p = blk >> 2, plane = blk & 3, s = i % kScoreTcRing, u = i / kScoreTcRing;
-                    if (!tc::mbar_wait(&sm.k_empty[s], (u & 1) ^ 1, abort_flag)) { ct = ct1; break; }
-                    tc::mbar_arrive_expect_tx(&sm.k_full[s], kBlockBytes);
-                    tc::tma_load_2d(&sm.kring[s][0][0], &tmK, p * 64, plane * n_rows + k_row0 + ct * kScoreTcCols, &sm.k_full[s]);
+            int i = 0;                                            // running block counter of this CTA
+            bool ok = true;
+            for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
+                const ScoreItem w = score_item(g, gt0, groups, cols_per_cta, it);
+                const int k_row0 = (w.b * g.Hkv + w.gk) * g.N_ld;
+                for (int ct = w.ct0; ok && ct < w.ct1; ++ct) {
+                    for (int blk = 0; blk < kBlocks; ++blk, ++i) {
+                        const int p = blk >> 2, plane = blk & 3, s = i % kScoreTcRing, u = i / kScoreTcRing;
+                        if (!(ok = tc::mbar_wait(&sm.k_empty[s], (u & 1) ^ 1, abort_flag))) break;
+                        tc::mbar_arrive_expect_tx(&sm.k_full[s], kBlockBytes);
+                        tc::tma_load_2d(&sm.kring[s][0][0], &tmK, p * 64, plane * n_rows + k_row0 + ct * kScoreTcCols, &sm.k_full[s]);
+                    }
                 }
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == 9) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             constexpr uint32_t kPlaneStep = (uint32_t)sizeof(sm.qd[0]) >> 4, kPanelStep = (128 * 64 * 2) >> 4;
             constexpr uint32_t kRingStep = (uint32_t)sizeof(sm.kring[0]) >> 4, kKStep = 32 >> 4;
             const uint32_t q_lo0 = tc::smem_desc_lo_sw128(smem_u32(&sm.qd[0][0][0][0]));
             const uint32_t k_lo0 = tc::smem_desc_lo_sw128(smem_u32(&sm.kring[0][0][0]));
-            bool ok = tc::mbar_wait(&sm.q_sliced, 0, abort_flag);
-            int i = 0;
-            for (int ct = ct0, t = 0; ok && ct < ct1; ++ct, ++t) {
-                if (t > 0 && !(ok = tc::mbar_wait(&sm.acc_free, (t - 1) & 1, abort_flag))) break;
-                tc::tc_fence_after_sync();
-                for (int blk = 0; blk < kBlocks; ++blk, ++i) {
-                    const int p = blk >> 2, plane = blk & 3, s = i % kScoreTcRing, u = i / kScoreTcRing;
-                    if (!(ok = tc::mbar_wait(&sm.k_full[s], u & 1, abort_flag))) break;
+            bool ok = true;
+            int i = 0, c = 0, n_done = 0;                         // running block / column-tile / item counters
+            for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
+                const ScoreItem w = score_item(g, gt0, groups, cols_per_cta, it);
+                if (w.ct0 >= w.ct1) continue;
+                if (!(ok = tc::mbar_wait(&sm.q_sliced, n_done & 1, abort_flag))) break;
+                for (int ct = w.ct0; ok && ct < w.ct1; ++ct, ++c) {
+                    if (c > 0 && !(ok = tc::mbar_wait(&sm.acc_free, (c - 1) & 1, abort_flag))) break;
                     tc::tc_fence_after_sync();
-                    const uint32_t kb = k_lo0 + s * kRingStep;
-                    for (int a = 0; a + plane <= 3; ++a) {        // level a + plane
-                        const uint32_t qa = q_lo0 + a * kPlaneStep + p * kPanelStep;
-                        const uint32_t dst = tbase + (a + plane) * 128;
+                    for (int blk = 0; blk < kBlocks; ++blk, ++i) {
+                        const int p = blk >> 2, plane = blk & 3, s = i % kScoreTcRing, u = i / kScoreTcRing;
+                        if (!(ok = tc::mbar_wait(&sm.k_full[s], u & 1, abort_flag))) break;
+                        tc::tc_fence_after_sync();
+                        const uint32_t kb = k_lo0 + s * kRingStep;
+                        for (int a = 0; a + plane <= 3; ++a) {    // level a + plane
+                            const uint32_t qa = q_lo0 + a * kPlaneStep + p * kPanelStep;
+                            const uint32_t dst = tbase + (a + plane) * 128;
 #pragma unroll
-                        for (int ks = 0; ks < 4; ++ks)
-                            tc::umma_ss(dst, tc::smem_desc_from_halves(qa + ks * kKStep, tc::kSmemDescHiSw128),
-                                        tc::smem_desc_from_halves(kb + ks * kKStep, tc::kSmemDescHiSw128), kIdesc,
-                                        !(blk == 0 && ks == 0));
+                            for (int ks = 0; ks < 4; ++ks)
+                                tc::umma_ss(dst, tc::smem_desc_from_halves(qa + ks * kKStep, tc::kSmemDescHiSw128),
+                                            tc::smem_desc_from_halves(kb + ks * kKStep, tc::kSmemDescHiSw128), kIdesc,
+                                            !(blk == 0 && ks == 0));
+                        }
+                        tc::umma_commit(&sm.k_empty[s]);
                     }
-                    tc::umma_commit(&sm.k_empty[s]);
+                    if (ok) tc::umma_commit(&sm.acc_full);
                 }
-                if (ok) tc::umma_commit(&sm.acc_full);
+                if (ok) tc::umma_commit(&sm.qd_free);             // the digit planes may be overwritten
+                ++n_done;
             }
         }
-    } else {
-        // ------------------------------------------------------------ slicing, then epilogue (thread = row)
-        const int r = tid;                                        // row of the tile = TMEM lane
-        bool ok = tc::mbar_wait(&sm.q_full, 0, abort_flag);
-        int e_q = 0;
-        if (ok) {
-            const unsigned char* raw = sm.qraw_or_stage;
+    } else if (warp >= 4) {
+// ------------------------------------------------------------ slicers (thread = row)
+        const int r = tid - 128;
+        bool ok = true;
+        int n_done = 0;
+        for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
+            const ScoreItem w = score_item(g, gt0, groups, cols_per_cta, it);
+            if (w.ct0 >= w.ct1) continue;
+            const int pos = w.tile * kTileRows + r;
+            const uint4* src = reinterpret_cast<const uint4*>(q_cube + ((size_t)(w.b * g.Hq + w.h) * g.S_cap + pos) * D);
+            uint4 v[D / 8];
+#pragma unroll
+            for (int c = 0; c < D / 8; ++c) v[c] = pos < g.S ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
             uint32_t mxbits = 0;
 #pragma unroll
             for (int c = 0; c < D / 8; ++c) {
-                const uint4 v = *reinterpret_cast<const uint4*>(raw + (c >> 3) * (128 * 128) + sw128(r, c & 7));
-                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+                const uint32_t wd[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
 #pragma unroll
-                for (int i = 0; i < 4; ++i) mxbits = max(mxbits, max(w[i] & 0x7fffu, (w[i] >> 16) & 0x7fffu));
+                for (int i = 0; i < 4; ++i) mxbits = max(mxbits, max(wd[i] & 0x7fffu, (wd[i] >> 16) & 0x7fffu));
             }
             const int ef = (int)(mxbits >> 7);
-            e_q = ef == 0 ? 0 : max(ef - 127, -90);
+            const int e_q = ef == 0 ? 0 : max(ef - 127, -90);
+            // the previous item's MMAs must have finished reading the digit planes
+            if (n_done > 0 && !(ok = tc::mbar_wait(&sm.qd_free, (n_done - 1) & 1, abort_flag))) break;
             unsigned char* dst = reinterpret_cast<unsigned char*>(&sm.qd[0][0][0][0]);
-#pragma unroll 2
+#pragma unroll
             for (int c = 0; c < D / 8; ++c) {
                 const int off = (c >> 3) * (128 * 128) + sw128(r, c & 7);
-                const uint4 v = *reinterpret_cast<const uint4*>(raw + off);
-                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+                const uint32_t wd[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
                 uint32_t out[4][4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     int lo[4], hi[4];
-                    digits256(fixed30(__uint_as_float(w[i] << 16), e_q), lo);
-                    digits256(fixed30(__uint_as_float(w[i] & 0xffff0000u), e_q), hi);
+                    digits256(fixed30(__uint_as_float(wd[i] << 16), e_q), lo);
+                    digits256(fixed30(__uint_as_float(wd[i] & 0xffff0000u), e_q), hi);
 #pragma unroll
                     for (int pl = 0; pl < 4; ++pl) out[pl][i] = bf16_bits_of_int(lo[pl]) | (bf16_bits_of_int(hi[pl]) << 16);
                 }
@@ -227,56 +251,72 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
                 for (int pl = 0; pl < 4; ++pl)
                     *reinterpret_cast<uint4*>(dst + (size_t)pl * sizeof(sm.qd[0]) + off) = make_uint4(out[pl][0], out[pl][1], out[pl][2], out[pl][3]);
             }
+            sm.row_exp[n_done & 1][r] = e_q;
             asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");   // digit planes visible to the tensor core
             tc::mbar_arrive(&sm.q_sliced);
+            ++n_done;
         }
-        const double rowf = __hiloint2double((1023 + e_q) << 20, 0);          // 2^e_q
-        double (*stage)[32] = reinterpret_cast<double (*)[32]>(sm.qraw_or_stage);
-        const int32_t* kexp = key_exp + (size_t)(b * g.Hkv + gk) * g.N_ld;
+    } else {
+// ------------------------------------------------------------ epilogue (thread = row = TMEM lane)
+        const int r = tid;
         const uint32_t lane_addr = tbase + ((uint32_t)(warp * 32) << 16);
-        double* out_rows = logits + (size_t)blockIdx.x * kTileRows * g.N_ld;
-        for (int ct = ct0, t = 0; ok && ct < ct1; ++ct, ++t) {
-            if (!(ok = tc::mbar_wait(&sm.acc_full, t & 1, abort_flag))) break;
-            tc::tc_fence_after_sync();
+        bool ok = true;
+        int c_run = 0, n_done = 0;
+        for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
+            const ScoreItem w = score_item(g, gt0, groups, cols_per_cta, it);
+            if (w.ct0 >= w.ct1) continue;
+            if (!(ok = tc::mbar_wait(&sm.q_sliced, n_done & 1, abort_flag))) break;
+            const int e_q = sm.row_exp[n_done & 1][r];
+            const double rowf = __hiloint2double((1023 + e_q) << 20, 0);          // 2^e_q
+            const int32_t* kexp = key_exp + (size_t)(w.b * g.Hkv + w.gk) * g.N_ld;
+            double* out_rows = logits + (size_t)w.tile_in_chunk * kTileRows * g.N_ld;
+            for (int ct = w.ct0; ok && ct < w.ct1; ++ct, ++c_run) {
+                if (!(ok = tc::mbar_wait(&sm.acc_full, c_run & 1, abort_flag))) break;
+                tc::tc_fence_after_sync();
 #pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                const int col0 = ct * kScoreTcCols + c * 32;
-                uint32_t lv[4][32];
+                for (int c = 0; c < 4; ++c) {
+                    const int col0 = ct * kScoreTcCols + c * 32;
+                    uint32_t lv[4][32];
 #pragma unroll
-                for (int L = 0; L < 4; ++L) tc::tmem_ld_32x32(lane_addr + L * 128 + c * 32, lv[L]);
-                tc::tmem_wait_ld();
-                if (c == 3) {                                     // last read of the accumulators: release them
-                    tc::tc_fence_before_sync();
-                    tc::mbar_arrive(&sm.acc_free);
-                }
-                // column factor 2^(e_k - 36) * scale, held by the lane that owns the column
-                const int jc = col0 + lane;
-                const int ek = jc < g.N_ld ? kexp[jc] : 0;
-                const double colf = __hiloint2double((1023 + ek - 36) << 20, 0) * g.scale_d;
-#pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const double v = fma((double)__uint_as_float(lv[0][i]), 16777216.0,
-                                         fma((double)__uint_as_float(lv[1][i]), 65536.0,
-                                             fma((double)__uint_as_float(lv[2][i]), 256.0, (double)__uint_as_float(lv[3][i]))));
-                    const double cf = __shfl_sync(0xffffffffu, colf, i);
-                    stage[r][i ^ (r & 31)] = (v * rowf) * cf;
-                }
-                __syncwarp();
-                if (col0 + lane < g.N_ld) {
-                    for (int rr = 0; rr < 32; ++rr) {
-                        const int row = warp * 32 + rr;
-                        out_rows[(size_t)row * g.N_ld + col0 + lane] = stage[row][lane ^ (row & 31)];
+                    for (int L = 0; L < 4; ++L) tc::tmem_ld_32x32(lane_addr + L * 128 + c * 32, lv[L]);
+                    tc::tmem_wait_ld();
+                    if (c == 3) {                                 // last read of the accumulators: release them
+                        tc::tc_fence_before_sync();
+                        tc::mbar_arrive(&sm.acc_free);
                     }
+                    // column factor 2^(e_k - 36) * scale, held by the lane that owns the column
+                    const int jc = col0 + lane;
+                    const int ek = jc < g.N_ld ? kexp[jc] : 0;
+                    const double colf = __hiloint2double((1023 + ek - 36) << 20, 0) * g.scale_d;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        // exact integer level sums: S0*2^24 + S1*2^16 + S2*2^8 + S3 = hi*2^16 + lo
+                        const int hi = __float2int_rn(__uint_as_float(lv[0][i])) * 256 + __float2int_rn(__uint_as_float(lv[1][i]));
+                        const int lo = __float2int_rn(__uint_as_float(lv[2][i])) * 256 + __float2int_rn(__uint_as_float(lv[3][i]));
+                        const double hd = __hiloint2double(0x43300000, hi ^ 0x80000000) - 4503601774854144.0;   // (double)hi
+                        const double ld = __hiloint2double(0x43300000, lo ^ 0x80000000) - 4503601774854144.0;   // 2^52 + 2^31
+                        const double v = fma(hd, 65536.0, ld);
+                        const double cf = __shfl_sync(0xffffffffu, colf, i);
+                        sm.stage[r][i ^ (r & 31)] = (v * rowf) * cf;
+                    }
+                    __syncwarp();
+                    if (col0 + lane < g.N_ld) {
+                        for (int rr = 0; rr < 32; ++rr) {
+                            const int row = warp * 32 + rr;
+                            out_rows[(size_t)row * g.N_ld + col0 + lane] = sm.stage[row][lane ^ (row & 31)];
+                        }
+                    }
+                    __syncwarp();
                 }
-                __syncwarp();
             }
+            ++n_done;
         }
     }
     // ---------------------------------------------------------------- teardown
     tc::tc_fence_before_sync();
     __syncthreads();
     if (tid == 0 && sm.abort_flag) atomicExch(status, 6);
-    if (warp == 4) tc::tmem_dealloc<512>(tbase);
+    if (warp == 8) tc::tmem_dealloc<512>(tbase);
 }
 
 }  // namespace adaspark
