@@ -333,7 +333,7 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
             const int n_rows = g.B * g.Hkv * g.N_ld;
             slice_keys_kernel<<<(n_rows + 3) / 4, 128, 0, st>>>(g, cube_keys, kplanes, key_exp);
             if (!launch_ok(h, "slice_keys_kernel")) return ADASPARK_ERR_CUDA;
-            if (!encode_bf16_2d(&tmKs, kplanes, (uint64_t)4 * n_rows + 128, D, 64, 128))
+            if (!encode_bf16_2d(&tmKs, kplanes, (uint64_t)4 * n_rows + 128, D, 64, kScoreTcCols))
                 return fail(h, ADASPARK_ERR_CUDA, "forward: cuTensorMapEncodeTiled failed");
             if (D == 128) { if (!set_smem(h, score_tc_kernel<128>, sizeof(ScoreTcSmem<128>) + 1024, "score_tc_kernel")) return ADASPARK_ERR_CUDA; }
             else { if (!set_smem(h, score_tc_kernel<64>, sizeof(ScoreTcSmem<64>) + 1024, "score_tc_kernel")) return ADASPARK_ERR_CUDA; }

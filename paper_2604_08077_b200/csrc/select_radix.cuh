@@ -265,7 +265,7 @@ __device__ unsigned long long nucleus_boundary_radix(const double* s, int n, dou
         m = (unsigned long long)__double_as_longlong(r) & 0xFFFFFFFFFFFFFull;
         const int top_bits = __double2hiint(r - 0x1p52) >> 19;        // (exponent << 1) | top mantissa bit of (double)m
         b = 2147 - top_bits;                                          // m = 2^50 -> 1, each half octave below -> +1
-        b = b > 31 ? 31 : b;
+        b = b > 31 ? 31 : (b < 0 ? 0 : b);                            // (non-finite scores must not index out of range)
         return (m << 13) | (unsigned long long)(4096 - jj);
     };
     j = gl;
