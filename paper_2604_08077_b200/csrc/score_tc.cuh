@@ -105,7 +105,7 @@ struct ScoreTcSmem {
     __nv_bfloat16 qd[4][D / 64][128][64];               // digit planes of the Q tile, UMMA layout (128-B swizzle)
     __nv_bfloat16 kring[kScoreTcRing][kScoreTcCols][64];   // key digit blocks: [cube][64 d of one panel of one plane]
     double stage[128][32];                              // epilogue: scores of 32 columns, column index ^ (row & 31)
-    uint64_t q_sliced, qd_free, k_full[kScoreTcRing], k_empty[kScoreTcRing], acc_full[2], acc_free[2];
+    uint64_t q_sliced, qd_free, k_full[kScoreTcRing], k_group_empty[kScoreTcRing / 4], acc_full[2], acc_free[2];
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -151,8 +151,10 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
         tc::mbar_init(&sm.qd_free, 1);
         for (int i = 0; i < kScoreTcRing; ++i) {
             tc::mbar_init(&sm.k_full[i], 1);
-            tc::mbar_init(&sm.k_empty[i], 1);
         }
+        // a tcgen05.commit costs about two MMA slots: the ring is released four blocks (one panel's
+        // digit planes) at a time
+        for (int i = 0; i < kScoreTcRing / 4; ++i) tc::mbar_init(&sm.k_group_empty[i], 1);
         for (int i = 0; i < 2; ++i) {
             tc::mbar_init(&sm.acc_full[i], 1);
             tc::mbar_init(&sm.acc_free[i], 128);
@@ -182,7 +184,7 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
                 for (int ct = w.ct0; ok && ct < w.ct1; ++ct) {
                     for (int blk = 0; blk < kBlocks; ++blk, ++i) {
                         const int p = blk >> 2, plane = blk & 3, s = i % kScoreTcRing, u = i / kScoreTcRing;
-                        if (!(ok = tc::mbar_wait(&sm.k_empty[s], (u & 1) ^ 1, abort_flag))) break;
+                        if ((blk & 3) == 0 && !(ok = tc::mbar_wait(&sm.k_group_empty[s >> 2], (u & 1) ^ 1, abort_flag))) break;
                         tc::mbar_arrive_expect_tx(&sm.k_full[s], kBlockBytes);
                         tc::tma_load_2d(&sm.kring[s][0][0], &tmK, p * 64, plane * n_rows + k_row0 + ct * kScoreTcCols, &sm.k_full[s]);
                     }
@@ -220,7 +222,7 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
                                             tc::smem_desc_from_halves(kb + ks * kKStep, tc::kSmemDescHiSw128), kIdesc,
                                             !(blk == 0 && ks == 0));
                         }
-                        tc::umma_commit(&sm.k_empty[s]);
+                        if ((blk & 3) == 3) tc::umma_commit(&sm.k_group_empty[s >> 2]);
                     }
                     if (ok) tc::umma_commit(&sm.acc_full[buf]);
                 }
