@@ -23,6 +23,11 @@ adaspark_status_t adaspark_attn_debug_umma_selftest(const void *a, const void *b
                                                     float *d_out, float *e_out, int32_t *status,
                                                     void *cuda_stream);
 
+/* One 128x128x128 product through the int8 tcgen05 path: d_out = A * B^T (int32 [128,128]) with A, B
+ * signed 8-bit row-major [128,128] device buffers (16-byte aligned).  `status` as above. */
+adaspark_status_t adaspark_attn_debug_imma_selftest(const void *a, const void *b, int32_t *d_out,
+                                                    int32_t *status, void *cuda_stream);
+
 /* Host only: n / d computed by the multiply-shift routine the kernels use for their index
  * arithmetic (0 <= n < 2^31, 1 <= d < 2^31); -1 for arguments outside that range. */
 int32_t adaspark_attn_debug_fastdiv(int32_t n, int32_t d);

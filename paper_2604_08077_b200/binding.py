@@ -47,7 +47,8 @@ EXPORTS = ["adaspark_attn_create", "adaspark_attn_partition", "adaspark_attn_get
            "adaspark_attn_last_error", "adaspark_attn_last_launch_count",
            "adaspark_attn_set_prefill_kernel", "adaspark_attn_enable_stage_timing",
            "adaspark_attn_get_stage_times", "adaspark_attn_decode_static",
-           "adaspark_attn_debug_umma_selftest", "adaspark_attn_debug_fastdiv"]
+           "adaspark_attn_debug_umma_selftest", "adaspark_attn_debug_imma_selftest",
+           "adaspark_attn_debug_fastdiv"]
 
 
 def load() -> ctypes.CDLL:
@@ -67,6 +68,7 @@ def load() -> ctypes.CDLL:
     lib.adaspark_attn_decode.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.adaspark_attn_decode_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.adaspark_attn_debug_umma_selftest.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    lib.adaspark_attn_debug_imma_selftest.argtypes = [vp, vp, vp, vp, vp]
     lib.adaspark_attn_debug_fastdiv.argtypes = [ctypes.c_int32, ctypes.c_int32]
     lib.adaspark_attn_debug_fastdiv.restype = ctypes.c_int32
     lib.adaspark_attn_destroy.argtypes = [vp]
@@ -163,6 +165,12 @@ def adaspark_attn_debug_umma_selftest(a, b, c, d_out, e_out, status, stream=None
     """128x128x128 tcgen05 self-test (see include/adaspark_attn_debug.h); returns the status code."""
     return int(load().adaspark_attn_debug_umma_selftest(_ptr(a), _ptr(b), _ptr(c), _ptr(d_out),
                                                        _ptr(e_out), _ptr(status), _stream_ptr(stream)))
+
+
+def adaspark_attn_debug_imma_selftest(a, b, d_out, status, stream=None) -> int:
+    """128x128x128 int8 tcgen05 self-test (see include/adaspark_attn_debug.h); returns the status code."""
+    return int(load().adaspark_attn_debug_imma_selftest(_ptr(a), _ptr(b), _ptr(d_out), _ptr(status),
+                                                       _stream_ptr(stream)))
 
 
 def adaspark_attn_debug_fastdiv(n: int, d: int) -> int:

@@ -609,6 +609,18 @@ extern "C" adaspark_status_t adaspark_attn_decode_static(adaspark_attn_t* h, con
 #include "../../include/adaspark_attn_debug.h"
 #include "umma_selftest.cuh"
 
+extern "C" adaspark_status_t adaspark_attn_debug_imma_selftest(const void* a, const void* b, int32_t* d_out, int32_t* status,
+                                                               void* cuda_stream) {
+    if (!a || !b || !d_out || !status) return ADASPARK_ERR_INVALID_ARG;
+    CUtensorMap tmA, tmB;
+    if (!encode_u8_2d(&tmA, a, 128, 128, 128, 128) || !encode_u8_2d(&tmB, b, 128, 128, 128, 128)) return ADASPARK_ERR_CUDA;
+    const size_t smem = sizeof(ImmaSelftestSmem) + 1024;
+    if (cudaFuncSetAttribute(imma_selftest_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return ADASPARK_ERR_CUDA;
+    imma_selftest_kernel<<<1, 128, smem, (cudaStream_t)cuda_stream>>>(tmA, tmB, d_out, status);
+    return cudaGetLastError() == cudaSuccess ? ADASPARK_OK : ADASPARK_ERR_CUDA;
+}
+
 extern "C" int32_t adaspark_attn_debug_fastdiv(int32_t n, int32_t d) {
     if (n < 0 || d <= 0) return -1;
     FastDiv f;

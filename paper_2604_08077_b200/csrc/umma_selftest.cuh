@@ -116,4 +116,71 @@ __global__ void __launch_bounds__(128) umma_selftest_kernel(const __grid_constan
     if (warp == 0) tc::tmem_dealloc<512>(tbase);
 }
 
+// Self-test of the int8 tensor path: D = A * B^T for int8 A, B [128,128] (row-major, 128 bytes per
+// row, TMA-staged with the 128-byte swizzle), int32 result.  Pins the kind::i8 instruction descriptor
+// and the signedness of the operands.
+struct ImmaSelftestSmem {
+    unsigned char a[128][128];
+    unsigned char b[128][128];
+    uint64_t full, mma_done;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+__global__ void __launch_bounds__(128) imma_selftest_kernel(const __grid_constant__ CUtensorMap tmA,
+                                                            const __grid_constant__ CUtensorMap tmB,
+                                                            int32_t* __restrict__ d_out, int32_t* __restrict__ status) {
+    extern __shared__ unsigned char imma_raw[];
+    ImmaSelftestSmem& sm = *reinterpret_cast<ImmaSelftestSmem*>((reinterpret_cast<uintptr_t>(imma_raw) + 1023) & ~(uintptr_t)1023);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr uint32_t kIdesc = tc::make_idesc_s8(128, 128);
+    if (tid == 0) {
+        tc::mbar_init(&sm.full, 1);
+        tc::mbar_init(&sm.mma_done, 1);
+        sm.abort_flag = 0;
+        tc::fence_barrier_init();
+    }
+    if (warp == 0) tc::tmem_alloc<128>(&sm.tmem_base);
+    tc::tc_fence_before_sync();
+    __syncthreads();
+    tc::tc_fence_after_sync();
+    const uint32_t tbase = sm.tmem_base;
+    volatile int* abort_flag = &sm.abort_flag;
+    bool ok = true;
+    if (tid == 0) {
+        tc::mbar_arrive_expect_tx(&sm.full, 2 * 128 * 128);
+        tc::tma_load_2d(&sm.a[0][0], &tmA, 0, 0, &sm.full);
+        tc::tma_load_2d(&sm.b[0][0], &tmB, 0, 0, &sm.full);
+        ok = tc::mbar_wait(&sm.full, 0, abort_flag);
+        if (ok) {
+            tc::tc_fence_after_sync();
+            for (int ks = 0; ks < 4; ++ks) {   // 32 bytes of k per step
+                uint64_t da = tc::make_smem_desc_sw128(smem_u32(&sm.a[0][0]) + ks * 32);
+                uint64_t db = tc::make_smem_desc_sw128(smem_u32(&sm.b[0][0]) + ks * 32);
+                tc::umma_ss_i8(tbase, da, db, kIdesc, ks > 0);
+            }
+            tc::umma_commit(&sm.mma_done);
+        }
+    }
+    __syncwarp();
+    ok = tc::mbar_wait(&sm.mma_done, 0, abort_flag);
+    if (ok) {
+        tc::tc_fence_after_sync();
+        const int row = warp * 32 + lane;
+        const uint32_t lane_addr = tbase + ((uint32_t)(warp * 32) << 16);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            uint32_t r[32];
+            tc::tmem_ld_32x32(lane_addr + c * 32, r);
+            tc::tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) d_out[row * 128 + c * 32 + i] = (int32_t)r[i];
+        }
+    }
+    if (!ok && lane == 0) atomicExch(status, 6);
+    tc::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) tc::tmem_dealloc<128>(tbase);
+}
+
 }  // namespace adaspark

@@ -21,3 +21,17 @@ def test_umma_selftest_matches_matmul():
     p = (d / 64).to(torch.bfloat16)
     e_ref = p.double() @ c.double().T
     assert torch.allclose(e.double(), e_ref, atol=1e-3, rtol=1e-4), (e.double() - e_ref).abs().max()
+
+
+def test_imma_selftest_is_an_exact_signed_product():
+    g = torch.Generator(device="cpu").manual_seed(4)
+    for lo, hi in [(-128, 128), (-128, -100), (100, 128)]:
+        a = torch.randint(lo, hi, (128, 128), generator=g, dtype=torch.int32).to(torch.int8)
+        b = torch.randint(-128, 128, (128, 128), generator=g, dtype=torch.int32).to(torch.int8)
+        d = torch.full((128, 128), -1, dtype=torch.int32, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        rc = binding.adaspark_attn_debug_imma_selftest(a.cuda(), b.cuda(), d, status)
+        torch.cuda.synchronize()
+        assert rc == binding.OK and int(status.item()) == 0
+        ref = a.to(torch.int64) @ b.to(torch.int64).T
+        assert torch.equal(d.cpu().to(torch.int64), ref)
