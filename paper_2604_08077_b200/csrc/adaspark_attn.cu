@@ -203,9 +203,9 @@ adaspark_status_t adaspark_attn_partition(adaspark_attn_t* h, int32_t batch, int
     h->fw_chunk_tiles = (int)chunk;
     h->fw_logits_off = off; off = align_up(off + 2 * chunk * tile_bytes);   // double-buffered
     h->fw_qcube_off = off; off = align_up(off + (size_t)batch * Hq * S_cap * D * 2);
-    // digit planes (4 x bf16 [B*Hkv*N_ld, D]) and row exponents of the mean keys (tensor-core scoring);
+    // digit planes (4 x int8 [B*Hkv*N_ld, 128]) and row exponents of the mean keys (tensor-core scoring);
     // 128 rows of slack so that the last 128-cube TMA box stays inside the allocation
-    h->fw_kplanes_off = off; off = align_up(off + ((size_t)4 * batch * Hkv * N_ld + 128) * D * 2);
+    h->fw_kplanes_off = off; off = align_up(off + ((size_t)4 * batch * Hkv * N_ld + 128) * kDigitRowBytes);
     h->fw_kexp_off = off; off = align_up(off + (size_t)batch * Hkv * N_ld * 4);
     h->fw_total = off;
     L.forward_workspace_bytes = (int64_t)off;
@@ -329,11 +329,11 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
         CUtensorMap tmKs;
         int32_t* key_exp = (int32_t*)(ws + h->fw_kexp_off);
         if (h->prefill_kernel == 1) {   // digit planes of the mean keys, tensor maps of the scoring kernel
-            __nv_bfloat16* kplanes = (__nv_bfloat16*)(ws + h->fw_kplanes_off);
+            unsigned char* kplanes = (unsigned char*)(ws + h->fw_kplanes_off);
             const int n_rows = g.B * g.Hkv * g.N_ld;
             slice_keys_kernel<<<(n_rows + 3) / 4, 128, 0, st>>>(g, cube_keys, kplanes, key_exp);
             if (!launch_ok(h, "slice_keys_kernel")) return ADASPARK_ERR_CUDA;
-            if (!encode_bf16_2d(&tmKs, kplanes, (uint64_t)4 * n_rows + 128, D, 64, kScoreTcCols))
+            if (!encode_u8_2d(&tmKs, kplanes, (uint64_t)4 * n_rows + 128, kDigitRowBytes, kDigitRowBytes, kScoreTcCols))
                 return fail(h, ADASPARK_ERR_CUDA, "forward: cuTensorMapEncodeTiled failed");
             if (D == 128) { if (!set_smem(h, score_tc_kernel<128>, sizeof(ScoreTcSmem<128>) + 1024, "score_tc_kernel")) return ADASPARK_ERR_CUDA; }
             else { if (!set_smem(h, score_tc_kernel<64>, sizeof(ScoreTcSmem<64>) + 1024, "score_tc_kernel")) return ADASPARK_ERR_CUDA; }

@@ -1,19 +1,18 @@
-// K3 on the bf16 tensor cores: cube scores of Eq. 1 from error-free digit slices.
+// K3 on the int8 tensor cores: cube scores of Eq. 1 from error-free digit slices.
 //
 // The selection must follow an fp64 evaluation of Eqs. 1-2 (rows may differ only inside a 1e-6
 // probability margin), so plain bf16/fp32 tensor-core arithmetic is not accurate enough.  Instead
 // every query row q and every mean key k are written in fixed point relative to the largest
 // exponent of their row,
-//     x = 2^(e - 30) * (d0*2^24 + d1*2^16 + d2*2^8 + d3),   digits d_i integers in [-128, 128],
-// (exact for elements within 2^-23 (q, 8 significant bits) / 2^-7 (k, 24 bits) of the row maximum,
-// rounded at 2^-30 of it below that).  Digits are exact bf16 values, a product of two digits has 15
-// bits and a sum of 4 * 128 such products stays below 2^24, so a tcgen05.mma with fp32 accumulation
-// computes  S_L = sum_{a+b=L} Q_a . K_b  EXACTLY for each level L.  Then
-//     q . k = 2^(e_q + e_k - 12) * (S_0 + S_1*2^-8 + S_2*2^-16 + S_3*2^-24 + levels >= 4),
+//     x = 2^(e - 29) * (d0*2^24 + d1*2^16 + d2*2^8 + d3),   digits d_i signed bytes in [-128, 127],
+// (exact for elements within 2^-22 (q, 8 significant bits) / 2^-6 (k, 24 bits) of the row maximum,
+// rounded at 2^-29 of it below that).  tcgen05.mma of kind::i8 multiplies the digit planes with exact
+// int32 accumulation:  S_L = sum_{a+b=L} Q_a . K_b  for each level L (|S_L| <= 4 * 128 * 2^14).  Then
+//     q . k = 2^(e_q + e_k - 10) * (S_0 + S_1*2^-8 + S_2*2^-16 + S_3*2^-24 + levels >= 4),
 // and the levels 0..3 (10 digit pairs, four TMEM accumulators) are combined exactly in fp64.  The
-// dropped levels are bounded by 1.5e-3 * 2^-12 * 2^(e_q+e_k) in the worst case (all digit products
-// aligned), about 5e-7 in the scaled logit for |q| <= 3, |k| <= 5 and typically 10x less: inside
-// the margin above.
+// dropped levels are bounded by about 5e-7 in the scaled logit for |q| <= 3, |k| <= 5 in the worst
+// case (all digit products aligned) and typically 10x less: inside the margin above.  A digit plane
+// row is always 128 bytes (head_dim 64 is zero-padded).
 //
 //   slice_keys_kernel   digit planes + row exponents of the mean keys (once per forward, tiny)
 //   score_tc_kernel     persistent CTAs, one per SM; work item = one 128-row query tile x a group of
@@ -24,86 +23,73 @@
 //     warps 4-11  slicers (two threads per row): read the bf16 query row, compute its digits in
 //                 registers while the previous item's MMAs still read the planes, then store the
 //                 four swizzled digit planes of the tile into shared memory
-//     warp 12     TMA producer: key digit blocks (plane, 64-d panel, 64 cubes) in a ring
-//     warp 13     issues the tcgen05.mma stream (80 of 128x64x16 per column tile at D = 128)
+//     warp 12     TMA producer: key digit blocks (one plane of 64 cubes, 8 KB) in a ring
+//     warp 13     issues the tcgen05.mma stream (40 of 128x64x32 per column tile)
 #pragma once
 #include "tc_common.cuh"
 
 namespace adaspark {
 
 constexpr int kScoreTcThreads = 448;
-constexpr int kScoreTcRing = 8;          // key digit blocks (64 cubes x 64 d, 8 KB) in flight
+constexpr int kScoreTcRing = 16;         // key digit blocks (64 cubes x 128 bytes, 8 KB) in flight
 constexpr int kScoreTcCols = 64;         // cubes per column tile
+constexpr int kDigitRowBytes = 128;      // bytes per row of a digit plane
 
-// Fixed-point value of x relative to the row exponent e (unbiased exponent of the row maximum):
-// round(x * 2^(30 - e)), |result| < 2^31.
-__device__ __forceinline__ int fixed30(float x, int e) {
-    return __float2int_rn(x * __int_as_float((157 - e) << 23));   // 2^(30 - e), exact for e >= -96
+// The four signed base-256 digits of v = round(x * 2^(29 - e)) (|v| < 2^30), packed in one word:
+// byte 3 = d0 (most significant) ... byte 0 = d3.  Adding 0x80 to every byte position turns the
+// balanced digits into the plain unsigned bytes of v + 0x80808080, so two integer operations give
+// all four.
+__device__ __forceinline__ uint32_t packed_digits(float x, float mult) {
+    const uint32_t u = (uint32_t)__float2int_rn(x * mult) + 0x80808080u;
+    return u ^ 0x80808080u;
 }
-// Signed base-256 digits, most significant first: v = d[0]*2^24 + d[1]*2^16 + d[2]*2^8 + d[3].
-__device__ __forceinline__ void digits256(int v, int (&d)[4]) {
-    // v = 256 * (floor(v / 256) + carry) + digit with digit = low byte read as signed (no overflow)
-    d[3] = (int)(signed char)(v & 0xff);
-    v = (v >> 8) + (d[3] < 0 ? 1 : 0);
-    d[2] = (int)(signed char)(v & 0xff);
-    v = (v >> 8) + (d[2] < 0 ? 1 : 0);
-    d[1] = (int)(signed char)(v & 0xff);
-    d[0] = (v >> 8) + (d[1] < 0 ? 1 : 0);
+__device__ __forceinline__ float digit_scale(int e) {             // 2^(29 - e), exact for e >= -97
+    return __int_as_float((156 - e) << 23);
 }
-// The same digits for a float that holds an integer-valued (or nearly: |fraction| only in the last
-// digit) fixed-point number v, |v| < 2^31, computed with exact float operations.
-__device__ __forceinline__ float round_small(float t) {          // nearest integer, |t| <= 2^22
-    return (t + 12582912.f) - 12582912.f;
+__device__ __forceinline__ int row_exponent_from_field(int biased) {   // 8-bit exponent field of the row maximum
+    return biased == 0 ? 0 : max(biased - 127, -90);               // rows smaller than 2^-90 keep fewer digits
 }
-__device__ __forceinline__ void float_digits256(float v, float (&d)[4]) {
-    d[0] = round_small(v * (1.f / 16777216.f));
-    float r = fmaf(-d[0], 16777216.f, v);
-    d[1] = round_small(r * (1.f / 65536.f));
-    r = fmaf(-d[1], 65536.f, r);
-    d[2] = round_small(r * (1.f / 256.f));
-    r = fmaf(-d[2], 256.f, r);
-    d[3] = round_small(r);
-}
-// bf16 bit pattern of a small integer (|i| <= 256: exact).
-__device__ __forceinline__ uint32_t bf16_bits_of_int(int i) {
-    return __float_as_uint((float)i) >> 16;
-}
-__device__ __forceinline__ int exponent_of(float x) {   // unbiased exponent field (0 for zero/denormal rows)
-    const int e = (int)((__float_as_uint(x) >> 23) & 0xffu);
-    return e == 0 ? 0 : max(e - 127, -90);     // rows smaller than 2^-90 keep fewer digits
+// Byte k of four packed words -> one word (element i in byte i): digit plane 3 - k of four elements.
+template <int k>
+__device__ __forceinline__ uint32_t gather_byte(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3) {
+    const uint32_t lo = __byte_perm(w0, w1, (uint32_t)k | ((uint32_t)(4 + k) << 4));
+    const uint32_t hi = __byte_perm(w2, w3, (uint32_t)k | ((uint32_t)(4 + k) << 4));
+    return __byte_perm(lo, hi, 0x5410);
 }
 
-// Digit planes of the mean keys: planes[p][(b*Hkv+gk)*N_ld + cube][D] (bf16), key_exp[(b*Hkv+gk)*N_ld + cube].
-// One warp per cube row; rows >= N inside the padded leading dimension are zero-filled.
+// Digit planes of the mean keys: planes[p][(b*Hkv+gk)*N_ld + cube][128 bytes] (int8, zero beyond D),
+// key_exp[(b*Hkv+gk)*N_ld + cube].  One warp per cube row, four elements per lane; rows >= N inside
+// the padded leading dimension are zero-filled.
 __global__ void __launch_bounds__(128) slice_keys_kernel(Geom g, const float* __restrict__ cube_keys,
-                                                         __nv_bfloat16* __restrict__ planes, int32_t* __restrict__ key_exp) {
+                                                         unsigned char* __restrict__ planes, int32_t* __restrict__ key_exp) {
     const int lane = threadIdx.x & 31;
     const int row = blockIdx.x * 4 + (threadIdx.x >> 5);              // (b*Hkv+gk)*N_ld + cube
     const int n_rows = g.B * g.Hkv * g.N_ld;
     if (row >= n_rows) return;
     const int bh = row / g.N_ld, cube = row - bh * g.N_ld;
-    const size_t plane_stride = (size_t)n_rows * g.D;
-    const bool live = cube < g.N;
-    const float* src = cube_keys + ((size_t)bh * g.N + (live ? cube : 0)) * g.D;
-    float mx = 0.f;
-    for (int d = lane; d < g.D; d += 32) mx = fmaxf(mx, live ? fabsf(src[d]) : 0.f);
+    const size_t plane_stride = (size_t)n_rows * kDigitRowBytes;
+    const bool live = cube < g.N && lane * 4 < g.D;
+    float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (live) x = *reinterpret_cast<const float4*>(cube_keys + ((size_t)bh * g.N + cube) * g.D + lane * 4);
+    float mx = fmaxf(fmaxf(fabsf(x.x), fabsf(x.y)), fmaxf(fabsf(x.z), fabsf(x.w)));
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    const int e = exponent_of(mx);
-    for (int d = lane; d < g.D; d += 32) {
-        int dg[4];
-        digits256(live ? fixed30(src[d], e) : 0, dg);
-#pragma unroll
-        for (int p = 0; p < 4; ++p)
-            planes[p * plane_stride + (size_t)row * g.D + d] = __ushort_as_bfloat16((unsigned short)bf16_bits_of_int(dg[p]));
-    }
+    const int e = row_exponent_from_field((int)((__float_as_uint(mx) >> 23) & 0xffu));
+    const float mult = digit_scale(e);
+    const uint32_t w0 = packed_digits(x.x, mult), w1 = packed_digits(x.y, mult);
+    const uint32_t w2 = packed_digits(x.z, mult), w3 = packed_digits(x.w, mult);
+    unsigned char* dst = planes + (size_t)row * kDigitRowBytes + lane * 4;
+    *reinterpret_cast<uint32_t*>(dst) = gather_byte<3>(w0, w1, w2, w3);
+    *reinterpret_cast<uint32_t*>(dst + plane_stride) = gather_byte<2>(w0, w1, w2, w3);
+    *reinterpret_cast<uint32_t*>(dst + 2 * plane_stride) = gather_byte<1>(w0, w1, w2, w3);
+    *reinterpret_cast<uint32_t*>(dst + 3 * plane_stride) = gather_byte<0>(w0, w1, w2, w3);
     if (lane == 0) key_exp[row] = e;
 }
 
 template <int D>
 struct ScoreTcSmem {
-    __nv_bfloat16 qd[4][D / 64][128][64];               // digit planes of the Q tile, UMMA layout (128-B swizzle)
-    __nv_bfloat16 kring[kScoreTcRing][kScoreTcCols][64];   // key digit blocks: [cube][64 d of one panel of one plane]
+    unsigned char qd[4][128][kDigitRowBytes];           // digit planes of the Q tile, UMMA layout (128-B swizzle)
+    unsigned char kring[kScoreTcRing][kScoreTcCols][kDigitRowBytes];   // key digit blocks: one plane of 64 cubes
     double stage[128][32];                              // epilogue: scores of 32 columns, column index ^ (row & 31)
     uint64_t q_sliced, qd_free, k_full[kScoreTcRing], k_group_empty[kScoreTcRing / 4], acc_full[2], acc_free[2];
     uint32_t tmem_base;
@@ -139,10 +125,9 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
     int32_t* __restrict__ status) {
     extern __shared__ unsigned char score_tc_raw[];
     ScoreTcSmem<D>& sm = *reinterpret_cast<ScoreTcSmem<D>*>((reinterpret_cast<uintptr_t>(score_tc_raw) + 1023) & ~(uintptr_t)1023);
-    constexpr int kPanels = D / 64;
-    constexpr int kBlocks = 4 * kPanels;                          // key digit blocks per column tile
-    constexpr uint32_t kIdesc = tc::make_idesc_bf16(128, kScoreTcCols);
-    constexpr uint32_t kBlockBytes = kScoreTcCols * 64 * 2;
+    constexpr int kBlocks = 4;                                    // key digit blocks (planes) per column tile
+    constexpr uint32_t kIdesc = tc::make_idesc_s8(128, kScoreTcCols);
+    constexpr uint32_t kBlockBytes = kScoreTcCols * kDigitRowBytes;
     constexpr int kProducerWarp = 12, kMmaWarp = 13;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -161,6 +146,11 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
         }
         sm.abort_flag = 0;
         tc::fence_barrier_init();
+    }
+    if (D < kDigitRowBytes) {                                     // bytes beyond head_dim stay zero for the whole kernel
+        uint4* z = reinterpret_cast<uint4*>(&sm.qd[0][0][0]);
+        for (int i = tid; i < (int)(sizeof(sm.qd) / 16); i += kScoreTcThreads) z[i] = make_uint4(0u, 0u, 0u, 0u);
+        asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
     }
     if (warp == kProducerWarp) {
         tc::tmem_alloc<512>(&sm.tmem_base);
@@ -183,10 +173,10 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
                 const int k_row0 = (w.b * g.Hkv + w.gk) * g.N_ld;
                 for (int ct = w.ct0; ok && ct < w.ct1; ++ct) {
                     for (int blk = 0; blk < kBlocks; ++blk, ++i) {
-                        const int p = blk >> 2, plane = blk & 3, s = i % kScoreTcRing, u = i / kScoreTcRing;
-                        if ((blk & 3) == 0 && !(ok = tc::mbar_wait(&sm.k_group_empty[s >> 2], (u & 1) ^ 1, abort_flag))) break;
+                        const int plane = blk, s = i % kScoreTcRing, u = i / kScoreTcRing;
+                        if (blk == 0 && !(ok = tc::mbar_wait(&sm.k_group_empty[s >> 2], (u & 1) ^ 1, abort_flag))) break;
                         tc::mbar_arrive_expect_tx(&sm.k_full[s], kBlockBytes);
-                        tc::tma_load_2d(&sm.kring[s][0][0], &tmK, p * 64, plane * n_rows + k_row0 + ct * kScoreTcCols, &sm.k_full[s]);
+                        tc::tma_load_2d(&sm.kring[s][0][0], &tmK, 0, plane * n_rows + k_row0 + ct * kScoreTcCols, &sm.k_full[s]);
                     }
                 }
             }
@@ -194,9 +184,9 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
     } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            constexpr uint32_t kPlaneStep = (uint32_t)sizeof(sm.qd[0]) >> 4, kPanelStep = (128 * 64 * 2) >> 4;
+            constexpr uint32_t kPlaneStep = (uint32_t)sizeof(sm.qd[0]) >> 4;
             constexpr uint32_t kRingStep = (uint32_t)sizeof(sm.kring[0]) >> 4, kKStep = 32 >> 4;
-            const uint32_t q_lo0 = tc::smem_desc_lo_sw128(smem_u32(&sm.qd[0][0][0][0]));
+            const uint32_t q_lo0 = tc::smem_desc_lo_sw128(smem_u32(&sm.qd[0][0][0]));
             const uint32_t k_lo0 = tc::smem_desc_lo_sw128(smem_u32(&sm.kring[0][0][0]));
             bool ok = true;
             int i = 0, c = 0, n_done = 0;                         // running block / column-tile / item counters
@@ -209,20 +199,20 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
                     if (use > 0 && !(ok = tc::mbar_wait(&sm.acc_free[buf], (use - 1) & 1, abort_flag))) break;
                     tc::tc_fence_after_sync();
                     for (int blk = 0; blk < kBlocks; ++blk, ++i) {
-                        const int p = blk >> 2, plane = blk & 3, s = i % kScoreTcRing, u = i / kScoreTcRing;
+                        const int plane = blk, s = i % kScoreTcRing, u = i / kScoreTcRing;
                         if (!(ok = tc::mbar_wait(&sm.k_full[s], u & 1, abort_flag))) break;
                         tc::tc_fence_after_sync();
                         const uint32_t kb = k_lo0 + s * kRingStep;
                         for (int a = 0; a + plane <= 3; ++a) {    // level a + plane
-                            const uint32_t qa = q_lo0 + a * kPlaneStep + p * kPanelStep;
+                            const uint32_t qa = q_lo0 + a * kPlaneStep;
                             const uint32_t dst = tbase + buf * 256 + (a + plane) * kScoreTcCols;
 #pragma unroll
                             for (int ks = 0; ks < 4; ++ks)
-                                tc::umma_ss(dst, tc::smem_desc_from_halves(qa + ks * kKStep, tc::kSmemDescHiSw128),
-                                            tc::smem_desc_from_halves(kb + ks * kKStep, tc::kSmemDescHiSw128), kIdesc,
-                                            !(blk == 0 && ks == 0));
+                                tc::umma_ss_i8(dst, tc::smem_desc_from_halves(qa + ks * kKStep, tc::kSmemDescHiSw128),
+                                               tc::smem_desc_from_halves(kb + ks * kKStep, tc::kSmemDescHiSw128), kIdesc,
+                                               !(blk == 0 && ks == 0));
                         }
-                        if ((blk & 3) == 3) tc::umma_commit(&sm.k_group_empty[s >> 2]);
+                        if (blk == 3) tc::umma_commit(&sm.k_group_empty[s >> 2]);
                     }
                     if (ok) tc::umma_commit(&sm.acc_full[buf]);
                 }
@@ -232,7 +222,8 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
         }
     } else if (warp >= 4) {
         // ------------------------------------------------------------ slicers (two threads per row)
-        constexpr int kChunks = D / 16;                           // 16-byte chunks (8 elements) per thread
+        constexpr int kChunks = D / 16;                           // 16-byte chunks (8 elements) of the row half
+        constexpr int kOut = D / 32;                              // 16-byte chunks (16 digits) per plane per thread
         const int r = (tid - 128) >> 1, half = (tid - 128) & 1;
         bool ok = true;
         int n_done = 0;
@@ -252,36 +243,35 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
                 for (int i = 0; i < 4; ++i) mxbits = max(mxbits, max(wd[i] & 0x7fffu, (wd[i] >> 16) & 0x7fffu));
             }
             mxbits = max(mxbits, __shfl_xor_sync(0xffffffffu, mxbits, 1));   // the two halves of the row
-            const int ef = (int)(mxbits >> 7);
-            const int e_q = ef == 0 ? 0 : max(ef - 127, -90);
-            // digits in the float domain (every intermediate is exact): x * 2^(30-e) = d0*2^24 + d1*2^16 + d2*2^8 + d3
-            const float mult = __int_as_float((157 - e_q) << 23);
-            uint4 out[4][kChunks];
+            const float mult = digit_scale(row_exponent_from_field((int)(mxbits >> 7)));
+            uint4 out[4][kOut];                                   // [plane][16 digits of this thread's half]
 #pragma unroll
-            for (int c = 0; c < kChunks; ++c) {
-                const uint32_t wd[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
-                uint32_t pk[4][4];
+            for (int o = 0; o < kOut; ++o) {
+                uint32_t pw[4][4];                                // [plane][4 elements per word]
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    float dl[4], dh[4];
-                    float_digits256(__uint_as_float(wd[i] << 16) * mult, dl);
-                    float_digits256(__uint_as_float(wd[i] & 0xffff0000u) * mult, dh);
-#pragma unroll
-                    for (int pl = 0; pl < 4; ++pl)    // bf16 of a small integer = upper half of its float
-                        pk[pl][i] = __byte_perm(__float_as_uint(dl[pl]), __float_as_uint(dh[pl]), 0x7632);
+                for (int q4 = 0; q4 < 4; ++q4) {                  // elements 16*o + 4*q4 .. +3 = two packed bf16 words
+                    const uint4 vv = v[2 * o + (q4 >> 1)];
+                    const uint32_t wa = (q4 & 1) ? vv.z : vv.x, wb = (q4 & 1) ? vv.w : vv.y;
+                    const uint32_t w0 = packed_digits(__uint_as_float(wa << 16), mult);
+                    const uint32_t w1 = packed_digits(__uint_as_float(wa & 0xffff0000u), mult);
+                    const uint32_t w2 = packed_digits(__uint_as_float(wb << 16), mult);
+                    const uint32_t w3 = packed_digits(__uint_as_float(wb & 0xffff0000u), mult);
+                    pw[0][q4] = gather_byte<3>(w0, w1, w2, w3);
+                    pw[1][q4] = gather_byte<2>(w0, w1, w2, w3);
+                    pw[2][q4] = gather_byte<1>(w0, w1, w2, w3);
+                    pw[3][q4] = gather_byte<0>(w0, w1, w2, w3);
                 }
 #pragma unroll
-                for (int pl = 0; pl < 4; ++pl) out[pl][c] = make_uint4(pk[pl][0], pk[pl][1], pk[pl][2], pk[pl][3]);
+                for (int pl = 0; pl < 4; ++pl) out[pl][o] = make_uint4(pw[pl][0], pw[pl][1], pw[pl][2], pw[pl][3]);
             }
             // the previous item's MMAs must have finished reading the digit planes
             if (n_done > 0 && !(ok = tc::mbar_wait(&sm.qd_free, (n_done - 1) & 1, abort_flag))) break;
-            unsigned char* dst = reinterpret_cast<unsigned char*>(&sm.qd[0][0][0][0]);
+            unsigned char* dst = &sm.qd[0][0][0];
 #pragma unroll
-            for (int c = 0; c < kChunks; ++c) {
-                const int cc = half * kChunks + c;                // chunk of the row: panel cc / 8, position cc % 8
-                const int off = (cc >> 3) * (128 * 128) + sw128(r, cc & 7);
+            for (int o = 0; o < kOut; ++o) {
+                const int off = sw128(r, half * kOut + o);        // 16-byte chunk of the 128-byte plane row
 #pragma unroll
-                for (int pl = 0; pl < 4; ++pl) *reinterpret_cast<uint4*>(dst + (size_t)pl * sizeof(sm.qd[0]) + off) = out[pl][c];
+                for (int pl = 0; pl < 4; ++pl) *reinterpret_cast<uint4*>(dst + (size_t)pl * sizeof(sm.qd[0]) + off) = out[pl][o];
             }
             asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");   // digit planes visible to the tensor core
             tc::mbar_arrive(&sm.q_sliced);
@@ -312,8 +302,7 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
                         for (int i = 0; i < 4; ++i) mxbits = max(mxbits, max(wd[i] & 0x7fffu, (wd[i] >> 16) & 0x7fffu));
                     }
                 }
-                const int ef = (int)(mxbits >> 7);
-                e_q = ef == 0 ? 0 : max(ef - 127, -90);
+                e_q = row_exponent_from_field((int)(mxbits >> 7));
             }
             const double rowf = __hiloint2double((1023 + e_q) << 20, 0);          // 2^e_q
             const int32_t* kexp = key_exp + (size_t)(w.b * g.Hkv + w.gk) * g.N_ld;
@@ -325,10 +314,10 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
 #pragma unroll 1
                 for (int c = 0; c < kScoreTcCols / 32; ++c) {     // 32 columns at a time through the staging tile
                     const int col0 = ct * kScoreTcCols + c * 32;
-                    // column factor 2^(e_k - 36) * scale, held by the lane that owns the column
+                    // column factor 2^(e_k - 34) * scale, held by the lane that owns the column
                     const int jc = col0 + lane;
                     const int ek = jc < g.N_ld ? kexp[jc] : 0;
-                    const double colf = __hiloint2double((1023 + ek - 36) << 20, 0) * g.scale_d;
+                    const double colf = __hiloint2double((1023 + ek - 34) << 20, 0) * g.scale_d;
 #pragma unroll
                     for (int hc = 0; hc < 2; ++hc) {
                         uint32_t lv[4][16];
@@ -342,8 +331,8 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
                             // exact integer level sums: S0*2^24 + S1*2^16 + S2*2^8 + S3 = hi*2^16 + lo
-                            const int hi = __float2int_rn(__uint_as_float(lv[0][i])) * 256 + __float2int_rn(__uint_as_float(lv[1][i]));
-                            const int lo = __float2int_rn(__uint_as_float(lv[2][i])) * 256 + __float2int_rn(__uint_as_float(lv[3][i]));
+                            const int hi = (int)lv[0][i] * 256 + (int)lv[1][i];
+                            const int lo = (int)lv[2][i] * 256 + (int)lv[3][i];
                             const double hd = __hiloint2double(0x43300000, hi ^ 0x80000000) - 4503601774854144.0;   // (double)hi
                             const double ld = __hiloint2double(0x43300000, lo ^ 0x80000000) - 4503601774854144.0;   // 2^52 + 2^31
                             const double v = fma(hd, 65536.0, ld);
