@@ -16,22 +16,23 @@
 //
 //   slice_keys_kernel   digit planes + row exponents of the mean keys (once per forward, tiny)
 //   score_tc_kernel     persistent CTAs, one per SM; work item = one 128-row query tile x a group of
-//                       64-cube column tiles.  Roles (448 threads), pipelined across items:
-//     warps 0-3   epilogue (thread = row = TMEM lane): TMEM -> fp64 scores -> coalesced rows of the
-//                 score buffer.  The four level accumulators are double-buffered in TMEM (2 x 4 x 64
-//                 columns), so the epilogue of one column tile overlaps the MMAs of the next
-//     warps 4-11  slicers (two threads per row): read the bf16 query row, compute its digits in
-//                 registers while the previous item's MMAs still read the planes, then store the
-//                 four swizzled digit planes of the tile into shared memory
-//     warp 12     TMA producer: key digit blocks (one plane of 64 cubes, 8 KB) in a ring
-//     warp 13     issues the tcgen05.mma stream (40 of 128x64x32 per column tile)
+//                       64-cube column tiles.  Roles (576 threads), pipelined across items:
+//     warps 0-7   epilogue (thread = row = TMEM lane, 32 of the 64 columns): TMEM -> fp64 scores ->
+//                 coalesced rows of the score buffer.  The four level accumulators are double-buffered
+//                 in TMEM (2 x 4 x 64 columns), so the epilogue of one column tile overlaps the MMAs of
+//                 the next
+//     warps 8-15  slicers (two threads per row): read the bf16 query row early, then write the four
+//                 swizzled digit planes of the tile into shared memory once the previous item's MMAs
+//                 have released them
+//     warp 16     TMA producer: key digit blocks (one plane of 64 cubes, 8 KB) in a ring
+//     warp 17     issues the tcgen05.mma stream (40 of 128x64x32 per column tile)
 #pragma once
 #include "tc_common.cuh"
 
 namespace adaspark {
 
-constexpr int kScoreTcThreads = 448;
-constexpr int kScoreTcRing = 16;         // key digit blocks (64 cubes x 128 bytes, 8 KB) in flight
+constexpr int kScoreTcThreads = 576;
+constexpr int kScoreTcRing = 12;         // key digit blocks (64 cubes x 128 bytes, 8 KB) in flight
 constexpr int kScoreTcCols = 64;         // cubes per column tile
 constexpr int kDigitRowBytes = 128;      // bytes per row of a digit plane
 
@@ -90,7 +91,7 @@ template <int D>
 struct ScoreTcSmem {
     unsigned char qd[4][128][kDigitRowBytes];           // digit planes of the Q tile, UMMA layout (128-B swizzle)
     unsigned char kring[kScoreTcRing][kScoreTcCols][kDigitRowBytes];   // key digit blocks: one plane of 64 cubes
-    double stage[128][32];                              // epilogue: scores of 32 columns, column index ^ (row & 31)
+    double stage[2][128][32];                           // epilogue, per column half: scores of 32 columns, index ^ (row & 31)
     uint64_t q_sliced, qd_free, k_full[kScoreTcRing], k_group_empty[kScoreTcRing / 4], acc_full[2], acc_free[2];
     uint32_t tmem_base;
     int abort_flag;
@@ -128,7 +129,7 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
     constexpr int kBlocks = 4;                                    // key digit blocks (planes) per column tile
     constexpr uint32_t kIdesc = tc::make_idesc_s8(128, kScoreTcCols);
     constexpr uint32_t kBlockBytes = kScoreTcCols * kDigitRowBytes;
-    constexpr int kProducerWarp = 12, kMmaWarp = 13;
+    constexpr int kProducerWarp = 16, kMmaWarp = 17;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid == 0) {
@@ -142,7 +143,7 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
         for (int i = 0; i < kScoreTcRing / 4; ++i) tc::mbar_init(&sm.k_group_empty[i], 1);
         for (int i = 0; i < 2; ++i) {
             tc::mbar_init(&sm.acc_full[i], 1);
-            tc::mbar_init(&sm.acc_free[i], 128);
+            tc::mbar_init(&sm.acc_free[i], 256);
         }
         sm.abort_flag = 0;
         tc::fence_barrier_init();
@@ -220,11 +221,11 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
                 ++n_done;
             }
         }
-    } else if (warp >= 4) {
+    } else if (warp >= 8) {
         // ------------------------------------------------------------ slicers (two threads per row)
         constexpr int kChunks = D / 16;                           // 16-byte chunks (8 elements) of the row half
         constexpr int kOut = D / 32;                              // 16-byte chunks (16 digits) per plane per thread
-        const int r = (tid - 128) >> 1, half = (tid - 128) & 1;
+        const int r = (tid - 256) >> 1, half = (tid - 256) & 1;
         bool ok = true;
         int n_done = 0;
         for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
@@ -244,7 +245,9 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
             }
             mxbits = max(mxbits, __shfl_xor_sync(0xffffffffu, mxbits, 1));   // the two halves of the row
             const float mult = digit_scale(row_exponent_from_field((int)(mxbits >> 7)));
-            uint4 out[4][kOut];                                   // [plane][16 digits of this thread's half]
+            // the previous item's MMAs must have finished reading the digit planes
+            if (n_done > 0 && !(ok = tc::mbar_wait(&sm.qd_free, (n_done - 1) & 1, abort_flag))) break;
+            unsigned char* dst = &sm.qd[0][0][0];
 #pragma unroll
             for (int o = 0; o < kOut; ++o) {
                 uint32_t pw[4][4];                                // [plane][4 elements per word]
@@ -261,17 +264,10 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
                     pw[2][q4] = gather_byte<1>(w0, w1, w2, w3);
                     pw[3][q4] = gather_byte<0>(w0, w1, w2, w3);
                 }
-#pragma unroll
-                for (int pl = 0; pl < 4; ++pl) out[pl][o] = make_uint4(pw[pl][0], pw[pl][1], pw[pl][2], pw[pl][3]);
-            }
-            // the previous item's MMAs must have finished reading the digit planes
-            if (n_done > 0 && !(ok = tc::mbar_wait(&sm.qd_free, (n_done - 1) & 1, abort_flag))) break;
-            unsigned char* dst = &sm.qd[0][0][0];
-#pragma unroll
-            for (int o = 0; o < kOut; ++o) {
                 const int off = sw128(r, half * kOut + o);        // 16-byte chunk of the 128-byte plane row
 #pragma unroll
-                for (int pl = 0; pl < 4; ++pl) *reinterpret_cast<uint4*>(dst + (size_t)pl * sizeof(sm.qd[0]) + off) = out[pl][o];
+                for (int pl = 0; pl < 4; ++pl)
+                    *reinterpret_cast<uint4*>(dst + (size_t)pl * sizeof(sm.qd[0]) + off) = make_uint4(pw[pl][0], pw[pl][1], pw[pl][2], pw[pl][3]);
             }
             asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");   // digit planes visible to the tensor core
             tc::mbar_arrive(&sm.q_sliced);
@@ -279,8 +275,10 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
         }
     } else {
         // ------------------------------------------------------------ epilogue (thread = row = TMEM lane)
-        const int r = tid;
-        const uint32_t lane_addr = tbase + ((uint32_t)(warp * 32) << 16);
+        const int lg = warp & 3, chalf = warp >> 2;               // TMEM lane group, column half of the tile
+        const int r = lg * 32 + lane;
+        const uint32_t lane_addr = tbase + ((uint32_t)(lg * 32) << 16);
+        double (*stage)[32] = sm.stage[chalf];
         bool ok = true;
         int c_run = 0, n_done = 0;
         for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
@@ -311,9 +309,8 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
                 const int buf = c_run & 1;
                 if (!(ok = tc::mbar_wait(&sm.acc_full[buf], (c_run >> 1) & 1, abort_flag))) break;
                 tc::tc_fence_after_sync();
-#pragma unroll 1
-                for (int c = 0; c < kScoreTcCols / 32; ++c) {     // 32 columns at a time through the staging tile
-                    const int col0 = ct * kScoreTcCols + c * 32;
+                {
+                    const int col0 = ct * kScoreTcCols + chalf * 32;   // this warp's 32 columns
                     // column factor 2^(e_k - 34) * scale, held by the lane that owns the column
                     const int jc = col0 + lane;
                     const int ek = jc < g.N_ld ? kexp[jc] : 0;
@@ -322,9 +319,9 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
                     for (int hc = 0; hc < 2; ++hc) {
                         uint32_t lv[4][16];
 #pragma unroll
-                        for (int L = 0; L < 4; ++L) tc::tmem_ld_32x16(lane_addr + buf * 256 + L * kScoreTcCols + c * 32 + hc * 16, lv[L]);
+                        for (int L = 0; L < 4; ++L) tc::tmem_ld_32x16(lane_addr + buf * 256 + L * kScoreTcCols + chalf * 32 + hc * 16, lv[L]);
                         tc::tmem_wait_ld();
-                        if (c == kScoreTcCols / 32 - 1 && hc == 1) {   // last read of this accumulator set: release it
+                        if (hc == 1) {                            // last read of this accumulator set: release it
                             tc::tc_fence_before_sync();
                             tc::mbar_arrive(&sm.acc_free[buf]);
                         }
@@ -338,14 +335,14 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
                             const double v = fma(hd, 65536.0, ld);
                             const int col = hc * 16 + i;
                             const double cf = __shfl_sync(0xffffffffu, colf, col);
-                            sm.stage[r][col ^ (r & 31)] = (v * rowf) * cf;
+                            stage[r][col ^ (r & 31)] = (v * rowf) * cf;
                         }
                     }
                     __syncwarp();
                     if (col0 + lane < g.N_ld) {
                         for (int rr = 0; rr < 32; ++rr) {
-                            const int row = warp * 32 + rr;
-                            out_rows[(size_t)row * g.N_ld + col0 + lane] = sm.stage[row][lane ^ (row & 31)];
+                            const int row = lg * 32 + rr;
+                            out_rows[(size_t)row * g.N_ld + col0 + lane] = stage[row][lane ^ (row & 31)];
                         }
                     }
                     __syncwarp();
