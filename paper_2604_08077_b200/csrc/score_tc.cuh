@@ -199,14 +199,18 @@ __global__ void __launch_bounds__(kScoreTcThreads, 1) score_tc_kernel(
                     const int buf = c & 1, use = c >> 1;          // accumulator set and how often it was used before
                     if (use > 0 && !(ok = tc::mbar_wait(&sm.acc_free[buf], (use - 1) & 1, abort_flag))) break;
                     tc::tc_fence_after_sync();
-                    for (int blk = 0; blk < kBlocks; ++blk, ++i) {
-                        const int plane = blk, s = i % kScoreTcRing, u = i / kScoreTcRing;
-                        if (!(ok = tc::mbar_wait(&sm.k_full[s], u & 1, abort_flag))) break;
+                    // fully unrolled: every descriptor is a base plus a compile-time offset
+#pragma unroll
+                    for (int blk = 0; blk < kBlocks; ++blk) {
+                        const int s = i % kScoreTcRing, u = i / kScoreTcRing;
+                        ++i;
+                        if (ok && !(ok = tc::mbar_wait(&sm.k_full[s], u & 1, abort_flag))) break;
                         tc::tc_fence_after_sync();
                         const uint32_t kb = k_lo0 + s * kRingStep;
-                        for (int a = 0; a + plane <= 3; ++a) {    // level a + plane
+#pragma unroll
+                        for (int a = 0; a + blk <= 3; ++a) {      // plane blk of the keys, plane a of the queries: level a + blk
                             const uint32_t qa = q_lo0 + a * kPlaneStep;
-                            const uint32_t dst = tbase + buf * 256 + (a + plane) * kScoreTcCols;
+                            const uint32_t dst = tbase + buf * 256 + (a + blk) * kScoreTcCols;
 #pragma unroll
                             for (int ks = 0; ks < 4; ++ks)
                                 tc::umma_ss_i8(dst, tc::smem_desc_from_halves(qa + ks * kKStep, tc::kSmemDescHiSw128),
