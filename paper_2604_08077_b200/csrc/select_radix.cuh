@@ -206,16 +206,15 @@ __device__ unsigned long long radix_boundary(const unsigned long long* keys, int
         mine[sl] = (i < count && count <= 32) ? cand[i] : 0ull;
         acc[sl] = 0ull;
     }
+    // every candidate of the group in turn, read from the list in shared memory (a broadcast load);
+    // the loop runs to the longest list among the groups of the warp
+    const int cmax = __reduce_max_sync(0xffffffffu, count <= 32 ? count : 0);
+    for (int e = 0; e < cmax; ++e) {
+        const unsigned long long other = e < count ? cand[e] : 0ull;
+        const unsigned long long om = other >> 13;
 #pragma unroll
-    for (int sl2 = 0; sl2 < kOwn; ++sl2) {
-#pragma unroll 8
-        for (int l = 0; l < G; ++l) {
-            const unsigned long long other = __shfl_sync(0xffffffffu, mine[sl2], gbase + l);
-            const unsigned long long om = other >> 13;
-#pragma unroll
-            for (int sl = 0; sl < kOwn; ++sl)
-                if (other >= mine[sl]) acc[sl] += om;
-        }
+        for (int sl = 0; sl < kOwn; ++sl)
+            if (other >= mine[sl]) acc[sl] += om;
     }
     unsigned long long best = 0ull;
 #pragma unroll
