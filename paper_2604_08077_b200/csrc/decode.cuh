@@ -77,21 +77,33 @@ __global__ void __launch_bounds__(256) decode_select_plan_kernel(
                 for (int s = 0; s < 4; ++s)
                     a[4 * S + s] = live ? (double)__bfloat162float(qsrc[16 * S + 4 * kq + s]) : 0.0;
         }
-        for (int c0 = warp * 8; c0 < g.N_ld; c0 += 64) {
-            double acc[2] = {0.0, 0.0};
-            const int cube = c0 + rq;
-            const float* ksrc = kbase + (size_t)(cube < g.N ? cube : 0) * D + 4 * kq;
+        // two groups of 8 cubes per iteration, all 16-byte loads of both issued before the tensor ops
+        // (the mean keys stream from HBM: bytes in flight decide the speed of this loop)
+        for (int c0 = warp * 8; c0 < g.N_ld; c0 += 128) {
+            float4 kv[2][D / 16];
 #pragma unroll
-            for (int S = 0; S < D / 16; ++S) {
-                float4 kv = cube < g.N ? *reinterpret_cast<const float4*>(ksrc + 16 * S) : make_float4(0.f, 0.f, 0.f, 0.f);
-                mma_f64_884(acc, a[4 * S + 0], (double)kv.x);
-                mma_f64_884(acc, a[4 * S + 1], (double)kv.y);
-                mma_f64_884(acc, a[4 * S + 2], (double)kv.z);
-                mma_f64_884(acc, a[4 * S + 3], (double)kv.w);
+            for (int u = 0; u < 2; ++u) {
+                const int cube = c0 + u * 64 + rq;
+                const float* ksrc = kbase + (size_t)(cube < g.N ? cube : 0) * D + 4 * kq;
+#pragma unroll
+                for (int S = 0; S < D / 16; ++S)
+                    kv[u][S] = cube < g.N ? *reinterpret_cast<const float4*>(ksrc + 16 * S) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
-            if (rq < rpp) {   // C fragment: row = lane/4, columns 2*(lane%4) + {0,1}
-                logit[(size_t)rq * g.N_ld + c0 + 2 * kq] = acc[0] * g.scale_d;
-                logit[(size_t)rq * g.N_ld + c0 + 2 * kq + 1] = acc[1] * g.scale_d;
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                if (c0 + u * 64 >= g.N_ld) break;
+                double acc[2] = {0.0, 0.0};
+#pragma unroll
+                for (int S = 0; S < D / 16; ++S) {
+                    mma_f64_884(acc, a[4 * S + 0], (double)kv[u][S].x);
+                    mma_f64_884(acc, a[4 * S + 1], (double)kv[u][S].y);
+                    mma_f64_884(acc, a[4 * S + 2], (double)kv[u][S].z);
+                    mma_f64_884(acc, a[4 * S + 3], (double)kv[u][S].w);
+                }
+                if (rq < rpp) {   // C fragment: row = lane/4, columns 2*(lane%4) + {0,1}
+                    logit[(size_t)rq * g.N_ld + c0 + u * 64 + 2 * kq] = acc[0] * g.scale_d;
+                    logit[(size_t)rq * g.N_ld + c0 + u * 64 + 2 * kq + 1] = acc[1] * g.scale_d;
+                }
             }
         }
         __syncthreads();
@@ -122,6 +134,13 @@ __global__ void __launch_bounds__(256) decode_select_plan_kernel(
     }
 
     // ---- plan: blocks that hold a selected cube of any head of the group, plus the text blocks
+    // (first the union of the group's bitmaps, written over the first head's row)
+    for (int w = threadIdx.x; w < g.n_words; w += blockDim.x) {
+        uint32_t u = 0;
+        for (int i = 0; i < g.G; ++i) u |= bm[i * g.n_words + w];
+        bm[w] = u;
+    }
+    __syncthreads();
     if (warp != 0) return;
     const int tl = text_len[b];
     const int last_pos = g.S_v + tl;                     // position of the new token
@@ -139,9 +158,7 @@ __global__ void __launch_bounds__(256) decode_select_plan_kernel(
                 int c_hi = min((kb * kBlockTok + kBlockTok - 1) >> g.c_shift, g.N - 1);
                 uint32_t span = c_hi - c_lo + 1;
                 uint32_t bits = (span >= 32 ? 0xffffffffu : ((1u << span) - 1u)) << (c_lo & 31);
-                uint32_t u = 0;
-                for (int i = 0; i < g.G; ++i) u |= bm[i * g.n_words + (c_lo >> 5)];
-                if (u & bits) need = true;
+                if (bm[c_lo >> 5] & bits) need = true;
             }
         }
         uint32_t ball = __ballot_sync(0xffffffffu, need);
