@@ -111,6 +111,20 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
+def max_over_ranks(value: float, dist, device) -> float:
+    """The slowest rank's figure (replicas run independently; the job is as slow as its slowest rank)."""
+    if dist is None:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(units_per_rank: float, world: int, ms_max: float) -> float:
+    """Whole-job units per second: every rank processes units_per_rank in the slowest rank's time."""
+    return world * units_per_rank / (ms_max * 1e-3)
+
+
 def timed_steps(step_fn, steps, warmup, flush, dist_barrier):
     """W warm-ups, then K steps each bracketed by CUDA events on the current stream, with an L2
     flush (not timed) before every step.  Returns per-step milliseconds."""
@@ -260,12 +274,9 @@ def main():
     launches_per_step = eng.launches()
     hdr = eng.header()
     ms = sum(times) / len(times)
-    ms_t = torch.tensor([ms], device="cuda")
-    if dist is not None:
-        dist.all_reduce(ms_t, op=dist.ReduceOp.MAX)
-    ms_max = float(ms_t.item())
+    ms_max = max_over_ranks(ms, dist, "cuda")
     tokens = wl.B * wl.S
-    value = world * tokens / (ms_max * 1e-3)
+    value = job_throughput(tokens, world, ms_max)
 
     # selection statistics -> useful FLOPs (4 * D * sum over rows of attended keys)
     _, bitmap, count = eng.forward(q, k, v, wl.n_text, out=out, want_selection=True)
@@ -294,10 +305,7 @@ def main():
 
     e2e_times, _ = timed_steps(e2e_step, max(3, args.steps // 2), 3, flush, barrier)
     e2e_ms = sum(e2e_times) / len(e2e_times)
-    e2e_t = torch.tensor([e2e_ms], device="cuda")
-    if dist is not None:
-        dist.all_reduce(e2e_t, op=dist.ReduceOp.MAX)
-    e2e_value = world * tokens / (float(e2e_t.item()) * 1e-3)
+    e2e_value = job_throughput(tokens, world, max_over_ranks(e2e_ms, dist, "cuda"))
     h2d = q_h.numel() * 2 + k_h.numel() * 2 + v_h.numel() * 2
     d2h = out_h.numel() * 2
 
@@ -407,10 +415,7 @@ def main():
 
         d_times, d_stages = timed_steps(dstep, args.steps, args.warmup, flush, barrier)
         d_ms = sum(d_times) / len(d_times)
-        d_t = torch.tensor([d_ms], device="cuda")
-        if dist is not None:
-            dist.all_reduce(d_t, op=dist.ReduceOp.MAX)
-        d_ms = float(d_t.item())
+        d_ms = max_over_ranks(d_ms, dist, "cuda")
         hd = engd.header()
         gathered = float(hd.decode_kv_blocks) * 2 * 64 * wd.D * 2
         keys_bytes = wd.B * wd.Hkv * wd.N * wd.D * 4
