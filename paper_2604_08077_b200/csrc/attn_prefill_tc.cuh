@@ -107,6 +107,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
             tc::prefetch_tensormap(&tmV);
         }
     }
+    __syncthreads();                                            // barriers initialised
+    if (warp == 8 && lane == 0) {
+        // the Q tiles do not depend on the block plan: their load overlaps the union computation below
+        const int q_row0 = (b * g.Hq + h) * g.S_cap + pair_pos0;
+        tc::mbar_arrive_expect_tx(&sm.q_full, kQBytes);
+        for (int t = 0; t < 2; ++t)
+            for (int p = 0; p < kPanels; ++p) tc::tma_load_2d(&sm.q[t][p][0][0], &tmQ, p * 64, q_row0 + t * 128, &sm.q_full);
+    }
     // union of the selection words of the 256 rows (two 128-row tiles of the mask matrix)
     for (int w = warp; w < g.n_words; w += kTcThreads / 32) {
         uint32_t u = 0;
@@ -155,12 +163,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     if (warp == 8) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            const int q_row0 = (b * g.Hq + h) * g.S_cap + pair_pos0;
             const int kv_row0 = (b * g.Hkv + gk) * g.S_cap;
             const int v_row0 = (b * g.Hkv + gk) * g.n_kv_blocks_cap * D;
-            tc::mbar_arrive_expect_tx(&sm.q_full, kQBytes);
-            for (int t = 0; t < 2; ++t)
-                for (int p = 0; p < kPanels; ++p) tc::tma_load_2d(&sm.q[t][p][0][0], &tmQ, p * 64, q_row0 + t * 128, &sm.q_full);
             BlockIter it(sm.blk_words);
             for (int j = 0; j < n_steps; ++j) {
                 const int st = j & 1, u = j >> 1;
