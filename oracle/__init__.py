@@ -28,7 +28,7 @@ class Shape(ctypes.Structure):
                 ("W", ctypes.c_int32), ("ct", ctypes.c_int32), ("ch", ctypes.c_int32),
                 ("cw", ctypes.c_int32), ("n_text", ctypes.c_int32), ("Hq", ctypes.c_int32),
                 ("Hkv", ctypes.c_int32), ("D", ctypes.c_int32), ("top_p", ctypes.c_double),
-                ("scale", ctypes.c_double)]
+                ("scale", ctypes.c_double), ("top_k", ctypes.c_int32)]
 
     @property
     def N(self) -> int:
@@ -65,7 +65,7 @@ def lib() -> ctypes.CDLL:
         _lib.adas_oracle_select_row.restype = ctypes.c_int64
         _lib.adas_oracle_select_row.argtypes = [
             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_double,
-            ctypes.c_double, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+            ctypes.c_double, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
     return _lib
 
 
@@ -75,16 +75,18 @@ def n_threads() -> int:
     return int(env) if env else (os.cpu_count() or 1)
 
 
-def make_shape(*, B, T, H, W, cube, n_text, Hq, Hkv, D, top_p, scale: Optional[float] = None) -> Shape:
+def make_shape(*, B, T, H, W, cube, n_text, Hq, Hkv, D, top_p, scale: Optional[float] = None,
+               top_k: int = 0) -> Shape:
     ct, ch, cw = cube
     return Shape(B, T, H, W, ct, ch, cw, n_text, Hq, Hkv, D, float(top_p),
-                 float(scale) if scale else 1.0 / float(np.sqrt(D)))
+                 float(scale) if scale else 1.0 / float(np.sqrt(D)), int(top_k))
 
 
-def shape_of(wl, top_p: Optional[float] = None) -> Shape:
+def shape_of(wl, top_p: Optional[float] = None, top_k: Optional[int] = None) -> Shape:
     """Shape of a ``paper_2604_08077_b200.inputs.Workload`` (duck-typed; no import)."""
     return make_shape(B=wl.B, T=wl.T, H=wl.H, W=wl.W, cube=wl.cube, n_text=wl.n_text, Hq=wl.Hq,
-                      Hkv=wl.Hkv, D=wl.D, top_p=wl.top_p if top_p is None else top_p)
+                      Hkv=wl.Hkv, D=wl.D, top_p=wl.top_p if top_p is None else top_p,
+                      top_k=getattr(wl, "top_k", 0) if top_k is None else top_k)
 
 
 def as_f32(t) -> np.ndarray:
@@ -116,7 +118,7 @@ def mean_keys(shape: Shape, k: np.ndarray) -> np.ndarray:
     return kbar
 
 
-def select_row(q: np.ndarray, kbar_g: np.ndarray, n_cand: int, scale: float, top_p: float):
+def select_row(q: np.ndarray, kbar_g: np.ndarray, n_cand: int, scale: float, top_p: float, top_k: int = 0):
     """One row of O3+O4.  Returns (sel uint8[n_cand], probs float64[n_cand], margin)."""
     q = as_f32(q)
     kbar_g = np.ascontiguousarray(kbar_g, np.float64)
@@ -124,7 +126,7 @@ def select_row(q: np.ndarray, kbar_g: np.ndarray, n_cand: int, scale: float, top
     sel = np.zeros(max(n_cand, 1), np.uint8)
     probs = np.zeros(max(n_cand, 1), np.float64)
     margin = ctypes.c_double(0.0)
-    lib().adas_oracle_select_row(_p(q), _p(kbar_g), n_cand, D, float(scale), float(top_p),
+    lib().adas_oracle_select_row(_p(q), _p(kbar_g), n_cand, D, float(scale), float(top_p), int(top_k),
                                  _p(sel), _p(probs), ctypes.addressof(margin))
     return sel[:n_cand], probs[:n_cand], margin.value
 
@@ -189,7 +191,7 @@ def decode(shape: Shape, k_cache, v_cache, text_len: Sequence[int], q_new, k_new
     for b in idx:
         tl = int(text_len[b])
         s1 = Shape(1, shape.T, shape.H, shape.W, shape.ct, shape.ch, shape.cw, tl + 1, shape.Hq,
-                   shape.Hkv, shape.D, shape.top_p, shape.scale)
+                   shape.Hkv, shape.D, shape.top_p, shape.scale, shape.top_k)
         Sv = shape.S_v
         k1 = np.concatenate([k_cache[b, :Sv + tl], k_new[b]], axis=0)[None]
         v1 = np.concatenate([v_cache[b, :Sv + tl], v_new[b]], axis=0)[None]

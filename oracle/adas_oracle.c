@@ -9,6 +9,8 @@
  *   O2  mean key per cube and KV head            Sec. 3.2, text under Eq. 1
  *   O3  selection scores + softmax over cubes    Eq. 1
  *   O4  nucleus (Top-p) cube selection           Eq. 2
+ *   O4k Top-K cube selection (the fixed-budget rule the paper compares Top-p with in its
+ *       selection-strategy ablation): the K most probable candidate cubes
  *   O5  attention over selected cubes + own-cube Eq. 3 and the text-token rule that follows it
  *       prefix (video) or text prefix (text)
  *   O6  decode = a text-rule row appended after the cached sequence (same code as O5)
@@ -45,6 +47,7 @@ typedef struct {
     int32_t Hq, Hkv, D;      /* query heads, KV heads, head dim                       */
     double top_p;            /* nucleus mass p                                        */
     double scale;            /* logit scale, 1/sqrt(D) in the paper                   */
+    int32_t top_k;           /* > 0: keep the K most probable cubes instead of Top-p  */
 } adas_shape;
 
 static int64_t n_cubes(const adas_shape *s) {
@@ -109,9 +112,11 @@ static int by_prob_desc_then_index(const void *a, const void *b) {
  * Outputs: sel[j] in {0,1} for j < n_cand (caller zeroes beyond), returns |S|.
  *   probs   (nullable) [n_cand] the softmax P
  *   margin  (nullable) tie margin of the row: min(|c_k* - p|, |c_(k*-1) - p|,
- *           p_(k*) - p_(k*+1)); +inf when nothing can tie (no candidates, or p >= 1). */
+ *           p_(k*) - p_(k*+1)); +inf when nothing can tie (no candidates, or p >= 1).
+ *   top_k   > 0: Top-K rule instead of Eq. 2: the first min(K, n_cand) cubes of the same order
+ *           (probability descending, index ascending); margin = p_(K) - p_(K+1). */
 int64_t adas_oracle_select_row(const float *q, const double *kbar_g, int64_t n_cand, int64_t D,
-                               double scale, double top_p, uint8_t *sel, double *probs,
+                               double scale, double top_p, int64_t top_k, uint8_t *sel, double *probs,
                                double *margin) {
     if (margin) *margin = INFINITY;
     if (n_cand <= 0) return 0;
@@ -136,7 +141,10 @@ int64_t adas_oracle_select_row(const float *q, const double *kbar_g, int64_t n_c
     qsort(order, (size_t)n_cand, sizeof(prob_idx), by_prob_desc_then_index);
     int64_t kstar = n_cand;
     double cum = 0.0, cum_before = 0.0;
-    if (top_p < 1.0) {
+    if (top_k > 0) {
+        kstar = top_k < n_cand ? top_k : n_cand;
+        if (margin && kstar < n_cand) *margin = order[kstar - 1].p - order[kstar].p;
+    } else if (top_p < 1.0) {
         for (int64_t k = 0; k < n_cand; ++k) {
             double before = cum;
             cum += order[k].p;
@@ -229,7 +237,7 @@ void adas_oracle_rows(const adas_shape *s, const float *Q, const float *K, const
         const double *kbar_g = kbar + ((b * s->Hkv + h / G) * N) * D;
         uint8_t *sel_i = sel + i * N;
         memset(sel_i, 0, (size_t)N);
-        int64_t cnt = adas_oracle_select_row(q, kbar_g, n_cand, D, s->scale, s->top_p, sel_i,
+        int64_t cnt = adas_oracle_select_row(q, kbar_g, n_cand, D, s->scale, s->top_p, s->top_k, sel_i,
                                              NULL, margin ? margin + i : NULL);
         count[i] = (int32_t)cnt;
         if (n_attended)

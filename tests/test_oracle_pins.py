@@ -340,3 +340,57 @@ def test_decode_is_a_text_row_of_the_appended_sequence():
             w = np.exp(s - s.max())
             w /= w.sum()
             np.testing.assert_allclose(res["out"][b, h], w @ vs[toks, g], rtol=1e-11, atol=1e-14)
+
+
+# ------------------------------------------------------------------ O4k: Top-K rule
+@pytest.mark.parametrize("w,k,expected", [
+    ([1, 5, 3, 2], 1, [1]),                 # K = 1 is the argmax cube
+    ([1, 5, 3, 2], 2, [1, 2]),
+    ([1, 5, 3, 2], 3, [1, 2, 3]),
+    ([1, 5, 3, 2], 4, [0, 1, 2, 3]),
+    ([1, 5, 3, 2], 9, [0, 1, 2, 3]),        # K beyond the candidate count keeps every candidate
+    ([2, 2, 2, 1], 2, [0, 1]),              # equal probabilities: lower cube index first
+    ([1, 2, 2, 2], 2, [1, 2]),
+])
+def test_top_k_closed_form(w, k, expected):
+    q = np.array([2, 0, 0, 0], np.float32)
+    kbar = np.zeros((len(w), 4))
+    kbar[:, 0] = np.log(w)
+    sel, probs, _ = oracle.select_row(q, kbar, len(w), 0.5, 0.9, top_k=k)
+    np.testing.assert_allclose(probs, np.array(w) / np.sum(w), rtol=1e-14)
+    assert np.flatnonzero(sel).tolist() == expected
+
+
+def test_top_k_brute_force_and_margin():
+    """On random rows the Top-K set is the subset of size min(K, n) with the largest total mass
+    (checked against every subset of that size), and the margin is the gap to the next cube."""
+    rng = np.random.default_rng(3)
+    for trial in range(40):
+        n, D = int(rng.integers(1, 11)), 8
+        k = int(rng.integers(1, 13))
+        q = rng.standard_normal(D).astype(np.float32)
+        kbar = rng.standard_normal((n, D)) * 2.0
+        sel, probs, margin = oracle.select_row(q, kbar, n, 1.0 / np.sqrt(D), 0.9, top_k=k)
+        size = min(k, n)
+        assert sel.sum() == size
+        best = max(sum(probs[list(c)]) for c in itertools.combinations(range(n), size))
+        assert abs(probs[sel.astype(bool)].sum() - best) < 1e-15
+        srt = np.sort(probs)[::-1]
+        if size < n:
+            assert abs(margin - (srt[size - 1] - srt[size])) < 1e-15
+        else:
+            assert np.isinf(margin)
+
+
+def test_top_k_rows_use_the_rule_inside_the_full_path():
+    """oracle.rows with top_k set: every row keeps min(K, candidates) cubes, and the attention over
+    them equals attend_given with that selection."""
+    wl = inputs.small_prefill(seed=51, T=8, H=8, W=8, n_text=6)
+    sh = oracle.shape_of(wl, top_k=3)
+    rows = oracle.all_rows(sh)[::7]
+    res = oracle.rows(sh, wl.q, wl.k, wl.v, rows)
+    pos, _ = oracle.positions(sh)
+    n_cand = np.where(rows[:, 2] < wl.S_v, pos[rows[:, 2]] // wl.C, wl.N)
+    assert np.array_equal(res["count"], np.minimum(n_cand, 3))
+    out2 = oracle.attend_given(sh, wl.q, wl.k, wl.v, rows, res["sel"])
+    np.testing.assert_allclose(res["out"], out2, rtol=0, atol=1e-15)
