@@ -57,6 +57,10 @@ typedef struct {
     float top_p;                    /* in (0, 1]; >= 1 selects every candidate cube (dense)    */
     float softmax_scale;            /* 0 => 1/sqrt(head_dim) (Eqs. 1, 3); used for both        */
     int32_t device;                 /* CUDA ordinal                                            */
+    int32_t top_k;                  /* 0: Top-p (Eq. 2).  > 0: keep the top_k most probable
+                                       candidate cubes instead (all of them if fewer exist), the
+                                       fixed-budget rule of the paper's selection ablation;
+                                       top_p is then ignored                                    */
 } adaspark_attn_config_t;
 
 /* Sizes fixed by _partition.  "pos" below is the cube-major position of a token:
@@ -88,7 +92,7 @@ typedef struct {
 /* Create a handle for one configuration.  Host only.  Fails with ERR_UNSUPPORTED for a
  * head_dim other than 64/128, a cube window whose token count C is not one of
  * {16, 32, 64, 128, 256, 512}, or a GQA group size above 16; with ERR_INVALID_ARG for
- * non-positive sizes, top_p <= 0, or a NULL pointer. */
+ * non-positive sizes, top_p <= 0, top_k < 0, or a NULL pointer. */
 adaspark_status_t adaspark_attn_create(const adaspark_attn_config_t *config,
                                        adaspark_attn_t **out_handle);
 

@@ -25,7 +25,7 @@ class Config(ctypes.Structure):
     _fields_ = [("cube_t", ctypes.c_int32), ("cube_h", ctypes.c_int32), ("cube_w", ctypes.c_int32),
                 ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
                 ("head_dim", ctypes.c_int32), ("top_p", ctypes.c_float),
-                ("softmax_scale", ctypes.c_float), ("device", ctypes.c_int32)]
+                ("softmax_scale", ctypes.c_float), ("device", ctypes.c_int32), ("top_k", ctypes.c_int32)]
 
 
 class Layout(ctypes.Structure):
@@ -212,9 +212,9 @@ class AdaSAttn:
     """Owns a handle plus the torch-allocated caches and workspace for one partition."""
 
     def __init__(self, *, cube, n_q_heads, n_kv_heads, head_dim, top_p, softmax_scale=0.0,
-                 device: int = 0):
+                 device: int = 0, top_k: int = 0):
         self.cfg = Config(cube[0], cube[1], cube[2], n_q_heads, n_kv_heads, head_dim, float(top_p),
-                          float(softmax_scale), device)
+                          float(softmax_scale), device, int(top_k))
         self.handle = adaspark_attn_create(self.cfg)
         self.device = torch.device("cuda", device)
         self.layout: Optional[Layout] = None

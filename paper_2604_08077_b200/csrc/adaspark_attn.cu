@@ -97,6 +97,7 @@ Geom make_geom(const adaspark_attn* h, int n_text) {
     g.scale = (float)scale;
     g.scale_log2 = (float)(scale * 1.4426950408889634);
     g.top_p = (double)h->cfg.top_p;
+    g.top_k = h->cfg.top_k;
     return g;
 }
 
@@ -137,7 +138,7 @@ adaspark_status_t adaspark_attn_create(const adaspark_attn_config_t* config, ada
     *out_handle = nullptr;
     if (config->cube_t <= 0 || config->cube_h <= 0 || config->cube_w <= 0 || config->n_q_heads <= 0 ||
         config->n_kv_heads <= 0 || config->head_dim <= 0 || !(config->top_p > 0.f) ||
-        config->softmax_scale < 0.f || config->device < 0)
+        config->softmax_scale < 0.f || config->device < 0 || config->top_k < 0)
         return ADASPARK_ERR_INVALID_ARG;
     if (config->n_q_heads % config->n_kv_heads != 0) return ADASPARK_ERR_INVALID_ARG;
     if (config->head_dim != 64 && config->head_dim != 128) return ADASPARK_ERR_UNSUPPORTED;

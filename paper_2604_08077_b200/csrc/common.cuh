@@ -55,6 +55,7 @@ struct Geom {
     float scale_log2;    // scale * log2(e)
     double scale_d;      // logit scale in double (selection scores)
     double top_p;
+    int top_k;           // > 0: Top-K rule instead of Top-p
 };
 
 // O1 inverse: cube-major position -> raster token index.

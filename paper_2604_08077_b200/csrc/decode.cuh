@@ -114,10 +114,10 @@ __global__ void __launch_bounds__(256) decode_select_plan_kernel(
             unsigned long long* keys = reinterpret_cast<unsigned long long*>(row);
             const int n = g.N;
             unsigned long long bd = 0ull;
-            const bool all = !(g.top_p < 1.0);
+            const bool all = g.top_k <= 0 && !(g.top_p < 1.0);
             if (!all) {
                 unsigned long long* hist = sel_scratch + (size_t)warp * (kSelHistWords + kDecodeCandCap);
-                bd = nucleus_boundary_radix<32, true>(row, n, g.top_p, keys, hist, hist + kSelHistWords, kDecodeCandCap, lane);
+                bd = nucleus_boundary_radix<32, true>(row, n, g.top_p, g.top_k, keys, hist, hist + kSelHistWords, kDecodeCandCap, lane);
             }
             for (int w = 0; w < g.n_words; ++w) {
                 int j = w * 32 + lane;

@@ -146,9 +146,9 @@ __global__ void __launch_bounds__(kSelectWarps * 32) select_kernel(Geom g, int g
     unsigned long long* keys = kInPlace ? reinterpret_cast<unsigned long long*>(s) : hist + kSelHistWords + (size_t)gi * g.N_ld;
 
     const int n = pos < g.S ? n_candidates(g, pos) : 0;
-    const bool all = !(g.top_p < 1.0);
+    const bool all = g.top_k <= 0 && !(g.top_p < 1.0);
     unsigned long long bd = 0ull;                    // 0: every candidate is selected
-    if (!all) bd = nucleus_boundary_radix<G, kInPlace>(s, n, g.top_p, keys, hist, cand, cand_cap, lane);
+    if (!all) bd = nucleus_boundary_radix<G, kInPlace>(s, n, g.top_p, g.top_k, keys, hist, cand, cand_cap, lane);
 
     const bool extra = (sel_bitmap != nullptr || sel_count != nullptr) && pos < g.S;
     const int raster = extra ? pos_to_raster(g, pos) : 0;

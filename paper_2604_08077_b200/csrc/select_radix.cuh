@@ -154,11 +154,12 @@ __device__ __forceinline__ unsigned long long group_sum_u64(unsigned long long x
 // Boundary key of each group's row.  On entry keys[0..n) of the group hold its order keys and the
 // group's columns of `hist` hold the first-level histogram (half-octave buckets, top = 63);
 // `target` = T.  `cand` is the group's scratch list of `cand_cap` entries.  A group with n = 0
-// takes part in the collectives and returns 0.
+// takes part in the collectives and returns 0.  by_count: every key weighs 1 instead of its mass (the
+// histogram then counts keys and `target` is a rank: the Top-K rule).
 template <int G>
 __device__ unsigned long long radix_boundary(const unsigned long long* keys, int n, unsigned long long target,
                                              unsigned long long* hist, unsigned long long* cand, int cand_cap,
-                                             int lane) {
+                                             int lane, bool by_count) {
     constexpr int kOwn = SelGeom<G>::kOwn;
     const int gl = lane & (G - 1), gbase = lane & ~(G - 1);
     const uint32_t gmask = G == 32 ? 0xffffffffu : (((1u << G) - 1u) << gbase);
@@ -201,7 +202,7 @@ __device__ unsigned long long radix_boundary(const unsigned long long* keys, int
                 const unsigned long long k = src[i];
                 if (k >= lo && k <= hi) {
                     const int b = octave_split ? octave_bucket_of(top, k) : 31 - (int)((k >> shift) & 31ull);
-                    hist[hist_index<G>(b, lane)] += k >> 13;
+                    hist[hist_index<G>(b, lane)] += by_count ? 1ull : (k >> 13);
                 }
             }
         }
@@ -237,7 +238,7 @@ __device__ unsigned long long radix_boundary(const unsigned long long* keys, int
     const int cmax = __reduce_max_sync(0xffffffffu, count <= 32 ? count : 0);
     for (int e = 0; e < cmax; ++e) {
         const unsigned long long other = e < count ? cand[e] : 0ull;
-        const unsigned long long om = other >> 13;
+        const unsigned long long om = by_count ? (other != 0ull ? 1ull : 0ull) : (other >> 13);
 #pragma unroll
         for (int sl = 0; sl < kOwn; ++sl)
             if (other >= mine[sl]) acc[sl] += om;
@@ -256,15 +257,17 @@ __device__ unsigned long long radix_boundary(const unsigned long long* keys, int
 
 // Builds the order keys of the group's row from its scaled scores s[0..n) (fp64), fills the
 // first-level histogram and returns the boundary key: cube j is selected iff keys[j] >= boundary.
-// A group with n = 0 (no candidates, or nothing to search) returns 0.  Requires p < 1.
+// A group with n = 0 (no candidates, or nothing to search) returns 0.  Requires p < 1 or top_k > 0
+// (top_k > 0 selects the min(top_k, n) first keys of the order instead of the nucleus).
 // hist: kSelHistWords entries shared by the warp (zeroed here); keys / cand: the group's own.
 // keys may be the score row itself (kInPlace: every score is replaced by its key, e.g. a row of the
 // L2-resident score buffer) or separate storage (shared memory for short rows).
 template <int G, bool kInPlace>
-__device__ unsigned long long nucleus_boundary_radix(const double* s, int n, double top_p,
+__device__ unsigned long long nucleus_boundary_radix(const double* s, int n, double top_p, int top_k,
                                                      unsigned long long* keys, unsigned long long* hist,
                                                      unsigned long long* cand, int cand_cap, int lane) {
     const int gl = lane & (G - 1);
+    const bool by_count = top_k > 0;
     zero_hist(hist, lane);
     double* sd = reinterpret_cast<double*>(keys);
     double mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
@@ -302,21 +305,23 @@ __device__ unsigned long long nucleus_boundary_radix(const double* s, int n, dou
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             keys[j + u * G] = k[u];
-            hist[hist_index<G>(b[u], lane)] += m[u];
-            z += m[u];
+            hist[hist_index<G>(b[u], lane)] += by_count ? 1ull : m[u];
+            z += by_count ? 1ull : m[u];
         }
     }
     for (; j < n; j += G) {
         unsigned long long m;
         int b;
         keys[j] = make_key(sd[j], j, m, b);
-        hist[hist_index<G>(b, lane)] += m;
-        z += m;
+        hist[hist_index<G>(b, lane)] += by_count ? 1ull : m;
+        z += by_count ? 1ull : m;
     }
     z = group_sum_u64<G>(z);
     __syncwarp();
-    const unsigned long long target = (unsigned long long)ceil((double)z * top_p);
-    return radix_boundary<G>(keys, n, target, hist, cand, cand_cap, lane);
+    // Top-p: mass target ceil(p * Z);  Top-K: the K-th key of the order (all of them if fewer exist)
+    const unsigned long long target = by_count ? (z < (unsigned long long)top_k ? z : (unsigned long long)top_k)
+                                               : (unsigned long long)ceil((double)z * top_p);
+    return radix_boundary<G>(keys, n, target, hist, cand, cand_cap, lane, by_count);
 }
 
 }  // namespace adaspark

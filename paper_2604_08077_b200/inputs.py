@@ -38,6 +38,7 @@ class Workload:
     Hkv: int
     D: int
     top_p: float
+    top_k: int = 0  # > 0: Top-K selection instead of Top-p
     q: Optional[torch.Tensor] = None  # bf16 [B, S, Hq, D]   (None for cache-only workloads)
     k: Optional[torch.Tensor] = None  # bf16 [B, S, Hkv, D]
     v: Optional[torch.Tensor] = None  # bf16 [B, S, Hkv, D]

@@ -15,7 +15,7 @@ TIE_MARGIN = 1e-6        # rows whose cumulative-probability margin is below thi
 
 def make_engine(wl, n_text_max=None, top_p=None, prefill_kernel=None):
     eng = binding.AdaSAttn(cube=wl.cube, n_q_heads=wl.Hq, n_kv_heads=wl.Hkv, head_dim=wl.D,
-                           top_p=wl.top_p if top_p is None else top_p)
+                           top_p=wl.top_p if top_p is None else top_p, top_k=getattr(wl, "top_k", 0))
     eng.partition(wl.B, wl.T, wl.H, wl.W, wl.n_text if n_text_max is None else n_text_max)
     if prefill_kernel is not None:
         binding.adaspark_attn_set_prefill_kernel(eng.handle, prefill_kernel)

@@ -20,7 +20,7 @@ def lib():
 
 def cfg(**kw):
     base = dict(cube_t=4, cube_h=4, cube_w=4, n_q_heads=28, n_kv_heads=4, head_dim=128, top_p=0.9,
-                softmax_scale=0.0, device=0)
+                softmax_scale=0.0, device=0, top_k=0)
     base.update(kw)
     return binding.Config(*[base[f[0]] for f in binding.Config._fields_])
 
@@ -48,6 +48,7 @@ def test_create_validation(lib):
                       (dict(n_q_heads=30), binding.ERR_INVALID_ARG),      # 30 % 4 != 0
                       (dict(n_q_heads=68, n_kv_heads=4), binding.ERR_UNSUPPORTED),  # group 17
                       (dict(top_p=0.0), binding.ERR_INVALID_ARG),
+                      (dict(top_k=-1), binding.ERR_INVALID_ARG),
                       (dict(cube_h=0), binding.ERR_INVALID_ARG)]:
         c = cfg(**bad)
         assert lib.adaspark_attn_create(ctypes.byref(c), ctypes.byref(h)) == code, bad
