@@ -91,7 +91,7 @@ typedef struct {
 
 /* Create a handle for one configuration.  Host only.  Fails with ERR_UNSUPPORTED for a
  * head_dim other than 64/128, a cube window whose token count C is not one of
- * {16, 32, 64, 128, 256, 512}, or a GQA group size above 16; with ERR_INVALID_ARG for
+ * {16, 32, 64, 128, 256, 512, 1024}, or a GQA group size above 16; with ERR_INVALID_ARG for
  * non-positive sizes, top_p <= 0, top_k < 0, or a NULL pointer. */
 adaspark_status_t adaspark_attn_create(const adaspark_attn_config_t *config,
                                        adaspark_attn_t **out_handle);

@@ -144,7 +144,7 @@ adaspark_status_t adaspark_attn_create(const adaspark_attn_config_t* config, ada
     if (config->head_dim != 64 && config->head_dim != 128) return ADASPARK_ERR_UNSUPPORTED;
     if (config->n_q_heads / config->n_kv_heads > 16) return ADASPARK_ERR_UNSUPPORTED;
     long long C = (long long)config->cube_t * config->cube_h * config->cube_w;
-    if (C != 16 && C != 32 && C != 64 && C != 128 && C != 256 && C != 512) return ADASPARK_ERR_UNSUPPORTED;
+    if (C != 16 && C != 32 && C != 64 && C != 128 && C != 256 && C != 512 && C != 1024) return ADASPARK_ERR_UNSUPPORTED;
     adaspark_attn* h = new (std::nothrow) adaspark_attn();
     if (!h) return ADASPARK_ERR_INVALID_ARG;
     std::memset(h, 0, sizeof(*h));

@@ -41,6 +41,14 @@ SMALL_CASES = {
                                                          n_text=130, Hq=2, Hkv=1, D=64, top_p=0.9),
     "single_cube": lambda: inputs.small_prefill(seed=11, T=4, H=4, W=4, cube=(4, 4, 4), n_text=3,
                                                 Hq=1, Hkv=1, D=128, top_p=0.9),
+    # the paper's cube-size ablation runs from 64 to 1024 tokens per cube; 1x1x64 and 8x8x1 are its
+    # temporal-only and spatial-only shapes
+    "c1024": lambda: inputs.small_prefill(seed=15, T=16, H=16, W=16, cube=(4, 16, 16), n_text=11, Hq=2,
+                                          Hkv=1, D=128, top_p=0.7),
+    "c64_temporal_only": lambda: inputs.small_prefill(seed=16, T=128, H=2, W=4, cube=(64, 1, 1), n_text=7,
+                                                      Hq=2, Hkv=2, D=64, top_p=0.8),
+    "c64_spatial_only": lambda: inputs.small_prefill(seed=17, T=6, H=16, W=8, cube=(1, 8, 8), n_text=0,
+                                                     Hq=2, Hkv=1, D=128, top_p=0.9),
     "sharp_scores": lambda: inputs.small_prefill(seed=12, T=16, H=8, W=8, n_text=17, top_p=0.5,
                                                  offset_std=3.0),
     # nucleus boundaries far down the tail of a sharp distribution (many octaves below the maximum)
