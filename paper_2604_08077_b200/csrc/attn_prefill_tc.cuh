@@ -115,13 +115,18 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
         for (int t = 0; t < 2; ++t)
             for (int p = 0; p < kPanels; ++p) tc::tma_load_2d(&sm.q[t][p][0][0], &tmQ, p * 64, q_row0 + t * 128, &sm.q_full);
     }
-    // union of the selection words of the 256 rows (two 128-row tiles of the mask matrix)
+    // union of the selection words of the 256 rows (two 128-row tiles of the mask matrix): the eight
+    // loads of a lane are issued together
     for (int w = warp; w < g.n_words; w += kTcThreads / 32) {
-        uint32_t u = 0;
-        for (int r = lane; r < kPairRows; r += 32) {
-            int tile = pair * 2 + (r >> 7);
-            if (tile < g.n_tiles) u |= tile_mask[mask_index(g, b, h, tile, w, r & 127)];
+        uint32_t v[kPairRows / 32];
+#pragma unroll
+        for (int i = 0; i < kPairRows / 32; ++i) {
+            const int r = lane + 32 * i, tile = pair * 2 + (r >> 7);
+            v[i] = tile < g.n_tiles ? __ldg(tile_mask + mask_index(g, b, h, tile, w, r & 127)) : 0u;
         }
+        uint32_t u = 0;
+#pragma unroll
+        for (int i = 0; i < kPairRows / 32; ++i) u |= v[i];
         u = __reduce_or_sync(0xffffffffu, u);
         if (lane == 0) sm.union_words[w] = u;
     }
@@ -132,17 +137,21 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     const int n_blk_words = (n_blk + 31) / 32;
     for (int wi = tid; wi < n_blk_words; wi += kTcThreads) {
         uint32_t bits = 0;
-        for (int i = 0; i < 32; ++i) {
-            int kb = wi * 32 + i;
-            if (kb >= n_blk) break;
-            bool need = kb >= first_local_blk;
-            if (!need) {
-                int c_lo = (kb * kBlockTok) >> g.c_shift, c_hi = (kb * kBlockTok + kBlockTok - 1) >> g.c_shift;
-                uint32_t span = c_hi - c_lo + 1;   // <= 4 cubes, aligned: never crosses a word
-                uint32_t m = (span >= 32 ? 0xffffffffu : ((1u << span) - 1u)) << (c_lo & 31);
-                need = (sm.union_words[c_lo >> 5] & m) != 0;
+        if (g.c_shift == 6 && wi * 32 + 31 < first_local_blk) {
+            bits = sm.union_words[wi];             // 64-token cubes: key block = cube, the word is the union word
+        } else {
+            for (int i = 0; i < 32; ++i) {
+                int kb = wi * 32 + i;
+                if (kb >= n_blk) break;
+                bool need = kb >= first_local_blk;
+                if (!need) {
+                    int c_lo = (kb * kBlockTok) >> g.c_shift, c_hi = (kb * kBlockTok + kBlockTok - 1) >> g.c_shift;
+                    uint32_t span = c_hi - c_lo + 1;   // <= 4 cubes, aligned: never crosses a word
+                    uint32_t m = (span >= 32 ? 0xffffffffu : ((1u << span) - 1u)) << (c_lo & 31);
+                    need = (sm.union_words[c_lo >> 5] & m) != 0;
+                }
+                if (need) bits |= 1u << i;
             }
-            if (need) bits |= 1u << i;
         }
         sm.blk_words[wi] = bits;
     }
@@ -441,19 +450,20 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
             const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
             const bool live = pr < g.S;
             __nv_bfloat16* dst = out + ((size_t)(b * g.S + (live ? pos_to_raster(g, pr) : 0)) * g.Hq + h) * D;
+            uint32_t o[D / 32][32];                                // the whole output row in one round of loads
 #pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
-                uint32_t o[32];
-                tc::tmem_ld_32x32(lane_addr + 128 + c * 32, o);
-                tc::tmem_wait_ld();
-                if (live) {
+            for (int c = 0; c < D / 32; ++c) tc::tmem_ld_32x32(lane_addr + 128 + c * 32, o[c]);
+            tc::tmem_wait_ld();
+            if (live) {
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) {
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         uint4 val;
-                        val.x = pack_bf16x2(__uint_as_float(o[8 * i + 0]) * inv, __uint_as_float(o[8 * i + 1]) * inv);
-                        val.y = pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv, __uint_as_float(o[8 * i + 3]) * inv);
-                        val.z = pack_bf16x2(__uint_as_float(o[8 * i + 4]) * inv, __uint_as_float(o[8 * i + 5]) * inv);
-                        val.w = pack_bf16x2(__uint_as_float(o[8 * i + 6]) * inv, __uint_as_float(o[8 * i + 7]) * inv);
+                        val.x = pack_bf16x2(__uint_as_float(o[c][8 * i + 0]) * inv, __uint_as_float(o[c][8 * i + 1]) * inv);
+                        val.y = pack_bf16x2(__uint_as_float(o[c][8 * i + 2]) * inv, __uint_as_float(o[c][8 * i + 3]) * inv);
+                        val.z = pack_bf16x2(__uint_as_float(o[c][8 * i + 4]) * inv, __uint_as_float(o[c][8 * i + 5]) * inv);
+                        val.w = pack_bf16x2(__uint_as_float(o[c][8 * i + 6]) * inv, __uint_as_float(o[c][8 * i + 7]) * inv);
                         *reinterpret_cast<uint4*>(dst + c * 32 + i * 8) = val;
                     }
                 }
