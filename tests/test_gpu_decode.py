@@ -61,6 +61,16 @@ def test_small_decode(case):
         assert torch.equal(eng.v_cube[b, :, pos // 64, :, pos % 64].cpu(), wl.v_new[b, 0])
 
 
+def test_decode_largest_gqa_group_and_cube_count():
+    """16 query heads per KV head (the largest group the library takes) over 4096 cubes."""
+    wl = inputs.small_decode(seed=44, B=2, T=256, H=16, W=16, cube=(1, 4, 4), n_text=9, Hq=16, Hkv=1, D=64,
+                             top_p=0.85)
+    assert wl.N == 4096
+    text_len = [9, 2]
+    eng, out, bitmap = run_decode(wl, text_len)
+    print(compare_decode(wl, text_len, out, bitmap, label="g16_n4096"))
+
+
 def test_decode_without_append_uses_the_cached_token():
     wl = inputs.small_decode(seed=41)
     text_len = [wl.n_text, wl.n_text - 1]

@@ -74,6 +74,24 @@ def test_cohesive_queries_256_token_cubes():
     _free()
 
 
+def test_maximum_cube_count_and_smallest_cubes():
+    """4096 cubes (the partition limit) of 16 tokens (the smallest cube): 65536 video tokens.  Every
+    64-key block then holds four cubes, so the attention kernel's per-chunk masks are mixed almost
+    everywhere, and the selection runs on the longest rows the library accepts."""
+    wl = inputs.make_prefill("n4096_c16", seed=77, B=1, T=256, H=16, W=16, cube=(1, 4, 4), n_text=33,
+                             Hq=4, Hkv=2, D=128, top_p=0.8, offset_std=1.5)
+    assert wl.N == 4096
+    eng, out, bitmap, count = pu.run_forward(wl)
+    n_tiles = (wl.S + 127) // 128
+    rows = pu.sample_rows(wl, 300, seed=8, whole_tiles=[(0, 0, 3), (0, 3, n_tiles - 1)])
+    rep = pu.compare_rows(wl, rows, out, bitmap, count, label="n4096")
+    print("n4096", rep)
+    print("n4096 selection", _selection_sample(wl, bitmap, 6000, seed=88))
+    assert eng.header().status == 0
+    del eng, out, bitmap, count
+    _free()
+
+
 def test_config4_full_size_sampled_rows():
     """Config 4 (131072 video tokens in 2048 cubes, half of the frames static, no text)."""
     wl = inputs.config4()
