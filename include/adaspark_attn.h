@@ -100,7 +100,10 @@ adaspark_status_t adaspark_attn_create(const adaspark_attn_config_t *config,
  * buffer size.  `batch`, `frames`, `grid_h`, `grid_w` describe the video token grid;
  * `n_text_max` is the largest number of text tokens any later _forward/_decode will hold.
  * `*workspace_bytes` (nullable) receives max(forward, decode) workspace size.  Host only.
- * ERR_UNSUPPORTED if the grid is not divisible by the cube window or N > 4096. */
+ * ERR_UNSUPPORTED if the grid is not divisible by the cube window or N > 4096.
+ * The forward workspace holds two buffers of fp64 cube scores for a chunk of query tiles each
+ * (512 MB each by default, less when the whole problem is smaller); the environment variable
+ * ADASPARK_SCORE_BUFFER_MB, read here, overrides the size of one buffer (1 .. 65536). */
 adaspark_status_t adaspark_attn_partition(adaspark_attn_t *handle, int32_t batch, int32_t frames,
                                           int32_t grid_h, int32_t grid_w, int32_t n_text_max,
                                           size_t *workspace_bytes);
