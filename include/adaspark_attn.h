@@ -202,7 +202,8 @@ int64_t adaspark_attn_last_launch_count(const adaspark_attn_t *handle);
  * caller's stream around their stages.  adaspark_attn_get_stage_times waits for the last
  * recorded event (the only host synchronisation in the library, and only in this call) and
  * returns milliseconds: prefill {re-layout+pooling, scoring+selection, attention, 0};
- * decode {append, scoring+selection+plan, split-KV attention, combine}. */
+ * decode {0, append+scoring+selection+plan, split-KV attention, combine} (the append of the new
+ * token is fused into the selection kernel). */
 adaspark_status_t adaspark_attn_enable_stage_timing(adaspark_attn_t *handle, int32_t enable);
 adaspark_status_t adaspark_attn_get_stage_times(adaspark_attn_t *handle, float *ms_out /* host [4] */);
 

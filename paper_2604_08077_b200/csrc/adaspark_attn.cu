@@ -458,20 +458,16 @@ adaspark_status_t adaspark_attn_decode(adaspark_attn_t* h, const void* q_new, co
     auto* vc = (__nv_bfloat16*)v_cube;
     auto* qn = (const __nv_bfloat16*)q_new;
 
-    if (k_new) {
-        decode_append_kernel<<<g.B, 256, 0, st>>>(g, (const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new, kc, vc, text_len, status);
-        if (!launch_ok(h, "decode_append_kernel")) return ADASPARK_ERR_CUDA;
-    }
     mark(h, 1, st);
     {
         size_t smem = decode_select_smem_bytes(g.N_ld, g.G, g.n_words);
         auto* blocks = (unsigned long long*)&hdr->decode_kv_blocks;
         if (D == 128) {
             if (!set_smem(h, decode_select_plan_kernel<128>, smem, "decode_select_plan_kernel")) return ADASPARK_ERR_CUDA;
-            decode_select_plan_kernel<128><<<dim3(g.Hkv, g.B), 256, smem, st>>>(g, qn, cube_keys, text_len, dec_bitmap, sel_bitmap, items, n_items, blocks);
+            decode_select_plan_kernel<128><<<dim3(g.Hkv, g.B), 256, smem, st>>>(g, qn, (const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new, kc, vc, cube_keys, text_len, dec_bitmap, sel_bitmap, items, n_items, blocks, status);
         } else {
             if (!set_smem(h, decode_select_plan_kernel<64>, smem, "decode_select_plan_kernel")) return ADASPARK_ERR_CUDA;
-            decode_select_plan_kernel<64><<<dim3(g.Hkv, g.B), 256, smem, st>>>(g, qn, cube_keys, text_len, dec_bitmap, sel_bitmap, items, n_items, blocks);
+            decode_select_plan_kernel<64><<<dim3(g.Hkv, g.B), 256, smem, st>>>(g, qn, (const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new, kc, vc, cube_keys, text_len, dec_bitmap, sel_bitmap, items, n_items, blocks, status);
         }
         if (!launch_ok(h, "decode_select_plan_kernel")) return ADASPARK_ERR_CUDA;
     }

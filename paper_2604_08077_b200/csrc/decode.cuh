@@ -1,7 +1,7 @@
 // K5 / K7: decode step = one new text token per sequence (text-token rule after Eq. 3).
 //
-//   decode_append_kernel       append the new token's K / V to the cube-major caches
-//   decode_select_plan_kernel  per (b, kv head): Eq. 1 scores of all heads of the GQA group against
+//   decode_select_plan_kernel  per (b, kv head): appends the new token's K / V to the cube-major caches,
+//                              then Eq. 1 scores of all heads of the GQA group against
 //                              the N cube keys (fp64 tensor op, the cube keys are read once per
 //                              group), Eq. 2 per head, then the list of 64-key blocks to visit =
 //                              blocks holding a cube selected by any head of the group + text blocks
@@ -13,20 +13,21 @@
 
 namespace adaspark {
 
-__global__ void decode_append_kernel(Geom g, const __nv_bfloat16* __restrict__ k_new,
-                                     const __nv_bfloat16* __restrict__ v_new,
-                                     __nv_bfloat16* __restrict__ k_cube, __nv_bfloat16* __restrict__ v_cube,
-                                     const int32_t* __restrict__ text_len, int32_t* __restrict__ status) {
-    const int b = blockIdx.x;
+// Appends the new token's K / V of one (batch, kv head) to the cube-major caches at text slot
+// text_len[b] (the V cache holds every 64-position block transposed).  A slot outside the cache sets
+// status 1 and writes nothing.  Called by all threads of a CTA.
+__device__ __forceinline__ void decode_append(const Geom& g, int b, int gk, const __nv_bfloat16* __restrict__ k_new,
+                                              const __nv_bfloat16* __restrict__ v_new, __nv_bfloat16* __restrict__ k_cube,
+                                              __nv_bfloat16* __restrict__ v_cube, const int32_t* __restrict__ text_len,
+                                              int32_t* __restrict__ status) {
     const int tl = text_len[b];
     if (tl < 0 || g.S_v + tl + 1 > g.S_cap) {
         if (threadIdx.x == 0) atomicExch(status, 1);
         return;
     }
     const int pos = g.S_v + tl, blk = pos / kBlockTok, tok = pos % kBlockTok;
-    for (int idx = threadIdx.x; idx < g.Hkv * g.D; idx += blockDim.x) {
-        int gk = idx / g.D, d = idx - gk * g.D;
-        size_t src = ((size_t)b * g.Hkv + gk) * g.D + d;
+    for (int d = threadIdx.x; d < g.D; d += blockDim.x) {
+        const size_t src = ((size_t)b * g.Hkv + gk) * g.D + d;
         k_cube[((size_t)(b * g.Hkv + gk) * g.S_cap + pos) * g.D + d] = k_new[src];
         v_cube[(((size_t)(b * g.Hkv + gk) * g.n_kv_blocks_cap + blk) * g.D + d) * kBlockTok + tok] = v_new[src];
     }
@@ -49,12 +50,15 @@ __host__ __device__ inline size_t decode_select_smem_bytes(int N_ld, int G, int 
 // items[(b*Hkv+gk) * n_kv_blocks_cap + i] = index of the i-th block to visit.
 template <int D>
 __global__ void __launch_bounds__(256) decode_select_plan_kernel(
-    Geom g, const __nv_bfloat16* __restrict__ q_new, const float* __restrict__ cube_keys,
-    const int32_t* __restrict__ text_len, uint32_t* __restrict__ dec_bitmap, uint32_t* __restrict__ sel_bitmap,
-    int32_t* __restrict__ items, int32_t* __restrict__ n_items, unsigned long long* __restrict__ total_blocks) {
+    Geom g, const __nv_bfloat16* __restrict__ q_new, const __nv_bfloat16* __restrict__ k_new,
+    const __nv_bfloat16* __restrict__ v_new, __nv_bfloat16* __restrict__ k_cube, __nv_bfloat16* __restrict__ v_cube,
+    const float* __restrict__ cube_keys, const int32_t* __restrict__ text_len, uint32_t* __restrict__ dec_bitmap,
+    uint32_t* __restrict__ sel_bitmap, int32_t* __restrict__ items, int32_t* __restrict__ n_items,
+    unsigned long long* __restrict__ total_blocks, int32_t* __restrict__ status) {
     extern __shared__ double dsp_smem[];
     const int gk = blockIdx.x, b = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (k_new != nullptr) decode_append(g, b, gk, k_new, v_new, k_cube, v_cube, text_len, status);   // read by the next kernel
     const int rpp = decode_rows_per_pass(g.N_ld);
     double* logit = dsp_smem;                                              // [rpp][N_ld]
     unsigned long long* sel_scratch = reinterpret_cast<unsigned long long*>(dsp_smem + (size_t)rpp * g.N_ld);   // [rpp][hist + cand]
