@@ -128,3 +128,25 @@ def test_config2_full_size_sampled_rows():
     assert not (diff & (res["margin"] >= pu.TIE_MARGIN)).any()
     print("cfg2 selection rows", len(rows), "tie-exempt", int(diff.sum()),
           "near-tie", int((res["margin"] < pu.TIE_MARGIN).sum()))
+
+
+def test_two_handles_on_two_streams_do_not_interfere():
+    """Two engines with different shapes run interleaved on their own streams (each handle also owns
+    a private side stream): the results equal those of running them one after the other."""
+    wa = inputs.small_prefill(seed=71, T=16, H=8, W=8, n_text=13)
+    wb = inputs.small_prefill(seed=72, T=8, H=16, W=8, cube=(2, 4, 4), n_text=40, Hq=6, Hkv=2, D=64, top_p=0.7)
+    ea, oa, _, _ = pu.run_forward(wa)
+    eb, ob, _, _ = pu.run_forward(wb)
+    sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+    qa, ka, va = wa.q.cuda(), wa.k.cuda(), wa.v.cuda()
+    qb, kb, vb = wb.q.cuda(), wb.k.cuda(), wb.v.cuda()
+    torch.cuda.synchronize()
+    outs = []
+    for _ in range(3):
+        xa, _, _ = ea.forward(qa, ka, va, wa.n_text, stream=sa)
+        xb, _, _ = eb.forward(qb, kb, vb, wb.n_text, stream=sb)
+        outs.append((xa, xb))
+    torch.cuda.synchronize()
+    for xa, xb in outs:
+        assert torch.equal(xa, oa) and torch.equal(xb, ob)
+    assert ea.header().status == 0 and eb.header().status == 0
