@@ -89,6 +89,15 @@ def test_degenerate_p(p):
     print(rep)
 
 
+@pytest.mark.parametrize("case", ["cfg1", "d128_c64_ragged_text", "deep_tail"])
+def test_tcgen05_attention_with_fp64_scoring(case):
+    """Kernel option 2: the tcgen05 attention kernel fed by the fp64 (mma.m8n8k4.f64) scoring kernel."""
+    wl = SMALL_CASES[case]()
+    eng, out, bitmap, count = pu.run_forward(wl, prefill_kernel=2)
+    rep = pu.compare_rows(wl, oracle.all_rows(oracle.shape_of(wl)), out, bitmap, count, label=case)
+    assert rep["rows"] == wl.B * wl.Hq * wl.S
+
+
 def test_cache_only_forward_builds_the_caches():
     wl = inputs.small_prefill(seed=31)
     eng = pu.make_engine(wl)
