@@ -454,20 +454,28 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) tc::tmem_ld_32x32(lane_addr + 128 + c * 32, o[c]);
             tc::tmem_wait_ld();
-            if (live) {
+            // The row goes to shared memory (the Q / K tiles are no longer read: every MMA has completed)
+            // and from there to its raster position as ONE 2*D-byte bulk copy: scattered 16-byte stores of
+            // 32 different rows per instruction touch twice as many sectors (measured 1.7 % slower).
+            constexpr int kRowPitch = 2 * D + 16;                 // bytes; keeps 16-byte alignment, spreads the banks
+            unsigned char* srow = reinterpret_cast<unsigned char*>(&sm.q[0][0][0][0]) + (size_t)(t * 128 + row) * kRowPitch;
 #pragma unroll
-                for (int c = 0; c < D / 32; ++c) {
+            for (int c = 0; c < D / 32; ++c) {
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        uint4 val;
-                        val.x = pack_bf16x2(__uint_as_float(o[c][8 * i + 0]) * inv, __uint_as_float(o[c][8 * i + 1]) * inv);
-                        val.y = pack_bf16x2(__uint_as_float(o[c][8 * i + 2]) * inv, __uint_as_float(o[c][8 * i + 3]) * inv);
-                        val.z = pack_bf16x2(__uint_as_float(o[c][8 * i + 4]) * inv, __uint_as_float(o[c][8 * i + 5]) * inv);
-                        val.w = pack_bf16x2(__uint_as_float(o[c][8 * i + 6]) * inv, __uint_as_float(o[c][8 * i + 7]) * inv);
-                        *reinterpret_cast<uint4*>(dst + c * 32 + i * 8) = val;
-                    }
+                for (int i = 0; i < 4; ++i) {
+                    uint4 val;
+                    val.x = pack_bf16x2(__uint_as_float(o[c][8 * i + 0]) * inv, __uint_as_float(o[c][8 * i + 1]) * inv);
+                    val.y = pack_bf16x2(__uint_as_float(o[c][8 * i + 2]) * inv, __uint_as_float(o[c][8 * i + 3]) * inv);
+                    val.z = pack_bf16x2(__uint_as_float(o[c][8 * i + 4]) * inv, __uint_as_float(o[c][8 * i + 5]) * inv);
+                    val.w = pack_bf16x2(__uint_as_float(o[c][8 * i + 6]) * inv, __uint_as_float(o[c][8 * i + 7]) * inv);
+                    *reinterpret_cast<uint4*>(srow + (c * 4 + i) * 16) = val;
                 }
             }
+            asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+            if (live)
+                asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;\n" ::"l"(dst), "r"(smem_u32(srow)), "n"(2 * D) : "memory");
+            asm volatile("cp.async.bulk.commit_group;\n" ::: "memory");
+            asm volatile("cp.async.bulk.wait_group.read 0;\n" ::: "memory");   // the row has left shared memory
         }
     }
     // ---------------------------------------------------------------- teardown
