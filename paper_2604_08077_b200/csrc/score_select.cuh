@@ -108,7 +108,7 @@ __global__ void __launch_bounds__(256) score_kernel(Geom g, int gt0,
 // in shared memory; long rows (G = 32) overwrite their scores in the L2-resident score buffer with
 // the keys, so that shared memory per warp stays small and many warps hide the latency of the passes.
 // dynamic smem per warp: kSelHistWords + (32/G) * (keys in smem ? N_ld : 0 + cand_cap) words of 8 bytes.
-constexpr int kSelectWarps = 2;     // small CTAs pack shared memory best (measured)
+constexpr int kSelectWarps = 1;     // one-warp CTAs pack shared memory best (measured)
 __host__ __device__ inline int select_lanes_per_row(int N_ld) { return N_ld <= 256 ? 8 : (N_ld <= 512 ? 16 : 32); }
 __host__ __device__ inline int select_cand_cap(int N_ld) { return N_ld <= 256 ? 64 : (N_ld <= 512 ? 128 : (N_ld <= 1024 ? 256 : 512)); }
 __host__ __device__ inline size_t select_smem_bytes(int N_ld) {
