@@ -289,7 +289,7 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
     }
 #ifdef ADASPARK_WITH_TCGEN05
     if (!cache_only && h->prefill_kernel != 0) {   // cube-major staging of Q for the TMA loads of K3 / K4
-        dim3 rgrid((g.S + 31) / 32, g.B);
+        dim3 rgrid((g.S + 3) / 4, g.B);
         __nv_bfloat16* q_cube = (__nv_bfloat16*)((char*)workspace + h->fw_qcube_off);
         if (D == 128) relayout_q_kernel<128><<<rgrid, 256, 0, st>>>(g, (const __nv_bfloat16*)q, q_cube);
         else relayout_q_kernel<64><<<rgrid, 256, 0, st>>>(g, (const __nv_bfloat16*)q, q_cube);

@@ -494,10 +494,10 @@ template <int D>
 __global__ void __launch_bounds__(256) relayout_q_kernel(Geom g, const __nv_bfloat16* __restrict__ q,
                                                          __nv_bfloat16* __restrict__ q_cube) {
     constexpr int kChunks = D / 8;
-    const int pos0 = blockIdx.x * 32;                   // 32 positions x all heads per CTA
+    const int pos0 = blockIdx.x * 4;                    // 4 positions x all heads per CTA: many small CTAs
     const int b = blockIdx.y;
     const int per_pos = g.Hq * kChunks;
-    for (int idx = threadIdx.x; idx < 32 * per_pos; idx += 256) {
+    for (int idx = threadIdx.x; idx < 4 * per_pos; idx += 256) {
         int p = idx / per_pos, rem = idx - p * per_pos;
         int h = rem / kChunks, c = rem - h * kChunks;
         int pos = pos0 + p;

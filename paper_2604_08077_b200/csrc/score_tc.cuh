@@ -32,7 +32,7 @@
 namespace adaspark {
 
 constexpr int kScoreTcThreads = 576;
-constexpr int kScoreTcRing = 12;         // key digit blocks (64 cubes x 128 bytes, 8 KB) in flight
+constexpr int kScoreTcRing = 8;          // key digit blocks (64 cubes x 128 bytes, 8 KB) in flight
 constexpr int kScoreTcCols = 64;         // cubes per column tile
 constexpr int kDigitRowBytes = 128;      // bytes per row of a digit plane
 
