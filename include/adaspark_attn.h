@@ -82,7 +82,8 @@ typedef struct {
 /* Header the library keeps in the first bytes of the workspace of _forward / _decode.  It is
  * reset at the start of every call; the caller may copy it to the host after synchronising. */
 typedef struct {
-    int32_t status;               /* 0 = ok; 1 = text_len out of range (decode)              */
+    int32_t status;               /* 0 = ok; 1 = text_len out of range (decode); 6 = a bounded
+                                     device wait expired (ADASPARK_ERR_TIMEOUT)               */
     int32_t reserved;
     uint64_t executed_kv_blocks;  /* prefill: (query tile, 64-key block) pairs the attention
                                      kernel computed; executed FLOPs = this * 128*64*D*4    */
@@ -100,7 +101,8 @@ adaspark_status_t adaspark_attn_create(const adaspark_attn_config_t *config,
  * buffer size.  `batch`, `frames`, `grid_h`, `grid_w` describe the video token grid;
  * `n_text_max` is the largest number of text tokens any later _forward/_decode will hold.
  * `*workspace_bytes` (nullable) receives max(forward, decode) workspace size.  Host only.
- * ERR_UNSUPPORTED if the grid is not divisible by the cube window or N > 4096.
+ * ERR_UNSUPPORTED if the grid is not divisible by the cube window, N > 4096, or the cache would
+ * hold more than 2097152 rows per sequence (s_video + n_text_max + 1).
  * The forward workspace holds two buffers of fp64 cube scores for a chunk of query tiles each
  * (512 MB each by default, less when the whole problem is smaller); the environment variable
  * ADASPARK_SCORE_BUFFER_MB, read here, overrides the size of one buffer (1 .. 65536). */
@@ -144,8 +146,9 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t *handle, const void *q, 
  *   k_cube, v_cube  in/out, cube_keys in: caches written by _forward.
  *   text_len     in : device int32 [B], text tokens cached before this step, 0 <= text_len[b]
  *                     <= n_text_max.  The row attends text slots 0..text_len[b] (itself included).
- *                     A value outside that range sets `status` in the workspace header to 1 and
- *                     yields a zero output row for that sequence.
+ *                     A value outside that range (checked on the device, with or without k_new)
+ *                     sets `status` in the workspace header to 1, writes nothing to the caches
+ *                     and yields a zero output row for that sequence.
  *   out          out: bf16 [B, 1, Hq, D].
  *   sel_bitmap   out, nullable: uint32 [B, Hq, bitmap_words].
  *   workspace    device scratch of at least decode_workspace_bytes, 256-byte aligned. */
@@ -177,6 +180,9 @@ adaspark_status_t adaspark_attn_decode(adaspark_attn_t *handle, const void *q_ne
  *     it needs about 10 MiB); use adaspark_attn_decode then.
  *   - The first call on each device looks up the array's device address (a one-time host-side
  *     set-up with that device current); make that first call before any stream capture begins.
+ *     The address is cached for the life of the process and is valid only while the device's
+ *     primary context lives: after a cudaDeviceReset by the host program it is stale, and this
+ *     entry point must not be called again in that process.
  *   - The call performs no cudaMalloc / cudaFree and uses no allocating library routine.
  *   - All calls on a device share the one array, which keeps whatever the previous call left in
  *     it; the header that must start at zero is cleared by every call.  Two calls whose kernels

@@ -32,6 +32,16 @@ adaspark_status_t adaspark_attn_debug_imma_selftest(const void *a, const void *b
  * arithmetic (0 <= n < 2^31, 1 <= d < 2^31); -1 for arguments outside that range. */
 int32_t adaspark_attn_debug_fastdiv(int32_t n, int32_t d);
 
+/* Exercises the give-up path of the kernels' bounded waits without disturbing a real kernel: one
+ * small CTA waits on a barrier at which nothing ever arrives.  After `limit_ns` nanoseconds
+ * (1000 <= limit_ns <= 100 000 000, else ERR_INVALID_ARG) the wait expires, the kernel stores
+ * ADASPARK_ERR_TIMEOUT in status[0], 1 in status[1] (a second waiting thread was released through
+ * the shared abort flag) and the time it waited in *waited_ns, and returns normally; the context
+ * stays usable.  `status` is a device int32[2] and `waited_ns` a device uint64, both zeroed by the
+ * caller. */
+adaspark_status_t adaspark_attn_debug_wait_timeout(uint64_t limit_ns, int32_t *status,
+                                                   uint64_t *waited_ns, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -48,7 +48,7 @@ EXPORTS = ["adaspark_attn_create", "adaspark_attn_partition", "adaspark_attn_get
            "adaspark_attn_set_prefill_kernel", "adaspark_attn_enable_stage_timing",
            "adaspark_attn_get_stage_times", "adaspark_attn_decode_static",
            "adaspark_attn_debug_umma_selftest", "adaspark_attn_debug_imma_selftest",
-           "adaspark_attn_debug_fastdiv"]
+           "adaspark_attn_debug_fastdiv", "adaspark_attn_debug_wait_timeout"]
 
 
 def load() -> ctypes.CDLL:
@@ -69,6 +69,7 @@ def load() -> ctypes.CDLL:
     lib.adaspark_attn_decode_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.adaspark_attn_debug_umma_selftest.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     lib.adaspark_attn_debug_imma_selftest.argtypes = [vp, vp, vp, vp, vp]
+    lib.adaspark_attn_debug_wait_timeout.argtypes = [ctypes.c_uint64, vp, vp, vp]
     lib.adaspark_attn_debug_fastdiv.argtypes = [ctypes.c_int32, ctypes.c_int32]
     lib.adaspark_attn_debug_fastdiv.restype = ctypes.c_int32
     lib.adaspark_attn_destroy.argtypes = [vp]
@@ -170,6 +171,12 @@ def adaspark_attn_debug_umma_selftest(a, b, c, d_out, e_out, status, stream=None
 def adaspark_attn_debug_imma_selftest(a, b, d_out, status, stream=None) -> int:
     """128x128x128 int8 tcgen05 self-test (see include/adaspark_attn_debug.h); returns the status code."""
     return int(load().adaspark_attn_debug_imma_selftest(_ptr(a), _ptr(b), _ptr(d_out), _ptr(status),
+                                                       _stream_ptr(stream)))
+
+
+def adaspark_attn_debug_wait_timeout(limit_ns: int, status, waited_ns, stream=None) -> int:
+    """A bounded device wait that is made to expire (see include/adaspark_attn_debug.h)."""
+    return int(load().adaspark_attn_debug_wait_timeout(int(limit_ns), _ptr(status), _ptr(waited_ns),
                                                        _stream_ptr(stream)))
 
 

@@ -174,6 +174,12 @@ adaspark_status_t adaspark_attn_partition(adaspark_attn_t* h, int32_t batch, int
     long long S_cap = (S_v + n_text_max + 1 + 127) / 128 * 128;
     if ((long long)batch * S_cap * c.n_q_heads * c.head_dim >= (1ll << 40) || S_cap >= (1ll << 30))
         return fail(h, ADASPARK_ERR_UNSUPPORTED, "partition: problem too large");
+#ifdef ADASPARK_WITH_TCGEN05
+    // the attention kernel keeps one bit per 64-key block of a sequence in shared memory
+    if (S_cap / kBlockTok > 32ll * kMaxBlockWords)
+        return fail(h, ADASPARK_ERR_UNSUPPORTED, "partition: %lld cache rows per sequence > %d", S_cap,
+                    32 * kMaxBlockWords * kBlockTok);
+#endif
     h->B = batch; h->T = frames; h->H = grid_h; h->W = grid_w; h->n_text_max = n_text_max;
     h->N = (int)N; h->S_v = (int)S_v; h->S_cap = (int)S_cap;
 
@@ -615,6 +621,14 @@ extern "C" adaspark_status_t adaspark_attn_debug_imma_selftest(const void* a, co
     if (cudaFuncSetAttribute(imma_selftest_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return ADASPARK_ERR_CUDA;
     imma_selftest_kernel<<<1, 128, smem, (cudaStream_t)cuda_stream>>>(tmA, tmB, d_out, status);
+    return cudaGetLastError() == cudaSuccess ? ADASPARK_OK : ADASPARK_ERR_CUDA;
+}
+
+extern "C" adaspark_status_t adaspark_attn_debug_wait_timeout(uint64_t limit_ns, int32_t* status, uint64_t* waited_ns,
+                                                              void* cuda_stream) {
+    if (!status || !waited_ns || limit_ns < 1000ull || limit_ns > 100000000ull) return ADASPARK_ERR_INVALID_ARG;
+    wait_timeout_selftest_kernel<<<1, 64, 0, (cudaStream_t)cuda_stream>>>((unsigned long long)limit_ns, status,
+                                                                          (unsigned long long*)waited_ns);
     return cudaGetLastError() == cudaSuccess ? ADASPARK_OK : ADASPARK_ERR_CUDA;
 }
 

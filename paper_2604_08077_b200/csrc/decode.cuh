@@ -14,17 +14,13 @@
 namespace adaspark {
 
 // Appends the new token's K / V of one (batch, kv head) to the cube-major caches at text slot
-// text_len[b] (the V cache holds every 64-position block transposed).  A slot outside the cache sets
-// status 1 and writes nothing.  Called by all threads of a CTA.
+// text_len[b] (the V cache holds every 64-position block transposed).  A text_len outside
+// [0, n_text_max] writes nothing (the caller reports status 1).  Called by all threads of a CTA.
 __device__ __forceinline__ void decode_append(const Geom& g, int b, int gk, const __nv_bfloat16* __restrict__ k_new,
                                               const __nv_bfloat16* __restrict__ v_new, __nv_bfloat16* __restrict__ k_cube,
-                                              __nv_bfloat16* __restrict__ v_cube, const int32_t* __restrict__ text_len,
-                                              int32_t* __restrict__ status) {
+                                              __nv_bfloat16* __restrict__ v_cube, const int32_t* __restrict__ text_len) {
     const int tl = text_len[b];
-    if (tl < 0 || g.S_v + tl + 1 > g.S_cap) {
-        if (threadIdx.x == 0) atomicExch(status, 1);
-        return;
-    }
+    if (tl < 0 || tl > g.n_text) return;             // g.n_text = n_text_max of the partition
     const int pos = g.S_v + tl, blk = pos / kBlockTok, tok = pos % kBlockTok;
     for (int d = threadIdx.x; d < g.D; d += blockDim.x) {
         const size_t src = ((size_t)b * g.Hkv + gk) * g.D + d;
@@ -58,7 +54,10 @@ __global__ void __launch_bounds__(256) decode_select_plan_kernel(
     extern __shared__ double dsp_smem[];
     const int gk = blockIdx.x, b = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (k_new != nullptr) decode_append(g, b, gk, k_new, v_new, k_cube, v_cube, text_len, status);   // read by the next kernel
+    // a text_len outside [0, n_text_max] is reported whether or not a token is appended; the
+    // sequence then gets an empty block list and a zero output row
+    if (threadIdx.x == 0 && (text_len[b] < 0 || text_len[b] > g.n_text)) atomicExch(status, 1);
+    if (k_new != nullptr) decode_append(g, b, gk, k_new, v_new, k_cube, v_cube, text_len);   // read by the next kernel
     const int rpp = decode_rows_per_pass(g.N_ld);
     double* logit = dsp_smem;                                              // [rpp][N_ld]
     unsigned long long* sel_scratch = reinterpret_cast<unsigned long long*>(dsp_smem + (size_t)rpp * g.N_ld);   // [rpp][hist + cand]
@@ -149,7 +148,7 @@ __global__ void __launch_bounds__(256) decode_select_plan_kernel(
     const int tl = text_len[b];
     const int last_pos = g.S_v + tl;                     // position of the new token
     int n_blk = 0;
-    if (tl >= 0 && last_pos < g.S_cap) n_blk = last_pos / kBlockTok + 1;
+    if (tl >= 0 && tl <= g.n_text) n_blk = last_pos / kBlockTok + 1;
     int32_t* dst = items + (size_t)(b * g.Hkv + gk) * g.n_kv_blocks_cap;
     int count = 0;
     for (int kb0 = 0; kb0 < n_blk; kb0 += 32) {

@@ -183,4 +183,28 @@ __global__ void __launch_bounds__(128) imma_selftest_kernel(const __grid_constan
     if (warp == 0) tc::tmem_dealloc<128>(tbase);
 }
 
+// One CTA waits, with the kernels' bounded mbarrier wait, on a barrier at which nothing ever arrives.
+// The wait gives up after limit_ns, the abort flag makes the second thread leave its wait too, and
+// the kernel reports ADASPARK_ERR_TIMEOUT (6) through `status` and returns normally: the same
+// give-up path the attention and scoring kernels take when a protocol error starves a wait.
+__global__ void wait_timeout_selftest_kernel(unsigned long long limit_ns, int32_t* status, unsigned long long* waited_ns) {
+    __shared__ uint64_t never;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        tc::mbar_init(&never, 1);
+        abort_flag = 0;
+        tc::fence_barrier_init();
+    }
+    __syncthreads();
+    const uint64_t t0 = tc::global_timer_ns();
+    // thread 0 owns the limit; thread 32 waits far longer and must be released by the abort flag
+    const bool ok = tc::mbar_wait(&never, 0, &abort_flag, threadIdx.x == 0 ? limit_ns : 1000ull * limit_ns);
+    const uint64_t t1 = tc::global_timer_ns();
+    if (!ok && threadIdx.x == 0) {
+        atomicExch(status, 6);
+        *waited_ns = t1 - t0;
+    }
+    if (!ok && threadIdx.x == 32) atomicAdd(status + 1, 1);
+}
+
 }  // namespace adaspark

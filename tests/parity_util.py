@@ -43,38 +43,110 @@ def run_forward(wl, *, top_p=None, prefill_kernel=None, want_selection=True):
     return eng, out, bitmap, count
 
 
-def compare_rows(wl, rows, gpu_out, gpu_bitmap, gpu_count=None, *, top_p=None, label=""):
+def check_nucleus_legal(probs, oracle_sel, gpu_sel, top_p, top_k=0, tol=TIE_MARGIN):
+    """Is ``gpu_sel`` a legal answer for a row whose oracle answer is ``oracle_sel``?
+
+    A row may differ from the oracle only because of a tie inside ``tol``: the two sets then have
+    sizes within one of each other, differ only in cubes whose probability lies within ``tol`` of the
+    probability of the oracle's last selected cube, and the GPU set is itself a top-prefix whose mass
+    reaches p while dropping its least probable member falls below p (both within ``tol``).  Returns
+    None when legal, else a string saying what is wrong."""
+    n = len(probs)
+    o, g = oracle_sel[:n].astype(bool), gpu_sel[:n].astype(bool)
+    if gpu_sel[n:].any():
+        return "a cube outside the row's candidates is selected"
+    if abs(int(o.sum()) - int(g.sum())) > 1:
+        return f"set sizes {int(g.sum())} vs {int(o.sum())}"
+    if not o.any() or not g.any():
+        return "empty set on one side only"
+    p_edge = probs[o].min()
+    diff = o ^ g
+    if (np.abs(probs[diff] - p_edge) > tol).any():
+        return "sets differ in a cube that is not tied with the boundary cube"
+    if (~g).any() and probs[g].min() < probs[~g].max() - tol:
+        return "not a prefix of the probability order"
+    if top_k > 0:
+        return None if int(g.sum()) == int(o.sum()) else "Top-K size"
+    mass = probs[g].sum()
+    if mass < top_p - tol:
+        return f"mass {mass} below p"
+    if mass - probs[g].min() >= top_p + tol:
+        return "not minimal: the set without its least probable cube still reaches p"
+    return None
+
+
+def check_selection(sh, wl, rows, got_sel, res, *, label=""):
+    """Selection parity on the listed rows (res = oracle.rows(...) of the same rows).
+
+    Bit-exact sets are required on every row whose oracle tie margin is >= 1e-6.  Rows inside the
+    margin may differ, but then (a) the GPU set must still be a legal nucleus (check_nucleus_legal),
+    and (b) there may be only few of them: the GPU evaluates Eqs. 1-2 with an absolute error far
+    below the margin, so it can flip only a small share of the near-tie rows -- at most
+    max(2, 5 %) of them is accepted.  Returns (same mask, counts dict)."""
+    rows = np.asarray(rows, dtype=np.int64).reshape(-1, 3)
+    same = (got_sel == res["sel"]).all(axis=1)
+    near = res["margin"] < TIE_MARGIN
+    bad = ~same & ~near
+    assert not bad.any(), (f"{label}: {bad.sum()} rows differ from the oracle selection with margin "
+                           f">= {TIE_MARGIN}; first {rows[bad][:5].tolist()} margins {res['margin'][bad][:5]}")
+    differing = np.flatnonzero(~same)
+    limit = max(2, int(0.05 * near.sum()))
+    assert len(differing) <= limit, (f"{label}: {len(differing)} rows differ from the oracle (all inside "
+                                     f"the tie margin) but only {limit} of the {int(near.sum())} near-tie "
+                                     f"rows may")
+    if len(differing):
+        kbar = res["kbar"]
+        G = sh.Hq // sh.Hkv
+        pos_of, _ = oracle.positions(sh)
+        qf = oracle.as_f32(wl.q)
+        for i in differing:
+            b, h, n = (int(x) for x in rows[i])
+            pos = int(pos_of[n])
+            n_cand = pos // sh.C if pos < sh.S_v else sh.N
+            _, probs, _ = oracle.select_row(qf[b, n, h], kbar[b, h // G], n_cand, sh.scale, sh.top_p, sh.top_k)
+            why = check_nucleus_legal(probs, res["sel"][i], got_sel[i], sh.top_p, sh.top_k)
+            assert why is None, f"{label}: row {rows[i].tolist()} differs from the oracle illegally: {why}"
+    return same, {"rows": int(len(rows)), "differing": int(len(differing)), "near_tie": int(near.sum())}
+
+
+def compare_rows(wl, rows, gpu_out, gpu_bitmap, gpu_count=None, *, top_p=None, label="", attend=True):
     """Oracle vs CUDA on the listed (b, h, raster token) rows.  Returns a report dict.
 
-    Selection must be bit-exact except on rows whose oracle tie margin is < 1e-6 (counted);
-    outputs are compared on the rows with identical selection."""
+    Selection: see check_selection.  Outputs: every row is compared -- rows with the oracle's
+    selection against the oracle's output, rows that legally differ against the oracle's attention
+    evaluated on the GPU's own set (Eq. 3 with that set)."""
     sh = oracle_shape(wl, top_p)
     rows = np.asarray(rows, dtype=np.int64).reshape(-1, 3)
-    res = oracle.rows(sh, wl.q, wl.k, wl.v, rows)
-    dev = gpu_out.device
+    res = oracle.rows(sh, wl.q, wl.k, wl.v, rows, attend=attend)
+    dev = gpu_bitmap.device
     b, h, n = (torch.from_numpy(np.ascontiguousarray(rows[:, i])).to(dev) for i in range(3))
     words = gpu_bitmap[b, h, n]
     got_sel = unpack_bitmap(words, sh.N)
-    same = (got_sel == res["sel"]).all(axis=1)
-    exempt = ~same & (res["margin"] < TIE_MARGIN)
-    bad = ~same & ~exempt
-    assert not bad.any(), (f"{label}: {bad.sum()} rows differ from the oracle selection with margin "
-                           f">= {TIE_MARGIN}; first {rows[bad][:5].tolist()} margins {res['margin'][bad][:5]}")
+    same, rep = check_selection(sh, wl, rows, got_sel, res, label=label)
     if gpu_count is not None:
         got_cnt = gpu_count[b, h, n].cpu().numpy()
         assert np.array_equal(got_cnt, got_sel.sum(axis=1)), f"{label}: sel_count != popcount(bitmap)"
+    rep.update({"mean_selected": float(res["count"].mean()),
+                "mean_attended": float(res["n_attended"].mean())})
+    if not attend:
+        return rep
     got = gpu_out[b, n, h].float().cpu().numpy()
-    ref = res["out"]
-    ok = same
-    max_abs = float(np.abs(got[ok] - ref[ok]).max()) if ok.any() else 0.0
-    mean_rel = float(np.abs(got[ok] - ref[ok]).mean() / np.abs(ref[ok]).mean()) if ok.any() else 0.0
+    ref = res["out"].copy()
+    if not same.all():
+        ref[~same] = oracle.attend_given(sh, wl.q, wl.k, wl.v, rows[~same], got_sel[~same])
+    max_abs = float(np.abs(got - ref).max()) if len(rows) else 0.0
+    mean_rel = float(np.abs(got - ref).mean() / np.abs(ref).mean()) if len(rows) else 0.0
     assert max_abs <= MAX_ABS_TOL, f"{label}: max-abs error {max_abs} > {MAX_ABS_TOL}"
     assert mean_rel <= MEAN_REL_TOL, f"{label}: mean-relative error {mean_rel} > {MEAN_REL_TOL}"
     assert np.isfinite(got).all()
-    return {"rows": len(rows), "tie_exempt": int(exempt.sum()),
-            "near_tie_rows": int((res["margin"] < TIE_MARGIN).sum()), "max_abs": max_abs,
-            "mean_rel": mean_rel, "mean_selected": float(res["count"].mean()),
-            "mean_attended": float(res["n_attended"].mean())}
+    rep.update({"max_abs": max_abs, "mean_rel": mean_rel})
+    return rep
+
+
+def random_rows(wl, n_rows, seed):
+    rng = np.random.default_rng(seed)
+    return np.stack([rng.integers(0, wl.B, n_rows), rng.integers(0, wl.Hq, n_rows),
+                     rng.integers(0, wl.S, n_rows)], axis=1)
 
 
 def sample_rows(wl, n_random, seed=0, whole_tiles=()):

@@ -163,3 +163,25 @@ def test_index_division_matches_integer_division(lib):
             assert binding.adaspark_attn_debug_fastdiv(n, d) == n // d, (n, d)
     assert binding.adaspark_attn_debug_fastdiv(-1, 3) == -1
     assert binding.adaspark_attn_debug_fastdiv(5, 0) == -1
+
+
+def test_wait_timeout_selftest_rejects_limits_outside_its_range(lib):
+    """Host-side argument check only (no launch): the limit must lie in [1 us, 100 ms]."""
+    fake = 0x1000
+    for bad in (0, 999, 100_000_001):
+        assert binding.adaspark_attn_debug_wait_timeout(bad, fake, fake) == binding.ERR_INVALID_ARG
+    assert binding.adaspark_attn_debug_wait_timeout(1000, None, fake) == binding.ERR_INVALID_ARG
+
+
+def test_partition_rejects_sequences_beyond_the_block_bitmap(lib):
+    """The attention kernel keeps one bit per 64-key block of a sequence (32768 blocks = 2097152
+    cache rows); a legal-looking partition beyond that is refused instead of overrunning it."""
+    hd = binding.adaspark_attn_create(cfg(cube_t=4, cube_h=16, cube_w=16, n_q_heads=1, n_kv_heads=1))
+    with pytest.raises(binding.AdasparkError) as e:                     # 4096 cubes of 1024 tokens
+        binding.adaspark_attn_partition(hd, 1, 4 * 4096, 16, 16, 0)
+    assert e.value.status == binding.ERR_UNSUPPORTED
+    assert binding.adaspark_attn_partition(hd, 1, 4 * 2047, 16, 16, 100) > 0   # just below the limit
+    with pytest.raises(binding.AdasparkError) as e:                     # a large text capacity
+        binding.adaspark_attn_partition(hd, 1, 4 * 2047, 16, 16, 2 * 1024 * 1024)
+    assert e.value.status == binding.ERR_UNSUPPORTED
+    binding.adaspark_attn_destroy(hd)

@@ -27,20 +27,43 @@ def run_decode(wl, text_len, *, top_p=None, n_text_max=None, append=True):
 
 
 def compare_decode(wl, text_len, out, bitmap, *, top_p=None, batch_index=None, label=""):
+    """Decode step vs the oracle, one row per (sequence, head).  Selection: bit-exact outside the
+    1e-6 tie margin; a row inside it may differ only as a legal nucleus (few of them, see
+    parity_util.check_selection).  Outputs: every row, a legally differing row against the oracle's
+    attention on the GPU's own set."""
     sh = pu.oracle_shape(wl, top_p)
     res = oracle.decode(sh, wl.k, wl.v, text_len, wl.q_new, wl.k_new, wl.v_new,
                         batch_index=batch_index)
     idx = list(range(wl.B)) if batch_index is None else list(batch_index)
-    got_sel = pu.unpack_bitmap(bitmap, sh.N)[idx]
-    same = (got_sel == res["sel"]).all(axis=-1)
-    bad = ~same & (res["margin"] >= pu.TIE_MARGIN)
-    assert not bad.any(), f"{label}: selection differs on rows {np.argwhere(bad)[:5].tolist()}"
+    got_sel = pu.unpack_bitmap(bitmap, sh.N)[idx]                     # [n_seq, Hq, N]
     got = out[idx, 0].float().cpu().numpy()
-    ref = res["out"]
-    max_abs = float(np.abs(got[same] - ref[same]).max())
-    mean_rel = float(np.abs(got[same] - ref[same]).mean() / np.abs(ref[same]).mean())
+    same = (got_sel == res["sel"]).all(axis=-1)
+    near = res["margin"] < pu.TIE_MARGIN
+    bad = ~same & ~near
+    assert not bad.any(), f"{label}: selection differs on rows {np.argwhere(bad)[:5].tolist()}"
+    n_diff = int((~same).sum())
+    assert n_diff <= max(2, int(0.05 * near.sum())), f"{label}: {n_diff} differing rows of {int(near.sum())} near ties"
+    ref = res["out"].copy()
+    G = sh.Hq // sh.Hkv
+    kf, qf = oracle.as_f32(wl.k), oracle.as_f32(wl.q_new)
+    for i, h in np.argwhere(~same):
+        b = idx[i]
+        tl = int(text_len[b])
+        s1 = oracle.Shape(1, sh.T, sh.H, sh.W, sh.ct, sh.ch, sh.cw, tl + 1, sh.Hq, sh.Hkv, sh.D, sh.top_p,
+                          sh.scale, sh.top_k)
+        k1 = np.concatenate([kf[b, :sh.S_v + tl], oracle.as_f32(wl.k_new)[b]], axis=0)[None]
+        v1 = np.concatenate([oracle.as_f32(wl.v)[b, :sh.S_v + tl], oracle.as_f32(wl.v_new)[b]], axis=0)[None]
+        q1 = np.zeros((1, sh.S_v + tl + 1, sh.Hq, sh.D), np.float32)
+        q1[0, -1] = qf[b, 0]
+        kbar = oracle.mean_keys(s1, k1)
+        _, probs, _ = oracle.select_row(q1[0, -1, h], kbar[0, h // G], sh.N, sh.scale, sh.top_p, sh.top_k)
+        why = pu.check_nucleus_legal(probs, res["sel"][i, h], got_sel[i, h], sh.top_p, sh.top_k)
+        assert why is None, f"{label}: sequence {b} head {h} differs illegally: {why}"
+        ref[i, h] = oracle.attend_given(s1, q1, k1, v1, [(0, h, sh.S_v + tl)], got_sel[i, h][None])[0]
+    max_abs = float(np.abs(got - ref).max())
+    mean_rel = float(np.abs(got - ref).mean() / np.abs(ref).mean())
     assert max_abs <= pu.MAX_ABS_TOL and mean_rel <= pu.MEAN_REL_TOL, (label, max_abs, mean_rel)
-    return {"rows": int(same.size), "tie_exempt": int((~same).sum()), "max_abs": max_abs,
+    return {"rows": int(same.size), "differing": n_diff, "near_tie": int(near.sum()), "max_abs": max_abs,
             "mean_rel": mean_rel, "mean_selected": float(res["count"].mean())}
 
 
@@ -111,3 +134,34 @@ def test_config5_shape_reduced_batch():
     eng, out, bitmap = run_decode(wl, text_len)
     rep = compare_decode(wl, text_len, out, bitmap, label="cfg5")
     print("cfg5", rep)
+
+
+@pytest.mark.parametrize("append", [True, False])
+def test_text_len_outside_the_partition_is_reported(append):
+    """text_len[b] < 0 or > n_text_max: header status 1, a zero output row for that sequence, the
+    cache untouched -- with and without an appended token; the other sequence is unaffected."""
+    wl = inputs.small_decode(seed=45, B=3, n_text=20)
+    n_text_max = wl.n_text + 2
+    good = wl.n_text
+    text_len = [-1, good, n_text_max + 1]
+    eng = pu.make_engine(wl, n_text_max=n_text_max)
+    eng.forward(None, wl.k.cuda(), wl.v.cuda(), wl.n_text)
+    torch.cuda.synchronize()
+    k_before = eng.k_cube.clone()
+    tl = torch.tensor(text_len, dtype=torch.int32, device="cuda")
+    if append:
+        out, bitmap = eng.decode(wl.q_new.cuda(), wl.k_new.cuda(), wl.v_new.cuda(), tl, want_selection=True)
+    else:
+        # store the middle sequence's token by hand, as a caller that keeps its own cache would
+        pos = wl.S_v + good
+        eng.k_cube[1, :, pos] = wl.k_new[1, 0].cuda()
+        eng.v_cube[1, :, pos // 64, :, pos % 64] = wl.v_new[1, 0].cuda()
+        k_before = eng.k_cube.clone()
+        out, bitmap = eng.decode(wl.q_new.cuda(), None, None, tl, want_selection=True)
+    torch.cuda.synchronize()
+    assert eng.header().status == 1
+    assert (out[0] == 0).all() and (out[2] == 0).all()
+    changed = (eng.k_cube != k_before).flatten(2).any(-1).any(-1)        # per sequence
+    assert changed.tolist() == [False, append, False]
+    rep = compare_decode(wl, text_len, out, bitmap, batch_index=[1], label="valid sequence beside bad ones")
+    assert rep["rows"] == wl.Hq

@@ -35,3 +35,24 @@ def test_imma_selftest_is_an_exact_signed_product():
         assert rc == binding.OK and int(status.item()) == 0
         ref = a.to(torch.int64) @ b.to(torch.int64).T
         assert torch.equal(d.cpu().to(torch.int64), ref)
+
+
+def test_bounded_wait_expires_and_the_context_survives():
+    """A wait on a barrier nobody arrives at gives up after its limit (1 ms here), reports
+    ERR_TIMEOUT through the status word, releases the other waiting threads through the abort flag,
+    and leaves the device usable: the path every mbarrier wait of the tcgen05 kernels takes if its
+    protocol is ever starved."""
+    status = torch.zeros(2, dtype=torch.int32, device="cuda")
+    waited = torch.zeros(1, dtype=torch.int64, device="cuda")
+    rc = binding.adaspark_attn_debug_wait_timeout(1_000_000, status, waited)
+    torch.cuda.synchronize()
+    assert rc == binding.OK
+    assert status.tolist() == [binding.ERR_TIMEOUT, 1]
+    assert 1_000_000 <= int(waited.item()) < 50_000_000
+    # the context is intact: another kernel of the library runs and is correct
+    a = torch.ones(128, 128, dtype=torch.int8, device="cuda")
+    d = torch.zeros(128, 128, dtype=torch.int32, device="cuda")
+    st2 = torch.zeros(1, dtype=torch.int32, device="cuda")
+    assert binding.adaspark_attn_debug_imma_selftest(a, a, d, st2) == binding.OK
+    torch.cuda.synchronize()
+    assert int(st2.item()) == 0 and bool((d == 128).all())
