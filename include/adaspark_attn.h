@@ -88,6 +88,9 @@ typedef struct {
     uint64_t executed_kv_blocks;  /* prefill: (query tile, 64-key block) pairs the attention
                                      kernel computed; executed FLOPs = this * 128*64*D*4    */
     uint64_t decode_kv_blocks;    /* decode: 64-key blocks gathered, summed over (b, kv head) */
+    uint32_t fallback_rows;       /* prefill: query rows whose selection the tensor-core kernel
+                                     left to the fp64 selection kernel (normally 0)           */
+    uint32_t reserved2;
 } adaspark_attn_workspace_header_t;
 
 /* Create a handle for one configuration.  Host only.  Fails with ERR_UNSUPPORTED for a

@@ -210,7 +210,8 @@ def adaspark_attn_get_stage_times(handle: int):
 
 class WorkspaceHeader(ctypes.Structure):
     _fields_ = [("status", ctypes.c_int32), ("reserved", ctypes.c_int32),
-                ("executed_kv_blocks", ctypes.c_uint64), ("decode_kv_blocks", ctypes.c_uint64)]
+                ("executed_kv_blocks", ctypes.c_uint64), ("decode_kv_blocks", ctypes.c_uint64),
+                ("fallback_rows", ctypes.c_uint32), ("reserved2", ctypes.c_uint32)]
 
 
 # ---- a small convenience owner of the handle and of the caller-side buffers --------------------

@@ -12,14 +12,14 @@
 
 #include "common.cuh"
 #include "relayout_pool.cuh"
-#include "score_select.cuh"
+#include "select_exact.cuh"
 #include "attn_prefill_mma.cuh"
 #include "tc_common.cuh"
 #include "decode.cuh"
 #include "decode_splitkv.cuh"
 #ifdef ADASPARK_WITH_TCGEN05
 #include "attn_prefill_tc.cuh"
-#include "score_tc.cuh"
+#include "score_select_fused.cuh"
 #endif
 
 using namespace adaspark;
@@ -31,8 +31,8 @@ struct adaspark_attn {
     int C, N, S_v, S_cap;
     adaspark_attn_layout_t layout;
     // workspace carving (byte offsets)
-    size_t fw_status_off, fw_mask_off, fw_logits_off, fw_qcube_off, fw_kplanes_off, fw_kexp_off, fw_total;
-    int fw_chunk_tiles;
+    size_t fw_status_off, fw_headmax_off, fw_mask_off, fw_union_off, fw_fallback_off, fw_scratch_off, fw_qcube_off,
+        fw_kplanes_off, fw_total;
     size_t dc_status_off, dc_bitmap_off, dc_items_off, dc_nitems_off, dc_partial_off, dc_total;
     int dc_splits;
     int prefill_kernel;
@@ -41,21 +41,13 @@ struct adaspark_attn {
     bool timing;
     cudaEvent_t ev[5];
     bool ev_recorded;
-    // scoring of one chunk of query tiles overlaps the selection of the previous chunk: the
-    // selection kernels run on this handle-private stream, ordered against the caller's by events
-    cudaStream_t side;
-    cudaEvent_t ev_fork, ev_score[2], ev_select[2];
-    bool side_ready;
     char err[256];
 };
 
 namespace {
 
 constexpr size_t kAlign = 256;
-// Per score buffer (there are two).  Large buffers mean few, many-wave launches of the scoring and
-// selection kernels: measured faster than L2-sized chunks whose launches are latency-bound, although
-// the scores then travel through HBM (config 4: 117 ms at 40 MB, 78 ms at 640 MB).
-constexpr size_t kLogitsBudget = 512ull << 20;
+constexpr int kExactCtas = 296;   // CTAs of the fp64 selection kernel (its scratch rows are sized for them)
 size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 
 adaspark_status_t fail(adaspark_attn* h, adaspark_status_t st, const char* fmt, ...) {
@@ -192,28 +184,19 @@ adaspark_status_t adaspark_attn_partition(adaspark_attn_t* h, int32_t batch, int
     L.v_cube_bytes = L.k_cube_bytes;
     L.cube_keys_bytes = (int64_t)((size_t)batch * Hkv * N * D * 4);
 
-    // forward workspace: status | per-tile mask matrix | score scratch | cube-major Q (tcgen05 path)
+    // forward workspace: header | head exponents | per-tile mask matrix | per-tile union words | rows left to
+    // the fp64 selection kernel | its score scratch | cube-major Q | key digit planes (tcgen05 path)
     size_t off = 0;
     h->fw_status_off = off; off = align_up(off + 256);
+    h->fw_headmax_off = off; off = align_up(off + (size_t)batch * Hkv * 4);
     h->fw_mask_off = off; off = align_up(off + (size_t)batch * Hq * n_tiles_cap * n_words * kTileRows * 4);
-    size_t total_tiles = (size_t)batch * Hq * n_tiles_cap;
-    size_t tile_bytes = (size_t)kTileRows * N_ld * 8;
-    size_t budget = kLogitsBudget;
-    if (const char* env = std::getenv("ADASPARK_SCORE_BUFFER_MB")) {   // tuning knob: size of each of the two score buffers
-        long mb = std::atol(env);
-        if (mb >= 1 && mb <= 65536) budget = (size_t)mb << 20;
-    }
-    size_t chunk = budget / tile_bytes;
-    if (chunk < 1) chunk = 1;
-    if (chunk > total_tiles) chunk = total_tiles;
-    if (chunk > 148) chunk = chunk / 148 * 148;    // whole waves of one-CTA-per-SM scoring tiles
-    h->fw_chunk_tiles = (int)chunk;
-    h->fw_logits_off = off; off = align_up(off + 2 * chunk * tile_bytes);   // double-buffered
+    h->fw_union_off = off; off = align_up(off + (size_t)batch * Hq * n_tiles_cap * n_words * 4);
+    h->fw_fallback_off = off; off = align_up(off + (size_t)batch * Hq * n_tiles_cap * kTileRows * 4);
+    h->fw_scratch_off = off; off = align_up(off + (size_t)kExactCtas * kExactWarps * N_ld * 8);
     h->fw_qcube_off = off; off = align_up(off + (size_t)batch * Hq * S_cap * D * 2);
-    // digit planes (4 x int8 [B*Hkv*N_ld, 128]) and row exponents of the mean keys (tensor-core scoring);
-    // 128 rows of slack so that the last 128-cube TMA box stays inside the allocation
-    h->fw_kplanes_off = off; off = align_up(off + ((size_t)4 * batch * Hkv * N_ld + 128) * kDigitRowBytes);
-    h->fw_kexp_off = off; off = align_up(off + (size_t)batch * Hkv * N_ld * 4);
+    // digit planes (4 x int8 [B*Hkv*N_ld, 128]) of the mean keys; 128 rows of slack so that the last TMA box
+    // stays inside the allocation
+    h->fw_kplanes_off = off; off = align_up(off + ((size_t)4 * batch * Hkv * N_ld + 128) * 128);
     h->fw_total = off;
     L.forward_workspace_bytes = (int64_t)off;
 
@@ -280,7 +263,8 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
     auto* kc = (__nv_bfloat16*)k_cube;
     auto* vc = (__nv_bfloat16*)v_cube;
 
-    if (!cache_only) cudaMemsetAsync((char*)workspace + h->fw_status_off, 0, 256, st);
+    // header and head exponents start at zero
+    if (!cache_only) cudaMemsetAsync((char*)workspace + h->fw_status_off, 0, h->fw_mask_off - h->fw_status_off, st);
     mark(h, 0, st);
     // K1: re-layout + pooling
     {
@@ -308,87 +292,68 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
     char* ws = (char*)workspace;
     auto* hdr = (adaspark_attn_workspace_header_t*)(ws + h->fw_status_off);
     uint32_t* tile_mask = (uint32_t*)(ws + h->fw_mask_off);
-    double* logits = (double*)(ws + h->fw_logits_off);
+    uint32_t* tile_union = (uint32_t*)(ws + h->fw_union_off);
     auto* qb = (const __nv_bfloat16*)q;
 
-    // K3: scoring + selection, chunk by chunk
+    // K3: scoring + selection
     {
-        const int total_gt = g.B * g.Hq * g.n_tiles;
-        const size_t sel_smem = select_smem_bytes(g.N_ld);
-        const int lanes = select_lanes_per_row(g.N_ld);
-        auto* sel_fn = lanes == 8 ? select_kernel<8> : (lanes == 16 ? select_kernel<16> : select_kernel<32>);
-        if (!set_smem(h, sel_fn, sel_smem, "select_kernel")) return ADASPARK_ERR_CUDA;
-        const int rows_per_cta = kSelectWarps * (32 / lanes);
-        if (!h->side_ready) {   // first forward of this handle: create the side stream and its events
-            cudaError_t e = cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking);
-            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming);
-            for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
-                e = cudaEventCreateWithFlags(&h->ev_score[i], cudaEventDisableTiming);
-                if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_select[i], cudaEventDisableTiming);
-            }
-            if (e != cudaSuccess) return fail(h, ADASPARK_ERR_CUDA, "forward: side stream set-up: %s", cudaGetErrorString(e));
+        if (h->sm_count <= 0) {
             int sms = 0;
             if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->cfg.device) != cudaSuccess || sms <= 0) sms = 148;
             h->sm_count = sms;
-            h->side_ready = true;
+        }
+        int32_t* fallback_rows = (int32_t*)(ws + h->fw_fallback_off);
+        double* scratch = (double*)(ws + h->fw_scratch_off);
+        const bool all = g.top_k <= 0 && !(g.top_p < 1.0);
+        auto launch_exact = [&](const int32_t* rows, const uint32_t* n_list, long long n_ids) {
+            if (D == 128)
+                select_exact_kernel<128><<<kExactCtas, kExactWarps * 32, 0, st>>>(g, qb, cube_keys, rows, n_list, n_ids, scratch,
+                                                                                   tile_mask, tile_union, sel_bitmap, sel_count);
+            else
+                select_exact_kernel<64><<<kExactCtas, kExactWarps * 32, 0, st>>>(g, qb, cube_keys, rows, n_list, n_ids, scratch,
+                                                                                  tile_mask, tile_union, sel_bitmap, sel_count);
+            return launch_ok(h, "select_exact_kernel");
+        };
+        if (all) {
+            select_all_kernel<<<dim3(g.n_tiles, g.Hq, g.B), kTileRows, 0, st>>>(g, tile_mask, tile_union, sel_bitmap, sel_count);
+            if (!launch_ok(h, "select_all_kernel")) return ADASPARK_ERR_CUDA;
         }
 #ifdef ADASPARK_WITH_TCGEN05
-        CUtensorMap tmKs;
-        int32_t* key_exp = (int32_t*)(ws + h->fw_kexp_off);
-        if (h->prefill_kernel == 1) {   // digit planes of the mean keys, tensor maps of the scoring kernel
+        else if (h->prefill_kernel == 1) {
+            uint32_t* head_max = (uint32_t*)(ws + h->fw_headmax_off);
             unsigned char* kplanes = (unsigned char*)(ws + h->fw_kplanes_off);
             const int n_rows = g.B * g.Hkv * g.N_ld;
-            slice_keys_kernel<<<(n_rows + 3) / 4, 128, 0, st>>>(g, cube_keys, kplanes, key_exp);
+            key_exponent_kernel<<<dim3(g.B * g.Hkv, 8), 256, 0, st>>>(g, cube_keys, head_max);
+            if (!launch_ok(h, "key_exponent_kernel")) return ADASPARK_ERR_CUDA;
+            slice_keys_kernel<<<(n_rows + 3) / 4, 128, 0, st>>>(g, cube_keys, head_max, kplanes);
             if (!launch_ok(h, "slice_keys_kernel")) return ADASPARK_ERR_CUDA;
+            CUtensorMap tmKs;
             if (!encode_u8_2d(&tmKs, kplanes, (uint64_t)4 * n_rows + 128, kDigitRowBytes, kDigitRowBytes, kScoreTcCols))
                 return fail(h, ADASPARK_ERR_CUDA, "forward: cuTensorMapEncodeTiled failed");
-            if (D == 128) { if (!set_smem(h, score_tc_kernel<128>, sizeof(ScoreTcSmem<128>) + 1024, "score_tc_kernel")) return ADASPARK_ERR_CUDA; }
-            else { if (!set_smem(h, score_tc_kernel<64>, sizeof(ScoreTcSmem<64>) + 1024, "score_tc_kernel")) return ADASPARK_ERR_CUDA; }
+            const int n_items = g.B * g.Hq * g.n_tiles;
+            const int grid = n_items < h->sm_count ? n_items : h->sm_count;
+            const __nv_bfloat16* q_cube_c = (const __nv_bfloat16*)(ws + h->fw_qcube_off);
+            const bool by_count = g.top_k > 0;
+#define ADASPARK_LAUNCH_FUSED(DD, BC)                                                                                  \
+    do {                                                                                                               \
+        const size_t smem = sizeof(FusedSmem<DD>) + 1024;                                                              \
+        if (!set_smem(h, score_select_fused_kernel<DD, BC>, smem, "score_select_fused_kernel")) return ADASPARK_ERR_CUDA; \
+        score_select_fused_kernel<DD, BC><<<grid, kFusedThreads, smem, st>>>(                                           \
+            g, n_items, q_cube_c, tmKs, head_max, tile_mask, tile_union, sel_bitmap, sel_count, fallback_rows,         \
+            &hdr->fallback_rows, &hdr->status);                                                                        \
+    } while (0)
+            if (D == 128) { if (by_count) ADASPARK_LAUNCH_FUSED(128, true); else ADASPARK_LAUNCH_FUSED(128, false); }
+            else { if (by_count) ADASPARK_LAUNCH_FUSED(64, true); else ADASPARK_LAUNCH_FUSED(64, false); }
+#undef ADASPARK_LAUNCH_FUSED
+            if (!launch_ok(h, "score_select_fused_kernel")) return ADASPARK_ERR_CUDA;
+            // the rows it left over (normally none): list length is read on the device
+            if (!launch_exact(fallback_rows, &hdr->fallback_rows, 0)) return ADASPARK_ERR_CUDA;
         }
 #endif
-        const size_t buf_elems = (size_t)h->fw_chunk_tiles * kTileRows * g.N_ld;
-        cudaEventRecord(h->ev_fork, st);                       // the side stream starts after the re-layout
-        cudaStreamWaitEvent(h->side, h->ev_fork, 0);
-        int chunk_idx = 0;
-        for (int gt0 = 0; gt0 < total_gt; gt0 += h->fw_chunk_tiles, ++chunk_idx) {
-            int n_gt = total_gt - gt0 < h->fw_chunk_tiles ? total_gt - gt0 : h->fw_chunk_tiles;
-            const int buf = chunk_idx & 1;
-            double* chunk_logits = logits + (size_t)buf * buf_elems;
-            if (chunk_idx >= 2) cudaStreamWaitEvent(st, h->ev_select[buf], 0);   // the buffer has been consumed
-#ifdef ADASPARK_WITH_TCGEN05
-            if (h->prefill_kernel == 1) {
-                const int n_ct = (g.N + kScoreTcCols - 1) / kScoreTcCols;
-                int groups = (h->sm_count + n_gt - 1) / n_gt;      // split the columns when tiles alone cannot fill the SMs
-                if (groups > n_ct) groups = n_ct;
-                const int cols_per_cta = (n_ct + groups - 1) / groups;
-                groups = (n_ct + cols_per_cta - 1) / cols_per_cta;
-                const int n_items = n_gt * groups;
-                const int tgrid = n_items < h->sm_count ? n_items : h->sm_count;
-                const __nv_bfloat16* q_cube_c = (const __nv_bfloat16*)(ws + h->fw_qcube_off);
-                if (D == 128)
-                    score_tc_kernel<128><<<tgrid, kScoreTcThreads, sizeof(ScoreTcSmem<128>) + 1024, st>>>(
-                        g, gt0, n_items, groups, cols_per_cta, q_cube_c, tmKs, key_exp, chunk_logits, &hdr->status);
-                else
-                    score_tc_kernel<64><<<tgrid, kScoreTcThreads, sizeof(ScoreTcSmem<64>) + 1024, st>>>(
-                        g, gt0, n_items, groups, cols_per_cta, q_cube_c, tmKs, key_exp, chunk_logits, &hdr->status);
-                if (!launch_ok(h, "score_tc_kernel")) return ADASPARK_ERR_CUDA;
-            } else
-#endif
-            {
-                dim3 sgrid(n_gt, g.N_ld / kScoreCols);
-                if (D == 128) score_kernel<128><<<sgrid, 256, 0, st>>>(g, gt0, qb, cube_keys, chunk_logits);
-                else score_kernel<64><<<sgrid, 256, 0, st>>>(g, gt0, qb, cube_keys, chunk_logits);
-                if (!launch_ok(h, "score_kernel")) return ADASPARK_ERR_CUDA;
-            }
-            cudaEventRecord(h->ev_score[buf], st);
-            cudaStreamWaitEvent(h->side, h->ev_score[buf], 0);
-            sel_fn<<<n_gt * kTileRows / rows_per_cta, kSelectWarps * 32, sel_smem, h->side>>>(g, gt0, n_gt, chunk_logits, tile_mask, sel_bitmap, sel_count);
-            if (!launch_ok(h, "select_kernel")) return ADASPARK_ERR_CUDA;
-            cudaEventRecord(h->ev_select[buf], h->side);
+        else {
+            cudaMemsetAsync(tile_union, 0, h->fw_fallback_off - h->fw_union_off, st);
+            if (!launch_exact(nullptr, nullptr, (long long)g.B * g.Hq * g.n_tiles_cap * kTileRows)) return ADASPARK_ERR_CUDA;
         }
-        // join: the attention kernel needs every selection
-        cudaStreamWaitEvent(st, h->ev_select[0], 0);
-        if (chunk_idx >= 2) cudaStreamWaitEvent(st, h->ev_select[1], 0);
     }
 
     mark(h, 2, st);
@@ -405,12 +370,12 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
         if (D == 128) {
             size_t smem = sizeof(TcAttnSmem<128>) + 1024;
             if (!set_smem(h, attn_prefill_tc_kernel<128>, smem, "attn_prefill_tc_kernel")) return ADASPARK_ERR_CUDA;
-            attn_prefill_tc_kernel<128><<<grid, kTcThreads, smem, st>>>(g, tmQ, tmK, tmV, tile_mask, (__nv_bfloat16*)out,
+            attn_prefill_tc_kernel<128><<<grid, kTcThreads, smem, st>>>(g, tmQ, tmK, tmV, tile_mask, tile_union, (__nv_bfloat16*)out,
                                                                         (unsigned long long*)&hdr->executed_kv_blocks, &hdr->status);
         } else {
             size_t smem = sizeof(TcAttnSmem<64>) + 1024;
             if (!set_smem(h, attn_prefill_tc_kernel<64>, smem, "attn_prefill_tc_kernel")) return ADASPARK_ERR_CUDA;
-            attn_prefill_tc_kernel<64><<<grid, kTcThreads, smem, st>>>(g, tmQ, tmK, tmV, tile_mask, (__nv_bfloat16*)out,
+            attn_prefill_tc_kernel<64><<<grid, kTcThreads, smem, st>>>(g, tmQ, tmK, tmV, tile_mask, tile_union, (__nv_bfloat16*)out,
                                                                        (unsigned long long*)&hdr->executed_kv_blocks, &hdr->status);
         }
         if (!launch_ok(h, "attn_prefill_tc_kernel")) return ADASPARK_ERR_CUDA;
@@ -505,15 +470,6 @@ adaspark_status_t adaspark_attn_decode(adaspark_attn_t* h, const void* q_new, co
 adaspark_status_t adaspark_attn_destroy(adaspark_attn_t* h) {
     if (h && h->timing)
         for (int i = 0; i < 5; ++i) cudaEventDestroy(h->ev[i]);
-    if (h && h->side_ready) {
-        cudaStreamSynchronize(h->side);
-        cudaEventDestroy(h->ev_fork);
-        for (int i = 0; i < 2; ++i) {
-            cudaEventDestroy(h->ev_score[i]);
-            cudaEventDestroy(h->ev_select[i]);
-        }
-        cudaStreamDestroy(h->side);
-    }
     delete h;
     return ADASPARK_OK;
 }

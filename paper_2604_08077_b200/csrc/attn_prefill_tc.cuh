@@ -60,7 +60,8 @@ struct BlockIter {
 template <int D>
 __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     Geom g, const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-    const __grid_constant__ CUtensorMap tmV, const uint32_t* __restrict__ tile_mask, __nv_bfloat16* __restrict__ out,
+    const __grid_constant__ CUtensorMap tmV, const uint32_t* __restrict__ tile_mask,
+    const uint32_t* __restrict__ tile_union, __nv_bfloat16* __restrict__ out,
     unsigned long long* __restrict__ executed_blocks, int32_t* __restrict__ status) {
     extern __shared__ unsigned char tc_smem_raw[];
     TcAttnSmem<D>& sm = *reinterpret_cast<TcAttnSmem<D>*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -115,20 +116,16 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
         for (int t = 0; t < 2; ++t)
             for (int p = 0; p < kPanels; ++p) tc::tma_load_2d(&sm.q[t][p][0][0], &tmQ, p * 64, q_row0 + t * 128, &sm.q_full);
     }
-    // union of the selection words of the 256 rows (two 128-row tiles of the mask matrix): the eight
-    // loads of a lane are issued together
-    for (int w = warp; w < g.n_words; w += kTcThreads / 32) {
-        uint32_t v[kPairRows / 32];
-#pragma unroll
-        for (int i = 0; i < kPairRows / 32; ++i) {
-            const int r = lane + 32 * i, tile = pair * 2 + (r >> 7);
-            v[i] = tile < g.n_tiles ? __ldg(tile_mask + mask_index(g, b, h, tile, w, r & 127)) : 0u;
-        }
+    // union of the selection words of the 256 rows = OR of the two tiles' union words (written by the
+    // selection kernel)
+    for (int w = tid; w < g.n_words; w += kTcThreads) {
         uint32_t u = 0;
 #pragma unroll
-        for (int i = 0; i < kPairRows / 32; ++i) u |= v[i];
-        u = __reduce_or_sync(0xffffffffu, u);
-        if (lane == 0) sm.union_words[w] = u;
+        for (int t = 0; t < 2; ++t) {
+            const int tile = pair * 2 + t;
+            if (tile < g.n_tiles) u |= __ldg(tile_union + ((size_t)(b * g.Hq + h) * g.n_tiles_cap + tile) * g.n_words + w);
+        }
+        sm.union_words[w] = u;
     }
     tc::tc_fence_before_sync();
     __syncthreads();
