@@ -16,7 +16,7 @@
 // the margin (e_q + E_K > kMaxExponentSum) are not decided here: they go to the fp64 kernel of
 // select_exact.cuh through a list in the workspace, and so does any row this kernel gives up on.
 //
-// Selection (thread = query row = TMEM lane; nothing is exchanged between lanes).  The scores of a
+// Selection (query row = TMEM lane).  The scores of a
 // 128-row tile are far too many to keep (128 x up to 4096), and the tensor pipe is nearly idle, so
 // the kernel RECOMPUTES them: it makes several passes over the tile's column tiles (64 cubes each),
 // re-issuing the same MMAs, and each row narrows a key interval that holds its nucleus boundary:
@@ -34,25 +34,38 @@
 // probability by more than n * 2^-39.  Equal scores are ordered by lower cube index.
 // Top-K (top_k > 0): the same with every mass = 1 and T = min(top_k, candidates).
 //
-// Roles (512 threads, one persistent CTA per SM, work item = one 128-row query tile, long tiles first):
-//   warps 0-3    selection (above).  They free an accumulator set as soon as its values are in registers
-//   warps 4-11   slicers (two threads per row): digit planes of the next tile's queries into shared memory
-//   warp 12      TMA producer: key digit planes of one column tile (4 x 8 KB; 2 x 8 KB in pass A), 2 slots
-//   warp 13      issues the tcgen05.mma stream (40 of 128x64x32 per column tile, 12 in pass A) into
+// A row is served by FOUR threads (same TMEM lane, four warps): each takes 16 of the 64 columns of every
+// column tile, adds to the row's histogram with shared-memory atomics and appends to the row's candidate
+// list through an atomic counter; what the four must agree on (anchor, crossing bucket, boundary key)
+// goes through small shared arrays between barriers of the 512 selection threads.  The work of a row is
+// latency-bound (TMEM loads, fp64 chains, shared-memory atomics), so four warps per scheduler matter
+// more than instruction count: with one thread per row the MMA thread waited 3/4 of the time.
+//
+// Roles (768 threads, one persistent CTA per SM, work item = one 128-row query tile, long tiles first):
+//   warps 0-15   selection: warp w serves TMEM lane quarter w % 4 (rows 32*(w%4) + lane) and columns
+//                16*(w/4) .. +15 of every column tile.  An accumulator set is freed as soon as its values
+//                are in registers
+//   warps 16-19  slicers (one thread per row): digit planes of the next tile's queries into shared memory
+//   warp 20      TMA producer: key digit planes of one column tile (4 x 8 KB; 2 x 8 KB in pass A), 2 slots
+//   warp 21      issues the tcgen05.mma stream (40 of 128x64x32 per column tile, 12 in pass A) into
 //                double-buffered accumulator sets (2 x 4 levels x 64 columns = all 512 TMEM columns)
-//   warps 14-15  idle (they complete the fourth warpgroup for the register re-allocation)
+//   warps 22-23  idle (they complete the sixth warpgroup for the register re-allocation)
 #pragma once
 #include "tc_common.cuh"
 
 namespace adaspark {
 
-constexpr int kFusedThreads = 512;
+constexpr int kFusedThreads = 768;
+constexpr int kSelThreads = 512;         // selection threads: four per row
 constexpr int kScoreTcCols = 64;         // cubes per column tile
 constexpr int kDigitRowBytes = 128;      // bytes per row of a digit plane
 constexpr int kCandCap = 24;             // cubes a row may collect from its boundary interval
 constexpr int kMaxHistPasses = 10;       // histogram passes a row may take before it is handed to the fp64 kernel
 constexpr int kMaxExponentSum = 6;       // largest e_q + E_K this kernel decides itself
-constexpr int kSelRegs = 224, kSlicerRegs = 96, kIssueRegs = 56;   // per-thread registers after setmaxnreg
+// Per-thread registers after setmaxnreg.  The re-allocation only moves registers inside the CTA's launch
+// allocation (768 threads x 80): 4 * 88 + 88 + 40 = 6 * 80.  (A sum above it would block forever.)
+constexpr int kSelRegs = 88, kSlicerRegs = 88, kIssueRegs = 40;
+static_assert(4 * kSelRegs + kSlicerRegs + kIssueRegs <= 6 * 80, "setmaxnreg budget exceeds the launch allocation");
 
 // The four signed base-256 digits of v = round(x * 2^(29 - e)) (|v| < 2^30), packed in one word:
 // byte 3 = d0 (most significant) ... byte 0 = d3.  Adding 0x80 to every byte position turns the
@@ -151,10 +164,15 @@ struct FusedSmem {
     unsigned char kring[2][4][kScoreTcCols][kDigitRowBytes];       // key digit planes of a column tile, two slots
     unsigned long long hist[64][128];                              // [bucket][row]: (sum of masses << 13) | count
     unsigned long long cand[kCandCap][128];                        // [slot][row]: (delta << 12) | cube
+    unsigned long long part[4][128];                               // what the four threads of a row exchange
+    unsigned long long res_base[128];                              // crossing bucket of a row: mass before it ...
+    int32_t res_cb[128];                                           // ... and bucket | count << 8
+    int32_t cand_cnt[128];                                         // candidates appended by the row's threads
+    int32_t row_count[128];                                        // |S_i| of the row
     uint32_t tile_union[2][128];                                   // OR over the tile's rows of each selection word
     int32_t eq[2][128];                                            // exponent e_q of each row of the tile (by tile parity)
     int32_t need[4];                                               // decision ring: d + 1 = "another pass after the next"
-    uint64_t q_sliced, qd_free, k_full[2], acc_full[2], acc_free[2], decided[4], tile_sync;
+    uint64_t q_sliced, qd_free, k_full[2], acc_full[2], acc_free[2], decided[4], sel_sync;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -175,9 +193,16 @@ __device__ __forceinline__ FusedItem fused_item(const Geom& g, int it) {
     return w;
 }
 
+__device__ __forceinline__ void tmem_ld_32x8(uint32_t taddr, uint32_t (&r)[8]) {   // 8 consecutive columns
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];\n"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr)
+                 : "memory");
+}
+
 // q_cube: cube-major bf16 queries [B*Hq, S_cap, D].  tile_mask as mask_index() describes;
 // tile_union[((b*Hq+h)*n_tiles_cap + tile)*n_words + w] = OR of word w over the tile's rows.
-// fallback_rows[0 .. hdr->fallback_rows) receives ((b*Hq+h)*n_tiles_cap + tile)*128 + r of the rows left
+// fallback_rows[0 .. *fallback_count) receives ((b*Hq+h)*n_tiles_cap + tile)*128 + r of the rows left
 // to the fp64 kernel.
 template <int D, bool kByCount>
 __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
@@ -189,25 +214,28 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
     FusedSmem<D>& sm = *reinterpret_cast<FusedSmem<D>*>((reinterpret_cast<uintptr_t>(fused_raw) + 1023) & ~(uintptr_t)1023);
     constexpr uint32_t kIdesc = tc::make_idesc_s8(128, kScoreTcCols);
     constexpr uint32_t kPlaneBytes = kScoreTcCols * kDigitRowBytes;
-    constexpr int kProducerWarp = 12, kMmaWarp = 13;
+    constexpr int kSlicerWarp0 = 16, kProducerWarp = 20, kMmaWarp = 21;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid == 0) {
-        tc::mbar_init(&sm.q_sliced, 256);
+        tc::mbar_init(&sm.q_sliced, 128);
         tc::mbar_init(&sm.qd_free, 1);
         for (int i = 0; i < 2; ++i) {
             tc::mbar_init(&sm.k_full[i], 1);
             tc::mbar_init(&sm.acc_full[i], 1);
-            tc::mbar_init(&sm.acc_free[i], 128);
+            tc::mbar_init(&sm.acc_free[i], kSelThreads);
         }
         for (int i = 0; i < 4; ++i) {
-            tc::mbar_init(&sm.decided[i], 128);
+            tc::mbar_init(&sm.decided[i], kSelThreads);
             sm.need[i] = 0;
         }
-        tc::mbar_init(&sm.tile_sync, 128);
+        tc::mbar_init(&sm.sel_sync, kSelThreads);
         sm.abort_flag = 0;
         tc::fence_barrier_init();
     }
+    // selection state that must start at zero
+    for (int i = tid; i < 64 * 128; i += kFusedThreads) (&sm.hist[0][0])[i] = 0ull;
+    if (tid < 128) { sm.cand_cnt[tid] = 0; sm.row_count[tid] = 0; sm.tile_union[0][tid] = 0u; sm.tile_union[1][tid] = 0u; }
     if (D < kDigitRowBytes) {                                     // bytes beyond head_dim stay zero for the whole kernel
         uint4* z = reinterpret_cast<uint4*>(&sm.qd[0][0][0]);
         for (int i = tid; i < (int)(sizeof(sm.qd) / 16); i += kFusedThreads) z[i] = make_uint4(0u, 0u, 0u, 0u);
@@ -231,9 +259,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
         return ok && *reinterpret_cast<volatile int32_t*>(&sm.need[d & 3]) == d + 1;
     };
 
-    if (warp >= 4) {
-        if (warp >= kProducerWarp) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kIssueRegs));
-        else asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kSlicerRegs));
+    if (warp >= kProducerWarp) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kIssueRegs));
     }
 
     if (warp == kProducerWarp) {
@@ -317,42 +344,44 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
                 ++n_done;
             }
         }
-    } else if (warp >= 4 && warp < kProducerWarp) {
-        // ------------------------------------------------------------ slicers (two threads per row)
-        constexpr int kChunks = D / 16;                           // 16-byte chunks (8 elements) of the row half
-        constexpr int kOut = D / 32;                              // 16-byte chunks (16 digits) per plane per thread
-        const int r = (tid - 128) >> 1, half = (tid - 128) & 1;
+    } else if (warp >= kSlicerWarp0 && warp < kProducerWarp) {
+        // ------------------------------------------------------------ slicers (one thread per row)
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kSlicerRegs));
+        const int r = tid - kSlicerWarp0 * 32;
         bool ok = true;
         int n_done = 0;
         for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
             const FusedItem w = fused_item(g, it);
             if (w.n_ct == 0) continue;
             const int pos = w.tile * kTileRows + r;
-            const uint4* src = reinterpret_cast<const uint4*>(q_cube + ((size_t)(w.b * g.Hq + w.h) * g.S_cap + pos) * D) + half * kChunks;
-            uint4 v[kChunks];
-#pragma unroll
-            for (int c = 0; c < kChunks; ++c) v[c] = pos < g.S ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
+            const bool live = pos < g.S;
+            const uint4* src = reinterpret_cast<const uint4*>(q_cube + ((size_t)(w.b * g.Hq + w.h) * g.S_cap + pos) * D);
+            // first sweep over the row (before the planes are free): its largest exponent
             uint32_t mxbits = 0;
+            if (live) {
 #pragma unroll
-            for (int c = 0; c < kChunks; ++c) {
-                const uint32_t wd[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
+                for (int c = 0; c < D / 8; ++c) {
+                    const uint4 v = __ldg(src + c);
+                    const uint32_t wd[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-                for (int i = 0; i < 4; ++i) mxbits = max(mxbits, max(wd[i] & 0x7fffu, (wd[i] >> 16) & 0x7fffu));
+                    for (int i = 0; i < 4; ++i) mxbits = max(mxbits, max(wd[i] & 0x7fffu, (wd[i] >> 16) & 0x7fffu));
+                }
             }
-            mxbits = max(mxbits, __shfl_xor_sync(0xffffffffu, mxbits, 1));   // the two halves of the row
             const int e_q = row_exponent_from_field((int)(mxbits >> 7));
             const float mult = digit_scale(e_q);
             // the previous tile's MMAs must have finished reading the digit planes (and its selection
             // threads are past reading their exponents of the tile before that)
             if (n_done > 0 && !(ok = tc::mbar_wait(&sm.qd_free, (n_done - 1) & 1, abort_flag))) break;
-            if (half == 0) sm.eq[n_done & 1][r] = e_q;
+            sm.eq[n_done & 1][r] = e_q;
             unsigned char* dst = &sm.qd[0][0][0];
-#pragma unroll
-            for (int o = 0; o < kOut; ++o) {
+#pragma unroll 2
+            for (int o = 0; o < D / 16; ++o) {                    // 16 elements = one 16-byte chunk of every plane
+                const uint4 va = live ? __ldg(src + 2 * o) : make_uint4(0u, 0u, 0u, 0u);
+                const uint4 vb = live ? __ldg(src + 2 * o + 1) : make_uint4(0u, 0u, 0u, 0u);
                 uint32_t pw[4][4];                                // [plane][4 elements per word]
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4) {                  // elements 16*o + 4*q4 .. +3 = two packed bf16 words
-                    const uint4 vv = v[2 * o + (q4 >> 1)];
+                    const uint4 vv = (q4 >> 1) ? vb : va;
                     const uint32_t wa = (q4 & 1) ? vv.z : vv.x, wb = (q4 & 1) ? vv.w : vv.y;
                     const uint32_t w0 = packed_digits(__uint_as_float(wa << 16), mult);
                     const uint32_t w1 = packed_digits(__uint_as_float(wa & 0xffff0000u), mult);
@@ -363,7 +392,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
                     pw[2][q4] = gather_byte<1>(w0, w1, w2, w3);
                     pw[3][q4] = gather_byte<0>(w0, w1, w2, w3);
                 }
-                const int off = sw128(r, half * kOut + o);        // 16-byte chunk of the 128-byte plane row
+                const int off = sw128(r, o);                      // 16-byte chunk of the 128-byte plane row
 #pragma unroll
                 for (int pl = 0; pl < 4; ++pl)
                     *reinterpret_cast<uint4*>(dst + (size_t)pl * sizeof(sm.qd[0]) + off) = make_uint4(pw[pl][0], pw[pl][1], pw[pl][2], pw[pl][3]);
@@ -372,11 +401,12 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
             tc::mbar_arrive(&sm.q_sliced);
             ++n_done;
         }
-    } else if (warp < 4) {
-        // ------------------------------------------------------------ selection (thread = row = TMEM lane)
+    } else if (warp < kSlicerWarp0) {
+        // ------------------------------------------------------------ selection (4 threads per row)
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kSelRegs));
-        const int r = warp * 32 + lane;
-        const uint32_t lane_addr = tbase + ((uint32_t)(warp * 32) << 16);
+        const int quarter = warp & 3, part = warp >> 2;
+        const int r = quarter * 32 + lane;
+        const uint32_t lane_addr = tbase + ((uint32_t)(quarter * 32) << 16) + part * 16;
         unsigned long long* hist = &sm.hist[0][r];                // bucket b at hist[b * 128]
         unsigned long long* cand = &sm.cand[0][r];                // slot k at cand[k * 128]
         enum { kDone = 0, kHist = 1, kCollect = 2 };
@@ -384,13 +414,16 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
         constexpr unsigned long long kOpen = 1ull << 62;          // span of an interval without upper end
         bool ok = true;
         int c = 0, d0 = 0, n_done = 0, t_par = 0, n_sync = 0;
-        // barrier among the 128 selection threads (a bounded wait like every other one here)
+        // barrier among the 512 selection threads (a bounded wait like every other one here)
         auto sync_selection = [&]() -> bool {
             __threadfence_block();
-            tc::mbar_arrive(&sm.tile_sync);
-            const bool done = tc::mbar_wait(&sm.tile_sync, n_sync & 1, abort_flag);
+            tc::mbar_arrive(&sm.sel_sync);
+            const bool done = tc::mbar_wait(&sm.sel_sync, n_sync & 1, abort_flag);
             ++n_sync;
             return done;
+        };
+        auto to_double = [](unsigned long long d) -> double {     // exact for d < 2^52
+            return __hiloint2double(0x43300000 | (int)(d >> 32), (int)(uint32_t)d) - 4503599627370496.0;
         };
         for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x, t_par ^= 1) {
             const FusedItem w = fused_item(g, it);
@@ -403,15 +436,12 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
             const bool extra = live && (sel_bitmap != nullptr || sel_count != nullptr);
             const size_t raster_row = extra ? (size_t)(w.b * g.Hq + w.h) * g.S + pos_to_raster(g, pos) : 0;
             uint32_t* bm_row = (extra && sel_bitmap) ? sel_bitmap + raster_row * g.n_words : nullptr;
-            // words beyond the tile's column tiles are zero (all words of a row without candidates); the
-            // union of the tile starts empty
-            for (int wd = n > 0 ? 2 * w.n_ct : 0; wd < g.n_words; ++wd) {
+            // words beyond the tile's column tiles are zero (all words of a row without candidates)
+            for (int wd = (n > 0 ? 2 * w.n_ct : 0) + part; wd < g.n_words; wd += 4) {
                 mask_row[(size_t)wd * kTileRows] = 0u;
                 if (bm_row) bm_row[wd] = 0u;
             }
-            if (r < g.n_words) sm.tile_union[t_par][r] = 0u;
-            if (!(ok = sync_selection())) break;
-            int count = 0;                                        // |S_i| of this row
+            bool give_up = false;
             if (w.n_ct > 0) {
                 // ---------------- anchor pass: largest S_0*256 + S_1 over the row's candidates
                 int max_hi = INT_MIN;
@@ -419,24 +449,28 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
                     const int s = c & 1;
                     if (!(ok = tc::mbar_wait(&sm.acc_full[s], (c >> 1) & 1, abort_flag))) break;
                     tc::tc_fence_after_sync();
+                    const int col0 = ct * kScoreTcCols + part * 16;
+                    if (col0 < n_warp) {
+                        uint32_t l0[16], l1[16];
+                        tc::tmem_ld_32x16(lane_addr + s * 256, l0);
+                        tc::tmem_ld_32x16(lane_addr + s * 256 + kScoreTcCols, l1);
+                        tc::tmem_wait_ld();
+                        tc::tc_fence_before_sync();
+                        tc::mbar_arrive(&sm.acc_free[s]);
 #pragma unroll
-                    for (int ch = 0; ch < 4; ++ch) {
-                        const int col0 = ct * kScoreTcCols + ch * 16;
-                        if (col0 < n_warp) {
-                            uint32_t l0[16], l1[16];
-                            tc::tmem_ld_32x16(lane_addr + s * 256 + ch * 16, l0);
-                            tc::tmem_ld_32x16(lane_addr + s * 256 + kScoreTcCols + ch * 16, l1);
-                            tc::tmem_wait_ld();
-#pragma unroll
-                            for (int i = 0; i < 16; ++i)
-                                if (col0 + i < n) max_hi = max(max_hi, (int)l0[i] * 256 + (int)l1[i]);
-                        }
+                        for (int i = 0; i < 16; ++i)
+                            if (col0 + i < n) max_hi = max(max_hi, (int)l0[i] * 256 + (int)l1[i]);
+                    } else {
+                        tc::tc_fence_before_sync();
+                        tc::mbar_arrive(&sm.acc_free[s]);
                     }
-                    tc::tc_fence_before_sync();
-                    tc::mbar_arrive(&sm.acc_free[s]);
                 }
                 if (!ok) break;
-                // ---------------- per-row constants
+                sm.part[part][r] = (unsigned long long)(long long)max_hi;
+                if (!(ok = sync_selection())) break;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) max_hi = max(max_hi, (int)(long long)sm.part[k][r]);
+                // ---------------- per-row constants (the same in the row's four threads)
                 const int e_sum = sm.eq[n_done & 1][r] + head_exponent(head_max_bits[w.b * g.Hkv + w.gk]);
                 const double f = __hiloint2double((1023 + e_sum - 34) << 20, 0) * g.scale_d;   // score per unit of V
                 const double neg_f = -f;
@@ -448,39 +482,34 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
                 }
                 unsigned long long lo = 0ull, span = kOpen, base = 0ull, target = 0ull;
                 int state = n > 0 ? kHist : kDone;
-                bool first_level = true, give_up = false;
+                bool first_level = true;
                 if (n > 0 && e_sum > kMaxExponentSum) { state = kDone; give_up = true; }
-                int n_cand = 0, hist_passes = 0;
+                int hist_passes = 0;
                 // ---------------- passes
                 int fpass = 0;
                 while (ok) {
                     const int my = state;                         // what this row does in this pass
-                    if (my == kHist) {
-#pragma unroll 8
-                        for (int b = 0; b < 64; ++b) hist[b * 128] = 0ull;
-                    }
-                    n_cand = 0;
-                    uint32_t word = 0;
+                    const bool warp_idle = !__any_sync(0xffffffffu, my != kDone);
                     for (int ct = 0; ok && ct < w.n_ct; ++ct, ++c) {
                         const int s = c & 1;
                         if (!(ok = tc::mbar_wait(&sm.acc_full[s], (c >> 1) & 1, abort_flag))) break;
                         tc::tc_fence_after_sync();
-#pragma unroll 1
-                        for (int ch = 0; ch < 4; ++ch) {
-                            const int col0 = ct * kScoreTcCols + ch * 16;
-                            const bool any_work = col0 < n_warp && __any_sync(0xffffffffu, my != kDone);
-                            if (any_work) {
-                                uint32_t lv[4][16];
+                        const int col0 = ct * kScoreTcCols + part * 16;
+                        uint32_t word = 0;                        // 16 bits: cubes col0 .. col0 + 15
+                        if (col0 < n_warp && !warp_idle) {
 #pragma unroll
-                                for (int L = 0; L < 4; ++L) tc::tmem_ld_32x16(lane_addr + s * 256 + L * kScoreTcCols + ch * 16, lv[L]);
+                            for (int hf = 0; hf < 2; ++hf) {
+                                uint32_t lv[4][8];
+#pragma unroll
+                                for (int L = 0; L < 4; ++L) tmem_ld_32x8(lane_addr + s * 256 + L * kScoreTcCols + hf * 8, lv[L]);
                                 tc::tmem_wait_ld();
-                                if (ch == 3) {                    // last read of this accumulator set: release it
+                                if (hf == 1) {                    // last read of this accumulator set: release it
                                     tc::tc_fence_before_sync();
                                     tc::mbar_arrive(&sm.acc_free[s]);
                                 }
                                 if (my == kHist) {
 #pragma unroll
-                                    for (int i0 = 0; i0 < 16; i0 += 4) {       // four independent mass evaluations at a time
+                                    for (int i0 = 0; i0 < 8; i0 += 4) {        // four independent mass evaluations at a time
                                         unsigned long long delta[4];
                                         bool in[4];
                                         bool any_in = false;
@@ -490,83 +519,118 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
                                             const int hi = (int)lv[0][i] * 256 + (int)lv[1][i];
                                             const int lw = (int)lv[2][i] * 256 + (int)lv[3][i];
                                             delta[u] = (unsigned long long)(VA - ((long long)hi * 65536 + lw));
-                                            in[u] = col0 + i < n && delta[u] - lo <= span;
+                                            in[u] = col0 + hf * 8 + i < n && delta[u] - lo <= span;
                                             any_in |= in[u];
                                         }
                                         if (!any_in) continue;
                                         unsigned long long m[4];
 #pragma unroll
-                                        for (int u = 0; u < 4; ++u) {
-                                            m[u] = 1ull;
-                                            if (!kByCount) {
-                                                const double dd = __hiloint2double(0x43300000 | (int)(delta[u] >> 32), (int)(uint32_t)delta[u]) - 4503599627370496.0;
-                                                m[u] = mass38(dd * neg_f);
-                                            }
-                                        }
+                                        for (int u = 0; u < 4; ++u) m[u] = kByCount ? 1ull : mass38(to_double(delta[u]) * neg_f);
 #pragma unroll
                                         for (int u = 0; u < 4; ++u) {
                                             if (in[u]) {
                                                 const unsigned long long bq = (delta[u] - lo) >> sh;
                                                 const int b = bq > 63ull ? 63 : (int)bq;
-                                                hist[b * 128] += (m[u] << 13) | 1ull;
+                                                atomicAdd(&hist[b * 128], (m[u] << 13) | 1ull);
                                             }
                                         }
                                     }
                                 } else if (my == kCollect) {
 #pragma unroll
-                                    for (int i = 0; i < 16; ++i) {
+                                    for (int i = 0; i < 8; ++i) {
                                         const int hi = (int)lv[0][i] * 256 + (int)lv[1][i];
                                         const int lw = (int)lv[2][i] * 256 + (int)lv[3][i];
                                         const unsigned long long delta = (unsigned long long)(VA - ((long long)hi * 65536 + lw));
-                                        const bool in_row = col0 + i < n;
-                                        const bool above = in_row && delta < lo;
+                                        const int j = col0 + hf * 8 + i;
+                                        const bool in_row = j < n;
                                         if (in_row && delta - lo <= span) {
-                                            if (n_cand < kCandCap) cand[n_cand * 128] = (delta << 12) | (unsigned long long)(col0 + i);
-                                            ++n_cand;
+                                            const int slot = atomicAdd(&sm.cand_cnt[r], 1);
+                                            if (slot < kCandCap) cand[slot * 128] = (delta << 12) | (unsigned long long)j;
                                         }
-                                        word |= (above ? 1u : 0u) << ((ch & 1) * 16 + i);
+                                        word |= ((in_row && delta < lo) ? 1u : 0u) << (hf * 8 + i);
                                     }
                                 }
-                            } else if (ch == 3) {
-                                tc::tc_fence_before_sync();
-                                tc::mbar_arrive(&sm.acc_free[s]);
                             }
-                            if (ch & 1) {                         // a 32-cube word is complete
-                                const int wd = ct * 2 + (ch >> 1);
-                                if (wd < g.n_words) {
-                                    const bool wr = my == kCollect;
-                                    if (wr) {
-                                        mask_row[(size_t)wd * kTileRows] = word;
-                                        if (bm_row) bm_row[wd] = word;
-                                        count += __popc(word);
-                                    }
-                                    const uint32_t u = __reduce_or_sync(0xffffffffu, wr ? word : 0u);
-                                    if (lane == 0 && u) atomicOr(&sm.tile_union[t_par][wd], u);
-                                }
-                                word = 0;
+                        } else {
+                            tc::tc_fence_before_sync();
+                            tc::mbar_arrive(&sm.acc_free[s]);
+                        }
+                        // this thread's half of a 32-cube word
+                        const int wd = ct * 2 + (part >> 1);
+                        if (wd < g.n_words && !warp_idle) {
+                            const bool wr = my == kCollect;
+                            if (wr) {
+                                reinterpret_cast<uint16_t*>(mask_row + (size_t)wd * kTileRows)[part & 1] = (uint16_t)word;
+                                if (bm_row) reinterpret_cast<uint16_t*>(bm_row + wd)[part & 1] = (uint16_t)word;
+                                if (word) atomicAdd(&sm.row_count[r], __popc(word));
                             }
+                            const uint32_t u = __reduce_or_sync(0xffffffffu, wr ? word : 0u);
+                            if (lane == 0 && u) atomicOr(&sm.tile_union[t_par][wd], u << ((part & 1) * 16));
                         }
                     }
                     if (!ok) break;
-                    // ---------------- end of the pass: every row advances by itself
+                    // ---------------- end of the pass: the row's four threads combine (three barriers, whatever the rows do)
+                    if (!(ok = sync_selection())) break;          // A: histogram / candidate list complete
+                    int n_cand = 0;
                     if (my == kHist) {
-                        ++hist_passes;
+                        unsigned long long ps = 0ull;
+#pragma unroll
+                        for (int b = 0; b < 16; ++b) ps += hist[(part * 16 + b) * 128] >> 13;
+                        sm.part[part][r] = ps;
+                    } else if (my == kCollect) {
+                        n_cand = sm.cand_cnt[r];
+                        if (n_cand <= kCandCap)
+                            for (int k = part; k < n_cand; k += 4)
+                                hist[k * 128] = kByCount ? 1ull : mass38(to_double(cand[k * 128] >> 12) * neg_f);
+                    }
+                    if (!(ok = sync_selection())) break;          // B: partial sums / candidate masses visible
+                    if (my == kHist) {
+                        unsigned long long p4[4];
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) p4[k] = sm.part[k][r];
                         if (first_level) {                        // Z and the target
-                            unsigned long long z = 0ull;
-#pragma unroll 8
-                            for (int b = 0; b < 64; ++b) z += hist[b * 128] >> 13;
+                            const unsigned long long z = (p4[0] + p4[1]) + (p4[2] + p4[3]);
                             target = kByCount ? (z < (unsigned long long)g.top_k ? z : (unsigned long long)g.top_k)
                                               : (unsigned long long)ceil((double)z * g.top_p);
                             if (target == 0ull) target = 1ull;
                         }
                         unsigned long long cum = base;
-                        int cb = 63, cnt = 0;
-                        for (int b = 0; b < 64; ++b) {
-                            const unsigned long long e = hist[b * 128];
-                            if (cum + (e >> 13) >= target) { cb = b; cnt = (int)(e & 8191ull); break; }
-                            cum += e >> 13;
+                        int kk = 3;
+#pragma unroll
+                        for (int k = 0; k < 3; ++k)
+                            if (kk == 3 && cum + p4[k] >= target) kk = k; else if (kk == 3) cum += p4[k];
+                        if (part == kk) {                         // the crossing bucket is one of mine
+                            int cb = 15, cnt = 0;
+                            for (int b = 0; b < 16; ++b) {
+                                const unsigned long long e = hist[(part * 16 + b) * 128];
+                                if (cum + (e >> 13) >= target || b == 15) { cb = b; cnt = (int)(e & 8191ull); break; }
+                                cum += e >> 13;
+                            }
+                            sm.res_base[r] = cum;
+                            sm.res_cb[r] = (part * 16 + cb) | (cnt << 8);
                         }
-                        base = cum;
+#pragma unroll
+                        for (int b = 0; b < 16; ++b) hist[(part * 16 + b) * 128] = 0ull;   // ready for the next histogram pass
+                    } else if (my == kCollect) {
+                        // the crossing cube among the collected ones: the smallest key whose mass, added to
+                        // that of all smaller keys and of everything above the interval, reaches the target
+                        unsigned long long best = ~0ull;
+                        if (n_cand <= kCandCap) {
+                            for (int i = part; i < n_cand; i += 4) {
+                                const unsigned long long ki = cand[i * 128];
+                                unsigned long long acc = base;
+                                for (int k = 0; k < n_cand; ++k) acc += cand[k * 128] <= ki ? hist[k * 128] : 0ull;
+                                if (acc >= target && ki < best) best = ki;
+                            }
+                        }
+                        sm.part[part][r] = best;
+                    }
+                    if (!(ok = sync_selection())) break;          // C: results visible
+                    if (my == kHist) {
+                        ++hist_passes;
+                        const int rc = sm.res_cb[r];
+                        const int cb = rc & 63, cnt = rc >> 8;
+                        base = sm.res_base[r];
                         const bool open_end = span == kOpen && cb == 63;   // the crossing lies beyond the window
                         lo += (unsigned long long)cb << sh;
                         if (!open_end) {
@@ -580,38 +644,26 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
                         if (state == kCollect && cnt > kCandCap) { state = kDone; give_up = true; }   // more exact ties than slots
                         if (state == kHist && hist_passes >= kMaxHistPasses) { state = kDone; give_up = true; }
                     } else if (my == kCollect) {
-                        // the crossing cube among the collected ones: the smallest key whose mass, added to
-                        // that of all smaller keys and of everything above the interval, reaches the target
                         if (n_cand > kCandCap) {
                             give_up = true;
                         } else {
-                            for (int k = 0; k < n_cand; ++k) {
-                                unsigned long long m = 1ull;
-                                if (!kByCount) {
-                                    const unsigned long long delta = cand[k * 128] >> 12;
-                                    const double dd = __hiloint2double(0x43300000 | (int)(delta >> 32), (int)(uint32_t)delta) - 4503599627370496.0;
-                                    m = mass38(dd * neg_f);
-                                }
-                                hist[k * 128] = m;
-                            }
-                            unsigned long long best = ~0ull;
-                            for (int i = 0; i < n_cand; ++i) {
-                                const unsigned long long ki = cand[i * 128];
-                                unsigned long long acc = base;
-                                for (int k = 0; k < n_cand; ++k) acc += cand[k * 128] <= ki ? hist[k * 128] : 0ull;
-                                if (acc >= target && ki < best) best = ki;
-                            }
-                            for (int k = 0; k < n_cand; ++k) {
+                            unsigned long long best = sm.part[0][r];
+#pragma unroll
+                            for (int k = 1; k < 4; ++k) best = min(best, sm.part[k][r]);
+                            int added = 0;
+                            for (int k = part; k < n_cand; k += 4) {
                                 const unsigned long long kk = cand[k * 128];
                                 if (kk <= best) {
                                     const int j = (int)(kk & 4095ull);
                                     const uint32_t bit = 1u << (j & 31);
-                                    mask_row[(size_t)(j >> 5) * kTileRows] |= bit;
-                                    if (bm_row) bm_row[j >> 5] |= bit;
+                                    atomicOr(mask_row + (size_t)(j >> 5) * kTileRows, bit);
+                                    if (bm_row) atomicOr(bm_row + (j >> 5), bit);
                                     atomicOr(&sm.tile_union[t_par][j >> 5], bit);
-                                    ++count;
+                                    ++added;
                                 }
                             }
+                            if (added) atomicAdd(&sm.row_count[r], added);
+                            for (int k = part; k < kCandCap; k += 4) hist[k * 128] = 0ull;   // the masses kept there
                         }
                         state = kDone;
                     }
@@ -628,15 +680,21 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
                 if (!ok) break;
                 d0 += fpass;
                 ++n_done;
+            }
+            // ---------------- end of the tile: union words, counts, rows handed over
+            if (!(ok = sync_selection())) break;
+            if (part == 0) {
+                if (extra && sel_count) sel_count[raster_row] = sm.row_count[r];
+                sm.row_count[r] = 0;
+                sm.cand_cnt[r] = 0;
                 if (give_up) {
                     const uint32_t slot = atomicAdd(fallback_count, 1u);
                     fallback_rows[slot] = (int32_t)(gt_cap * kTileRows + r);
                 }
+            } else if (part == 1 && r < g.n_words) {
+                tile_union[gt_cap * g.n_words + r] = sm.tile_union[t_par][r];
+                sm.tile_union[t_par][r] = 0u;             // this buffer is used again by the tile after the next
             }
-            if (extra && sel_count) sel_count[raster_row] = count;
-            // ---------------- the tile's union words
-            if (!(ok = sync_selection())) break;
-            if (r < g.n_words) tile_union[gt_cap * g.n_words + r] = sm.tile_union[t_par][r];
         }
     }
     // ---------------------------------------------------------------- teardown
