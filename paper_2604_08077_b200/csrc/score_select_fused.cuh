@@ -47,9 +47,9 @@
 //                are in registers
 //   warps 16-19  slicers (one thread per row): digit planes of the next tile's queries into shared memory
 //   warp 20      TMA producer: key digit planes of one column tile (4 x 8 KB; 2 x 8 KB in pass A), 2 slots
-//   warp 21      issues the tcgen05.mma stream (40 of 128x64x32 per column tile, 12 in pass A) into
-//                double-buffered accumulator sets (2 x 4 levels x 64 columns = all 512 TMEM columns)
-//   warps 22-23  idle (they complete the sixth warpgroup for the register re-allocation)
+//   warps 21-22  issue the tcgen05.mma stream (40 of 128x64x32 per column tile, 12 in pass A; half each)
+//                into double-buffered accumulator sets (2 x 4 levels x 64 columns = all 512 TMEM columns)
+//   warp 23      idle (it completes the sixth warpgroup for the register re-allocation)
 #pragma once
 #include "tc_common.cuh"
 
@@ -172,7 +172,7 @@ struct FusedSmem {
     uint32_t tile_union[2][128];                                   // OR over the tile's rows of each selection word
     int32_t eq[2][128];                                            // exponent e_q of each row of the tile (by tile parity)
     int32_t need[4];                                               // decision ring: d + 1 = "another pass after the next"
-    uint64_t q_sliced, qd_free, k_full[2], acc_full[2], acc_free[2], decided[4], sel_sync;
+    uint64_t q_sliced, qd_free, k_full[2], acc_full[2], acc_free[2], decided[4], sel_sync, quarter_sync[4];
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -200,6 +200,13 @@ __device__ __forceinline__ void tmem_ld_32x8(uint32_t taddr, uint32_t (&r)[8]) {
                  : "memory");
 }
 
+__device__ __forceinline__ void tmem_ld_32x4(uint32_t taddr, uint32_t* r) {   // 4 consecutive columns
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];\n"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(taddr)
+                 : "memory");
+}
+
 // q_cube: cube-major bf16 queries [B*Hq, S_cap, D].  tile_mask as mask_index() describes;
 // tile_union[((b*Hq+h)*n_tiles_cap + tile)*n_words + w] = OR of word w over the tile's rows.
 // fallback_rows[0 .. *fallback_count) receives ((b*Hq+h)*n_tiles_cap + tile)*128 + r of the rows left
@@ -218,18 +225,20 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid == 0) {
-        tc::mbar_init(&sm.q_sliced, 128);
-        tc::mbar_init(&sm.qd_free, 1);
+        tc::mbar_init(&sm.q_sliced, 4);                     // one arrival per slicer warp
+        tc::mbar_init(&sm.qd_free, 2);
         for (int i = 0; i < 2; ++i) {
             tc::mbar_init(&sm.k_full[i], 1);
-            tc::mbar_init(&sm.acc_full[i], 1);
-            tc::mbar_init(&sm.acc_free[i], kSelThreads);
+            tc::mbar_init(&sm.acc_full[i], 2);                // one commit per MMA-issuing thread
+            tc::mbar_init(&sm.acc_free[i], kSelThreads / 32);   // one arrival per selection warp:
+            // 512 single arrivals on one barrier word serialise and cost more than the work between them
         }
         for (int i = 0; i < 4; ++i) {
-            tc::mbar_init(&sm.decided[i], kSelThreads);
+            tc::mbar_init(&sm.decided[i], kSelThreads / 32);
             sm.need[i] = 0;
         }
-        tc::mbar_init(&sm.sel_sync, kSelThreads);
+        tc::mbar_init(&sm.sel_sync, kSelThreads / 32);
+        for (int i = 0; i < 4; ++i) tc::mbar_init(&sm.quarter_sync[i], 4);   // the four warps that share 32 rows
         sm.abort_flag = 0;
         tc::fence_barrier_init();
     }
@@ -289,8 +298,12 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
                 d0 += f;
             }
         }
-    } else if (warp == kMmaWarp) {
-        // ------------------------------------------------------------ MMA issuer
+    } else if (warp == kMmaWarp || warp == kMmaWarp + 1) {
+        // ------------------------------------------------------------ MMA issuers
+        // Two threads issue the stream (one thread alone is the bottleneck: ~95 cycles per 128x64x32 MMA):
+        // issuer 0 owns the accumulators of levels 0 and 3, issuer 1 those of levels 1 and 2 (five digit
+        // pairs each, no accumulator shared); a job is ready when both have committed.
+        const int issuer = warp - kMmaWarp;
         if (lane == 0) {
             constexpr uint32_t kQPlaneStep = (uint32_t)sizeof(sm.qd[0]) >> 4, kKPlaneStep = (uint32_t)sizeof(sm.kring[0][0]) >> 4;
             constexpr uint32_t kSlotStep = (uint32_t)sizeof(sm.kring[0]) >> 4, kKStep = 32 >> 4;
@@ -310,29 +323,20 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
                         if (!(ok = tc::mbar_wait(&sm.k_full[s], use & 1, abort_flag))) break;
                         tc::tc_fence_after_sync();
                         const uint32_t kb0 = k_lo0 + s * kSlotStep;
-                        if (f < 0) {
-                            // anchor pass: S_0 = Q_0 K_0, S_1 = Q_0 K_1 + Q_1 K_0
+                        // level L = a + blk: plane a of the queries, plane blk of the keys; the anchor pass
+                        // computes levels 0 and 1 only (S_0 = Q_0 K_0, S_1 = Q_0 K_1 + Q_1 K_0)
+                        const int n_levels = f < 0 ? 2 : 4;
 #pragma unroll
-                            for (int blk = 0; blk < 2; ++blk)
+                        for (int L = 0; L < 4; ++L) {
+                            if (L >= n_levels || ((L == 0 || L == 3) ? 0 : 1) != issuer) continue;
 #pragma unroll
-                                for (int a = 0; a + blk <= 1; ++a)
+                            for (int a = 0; a <= L; ++a)
 #pragma unroll
-                                    for (int ks = 0; ks < 4; ++ks)
-                                        tc::umma_ss_i8(tbase + s * 256 + (a + blk) * kScoreTcCols,
-                                                       tc::smem_desc_from_halves(q_lo0 + a * kQPlaneStep + ks * kKStep, tc::kSmemDescHiSw128),
-                                                       tc::smem_desc_from_halves(kb0 + blk * kKPlaneStep + ks * kKStep, tc::kSmemDescHiSw128),
-                                                       kIdesc, !(blk == 0 && ks == 0));
-                        } else {
-#pragma unroll
-                            for (int blk = 0; blk < 4; ++blk)     // plane blk of the keys, plane a of the queries: level a + blk
-#pragma unroll
-                                for (int a = 0; a + blk <= 3; ++a)
-#pragma unroll
-                                    for (int ks = 0; ks < 4; ++ks)
-                                        tc::umma_ss_i8(tbase + s * 256 + (a + blk) * kScoreTcCols,
-                                                       tc::smem_desc_from_halves(q_lo0 + a * kQPlaneStep + ks * kKStep, tc::kSmemDescHiSw128),
-                                                       tc::smem_desc_from_halves(kb0 + blk * kKPlaneStep + ks * kKStep, tc::kSmemDescHiSw128),
-                                                       kIdesc, !(blk == 0 && ks == 0));
+                                for (int ks = 0; ks < 4; ++ks)
+                                    tc::umma_ss_i8(tbase + s * 256 + L * kScoreTcCols,
+                                                   tc::smem_desc_from_halves(q_lo0 + a * kQPlaneStep + ks * kKStep, tc::kSmemDescHiSw128),
+                                                   tc::smem_desc_from_halves(kb0 + (L - a) * kKPlaneStep + ks * kKStep, tc::kSmemDescHiSw128),
+                                                   kIdesc, !(a == 0 && ks == 0));
                         }
                         tc::umma_commit(&sm.acc_full[s]);         // accumulators ready; the key slot may be reloaded
                     }
@@ -340,7 +344,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
                     if (f >= 2 && !another_pass(d0 + f - 2, ok)) break;
                 }
                 d0 += f;
-                if (ok) tc::umma_commit(&sm.qd_free);             // the digit planes may be overwritten
+                if (ok) tc::umma_commit(&sm.qd_free);             // the digit planes may be overwritten (both issuers)
                 ++n_done;
             }
         }
@@ -398,7 +402,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
                     *reinterpret_cast<uint4*>(dst + (size_t)pl * sizeof(sm.qd[0]) + off) = make_uint4(pw[pl][0], pw[pl][1], pw[pl][2], pw[pl][3]);
             }
             asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");   // digit planes visible to the tensor core
-            tc::mbar_arrive(&sm.q_sliced);
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(&sm.q_sliced);
             ++n_done;
         }
     } else if (warp < kSlicerWarp0) {
@@ -406,21 +411,37 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kSelRegs));
         const int quarter = warp & 3, part = warp >> 2;
         const int r = quarter * 32 + lane;
-        const uint32_t lane_addr = tbase + ((uint32_t)(quarter * 32) << 16) + part * 16;
+        const uint32_t lane_addr = tbase + ((uint32_t)(quarter * 32) << 16);
         unsigned long long* hist = &sm.hist[0][r];                // bucket b at hist[b * 128]
         unsigned long long* cand = &sm.cand[0][r];                // slot k at cand[k * 128]
         enum { kDone = 0, kHist = 1, kCollect = 2 };
         constexpr long long kLoMax = 3ll * (1ll << 29) + (1ll << 23);      // >= |S_2*256 + S_3|
         constexpr unsigned long long kOpen = 1ull << 62;          // span of an interval without upper end
         bool ok = true;
-        int c = 0, d0 = 0, n_done = 0, t_par = 0, n_sync = 0;
-        // barrier among the 512 selection threads (a bounded wait like every other one here)
+        int c = 0, d0 = 0, n_done = 0, t_par = 0, n_sync = 0, n_qsync = 0;
+        // barrier among the four warps that serve the same 32 rows (bounded like every other wait here)
+        auto sync_rows = [&]() -> bool {
+            __threadfence_block();
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(&sm.quarter_sync[quarter]);
+            const bool done = tc::mbar_wait(&sm.quarter_sync[quarter], n_qsync & 1, abort_flag);
+            ++n_qsync;
+            return done;
+        };
+        // barrier among all 512 selection threads
         auto sync_selection = [&]() -> bool {
             __threadfence_block();
-            tc::mbar_arrive(&sm.sel_sync);
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(&sm.sel_sync);
             const bool done = tc::mbar_wait(&sm.sel_sync, n_sync & 1, abort_flag);
             ++n_sync;
             return done;
+        };
+        // this warp has read its part of accumulator set s (one arrival per warp)
+        auto release_acc = [&](int s) {
+            tc::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(&sm.acc_free[s]);
         };
         auto to_double = [](unsigned long long d) -> double {     // exact for d < 2^52
             return __hiloint2double(0x43300000 | (int)(d >> 32), (int)(uint32_t)d) - 4503599627370496.0;
@@ -436,8 +457,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
             const bool extra = live && (sel_bitmap != nullptr || sel_count != nullptr);
             const size_t raster_row = extra ? (size_t)(w.b * g.Hq + w.h) * g.S + pos_to_raster(g, pos) : 0;
             uint32_t* bm_row = (extra && sel_bitmap) ? sel_bitmap + raster_row * g.n_words : nullptr;
-            // words beyond the tile's column tiles are zero (all words of a row without candidates)
-            for (int wd = (n > 0 ? 2 * w.n_ct : 0) + part; wd < g.n_words; wd += 4) {
+            // every word starts at zero: the collect pass ORs the selected cubes' bits into them
+            for (int wd = part; wd < g.n_words; wd += 4) {
                 mask_row[(size_t)wd * kTileRows] = 0u;
                 if (bm_row) bm_row[wd] = 0u;
             }
@@ -452,22 +473,20 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
                     const int col0 = ct * kScoreTcCols + part * 16;
                     if (col0 < n_warp) {
                         uint32_t l0[16], l1[16];
-                        tc::tmem_ld_32x16(lane_addr + s * 256, l0);
-                        tc::tmem_ld_32x16(lane_addr + s * 256 + kScoreTcCols, l1);
+                        tc::tmem_ld_32x16(lane_addr + s * 256 + part * 16, l0);
+                        tc::tmem_ld_32x16(lane_addr + s * 256 + kScoreTcCols + part * 16, l1);
                         tc::tmem_wait_ld();
-                        tc::tc_fence_before_sync();
-                        tc::mbar_arrive(&sm.acc_free[s]);
+                        release_acc(s);
 #pragma unroll
                         for (int i = 0; i < 16; ++i)
                             if (col0 + i < n) max_hi = max(max_hi, (int)l0[i] * 256 + (int)l1[i]);
                     } else {
-                        tc::tc_fence_before_sync();
-                        tc::mbar_arrive(&sm.acc_free[s]);
+                        release_acc(s);
                     }
                 }
                 if (!ok) break;
                 sm.part[part][r] = (unsigned long long)(long long)max_hi;
-                if (!(ok = sync_selection())) break;
+                if (!(ok = sync_rows())) break;
 #pragma unroll
                 for (int k = 0; k < 4; ++k) max_hi = max(max_hi, (int)(long long)sm.part[k][r]);
                 // ---------------- per-row constants (the same in the row's four threads)
@@ -494,19 +513,21 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
                         const int s = c & 1;
                         if (!(ok = tc::mbar_wait(&sm.acc_full[s], (c >> 1) & 1, abort_flag))) break;
                         tc::tc_fence_after_sync();
-                        const int col0 = ct * kScoreTcCols + part * 16;
-                        uint32_t word = 0;                        // 16 bits: cubes col0 .. col0 + 15
-                        if (col0 < n_warp && !warp_idle) {
+                        // This thread's columns of the job: 4*part .. +3 of every group of 16 (interleaved, so
+                        // that a ragged last column tile loads the row's four threads alike); half hf = one 32-cube word
 #pragma unroll
-                            for (int hf = 0; hf < 2; ++hf) {
+                        for (int hf = 0; hf < 2; ++hf) {
+                            const int colh = ct * kScoreTcCols + hf * 32 + part * 4;    // first column of this half
+                            uint32_t bits = 0;
+                            if (colh < n_warp && !warp_idle) {
                                 uint32_t lv[4][8];
 #pragma unroll
-                                for (int L = 0; L < 4; ++L) tmem_ld_32x8(lane_addr + s * 256 + L * kScoreTcCols + hf * 8, lv[L]);
-                                tc::tmem_wait_ld();
-                                if (hf == 1) {                    // last read of this accumulator set: release it
-                                    tc::tc_fence_before_sync();
-                                    tc::mbar_arrive(&sm.acc_free[s]);
+                                for (int L = 0; L < 4; ++L) {
+                                    tmem_ld_32x4(lane_addr + s * 256 + L * kScoreTcCols + hf * 32 + part * 4, &lv[L][0]);
+                                    tmem_ld_32x4(lane_addr + s * 256 + L * kScoreTcCols + hf * 32 + 16 + part * 4, &lv[L][4]);
                                 }
+                                tc::tmem_wait_ld();
+                                if (hf == 1) release_acc(s);      // last read of this accumulator set
                                 if (my == kHist) {
 #pragma unroll
                                     for (int i0 = 0; i0 < 8; i0 += 4) {        // four independent mass evaluations at a time
@@ -519,7 +540,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
                                             const int hi = (int)lv[0][i] * 256 + (int)lv[1][i];
                                             const int lw = (int)lv[2][i] * 256 + (int)lv[3][i];
                                             delta[u] = (unsigned long long)(VA - ((long long)hi * 65536 + lw));
-                                            in[u] = col0 + hf * 8 + i < n && delta[u] - lo <= span;
+                                            in[u] = colh + (i0 >> 2) * 16 + u < n && delta[u] - lo <= span;
                                             any_in |= in[u];
                                         }
                                         if (!any_in) continue;
@@ -541,36 +562,33 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
                                         const int hi = (int)lv[0][i] * 256 + (int)lv[1][i];
                                         const int lw = (int)lv[2][i] * 256 + (int)lv[3][i];
                                         const unsigned long long delta = (unsigned long long)(VA - ((long long)hi * 65536 + lw));
-                                        const int j = col0 + hf * 8 + i;
+                                        const int j = colh + (i >> 2) * 16 + (i & 3);
                                         const bool in_row = j < n;
                                         if (in_row && delta - lo <= span) {
                                             const int slot = atomicAdd(&sm.cand_cnt[r], 1);
                                             if (slot < kCandCap) cand[slot * 128] = (delta << 12) | (unsigned long long)j;
                                         }
-                                        word |= ((in_row && delta < lo) ? 1u : 0u) << (hf * 8 + i);
+                                        bits |= ((in_row && delta < lo) ? 1u : 0u) << ((i >> 2) * 16 + part * 4 + (i & 3));
                                     }
                                 }
+                            } else if (hf == 1) {
+                                release_acc(s);
                             }
-                        } else {
-                            tc::tc_fence_before_sync();
-                            tc::mbar_arrive(&sm.acc_free[s]);
-                        }
-                        // this thread's half of a 32-cube word
-                        const int wd = ct * 2 + (part >> 1);
-                        if (wd < g.n_words && !warp_idle) {
-                            const bool wr = my == kCollect;
-                            if (wr) {
-                                reinterpret_cast<uint16_t*>(mask_row + (size_t)wd * kTileRows)[part & 1] = (uint16_t)word;
-                                if (bm_row) reinterpret_cast<uint16_t*>(bm_row + wd)[part & 1] = (uint16_t)word;
-                                if (word) atomicAdd(&sm.row_count[r], __popc(word));
+                            if (!warp_idle && my == kCollect && bits) {
+                                const int wd = ct * 2 + hf;
+                                atomicOr(mask_row + (size_t)wd * kTileRows, bits);
+                                if (bm_row) atomicOr(bm_row + wd, bits);
+                                atomicAdd(&sm.row_count[r], __popc(bits));
                             }
-                            const uint32_t u = __reduce_or_sync(0xffffffffu, wr ? word : 0u);
-                            if (lane == 0 && u) atomicOr(&sm.tile_union[t_par][wd], u << ((part & 1) * 16));
+                            if (!warp_idle) {
+                                const uint32_t u = __reduce_or_sync(0xffffffffu, bits);
+                                if (lane == 0 && u) atomicOr(&sm.tile_union[t_par][ct * 2 + hf], u);
+                            }
                         }
                     }
                     if (!ok) break;
                     // ---------------- end of the pass: the row's four threads combine (three barriers, whatever the rows do)
-                    if (!(ok = sync_selection())) break;          // A: histogram / candidate list complete
+                    if (!(ok = sync_rows())) break;               // A: histogram / candidate list complete
                     int n_cand = 0;
                     if (my == kHist) {
                         unsigned long long ps = 0ull;
@@ -583,7 +601,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
                             for (int k = part; k < n_cand; k += 4)
                                 hist[k * 128] = kByCount ? 1ull : mass38(to_double(cand[k * 128] >> 12) * neg_f);
                     }
-                    if (!(ok = sync_selection())) break;          // B: partial sums / candidate masses visible
+                    if (!(ok = sync_rows())) break;               // B: partial sums / candidate masses visible
                     if (my == kHist) {
                         unsigned long long p4[4];
 #pragma unroll
@@ -625,7 +643,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
                         }
                         sm.part[part][r] = best;
                     }
-                    if (!(ok = sync_selection())) break;          // C: results visible
+                    if (!(ok = sync_rows())) break;               // C: results visible
                     if (my == kHist) {
                         ++hist_passes;
                         const int rc = sm.res_cb[r];
@@ -671,7 +689,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
                     const int d = d0 + fpass;
                     if (state == kHist) *reinterpret_cast<volatile int32_t*>(&sm.need[d & 3]) = d + 1;
                     __threadfence_block();
-                    tc::mbar_arrive(&sm.decided[d & 3]);
+                    __syncwarp();
+                    if (lane == 0) tc::mbar_arrive(&sm.decided[d & 3]);
                     ++fpass;
                     bool more = true;
                     if (fpass >= 2) more = another_pass(d0 + fpass - 2, ok);
