@@ -391,18 +391,26 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
             // ---- P = 2^(s*scale - m_ref) on visible keys, 0 elsewhere; bf16 pairs into TMEM
             const float neg_ref = -m_ref;                          // finite whenever a key is visible
             if (uniform) {
-                float ps0 = 0.f, ps1 = 0.f, ps2 = 0.f, ps3 = 0.f;
+                // The softmax warps are issue-bound (moving exponentials to an FMA polynomial only slowed
+                // the kernel), so the scale-subtract and the row sums use the packed fp32x2 instructions:
+                // 10 instead of 14 instructions per four keys.
+                unsigned long long psA = 0ull, psB = 0ull;             // two packed pairs of partial row sums
+                const unsigned long long scale2 = pack_f32x2(scale_log2, scale_log2);
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     const float addend = amask[c] ? neg_ref : -INFINITY;   // 2^(-inf) = 0 hides the chunk
+                    const unsigned long long add2 = pack_f32x2(addend, addend);
                     uint32_t pk[16];
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
-                        const float p0 = fast_exp2(fmaf(__uint_as_float(s[c][4 * i]), scale_log2, addend));
-                        const float p1 = fast_exp2(fmaf(__uint_as_float(s[c][4 * i + 1]), scale_log2, addend));
-                        const float p2 = fast_exp2(fmaf(__uint_as_float(s[c][4 * i + 2]), scale_log2, addend));
-                        const float p3 = fast_exp2(fmaf(__uint_as_float(s[c][4 * i + 3]), scale_log2, addend));
-                        ps0 += p0; ps1 += p1; ps2 += p2; ps3 += p3;
+                        const unsigned long long x01 = fma_f32x2(pack_f32x2(__uint_as_float(s[c][4 * i]), __uint_as_float(s[c][4 * i + 1])), scale2, add2);
+                        const unsigned long long x23 = fma_f32x2(pack_f32x2(__uint_as_float(s[c][4 * i + 2]), __uint_as_float(s[c][4 * i + 3])), scale2, add2);
+                        float x0, x1, x2, x3;
+                        unpack_f32x2(x01, x0, x1);
+                        unpack_f32x2(x23, x2, x3);
+                        const float p0 = fast_exp2(x0), p1 = fast_exp2(x1), p2 = fast_exp2(x2), p3 = fast_exp2(x3);
+                        psA = add_f32x2(psA, pack_f32x2(p0, p1));
+                        psB = add_f32x2(psB, pack_f32x2(p2, p3));
                         pk[2 * i] = pack_bf16x2(p0, p1);
                         pk[2 * i + 1] = pack_bf16x2(p2, p3);
                     }
@@ -413,7 +421,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
                         tc::mbar_arrive(&sm.p_half[t][0]);
                     }
                 }
-                l_sum += (ps0 + ps1) + (ps2 + ps3);
+                float a0, a1, b0, b1;
+                unpack_f32x2(psA, a0, a1);
+                unpack_f32x2(psB, b0, b1);
+                l_sum += (a0 + a1) + (b0 + b1);
             } else {
                 float ps0 = 0.f, ps1 = 0.f;
 #pragma unroll
