@@ -37,10 +37,22 @@ WORKLOAD = ("config2: AdaS-Attn prefill, batch 1, 64x16x16 video tokens (cube 4x
             "+ 128 text, 28/4 heads, head_dim 128, p=0.9")
 
 
-# DRAM bytes (read + write) of one launch of the prefill attention kernel on this workload, from the
-# ncu capture summarised in profiles/attn_prefill_tc_kernel_config2.md.  Set to None whenever that
-# kernel changes until the counters are taken again.
-ATTN_DRAM_TRAFFIC_BYTES = 256.1e6
+def profiled_traffic(kernel_source: str, summary: str):
+    """DRAM bytes per launch of a kernel from its committed ncu summary, or None when the kernel's
+    source file no longer has the hash the summary was taken with (the counters are then stale).
+    The summary carries two lines: `dram_bytes_per_launch: <n>` and `kernel_source_sha256: <hex>`."""
+    import hashlib
+    import re
+    try:
+        text = open(os.path.join(ROOT, "profiles", summary)).read()
+        src = open(os.path.join(ROOT, "paper_2604_08077_b200", "csrc", kernel_source), "rb").read()
+    except OSError:
+        return None
+    m_bytes = re.search(r"dram_bytes_per_launch:\s*([0-9.eE+]+)", text)
+    m_hash = re.search(r"kernel_source_sha256:\s*([0-9a-f]{64})", text)
+    if not m_bytes or not m_hash or hashlib.sha256(src).hexdigest() != m_hash.group(1):
+        return None
+    return float(m_bytes.group(1))
 
 
 def load_peaks():
@@ -187,6 +199,43 @@ def run_reference(args):
                 "d2h_bytes_per_step": 0}}))
 
 
+def parity_check(wl, eng, q, k, v, n_rows=1200, n_sel_rows=12000):
+    """The CUDA path against the CPU oracle on seeded rows of the bench workload, before anything is
+    timed: selection on n_sel_rows rows, outputs on n_rows of them.  Rows outside the 1e-6 tie margin
+    must match bit for bit; rows inside it are counted (`differing`) and their outputs compared with
+    the oracle's attention on the GPU's own set.  Raises on a mismatch."""
+    import oracle
+    sh = oracle.shape_of(wl, top_p=float(np.float32(wl.top_p)))
+    out, bitmap, _ = eng.forward(q, k, v, wl.n_text, want_selection=True)
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(11)
+    rows = np.stack([np.zeros(n_sel_rows, np.int64), rng.integers(0, wl.Hq, n_sel_rows),
+                     rng.integers(0, wl.S, n_sel_rows)], axis=1)
+    kbar = oracle.mean_keys(sh, wl.k)
+    res = oracle.rows(sh, wl.q, wl.k, wl.v, rows, kbar=kbar, attend=False)
+    dev = bitmap.device
+    hh, nn = torch.from_numpy(rows[:, 1]).to(dev), torch.from_numpy(rows[:, 2]).to(dev)
+    words = bitmap[0, hh, nn].cpu().numpy().view(np.uint32)
+    got_sel = ((words[..., None] >> np.arange(32, dtype=np.uint32)) & 1).reshape(len(rows), -1)[:, :sh.N].astype(np.uint8)
+    same = (got_sel == res["sel"]).all(axis=1)
+    near = res["margin"] < 1e-6
+    if not (same | near).all():
+        raise SystemExit("bench: selection differs from the oracle outside the 1e-6 tie margin")
+    sub = rows[:n_rows]
+    ref = oracle.rows(sh, wl.q, wl.k, wl.v, sub, kbar=kbar)["out"]
+    if not same[:n_rows].all():
+        bad = ~same[:n_rows]
+        ref[bad] = oracle.attend_given(sh, wl.q, wl.k, wl.v, sub[bad], got_sel[:n_rows][bad])
+    got = out[0, nn[:n_rows], hh[:n_rows]].float().cpu().numpy()
+    max_abs = float(np.abs(got - ref).max())
+    mean_rel = float(np.abs(got - ref).mean() / np.abs(ref).mean())
+    if max_abs > 2e-2 or mean_rel > 1e-2:
+        raise SystemExit(f"bench: outputs differ from the oracle (max abs {max_abs}, mean rel {mean_rel})")
+    return {"rows": int(n_sel_rows), "output_rows": int(n_rows), "differing": int((~same).sum()),
+            "near_tie": int(near.sum()), "max_abs": max_abs, "mean_rel": mean_rel,
+            "fallback_rows": int(eng.header().fallback_rows)}
+
+
 def cpu_baseline(wl, n_rows=32768):
     import oracle
     sh = oracle.shape_of(wl, top_p=float(np.float32(wl.top_p)))
@@ -215,6 +264,8 @@ def main():
     ap.add_argument("--no-dense", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-cohesive", action="store_true")
+    ap.add_argument("--no-parity", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the config-3 sweep and config 4")
     ap.add_argument("--decode-batch", type=int, default=16)
     ap.add_argument("--prefill-kernel", type=int, default=None)
     args = ap.parse_args()
@@ -262,6 +313,10 @@ def main():
 
     def flush():
         flush_buf.fill_(1)
+
+    parity = None
+    if rank == 0 and not args.no_parity:
+        parity = parity_check(wl, eng, q, k, v)
 
     def step():
         eng.forward(q, k, v, wl.n_text, out=out)
@@ -358,11 +413,12 @@ def main():
         "gpu_launches": launches_per_step * args.steps,
         "roofline": {"kernel": "prefill attention", "bound": "tensor", "achieved": achieved_tflops,
                      "peak": peak_tflops, "unit": "TFLOP/s", "frac": achieved_tflops / peak_tflops,
-                     "traffic": ATTN_DRAM_TRAFFIC_BYTES,
+                     "traffic": profiled_traffic("attn_prefill_tc.cuh", "attn_prefill_tc_kernel_config2.md"),
                      "traffic_unit": "bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum)",
                      "peak_source": f"{peaks['source']} bf16 burst (kernel of ~ms inside a ~ms step)"},
         "stages_ms": {"relayout_pool": float(st_mean[0]), "score_select": float(st_mean[1]),
                       "attention": attn_ms},
+        "parity": parity,
         "flops": {"executed": executed_flops, "useful": useful_flops, "dense_causal": dense_flops,
                   "useful_over_executed": useful_flops / max(executed_flops, 1.0),
                   "effective_tflops_executed": executed_flops / (ms_max * 1e-3) / 1e12,
@@ -393,6 +449,99 @@ def main():
             del eng1
         except Exception as e:  # comparison only
             result["dense"] = {"error": repr(e)[:200]}
+
+    # ------------------------------------------------------------------ rooflines of the other stages
+    # re-layout + pooling (K/V once in, once out, fp32 keys) and the Q re-layout: HBM-bound copies
+    relayout_bytes = 2 * (k.numel() + v.numel()) * 2 + wl.B * wl.Hkv * wl.N * wl.D * 4 + 2 * q.numel() * 2
+    rl_gbs = relayout_bytes / (float(st_mean[0]) * 1e-3) / 1e9
+    # scoring + selection: candidate (row, cube) pairs; algorithmic bytes = Q once + mean keys + mask words
+    n_tiles = (wl.S + 127) // 128
+    pos = np.arange(wl.S)
+    cand_per_row = np.where(pos < wl.S_v, pos // C, wl.N)
+    pairs = float(cand_per_row.sum()) * wl.B * wl.Hq
+    ss_bytes = q.numel() * 2 + wl.B * wl.Hkv * wl.N * wl.D * 4 + wl.B * wl.Hq * n_tiles * 128 * ((wl.N + 31) // 32) * 4
+    ss_ms = float(st_mean[1])
+    result["stage_rooflines"] = {
+        "relayout": {"bound": "hbm", "bytes": relayout_bytes, "ms": float(st_mean[0]), "achieved": rl_gbs,
+                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": rl_gbs / peaks["hbm_gbs"]},
+        "score_select": {"bound": "alu", "candidate_pairs": pairs, "ms": ss_ms,
+                         "achieved": pairs / (ss_ms * 1e-3) / 1e9, "unit": "G candidate (row, cube) pairs/s",
+                         "algorithmic_bytes": ss_bytes, "hbm_floor_ms": ss_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3,
+                         "useful_flops": 2.0 * wl.D * pairs},
+    }
+
+    # ------------------------------------------------------------------ config 3 sweep and config 4
+    def one_config(wx, p, n_steps=3):
+        e = binding.AdaSAttn(cube=wx.cube, n_q_heads=wx.Hq, n_kv_heads=wx.Hkv, head_dim=wx.D, top_p=p,
+                             device=local_rank)
+        e.partition(wx.B, wx.T, wx.H, wx.W, wx.n_text)
+        binding.adaspark_attn_enable_stage_timing(e.handle, True)
+        ox = torch.empty_like(wx.q)
+
+        def stp():
+            e.forward(wx.q, wx.k, wx.v, wx.n_text, out=ox)
+            return lambda: binding.adaspark_attn_get_stage_times(e.handle)
+
+        t, stg = timed_steps(stp, n_steps, 3, flush, lambda: None)
+        stg = np.asarray(stg).mean(axis=0)
+        hx = e.header()
+        _, _, cnt = e.forward(wx.q, wx.k, wx.v, wx.n_text, out=ox, want_selection=True)
+        torch.cuda.synchronize()
+        sel = int(cnt.sum().item())
+        Cx = wx.C
+        local_x = wx.S_v // Cx * (Cx * (Cx + 1) // 2) + wx.n_text * (wx.n_text + 1) // 2
+        useful = 4.0 * wx.D * (sel * Cx + wx.B * wx.Hq * local_x)
+        executed = float(hx.executed_kv_blocks) * 128 * 64 * wx.D * 4
+        n_pairs = wx.B * wx.Hq * ((wx.S + 255) // 256)
+        rec = {"p": p, "forward_ms": sum(t) / len(t),
+               "stages_ms": {"relayout_pool": float(stg[0]), "score_select": float(stg[1]), "attention": float(stg[2])},
+               "mean_selected_cubes_per_row": sel / (wx.B * wx.Hq * wx.S),
+               "useful_over_executed": useful / max(executed, 1.0),
+               "executed_tflops": executed / (float(stg[2]) * 1e-3) / 1e12,
+               "kv_blocks_per_pair_tile": {"mean": float(hx.executed_kv_blocks) / 2 / n_pairs, "max": int(hx.max_tile_kv_blocks)},
+               "fallback_rows": int(hx.fallback_rows), "status": int(hx.status)}
+        e.close()
+        del e, ox, cnt
+        return rec
+
+    if not args.no_sweep and rank == 0:
+        try:
+            del bitmap, count
+            torch.cuda.empty_cache()
+            sweep = []
+            sdpa_ms = None
+            for sigma in (0.5, 1.5, 3.0):
+                w3 = inputs.config3(sigma=sigma, device="cuda")
+                if sdpa_ms is None and not args.no_dense:
+                    q3, k3, v3 = (t.permute(0, 2, 1, 3) for t in (w3.q, w3.k, w3.v))
+
+                    def sdpa3():
+                        torch.nn.functional.scaled_dot_product_attention(q3, k3, v3, is_causal=True, enable_gqa=True)
+
+                    sd3, _ = timed_steps(sdpa3, 3, 3, flush, lambda: None)
+                    del q3, k3, v3
+                    sdpa_ms = sum(sd3) / len(sd3)
+                recs = {p: one_config(w3, p) for p in (1.0, 0.95, 0.9, 0.7, 0.5)}
+                for p in (0.5, 0.7, 0.9, 0.95, 1.0):
+                    r3 = recs[p]
+                    r3["sigma"] = sigma
+                    r3["speedup_vs_own_p1"] = recs[1.0]["forward_ms"] / r3["forward_ms"]
+                    r3["speedup_vs_torch_sdpa"] = sdpa_ms / r3["forward_ms"] if sdpa_ms else None
+                    sweep.append(r3)
+                del w3
+                torch.cuda.empty_cache()
+            result["config3_sweep"] = {"workload": "config3: 256x16x16 video tokens (1024 cubes) + 256 text, 28/4 heads, "
+                                                   "head_dim 128; p=1.0 is the dense reference of the same kernels",
+                                       "torch_sdpa_causal_ms": sdpa_ms, "points": sweep}
+            w4 = inputs.config4(device="cuda")
+            r4 = one_config(w4, w4.top_p, n_steps=2)
+            r4["workload"] = "config4: 512x16x16 video tokens (2048 cubes), first half of the frames static, p=0.9"
+            r4["tokens_per_s"] = w4.B * w4.S / (r4["forward_ms"] * 1e-3)
+            result["config4"] = r4
+            del w4
+            torch.cuda.empty_cache()
+        except Exception as e:  # extra measurements only
+            result["config3_sweep"] = {"error": repr(e)[:300]}
 
     # ------------------------------------------------------------------ cohesive queries (extra workload)
     if not args.no_cohesive and rank == 0:
@@ -430,7 +579,7 @@ def main():
 
     # ------------------------------------------------------------------ decode (config 5)
     if not args.no_decode:
-        del q, k, v, out, bitmap, count
+        del q, k, v, out
         torch.cuda.empty_cache()
         wd = inputs.config5(variant=rank, B=args.decode_batch, device="cuda")
         engd = binding.AdaSAttn(cube=wd.cube, n_q_heads=wd.Hq, n_kv_heads=wd.Hkv, head_dim=wd.D,

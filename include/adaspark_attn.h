@@ -90,7 +90,9 @@ typedef struct {
     uint64_t decode_kv_blocks;    /* decode: 64-key blocks gathered, summed over (b, kv head) */
     uint32_t fallback_rows;       /* prefill: query rows whose selection the tensor-core kernel
                                      left to the fp64 selection kernel (normally 0)           */
-    uint32_t reserved2;
+    uint32_t max_tile_kv_blocks;  /* prefill: largest number of 64-key blocks one 256-row pair of
+                                     query tiles visited (load imbalance: compare with the mean
+                                     executed_kv_blocks / 2 / number of pair tiles)           */
 } adaspark_attn_workspace_header_t;
 
 /* Create a handle for one configuration.  Host only.  Fails with ERR_UNSUPPORTED for a
@@ -139,6 +141,31 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t *handle, const void *q, 
                                         void *v_cube, float *cube_keys, uint32_t *sel_bitmap,
                                         int32_t *sel_count, void *workspace,
                                         size_t workspace_bytes, void *cuda_stream);
+
+/* Chunked prefill: the same computation as adaspark_attn_forward, fed one run of frames at a time
+ * (the long-video setting of the paper: a later frame never changes an earlier row, because a video
+ * query of Eq. 1 only sees the cubes that precede its own and the text comes after the video).
+ * The call brings frames [frame_begin, frame_begin + frame_count) of every sequence: it appends
+ * their cubes to k_cube / v_cube / cube_keys and computes `out` for these tokens only, attending the
+ * cubes of earlier calls through the caches.
+ *   frame_begin, frame_count  multiples of cube_t (whole time blocks of cubes); frame_begin * H * W
+ *                must be a multiple of 256 (ERR_UNSUPPORTED otherwise).  Chunks must be fed in
+ *                order, without gaps, to the same caches; the library keeps no record of them.
+ *   n_text       < 0: more video follows (no text in this call).  >= 0: this is the last call of the
+ *                sequence: it must end the video (frame_begin + frame_count = T; frame_count may be 0
+ *                when the video is already complete), brings n_text text tokens after its frames,
+ *                and zero-fills the caches beyond the sequence up to their capacity.
+ *   q, k, v, out bf16 [B, frame_count*H*W + max(n_text, 0), H*, D]: this call's tokens in raster order
+ *                (then its text tokens).  q and out may both be NULL (caches only).
+ *   sel_bitmap / sel_count  nullable, rows of this call only: [B, Hq, tokens of the call, ...].
+ * Everything else as adaspark_attn_forward; adaspark_attn_forward(n_text) is the single chunk
+ * (0, T, n_text). */
+adaspark_status_t adaspark_attn_forward_chunk(adaspark_attn_t *handle, const void *q, const void *k,
+                                              const void *v, int32_t frame_begin, int32_t frame_count,
+                                              int32_t n_text, void *out, void *k_cube, void *v_cube,
+                                              float *cube_keys, uint32_t *sel_bitmap,
+                                              int32_t *sel_count, void *workspace,
+                                              size_t workspace_bytes, void *cuda_stream);
 
 /* Decode: one new text token per sequence (the text-token rule after Eq. 3 applied to a row
  * appended after the cached sequence; the new token attends itself).

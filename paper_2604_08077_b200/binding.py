@@ -43,7 +43,7 @@ class AdasparkError(RuntimeError):
 _lib: Optional[ctypes.CDLL] = None
 
 EXPORTS = ["adaspark_attn_create", "adaspark_attn_partition", "adaspark_attn_get_layout",
-           "adaspark_attn_forward", "adaspark_attn_decode", "adaspark_attn_destroy",
+           "adaspark_attn_forward", "adaspark_attn_forward_chunk", "adaspark_attn_decode", "adaspark_attn_destroy",
            "adaspark_attn_last_error", "adaspark_attn_last_launch_count",
            "adaspark_attn_set_prefill_kernel", "adaspark_attn_enable_stage_timing",
            "adaspark_attn_get_stage_times", "adaspark_attn_decode_static",
@@ -65,6 +65,7 @@ def load() -> ctypes.CDLL:
     lib.adaspark_attn_partition.argtypes = [vp, i32, i32, i32, i32, i32, ctypes.POINTER(sz)]
     lib.adaspark_attn_get_layout.argtypes = [vp, ctypes.POINTER(Layout)]
     lib.adaspark_attn_forward.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.adaspark_attn_forward_chunk.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.adaspark_attn_decode.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.adaspark_attn_decode_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.adaspark_attn_debug_umma_selftest.argtypes = [vp, vp, vp, vp, vp, vp, vp]
@@ -141,6 +142,15 @@ def adaspark_attn_forward(handle: int, q, k, v, n_text: int, out, k_cube, v_cube
         _stream_ptr(stream)))
 
 
+def adaspark_attn_forward_chunk(handle: int, q, k, v, frame_begin: int, frame_count: int, n_text: int, out,
+                                k_cube, v_cube, cube_keys, sel_bitmap, sel_count, workspace,
+                                workspace_bytes: int, stream=None):
+    _check(handle, load().adaspark_attn_forward_chunk(
+        handle, _ptr(q), _ptr(k), _ptr(v), frame_begin, frame_count, n_text, _ptr(out), _ptr(k_cube),
+        _ptr(v_cube), _ptr(cube_keys), _ptr(sel_bitmap), _ptr(sel_count), _ptr(workspace), workspace_bytes,
+        _stream_ptr(stream)))
+
+
 def adaspark_attn_decode(handle: int, q_new, k_new, v_new, k_cube, v_cube, cube_keys, text_len, out,
                          sel_bitmap, workspace, workspace_bytes: int, stream=None):
     _check(handle, load().adaspark_attn_decode(
@@ -211,7 +221,7 @@ def adaspark_attn_get_stage_times(handle: int):
 class WorkspaceHeader(ctypes.Structure):
     _fields_ = [("status", ctypes.c_int32), ("reserved", ctypes.c_int32),
                 ("executed_kv_blocks", ctypes.c_uint64), ("decode_kv_blocks", ctypes.c_uint64),
-                ("fallback_rows", ctypes.c_uint32), ("reserved2", ctypes.c_uint32)]
+                ("fallback_rows", ctypes.c_uint32), ("max_tile_kv_blocks", ctypes.c_uint32)]
 
 
 # ---- a small convenience owner of the handle and of the caller-side buffers --------------------
@@ -254,6 +264,23 @@ class AdaSAttn:
                 count = torch.empty(B, Hq, S, dtype=torch.int32, device=q.device)
         adaspark_attn_forward(self.handle, q, k, v, n_text, out, self.k_cube, self.v_cube,
                               self.cube_keys, bitmap, count, self.workspace, self.ws_bytes, stream)
+        return out, bitmap, count
+
+    def forward_chunk(self, q, k, v, frame_begin, frame_count, n_text, *, out=None, want_selection=False,
+                      stream=None):
+        """One chunk of a chunked prefill (n_text < 0: more video follows).  q may be None."""
+        lay = self.layout
+        bitmap = count = None
+        if q is not None:
+            if out is None:
+                out = torch.empty_like(q)
+            if want_selection:
+                B, S, Hq, _ = q.shape
+                bitmap = torch.empty(B, Hq, S, lay.bitmap_words, dtype=torch.int32, device=q.device)
+                count = torch.empty(B, Hq, S, dtype=torch.int32, device=q.device)
+        adaspark_attn_forward_chunk(self.handle, q, k, v, frame_begin, frame_count, n_text, out, self.k_cube,
+                                    self.v_cube, self.cube_keys, bitmap, count, self.workspace, self.ws_bytes,
+                                    stream)
         return out, bitmap, count
 
     def decode(self, q_new, k_new, v_new, text_len, *, out=None, want_selection=False, stream=None):

@@ -60,8 +60,11 @@ adaspark_status_t fail(adaspark_attn* h, adaspark_status_t st, const char* fmt, 
     return st;
 }
 
-Geom make_geom(const adaspark_attn* h, int n_text) {
+// Geometry of one call.  frame_begin / frame_end delimit the video frames this call brings (whole time
+// blocks of cubes); n_text text tokens are present after the call (0 while the video is incomplete).
+Geom make_geom(const adaspark_attn* h, int n_text, int frame_begin = 0, int frame_end = -1) {
     Geom g;
+    if (frame_end < 0) frame_end = h->T;
     g.B = h->B; g.T = h->T; g.H = h->H; g.W = h->W;
     g.ct = h->cfg.cube_t; g.ch = h->cfg.cube_h; g.cw = h->cfg.cube_w;
     g.nH = h->H / g.ch; g.nW = h->W / g.cw;
@@ -72,7 +75,12 @@ Geom make_geom(const adaspark_attn* h, int n_text) {
     while ((1 << g.cw_shift) < g.cw) ++g.cw_shift;
     g.ch_shift = 0;
     while ((1 << g.ch_shift) < g.ch) ++g.ch_shift;
-    g.S_v = h->S_v; g.n_text = n_text; g.S = h->S_v + n_text;
+    g.S_v = h->S_v; g.n_text = n_text;
+    g.S = frame_end * h->H * h->W + n_text;                  // n_text > 0 only once the video is complete
+    g.pos_begin = frame_begin * h->H * h->W;
+    g.S_io = g.S - g.pos_begin;
+    g.tile_begin = g.pos_begin / kTileRows;
+    g.N_live = (frame_end / h->cfg.cube_t) * (h->H / g.ch) * (h->W / g.cw);
     g.S_cap = h->S_cap;
     g.n_words = (h->N + 31) / 32;
     g.n_tiles = (g.S + kTileRows - 1) / kTileRows;
@@ -237,26 +245,46 @@ adaspark_status_t adaspark_attn_get_layout(const adaspark_attn_t* h, adaspark_at
     return ADASPARK_OK;
 }
 
-adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const void* k, const void* v,
-                                        int32_t n_text, void* out, void* k_cube, void* v_cube, float* cube_keys,
-                                        uint32_t* sel_bitmap, int32_t* sel_count, void* workspace,
-                                        size_t workspace_bytes, void* cuda_stream) {
+}  // extern "C"
+
+namespace {
+
+// Prefill of the frames [frame_begin, frame_begin + frame_count) plus, when n_text >= 0 (the last call of a
+// sequence), n_text text tokens; n_text < 0: more video follows.  The one-shot forward is the window
+// [0, T) with its text.
+adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* q, const void* k, const void* v,
+                               int32_t frame_begin, int32_t frame_count, int32_t n_text_arg, void* out, void* k_cube,
+                               void* v_cube, float* cube_keys, uint32_t* sel_bitmap, int32_t* sel_count, void* workspace,
+                               size_t workspace_bytes, void* cuda_stream) {
     if (!h) return ADASPARK_ERR_INVALID_ARG;
-    if (!h->partitioned) return fail(h, ADASPARK_ERR_NOT_PARTITIONED, "forward: call adaspark_attn_partition first");
-    if (!k || !v || !k_cube || !v_cube || !cube_keys) return fail(h, ADASPARK_ERR_INVALID_ARG, "forward: NULL k/v/cache pointer");
-    if ((q == nullptr) != (out == nullptr)) return fail(h, ADASPARK_ERR_INVALID_ARG, "forward: q and out must both be given or both be NULL");
-    if (n_text < 0 || n_text > h->n_text_max) return fail(h, ADASPARK_ERR_INVALID_ARG, "forward: n_text %d outside [0, %d]", n_text, h->n_text_max);
+    if (!h->partitioned) return fail(h, ADASPARK_ERR_NOT_PARTITIONED, "%s: call adaspark_attn_partition first", who);
+    if (!k || !v || !k_cube || !v_cube || !cube_keys) return fail(h, ADASPARK_ERR_INVALID_ARG, "%s: NULL k/v/cache pointer", who);
+    if ((q == nullptr) != (out == nullptr)) return fail(h, ADASPARK_ERR_INVALID_ARG, "%s: q and out must both be given or both be NULL", who);
+    const bool last_call = n_text_arg >= 0;
+    const int n_text = last_call ? n_text_arg : 0;
+    if (n_text > h->n_text_max) return fail(h, ADASPARK_ERR_INVALID_ARG, "%s: n_text %d outside [0, %d]", who, n_text, h->n_text_max);
+    const int ct = h->cfg.cube_t;
+    if (frame_begin < 0 || frame_count < 0 || frame_begin % ct || frame_count % ct || frame_begin + frame_count > h->T)
+        return fail(h, ADASPARK_ERR_INVALID_ARG, "%s: frames [%d, %d) are not whole time blocks of %d frames inside [0, %d)", who,
+                    frame_begin, frame_begin + frame_count, ct, h->T);
+    if (last_call && frame_begin + frame_count != h->T)
+        return fail(h, ADASPARK_ERR_INVALID_ARG, "%s: the call that brings the text must end the video (frame %d of %d)", who,
+                    frame_begin + frame_count, h->T);
+    if (frame_count == 0 && n_text == 0) return fail(h, ADASPARK_ERR_INVALID_ARG, "%s: empty call", who);
+    if (((long long)frame_begin * h->H * h->W) % 256)
+        return fail(h, ADASPARK_ERR_UNSUPPORTED, "%s: a chunk must start at a multiple of 256 tokens (frame_begin * H * W = %lld)", who,
+                    (long long)frame_begin * h->H * h->W);
     const bool cache_only = (q == nullptr);
     if (!cache_only) {
-        if (!workspace) return fail(h, ADASPARK_ERR_INVALID_ARG, "forward: NULL workspace");
-        if (workspace_bytes < h->fw_total) return fail(h, ADASPARK_ERR_WORKSPACE_TOO_SMALL, "forward: workspace %zu < %zu bytes", workspace_bytes, h->fw_total);
-        if ((uintptr_t)workspace % kAlign) return fail(h, ADASPARK_ERR_INVALID_ARG, "forward: workspace not 256-byte aligned");
+        if (!workspace) return fail(h, ADASPARK_ERR_INVALID_ARG, "%s: NULL workspace", who);
+        if (workspace_bytes < h->fw_total) return fail(h, ADASPARK_ERR_WORKSPACE_TOO_SMALL, "%s: workspace %zu < %zu bytes", who, workspace_bytes, h->fw_total);
+        if ((uintptr_t)workspace % kAlign) return fail(h, ADASPARK_ERR_INVALID_ARG, "%s: workspace not 256-byte aligned", who);
     }
     cudaError_t ce = cudaSetDevice(h->cfg.device);
-    if (ce != cudaSuccess) return fail(h, ADASPARK_ERR_CUDA, "forward: cudaSetDevice(%d): %s", h->cfg.device, cudaGetErrorString(ce));
+    if (ce != cudaSuccess) return fail(h, ADASPARK_ERR_CUDA, "%s: cudaSetDevice(%d): %s", who, h->cfg.device, cudaGetErrorString(ce));
     cudaStream_t st = (cudaStream_t)cuda_stream;
     h->launches = 0;
-    const Geom g = make_geom(h, n_text);
+    const Geom g = make_geom(h, n_text, frame_begin, frame_begin + frame_count);
     const int D = g.D;
     auto* kb = (const __nv_bfloat16*)k;
     auto* vb = (const __nv_bfloat16*)v;
@@ -268,18 +296,22 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
     mark(h, 0, st);
     // K1: re-layout + pooling
     {
-        dim3 grid(g.n_kv_blocks_cap, g.Hkv, g.B);
+        // blocks of this call's rows; the last call of a sequence also zero-fills the cache up to its capacity
+        const int blk_begin = g.pos_begin / kBlockTok;
+        const int blk_end = last_call ? g.n_kv_blocks_cap : (g.S + kBlockTok - 1) / kBlockTok;
+        dim3 grid(blk_end - blk_begin, g.Hkv, g.B);
         if (D == 128) relayout_pool_kernel<128><<<grid, 256, 0, st>>>(g, kb, vb, kc, vc, cube_keys);
         else relayout_pool_kernel<64><<<grid, 256, 0, st>>>(g, kb, vb, kc, vc, cube_keys);
         if (!launch_ok(h, "relayout_pool_kernel")) return ADASPARK_ERR_CUDA;
-        if (g.C > kBlockTok) {
-            pool_large_cubes_kernel<<<dim3(g.N, g.Hkv, g.B), D, 0, st>>>(g, kc, cube_keys);
+        const int cube_begin = g.pos_begin >> g.c_shift;
+        if (g.C > kBlockTok && g.N_live > cube_begin) {
+            pool_large_cubes_kernel<<<dim3(g.N_live - cube_begin, g.Hkv, g.B), D, 0, st>>>(g, kc, cube_keys);
             if (!launch_ok(h, "pool_large_cubes_kernel")) return ADASPARK_ERR_CUDA;
         }
     }
 #ifdef ADASPARK_WITH_TCGEN05
     if (!cache_only && h->prefill_kernel != 0) {   // cube-major staging of Q for the TMA loads of K3 / K4
-        dim3 rgrid((g.S + 3) / 4, g.B);
+        dim3 rgrid((g.S_io + 3) / 4, g.B);
         __nv_bfloat16* q_cube = (__nv_bfloat16*)((char*)workspace + h->fw_qcube_off);
         if (D == 128) relayout_q_kernel<128><<<rgrid, 256, 0, st>>>(g, (const __nv_bfloat16*)q, q_cube);
         else relayout_q_kernel<64><<<rgrid, 256, 0, st>>>(g, (const __nv_bfloat16*)q, q_cube);
@@ -315,7 +347,7 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
             return launch_ok(h, "select_exact_kernel");
         };
         if (all) {
-            select_all_kernel<<<dim3(g.n_tiles, g.Hq, g.B), kTileRows, 0, st>>>(g, tile_mask, tile_union, sel_bitmap, sel_count);
+            select_all_kernel<<<dim3(g.n_tiles - g.tile_begin, g.Hq, g.B), kTileRows, 0, st>>>(g, tile_mask, tile_union, sel_bitmap, sel_count);
             if (!launch_ok(h, "select_all_kernel")) return ADASPARK_ERR_CUDA;
         }
 #ifdef ADASPARK_WITH_TCGEN05
@@ -329,8 +361,8 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
             if (!launch_ok(h, "slice_keys_kernel")) return ADASPARK_ERR_CUDA;
             CUtensorMap tmKs;
             if (!encode_u8_2d(&tmKs, kplanes, (uint64_t)4 * n_rows + 128, kDigitRowBytes, kDigitRowBytes, kScoreTcCols))
-                return fail(h, ADASPARK_ERR_CUDA, "forward: cuTensorMapEncodeTiled failed");
-            const int n_items = g.B * g.Hq * g.n_tiles;
+                return fail(h, ADASPARK_ERR_CUDA, "%s: cuTensorMapEncodeTiled failed", who);
+            const int n_items = g.B * g.Hq * (g.n_tiles - g.tile_begin);
             const int grid = n_items < h->sm_count ? n_items : h->sm_count;
             const __nv_bfloat16* q_cube_c = (const __nv_bfloat16*)(ws + h->fw_qcube_off);
             const bool by_count = g.top_k > 0;
@@ -365,24 +397,24 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
         if (!encode_bf16_2d(&tmQ, q_cube, (uint64_t)g.B * g.Hq * g.S_cap, D, 64, 128) ||
             !encode_bf16_2d(&tmK, kc, (uint64_t)g.B * g.Hkv * g.S_cap, D, 64, 64) ||
             !encode_bf16_2d(&tmV, vc, (uint64_t)g.B * g.Hkv * g.n_kv_blocks_cap * D, 64, 64, D))
-            return fail(h, ADASPARK_ERR_CUDA, "forward: cuTensorMapEncodeTiled failed");
-        dim3 grid(((g.S + kPairRows - 1) / kPairRows) * g.Hq * g.B);
+            return fail(h, ADASPARK_ERR_CUDA, "%s: cuTensorMapEncodeTiled failed", who);
+        dim3 grid(((g.S + kPairRows - 1) / kPairRows - g.pos_begin / kPairRows) * g.Hq * g.B);
         if (D == 128) {
             size_t smem = sizeof(TcAttnSmem<128>) + 1024;
             if (!set_smem(h, attn_prefill_tc_kernel<128>, smem, "attn_prefill_tc_kernel")) return ADASPARK_ERR_CUDA;
             attn_prefill_tc_kernel<128><<<grid, kTcThreads, smem, st>>>(g, tmQ, tmK, tmV, tile_mask, tile_union, (__nv_bfloat16*)out,
-                                                                        (unsigned long long*)&hdr->executed_kv_blocks, &hdr->status);
+                                                                        (unsigned long long*)&hdr->executed_kv_blocks, &hdr->max_tile_kv_blocks, &hdr->status);
         } else {
             size_t smem = sizeof(TcAttnSmem<64>) + 1024;
             if (!set_smem(h, attn_prefill_tc_kernel<64>, smem, "attn_prefill_tc_kernel")) return ADASPARK_ERR_CUDA;
             attn_prefill_tc_kernel<64><<<grid, kTcThreads, smem, st>>>(g, tmQ, tmK, tmV, tile_mask, tile_union, (__nv_bfloat16*)out,
-                                                                       (unsigned long long*)&hdr->executed_kv_blocks, &hdr->status);
+                                                                       (unsigned long long*)&hdr->executed_kv_blocks, &hdr->max_tile_kv_blocks, &hdr->status);
         }
         if (!launch_ok(h, "attn_prefill_tc_kernel")) return ADASPARK_ERR_CUDA;
     } else
 #endif
     {
-        dim3 grid(g.n_tiles, g.Hq, g.B);
+        dim3 grid(g.n_tiles - g.tile_begin, g.Hq, g.B);
         if (D == 128) {
             size_t smem = sizeof(MmaAttnSmem<128>);
             if (!set_smem(h, attn_prefill_mma_kernel<128>, smem, "attn_prefill_mma_kernel")) return ADASPARK_ERR_CUDA;
@@ -397,6 +429,29 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
     mark(h, 3, st);
     mark(h, 4, st);
     return ADASPARK_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const void* k, const void* v,
+                                        int32_t n_text, void* out, void* k_cube, void* v_cube, float* cube_keys,
+                                        uint32_t* sel_bitmap, int32_t* sel_count, void* workspace,
+                                        size_t workspace_bytes, void* cuda_stream) {
+    if (!h) return ADASPARK_ERR_INVALID_ARG;
+    if (n_text < 0) return fail(h, ADASPARK_ERR_INVALID_ARG, "forward: n_text %d outside [0, %d]", n_text, h->n_text_max);
+    return forward_impl(h, "forward", q, k, v, 0, h->partitioned ? h->T : 0, n_text, out, k_cube, v_cube, cube_keys, sel_bitmap,
+                        sel_count, workspace, workspace_bytes, cuda_stream);
+}
+
+adaspark_status_t adaspark_attn_forward_chunk(adaspark_attn_t* h, const void* q, const void* k, const void* v,
+                                              int32_t frame_begin, int32_t frame_count, int32_t n_text, void* out,
+                                              void* k_cube, void* v_cube, float* cube_keys, uint32_t* sel_bitmap,
+                                              int32_t* sel_count, void* workspace, size_t workspace_bytes,
+                                              void* cuda_stream) {
+    return forward_impl(h, "forward_chunk", q, k, v, frame_begin, frame_count, n_text < 0 ? -1 : n_text, out, k_cube, v_cube,
+                        cube_keys, sel_bitmap, sel_count, workspace, workspace_bytes, cuda_stream);
 }
 
 adaspark_status_t adaspark_attn_decode(adaspark_attn_t* h, const void* q_new, const void* k_new, const void* v_new,

@@ -48,7 +48,7 @@ __global__ void __launch_bounds__(256) attn_prefill_mma_kernel(Geom g, const __n
         int pos = tile_pos0 + row;
         uint4 val = make_uint4(0, 0, 0, 0);
         if (pos < g.S)
-            val = *reinterpret_cast<const uint4*>(q + ((size_t)(b * g.S + pos_to_raster(g, pos)) * g.Hq + h) * D + c * 8);
+            val = *reinterpret_cast<const uint4*>(q + (io_row(g, b, pos) * g.Hq + h) * D + c * 8);
         *reinterpret_cast<uint4*>(&sm.q[row][swz(row, c) * 8]) = val;
     }
     // ---- union of the rows' selection words
@@ -221,13 +221,13 @@ __global__ void __launch_bounds__(256) attn_prefill_mma_kernel(Geom g, const __n
     lB += __shfl_xor_sync(0xffffffffu, lB, 2);
     float invA = lA > 0.f ? 1.f / lA : 0.f, invB = lB > 0.f ? 1.f / lB : 0.f;
     if (posA < g.S) {
-        __nv_bfloat16* dst = out + ((size_t)(b * g.S + pos_to_raster(g, posA)) * g.Hq + h) * D + 2 * (lane & 3);
+        __nv_bfloat16* dst = out + (io_row(g, b, posA) * g.Hq + h) * D + 2 * (lane & 3);
 #pragma unroll
         for (int dt = 0; dt < kDTiles; ++dt)
             *reinterpret_cast<uint32_t*>(dst + dt * 8) = pack_bf16x2(o[dt][0] * invA, o[dt][1] * invA);
     }
     if (posB < g.S) {
-        __nv_bfloat16* dst = out + ((size_t)(b * g.S + pos_to_raster(g, posB)) * g.Hq + h) * D + 2 * (lane & 3);
+        __nv_bfloat16* dst = out + (io_row(g, b, posB) * g.Hq + h) * D + 2 * (lane & 3);
 #pragma unroll
         for (int dt = 0; dt < kDTiles; ++dt)
             *reinterpret_cast<uint32_t*>(dst + dt * 8) = pack_bf16x2(o[dt][2] * invB, o[dt][3] * invB);

@@ -62,7 +62,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     Geom g, const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
     const __grid_constant__ CUtensorMap tmV, const uint32_t* __restrict__ tile_mask,
     const uint32_t* __restrict__ tile_union, __nv_bfloat16* __restrict__ out,
-    unsigned long long* __restrict__ executed_blocks, int32_t* __restrict__ status) {
+    unsigned long long* __restrict__ executed_blocks, uint32_t* __restrict__ max_tile_blocks, int32_t* __restrict__ status) {
     extern __shared__ unsigned char tc_smem_raw[];
     TcAttnSmem<D>& sm = *reinterpret_cast<TcAttnSmem<D>*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~(uintptr_t)1023);
     constexpr int kPanels = D / 64;
@@ -457,7 +457,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
             tc::tc_fence_after_sync();
             const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
             const bool live = pr < g.S;
-            __nv_bfloat16* dst = out + ((size_t)(b * g.S + (live ? pos_to_raster(g, pr) : 0)) * g.Hq + h) * D;
+            __nv_bfloat16* dst = out + ((live ? io_row(g, b, pr) : 0) * g.Hq + h) * D;
             uint32_t o[D / 32][32];                                // the whole output row in one round of loads
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) tc::tmem_ld_32x32(lane_addr + 128 + c * 32, o[c]);
@@ -491,7 +491,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     __syncthreads();
     if (tid == 0) {
         if (sm.abort_flag) atomicExch(status, 6);   // a bounded wait expired
-        else atomicAdd(executed_blocks, (unsigned long long)(2 * n_needed));
+        else {
+            atomicAdd(executed_blocks, (unsigned long long)(2 * n_needed));
+            atomicMax(max_tile_blocks, (uint32_t)n_needed);
+        }
     }
     if (warp == 8) tc::tmem_dealloc<512>(tbase);
 }
@@ -502,7 +505,7 @@ template <int D>
 __global__ void __launch_bounds__(256) relayout_q_kernel(Geom g, const __nv_bfloat16* __restrict__ q,
                                                          __nv_bfloat16* __restrict__ q_cube) {
     constexpr int kChunks = D / 8;
-    const int pos0 = blockIdx.x * 4;                    // 4 positions x all heads per CTA: many small CTAs
+    const int pos0 = g.pos_begin + blockIdx.x * 4;      // 4 positions x all heads per CTA: many small CTAs
     const int b = blockIdx.y;
     const int per_pos = g.Hq * kChunks;
     for (int idx = threadIdx.x; idx < 4 * per_pos; idx += 256) {
@@ -510,7 +513,7 @@ __global__ void __launch_bounds__(256) relayout_q_kernel(Geom g, const __nv_bflo
         int h = rem / kChunks, c = rem - h * kChunks;
         int pos = pos0 + p;
         if (pos >= g.S) break;
-        uint4 val = *reinterpret_cast<const uint4*>(q + ((size_t)(b * g.S + pos_to_raster(g, pos)) * g.Hq + h) * D + c * 8);
+        uint4 val = *reinterpret_cast<const uint4*>(q + (io_row(g, b, pos) * g.Hq + h) * D + c * 8);
         *reinterpret_cast<uint4*>(q_cube + ((size_t)(b * g.Hq + h) * g.S_cap + pos) * D + c * 8) = val;
     }
 }

@@ -43,7 +43,13 @@ struct Geom {
     int c_shift;         // log2(C)
     int cw_shift, ch_shift;   // log2(cw), log2(ch): C is a power of two, so every window side is one
     FastDiv div_nW, div_nH, div_n_tiles, div_Hq;
-    int S_v, n_text, S;  // video tokens, text tokens of this call, total
+    int S_v, n_text, S;  // video tokens of the partition, text tokens so far, positions present after this call
+    // Row window of this call (chunked prefill): the q/k/v/out tensors hold the S_io tokens whose
+    // cube-major positions are [pos_begin, S) -- whole time blocks of cubes, so they are also the raster
+    // tokens pos_begin .. -- and only those rows are computed.  One-shot prefill: pos_begin = 0, S_io = S.
+    int pos_begin, S_io;
+    int N_live;          // cubes present after this call (<= N)
+    int tile_begin;      // pos_begin / 128
     int S_cap;           // cache rows per (b, kv head), multiple of 128
     int n_words;         // ceil(N/32)
     int n_tiles;         // ceil(S/128) query tiles of this call
@@ -69,6 +75,11 @@ __device__ __forceinline__ int pos_to_raster(const Geom& g, int pos) {
     const int ry = (r >> g.cw_shift) & (g.ch - 1);
     const int rt = r >> (g.cw_shift + g.ch_shift);
     return ((cb * g.ct + rt) * g.H + (cy * g.ch + ry)) * g.W + (cx * g.cw + rx);
+}
+
+// Row of the call's q/k/v/out tensors (batch b) that holds the token at cube-major position pos.
+__device__ __forceinline__ size_t io_row(const Geom& g, int b, int pos) {
+    return (size_t)b * g.S_io + (pos_to_raster(g, pos) - g.pos_begin);
 }
 
 // Number of candidate cubes of the row at `pos`: preceding cubes for video, all cubes for text.

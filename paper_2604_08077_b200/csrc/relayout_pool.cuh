@@ -24,7 +24,7 @@ __global__ void __launch_bounds__(256) relayout_pool_kernel(Geom g, const __nv_b
     __shared__ __align__(16) __nv_bfloat16 Ks[kBlockTok][D];
     __shared__ __align__(16) __nv_bfloat16 Vs[kBlockTok][kVPitch];
 
-    const int blk = blockIdx.x, gk = blockIdx.y, b = blockIdx.z;
+    const int blk = blockIdx.x + g.pos_begin / kBlockTok, gk = blockIdx.y, b = blockIdx.z;   // blocks of this call's row window
     const int pos0 = blk * kBlockTok;
     const int tid = threadIdx.x;
 
@@ -33,7 +33,7 @@ __global__ void __launch_bounds__(256) relayout_pool_kernel(Geom g, const __nv_b
         int pos = pos0 + row;
         uint4 kv4 = make_uint4(0, 0, 0, 0), vv4 = make_uint4(0, 0, 0, 0);
         if (pos < g.S) {
-            size_t src = ((size_t)(b * g.S + pos_to_raster(g, pos)) * g.Hkv + gk) * D + c * 8;
+            size_t src = (io_row(g, b, pos) * g.Hkv + gk) * D + c * 8;
             kv4 = *reinterpret_cast<const uint4*>(k + src);
             vv4 = *reinterpret_cast<const uint4*>(v + src);
         }
@@ -60,7 +60,7 @@ __global__ void __launch_bounds__(256) relayout_pool_kernel(Geom g, const __nv_b
         for (int idx = tid; idx < cubes_here * D; idx += 256) {
             int cb = idx / D, d = idx - cb * D;
             int cube = pos0 / g.C + cb;
-            if (cube < g.N) {
+            if (cube < g.N_live) {
                 double acc = 0.0;
                 for (int r = 0; r < g.C; ++r) acc += (double)__bfloat162float(Ks[cb * g.C + r][d]);
                 cube_keys[((size_t)(b * g.Hkv + gk) * g.N + cube) * D + d] = (float)(acc / (double)g.C);
@@ -73,7 +73,7 @@ __global__ void __launch_bounds__(256) relayout_pool_kernel(Geom g, const __nv_b
 // reading the cube-major keys just written by relayout_pool_kernel.
 __global__ void pool_large_cubes_kernel(Geom g, const __nv_bfloat16* __restrict__ k_cube,
                                         float* __restrict__ cube_keys) {
-    const int cube = blockIdx.x, gk = blockIdx.y, b = blockIdx.z, d = threadIdx.x;
+    const int cube = blockIdx.x + (g.pos_begin >> g.c_shift), gk = blockIdx.y, b = blockIdx.z, d = threadIdx.x;
     if (d >= g.D) return;
     const __nv_bfloat16* src = k_cube + ((size_t)(b * g.Hkv + gk) * g.S_cap + (size_t)cube * g.C) * g.D + d;
     double acc = 0.0;

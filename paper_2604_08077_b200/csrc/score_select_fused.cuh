@@ -94,7 +94,7 @@ __device__ __forceinline__ uint32_t gather_byte(uint32_t w0, uint32_t w1, uint32
 __global__ void __launch_bounds__(256) key_exponent_kernel(Geom g, const float* __restrict__ cube_keys,
                                                            uint32_t* __restrict__ head_max_bits) {
     const int bh = blockIdx.x;
-    const size_t n4 = (size_t)g.N * g.D / 4;
+    const size_t n4 = (size_t)g.N_live * g.D / 4;             // the cubes present so far
     const float4* src = reinterpret_cast<const float4*>(cube_keys + (size_t)bh * g.N * g.D);
     uint32_t mx = 0;
     for (size_t i = (size_t)blockIdx.y * 256 + threadIdx.x; i < n4; i += (size_t)gridDim.y * 256) {
@@ -119,7 +119,7 @@ __global__ void __launch_bounds__(128) slice_keys_kernel(Geom g, const float* __
     if (row >= n_rows) return;
     const int bh = row / g.N_ld, cube = row - bh * g.N_ld;
     const size_t plane_stride = (size_t)n_rows * kDigitRowBytes;
-    const bool live = cube < g.N && lane * 4 < g.D;
+    const bool live = cube < g.N_live && lane * 4 < g.D;
     float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
     if (live) x = *reinterpret_cast<const float4*>(cube_keys + ((size_t)bh * g.N + cube) * g.D + lane * 4);
     const float mult = digit_scale(head_exponent(head_max_bits[bh]));
@@ -455,7 +455,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
             const size_t gt_cap = (size_t)(w.b * g.Hq + w.h) * g.n_tiles_cap + w.tile;
             uint32_t* mask_row = tile_mask + gt_cap * g.n_words * kTileRows + r;        // word w at mask_row[w * 128]
             const bool extra = live && (sel_bitmap != nullptr || sel_count != nullptr);
-            const size_t raster_row = extra ? (size_t)(w.b * g.Hq + w.h) * g.S + pos_to_raster(g, pos) : 0;
+            const size_t raster_row = extra ? (size_t)(w.b * g.Hq + w.h) * g.S_io + (pos_to_raster(g, pos) - g.pos_begin) : 0;
             uint32_t* bm_row = (extra && sel_bitmap) ? sel_bitmap + raster_row * g.n_words : nullptr;
             // every word starts at zero: the collect pass ORs the selected cubes' bits into them
             for (int wd = part; wd < g.n_words; wd += 4) {
@@ -723,17 +723,17 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
     if (warp == kProducerWarp) tc::tmem_dealloc<512>(tbase);
 }
 
-// p >= 1 without Top-K: every candidate cube is selected (Eq. 2 with p = 1).  grid (n_tiles, Hq, B),
+// p >= 1 without Top-K: every candidate cube is selected (Eq. 2 with p = 1).  grid (tiles of the call, Hq, B),
 // 128 threads = rows of the tile.
 __global__ void __launch_bounds__(128) select_all_kernel(Geom g, uint32_t* __restrict__ tile_mask,
                                                          uint32_t* __restrict__ tile_union, uint32_t* __restrict__ sel_bitmap,
                                                          int32_t* __restrict__ sel_count) {
-    const int tile = blockIdx.x, h = blockIdx.y, b = blockIdx.z, r = threadIdx.x;
+    const int tile = blockIdx.x + g.tile_begin, h = blockIdx.y, b = blockIdx.z, r = threadIdx.x;
     const int pos = tile * kTileRows + r;
     const bool live = pos < g.S;
     const int n = live ? n_candidates(g, pos) : 0;
     const size_t gt_cap = (size_t)(b * g.Hq + h) * g.n_tiles_cap + tile;
-    const size_t raster_row = live ? (size_t)(b * g.Hq + h) * g.S + pos_to_raster(g, pos) : 0;
+    const size_t raster_row = live ? (size_t)(b * g.Hq + h) * g.S_io + (pos_to_raster(g, pos) - g.pos_begin) : 0;
     const int n_max = n_candidates(g, min(tile * kTileRows + kTileRows, g.S) - 1);
     for (int w = 0; w < g.n_words; ++w) {
         const int rem = n - w * 32;

@@ -41,18 +41,18 @@ __global__ void __launch_bounds__(kExactWarps * 32) select_exact_kernel(
         const int r = (int)(id & (kTileRows - 1));
         const int gt_cap = (int)(id >> 7);
         const int bh = gt_cap / g.n_tiles_cap, tile = gt_cap - bh * g.n_tiles_cap;
-        if (tile >= g.n_tiles) continue;
+        if (tile >= g.n_tiles || tile < g.tile_begin) continue;
         int b, h;
         g.div_Hq.divmod(bh, b, h);
         const int gk = h / g.G;
         const int pos = tile * kTileRows + r;
         const bool live = pos < g.S;
         const int n = live ? n_candidates(g, pos) : 0;
-        const int raster = live ? pos_to_raster(g, pos) : 0;
+        const int raster = live ? pos_to_raster(g, pos) - g.pos_begin : 0;   // row of the call's tensors
         unsigned long long bd = 0ull;                    // 0: every candidate is selected
         if (!all && n > 0) {
             // ---- scores: s[j] = scale * <q, kbar_j> in fp64
-            const __nv_bfloat16* qsrc = q + ((size_t)(b * g.S + raster) * g.Hq + h) * D;
+            const __nv_bfloat16* qsrc = q + (((size_t)b * g.S_io + raster) * g.Hq + h) * D;
             for (int d = lane; d < D; d += 32) qd[d] = (double)__bfloat162float(qsrc[d]);
             __syncwarp();
             const float* kbase = cube_keys + (size_t)(b * g.Hkv + gk) * g.N * D;
@@ -83,10 +83,10 @@ __global__ void __launch_bounds__(kExactWarps * 32) select_exact_kernel(
             if (lane == 0) {
                 tile_mask[mask_index(g, b, h, tile, w, r)] = word;
                 if (word) atomicOr(tile_union + (size_t)gt_cap * g.n_words + w, word);
-                if (sel_bitmap && extra) sel_bitmap[((size_t)(b * g.Hq + h) * g.S + raster) * g.n_words + w] = word;
+                if (sel_bitmap && extra) sel_bitmap[((size_t)(b * g.Hq + h) * g.S_io + raster) * g.n_words + w] = word;
             }
         }
-        if (sel_count && lane == 0 && extra) sel_count[(size_t)(b * g.Hq + h) * g.S + raster] = count;
+        if (sel_count && lane == 0 && extra) sel_count[(size_t)(b * g.Hq + h) * g.S_io + raster] = count;
         __syncwarp();
     }
 }

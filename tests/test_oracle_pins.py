@@ -394,3 +394,23 @@ def test_top_k_rows_use_the_rule_inside_the_full_path():
     assert np.array_equal(res["count"], np.minimum(n_cand, 3))
     out2 = oracle.attend_given(sh, wl.q, wl.k, wl.v, rows, res["sel"])
     np.testing.assert_allclose(res["out"], out2, rtol=0, atol=1e-15)
+
+
+def test_chunked_prefill_rows_equal_one_shot_rows():
+    """A later chunk never changes an earlier row (Eq. 1: a video query sees only preceding cubes; the
+    text follows the video): evaluating the rows of frames [0, T') on the truncated problem gives the
+    same selection, bit for bit, and the same outputs as evaluating them on the whole sequence."""
+    from paper_2604_08077_b200 import inputs
+    wl = inputs.small_prefill(seed=93, T=16, H=8, W=8, n_text=9, Hq=2, Hkv=1, D=64, top_p=0.8)
+    full = oracle.shape_of(wl)
+    for t_cut in (4, 12):
+        s_cut = t_cut * wl.H * wl.W
+        part = oracle.make_shape(B=wl.B, T=t_cut, H=wl.H, W=wl.W, cube=wl.cube, n_text=0, Hq=wl.Hq, Hkv=wl.Hkv,
+                                 D=wl.D, top_p=wl.top_p)
+        rows = [(0, h, n) for h in range(wl.Hq) for n in range(0, s_cut, 7)]
+        a = oracle.rows(full, wl.q, wl.k, wl.v, rows)
+        b = oracle.rows(part, wl.q[:, :s_cut], wl.k[:, :s_cut], wl.v[:, :s_cut], rows)
+        n_part = part.N
+        assert np.array_equal(a["sel"][:, :n_part], b["sel"]) and not a["sel"][:, n_part:].any()
+        assert np.array_equal(a["count"], b["count"])
+        np.testing.assert_allclose(a["out"], b["out"], rtol=0, atol=1e-12)
