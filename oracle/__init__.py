@@ -28,11 +28,11 @@ class Shape(ctypes.Structure):
                 ("W", ctypes.c_int32), ("ct", ctypes.c_int32), ("ch", ctypes.c_int32),
                 ("cw", ctypes.c_int32), ("n_text", ctypes.c_int32), ("Hq", ctypes.c_int32),
                 ("Hkv", ctypes.c_int32), ("D", ctypes.c_int32), ("top_p", ctypes.c_double),
-                ("scale", ctypes.c_double), ("top_k", ctypes.c_int32)]
+                ("scale", ctypes.c_double), ("top_k", ctypes.c_int32), ("n_prefix", ctypes.c_int32)]
 
     @property
     def N(self) -> int:
-        return (self.T // self.ct) * (self.H // self.ch) * (self.W // self.cw)
+        return (-(-self.T // self.ct)) * (-(-self.H // self.ch)) * (-(-self.W // self.cw))
 
     @property
     def C(self) -> int:
@@ -44,7 +44,13 @@ class Shape(ctypes.Structure):
 
     @property
     def S(self) -> int:
-        return self.S_v + self.n_text
+        return self.n_prefix + self.S_v + self.n_text
+
+    @property
+    def n_positions(self) -> int:
+        """Slots of the causal order: prefix, N cubes of C slots (boundary cubes of a grid the window
+        does not divide hold fewer tokens than slots), text."""
+        return self.n_prefix + self.N * self.C + self.n_text
 
 
 def build(force: bool = False) -> str:
@@ -60,6 +66,7 @@ def lib() -> ctypes.CDLL:
     if _lib is None:
         _lib = ctypes.CDLL(build())
         _lib.adas_oracle_num_cubes.restype = ctypes.c_int64
+        _lib.adas_oracle_num_positions.restype = ctypes.c_int64
         _lib.adas_oracle_position.restype = ctypes.c_int64
         _lib.adas_oracle_position.argtypes = [ctypes.POINTER(Shape), ctypes.c_int64]
         _lib.adas_oracle_select_row.restype = ctypes.c_int64
@@ -76,17 +83,18 @@ def n_threads() -> int:
 
 
 def make_shape(*, B, T, H, W, cube, n_text, Hq, Hkv, D, top_p, scale: Optional[float] = None,
-               top_k: int = 0) -> Shape:
+               top_k: int = 0, n_prefix: int = 0) -> Shape:
     ct, ch, cw = cube
     return Shape(B, T, H, W, ct, ch, cw, n_text, Hq, Hkv, D, float(top_p),
-                 float(scale) if scale else 1.0 / float(np.sqrt(D)), int(top_k))
+                 float(scale) if scale else 1.0 / float(np.sqrt(D)), int(top_k), int(n_prefix))
 
 
 def shape_of(wl, top_p: Optional[float] = None, top_k: Optional[int] = None) -> Shape:
     """Shape of a ``paper_2604_08077_b200.inputs.Workload`` (duck-typed; no import)."""
     return make_shape(B=wl.B, T=wl.T, H=wl.H, W=wl.W, cube=wl.cube, n_text=wl.n_text, Hq=wl.Hq,
                       Hkv=wl.Hkv, D=wl.D, top_p=wl.top_p if top_p is None else top_p,
-                      top_k=getattr(wl, "top_k", 0) if top_k is None else top_k)
+                      top_k=getattr(wl, "top_k", 0) if top_k is None else top_k,
+                      n_prefix=getattr(wl, "n_prefix", 0))
 
 
 def as_f32(t) -> np.ndarray:
@@ -101,10 +109,10 @@ def _p(a: Optional[np.ndarray]):
 
 
 def positions(shape: Shape):
-    """(pos_of_raster, raster_of_pos): the cube-major permutation and its inverse (O1)."""
-    S = shape.S
-    pos = np.empty(S, np.int64)
-    inv = np.empty(S, np.int64)
+    """(pos_of_raster [S], raster_of_pos [n_positions], -1 where a slot holds no token): the order
+    of the tokens and its inverse (O1)."""
+    pos = np.empty(shape.S, np.int64)
+    inv = np.empty(shape.n_positions, np.int64)
     lib().adas_oracle_positions(ctypes.byref(shape), _p(pos), _p(inv))
     return pos, inv
 
@@ -191,7 +199,7 @@ def decode(shape: Shape, k_cache, v_cache, text_len: Sequence[int], q_new, k_new
     for b in idx:
         tl = int(text_len[b])
         s1 = Shape(1, shape.T, shape.H, shape.W, shape.ct, shape.ch, shape.cw, tl + 1, shape.Hq,
-                   shape.Hkv, shape.D, shape.top_p, shape.scale, shape.top_k)
+                   shape.Hkv, shape.D, shape.top_p, shape.scale, shape.top_k, 0)
         Sv = shape.S_v
         k1 = np.concatenate([k_cache[b, :Sv + tl], k_new[b]], axis=0)[None]
         v1 = np.concatenate([v_cache[b, :Sv + tl], v_new[b]], axis=0)[None]

@@ -24,7 +24,13 @@
  *     ascending) whose cumulative probability is >= p; p >= 1 selects every candidate;
  *   - the own cube is never a candidate; text queries see every video cube as a candidate;
  *   - with grouped-query attention the mean keys are per KV head, the selection per query
- *     head (kv head = query head / group size).
+ *     head (kv head = query head / group size);
+ *   - a video grid that the cube window does not divide is covered by ceil(T/ct) x ceil(H/ch) x
+ *     ceil(W/cw) cubes; the cubes at the far faces hold fewer tokens, their mean key is the mean
+ *     over the tokens they do hold, and only those tokens are attended when the cube is selected;
+ *   - text placed BEFORE the video (a prompt prefix; n_prefix tokens) is attended by every later
+ *     token always and in full, like the own cube: it is never a candidate of Eq. 1 and its
+ *     mass does not count toward p; prefix tokens themselves attend causally among themselves.
  *
  * Pins (tests/test_oracle_*.py): closed-form permutation examples, numpy reshape-mean,
  * brute force over all cube subsets, p -> 0 argmax, p = 1 equals an independently written
@@ -33,7 +39,12 @@
  * values are pinned only through those identities.
  *
  * All tensors are raster order, row-major:  Q [B,S,Hq,D], K,V [B,S,Hkv,D] as float (the
- * bf16-rounded inputs widened exactly), S = T*H*W + n_text, text after video.
+ * bf16-rounded inputs widened exactly), S = n_prefix + T*H*W + n_text: prefix text, video
+ * tokens (t, y, x) row-major, text.
+ *
+ * "Position" below is the place of a token in the causal order: prefix token u at u, the video
+ * token of cube c with in-window rank r at n_prefix + c*C + r (slots of a boundary cube that
+ * fall outside the grid hold no token), text token u at n_prefix + N*C + u.
  */
 #include <math.h>
 #include <stdint.h>
@@ -48,31 +59,41 @@ typedef struct {
     double top_p;            /* nucleus mass p                                        */
     double scale;            /* logit scale, 1/sqrt(D) in the paper                   */
     int32_t top_k;           /* > 0: keep the K most probable cubes instead of Top-p  */
+    int32_t n_prefix;        /* text tokens before the video                          */
 } adas_shape;
 
+static int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 static int64_t n_cubes(const adas_shape *s) {
-    return (int64_t)(s->T / s->ct) * (s->H / s->ch) * (s->W / s->cw);
+    return ceil_div(s->T, s->ct) * ceil_div(s->H, s->ch) * ceil_div(s->W, s->cw);
 }
 static int64_t cube_tokens(const adas_shape *s) { return (int64_t)s->ct * s->ch * s->cw; }
 static int64_t video_tokens(const adas_shape *s) { return (int64_t)s->T * s->H * s->W; }
-static int64_t seq_len(const adas_shape *s) { return video_tokens(s) + s->n_text; }
+static int64_t seq_len(const adas_shape *s) { return s->n_prefix + video_tokens(s) + s->n_text; }
+/* number of positions (slots of the causal order, including the empty slots of boundary cubes) */
+static int64_t n_positions(const adas_shape *s) { return s->n_prefix + n_cubes(s) * cube_tokens(s) + s->n_text; }
+int64_t adas_oracle_num_positions(const adas_shape *s) { return n_positions(s); }
 
 int64_t adas_oracle_num_cubes(const adas_shape *s) { return n_cubes(s); }
 
-/* O1 (Sec. 3.1): raster index n = (t*H + y)*W + x of a video token -> cube-major position
- * c*C + r; a text token u keeps position S_v + u. */
+/* O1 (Sec. 3.1): token n of the sequence -> its position.  Video token (t, y, x), raster index
+ * (t*H + y)*W + x after the prefix, lies in cube ((t/ct)*nH + y/ch)*nW + x/cw with rank
+ * ((t%ct)*ch + y%ch)*cw + x%cw. */
 int64_t adas_oracle_position(const adas_shape *s, int64_t n) {
     int64_t Sv = video_tokens(s);
-    if (n >= Sv) return n;
+    if (n < s->n_prefix) return n;
+    n -= s->n_prefix;
+    if (n >= Sv) return s->n_prefix + n_cubes(s) * cube_tokens(s) + (n - Sv);
     int64_t x = n % s->W, y = (n / s->W) % s->H, t = n / ((int64_t)s->W * s->H);
-    int64_t cube = ((t / s->ct) * (s->H / s->ch) + y / s->ch) * (s->W / s->cw) + x / s->cw;
+    int64_t cube = ((t / s->ct) * ceil_div(s->H, s->ch) + y / s->ch) * ceil_div(s->W, s->cw) + x / s->cw;
     int64_t rank = ((t % s->ct) * s->ch + y % s->ch) * s->cw + x % s->cw;
-    return cube * cube_tokens(s) + rank;
+    return s->n_prefix + cube * cube_tokens(s) + rank;
 }
 
-/* pos_of_raster[n] and its inverse raster_of_pos[pos], both length S. */
+/* pos_of_raster[n] (length S) and its inverse raster_of_pos[pos] (length adas_oracle_num_positions,
+ * -1 at the slots that hold no token). */
 void adas_oracle_positions(const adas_shape *s, int64_t *pos_of_raster, int64_t *raster_of_pos) {
-    int64_t S = seq_len(s);
+    int64_t S = seq_len(s), P = n_positions(s);
+    for (int64_t p = 0; p < P; ++p) raster_of_pos[p] = -1;
     for (int64_t n = 0; n < S; ++n) {
         int64_t pos = adas_oracle_position(s, n);
         pos_of_raster[n] = pos;
@@ -80,21 +101,27 @@ void adas_oracle_positions(const adas_shape *s, int64_t *pos_of_raster, int64_t 
     }
 }
 
-/* O2: kbar[b][g][c][:] = (1/C) * sum of the C keys of cube c (KV head g).  kbar: [B,Hkv,N,D]. */
+/* O2: kbar[b][g][c][:] = mean of the keys of the tokens of cube c (KV head g): C of them, fewer in
+ * a boundary cube of a grid the window does not divide.  kbar: [B,Hkv,N,D]. */
 void adas_oracle_mean_keys(const adas_shape *s, const float *K, double *kbar) {
     int64_t S = seq_len(s), Sv = video_tokens(s), N = n_cubes(s), C = cube_tokens(s);
     int64_t D = s->D, Hkv = s->Hkv;
+    int64_t *held = (int64_t *)calloc((size_t)N, sizeof(int64_t));
     memset(kbar, 0, sizeof(double) * (size_t)(s->B * Hkv * N * D));
+    for (int64_t n = 0; n < Sv; ++n) held[(adas_oracle_position(s, s->n_prefix + n) - s->n_prefix) / C] += 1;
     for (int64_t b = 0; b < s->B; ++b)
         for (int64_t n = 0; n < Sv; ++n) {
-            int64_t c = adas_oracle_position(s, n) / C;
+            int64_t c = (adas_oracle_position(s, s->n_prefix + n) - s->n_prefix) / C;
             for (int64_t g = 0; g < Hkv; ++g) {
-                const float *k = K + ((b * S + n) * Hkv + g) * D;
+                const float *k = K + ((b * S + s->n_prefix + n) * Hkv + g) * D;
                 double *m = kbar + ((b * Hkv + g) * N + c) * D;
                 for (int64_t d = 0; d < D; ++d) m[d] += (double)k[d];
             }
         }
-    for (int64_t i = 0; i < s->B * Hkv * N * D; ++i) kbar[i] /= (double)C;
+    for (int64_t b = 0; b < s->B * Hkv; ++b)
+        for (int64_t c = 0; c < N; ++c)
+            for (int64_t d = 0; d < D; ++d) kbar[(b * N + c) * D + d] /= (double)held[c];
+    free(held);
 }
 
 typedef struct { double p; int64_t j; } prob_idx;
@@ -171,25 +198,30 @@ int64_t adas_oracle_select_row(const float *q, const double *kbar_g, int64_t n_c
     return kstar;
 }
 
-/* O5 for one row whose selection is known.  Key set A = all tokens of every selected cube,
- * plus (video) the own-cube tokens at cube-major positions <= the query's, or (text) the
- * text tokens <= the query's.  One softmax over A (Eq. 3), output [D] in fp64. */
-static void attend_row(const adas_shape *s, const float *Q, const float *K, const float *V,
-                       const int64_t *raster_of_pos, int64_t b, int64_t h, int64_t n_raster,
-                       int64_t pos, const uint8_t *sel, int64_t n_cand, double *out) {
-    int64_t S = seq_len(s), Sv = video_tokens(s), C = cube_tokens(s), D = s->D;
+/* O5 for one row whose selection is known.  Key set A = every prefix token (a prefix row: those
+ * up to itself), all tokens of every selected cube, plus (video) the own-cube tokens at positions
+ * <= the query's, or (text) the text tokens <= the query's.  One softmax over A (Eq. 3), output
+ * [D] in fp64.  Returns |A|. */
+static int64_t attend_row(const adas_shape *s, const float *Q, const float *K, const float *V,
+                          const int64_t *raster_of_pos, int64_t b, int64_t h, int64_t n_raster,
+                          int64_t pos, const uint8_t *sel, int64_t n_cand, double *out) {
+    int64_t S = seq_len(s), N = n_cubes(s), C = cube_tokens(s), D = s->D, P0 = s->n_prefix;
+    int64_t vid_end = P0 + N * C;                       /* first text position */
     int64_t g = h / (s->Hq / s->Hkv);
     const float *q = Q + ((b * S + n_raster) * s->Hq + h) * D;
-    /* gather the cube-major positions of A */
-    int64_t cap = n_cand * C + (pos < Sv ? C : s->n_text) + 1, na = 0;
+    /* gather the positions of A (slots without a token are skipped) */
+    int64_t cap = P0 + n_cand * C + C + s->n_text + 1, na = 0;
     int64_t *att = (int64_t *)malloc(sizeof(int64_t) * (size_t)cap);
+    for (int64_t pp = 0; pp < P0 && pp <= pos; ++pp) att[na++] = pp;
     for (int64_t j = 0; j < n_cand; ++j)
         if (sel[j])
-            for (int64_t r = 0; r < C; ++r) att[na++] = j * C + r;
-    if (pos < Sv) {
-        for (int64_t pp = (pos / C) * C; pp <= pos; ++pp) att[na++] = pp;
-    } else {
-        for (int64_t pp = Sv; pp <= pos; ++pp) att[na++] = pp;
+            for (int64_t r = 0; r < C; ++r)
+                if (raster_of_pos[P0 + j * C + r] >= 0) att[na++] = P0 + j * C + r;
+    if (pos >= P0 && pos < vid_end) {
+        for (int64_t pp = P0 + ((pos - P0) / C) * C; pp <= pos; ++pp)
+            if (raster_of_pos[pp] >= 0) att[na++] = pp;
+    } else if (pos >= vid_end) {
+        for (int64_t pp = vid_end; pp <= pos; ++pp) att[na++] = pp;
     }
     double *w = (double *)malloc(sizeof(double) * (size_t)na);
     double mx = -INFINITY;
@@ -210,6 +242,16 @@ static void attend_row(const adas_shape *s, const float *Q, const float *K, cons
     }
     free(w);
     free(att);
+    return na;
+}
+
+/* candidate cubes of the row at `pos`: none for a prefix token, the preceding cubes for a video
+ * token, every cube for a text token */
+static int64_t candidates_of(const adas_shape *s, int64_t pos) {
+    int64_t N = n_cubes(s), C = cube_tokens(s);
+    if (pos < s->n_prefix) return 0;
+    if (pos < s->n_prefix + N * C) return (pos - s->n_prefix) / C;
+    return N;
 }
 
 /* Evaluate a list of rows.  rows[3*i + {0,1,2}] = (batch b, query head h, raster token n).
@@ -223,16 +265,16 @@ static void attend_row(const adas_shape *s, const float *Q, const float *K, cons
 void adas_oracle_rows(const adas_shape *s, const float *Q, const float *K, const float *V,
                       const double *kbar, int64_t nrows, const int64_t *rows, double *out,
                       uint8_t *sel, int32_t *count, double *margin, int64_t *n_attended) {
-    int64_t S = seq_len(s), Sv = video_tokens(s), N = n_cubes(s), C = cube_tokens(s), D = s->D;
+    int64_t S = seq_len(s), N = n_cubes(s), D = s->D;
     int64_t *pos_of_raster = (int64_t *)malloc(sizeof(int64_t) * (size_t)S);
-    int64_t *raster_of_pos = (int64_t *)malloc(sizeof(int64_t) * (size_t)S);
+    int64_t *raster_of_pos = (int64_t *)malloc(sizeof(int64_t) * (size_t)n_positions(s));
     adas_oracle_positions(s, pos_of_raster, raster_of_pos);
     int64_t G = s->Hq / s->Hkv;
 #pragma omp parallel for schedule(dynamic, 16)
     for (int64_t i = 0; i < nrows; ++i) {
         int64_t b = rows[3 * i], h = rows[3 * i + 1], n = rows[3 * i + 2];
         int64_t pos = pos_of_raster[n];
-        int64_t n_cand = pos < Sv ? pos / C : N;   /* preceding cubes; text sees all cubes */
+        int64_t n_cand = candidates_of(s, pos);
         const float *q = Q + ((b * S + n) * s->Hq + h) * D;
         const double *kbar_g = kbar + ((b * s->Hkv + h / G) * N) * D;
         uint8_t *sel_i = sel + i * N;
@@ -240,9 +282,23 @@ void adas_oracle_rows(const adas_shape *s, const float *Q, const float *K, const
         int64_t cnt = adas_oracle_select_row(q, kbar_g, n_cand, D, s->scale, s->top_p, s->top_k, sel_i,
                                              NULL, margin ? margin + i : NULL);
         count[i] = (int32_t)cnt;
-        if (n_attended)
-            n_attended[i] = cnt * C + (pos < Sv ? pos - (pos / C) * C + 1 : pos - Sv + 1);
-        if (out) attend_row(s, Q, K, V, raster_of_pos, b, h, n, pos, sel_i, n_cand, out + i * D);
+        int64_t na = -1;
+        if (out) na = attend_row(s, Q, K, V, raster_of_pos, b, h, n, pos, sel_i, n_cand, out + i * D);
+        if (n_attended) {
+            if (na < 0) {       /* selection only: count the attended tokens without attending */
+                int64_t P0 = s->n_prefix, C = cube_tokens(s), vid_end = P0 + N * C;
+                na = pos < P0 ? pos + 1 : P0;
+                for (int64_t j = 0; j < n_cand; ++j)
+                    if (sel_i[j])
+                        for (int64_t r = 0; r < C; ++r) na += raster_of_pos[P0 + j * C + r] >= 0;
+                if (pos >= P0 && pos < vid_end) {
+                    for (int64_t pp = P0 + ((pos - P0) / C) * C; pp <= pos; ++pp) na += raster_of_pos[pp] >= 0;
+                } else if (pos >= vid_end) {
+                    na += pos - vid_end + 1;
+                }
+            }
+            n_attended[i] = na;
+        }
     }
     free(pos_of_raster);
     free(raster_of_pos);
@@ -252,16 +308,15 @@ void adas_oracle_rows(const adas_shape *s, const float *Q, const float *K, const
  * (used by tests that plant a selection, e.g. "all cubes" for the dense identity). */
 void adas_oracle_attend_given(const adas_shape *s, const float *Q, const float *K, const float *V,
                               int64_t nrows, const int64_t *rows, const uint8_t *sel, double *out) {
-    int64_t S = seq_len(s), Sv = video_tokens(s), N = n_cubes(s), C = cube_tokens(s), D = s->D;
+    int64_t S = seq_len(s), N = n_cubes(s), D = s->D;
     int64_t *pos_of_raster = (int64_t *)malloc(sizeof(int64_t) * (size_t)S);
-    int64_t *raster_of_pos = (int64_t *)malloc(sizeof(int64_t) * (size_t)S);
+    int64_t *raster_of_pos = (int64_t *)malloc(sizeof(int64_t) * (size_t)n_positions(s));
     adas_oracle_positions(s, pos_of_raster, raster_of_pos);
 #pragma omp parallel for schedule(dynamic, 16)
     for (int64_t i = 0; i < nrows; ++i) {
         int64_t b = rows[3 * i], h = rows[3 * i + 1], n = rows[3 * i + 2];
         int64_t pos = pos_of_raster[n];
-        int64_t n_cand = pos < Sv ? pos / C : N;
-        attend_row(s, Q, K, V, raster_of_pos, b, h, n, pos, sel + i * N, n_cand, out + i * D);
+        attend_row(s, Q, K, V, raster_of_pos, b, h, n, pos, sel + i * N, candidates_of(s, pos), out + i * D);
     }
     free(pos_of_raster);
     free(raster_of_pos);

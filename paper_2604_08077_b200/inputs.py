@@ -11,9 +11,10 @@ bf16 exactly once.  The CUDA path consumes the bf16 bytes; the oracle consumes t
 values widened to fp32/fp64, so both sides see identical real numbers.
 
 Layout of every returned tensor: raster order ``[B, S, heads, D]`` with
-``S = T*H*W + n_text``; video token ``(t, y, x)`` sits at ``s = (t*H + y)*W + x`` and the text
-tokens follow the video tokens (Sec. 3.1 / Algorithm 1 of the paper: video cubes first, text
-after them).
+``S = n_prefix + T*H*W + n_text``; video token ``(t, y, x)`` sits at ``s = n_prefix + (t*H + y)*W + x``
+and the text tokens follow the video tokens (Sec. 3.1 / Algorithm 1 of the paper: video cubes
+first, text after them); ``n_prefix`` (0 in the benchmark configurations) text tokens may precede
+the video, as a prompt does.  The grid need not be a multiple of the cube window.
 """
 from __future__ import annotations
 
@@ -39,6 +40,7 @@ class Workload:
     D: int
     top_p: float
     top_k: int = 0  # > 0: Top-K selection instead of Top-p
+    n_prefix: int = 0  # text tokens before the video
     q: Optional[torch.Tensor] = None  # bf16 [B, S, Hq, D]   (None for cache-only workloads)
     k: Optional[torch.Tensor] = None  # bf16 [B, S, Hkv, D]
     v: Optional[torch.Tensor] = None  # bf16 [B, S, Hkv, D]
@@ -54,7 +56,7 @@ class Workload:
 
     @property
     def S(self) -> int:
-        return self.S_v + self.n_text
+        return self.n_prefix + self.S_v + self.n_text
 
     @property
     def C(self) -> int:
@@ -63,7 +65,7 @@ class Workload:
     @property
     def N(self) -> int:
         ct, ch, cw = self.cube
-        return (self.T // ct) * (self.H // ch) * (self.W // cw)
+        return (-(-self.T // ct)) * (-(-self.H // ch)) * (-(-self.W // cw))
 
 
 def _gen(seed: int, device: str = "cpu") -> torch.Generator:
@@ -89,15 +91,20 @@ def _add_cube_offsets(k_video: torch.Tensor, g: torch.Generator, T: int, H: int,
     """
     ct, ch, cw = cube
     B, _, Hkv, D = k_video.shape
-    view = k_video.view(B, T // ct, ct, H // ch, ch, W // cw, cw, Hkv, D)
-    off = _randn(g, B, T // ct, 1, H // ch, 1, W // cw, 1, Hkv, D, std=std)
-    view.add_(off)
+    nT, nH, nW = -(-T // ct), -(-H // ch), -(-W // cw)         # windows along each axis (the last may be cut)
+    off = _randn(g, B, nT, 1, nH, 1, nW, 1, Hkv, D, std=std)
+    if (nT * ct, nH * ch, nW * cw) == (T, H, W):
+        k_video.view(B, nT, ct, nH, ch, nW, cw, Hkv, D).add_(off)
+    else:   # broadcast over whole windows, then keep the part of the grid that exists
+        full = off.expand(B, nT, ct, nH, ch, nW, cw, Hkv, D).reshape(B, nT * ct, nH * ch, nW * cw, Hkv, D)
+        k_video.view(B, T, H, W, Hkv, D).add_(full[:, :T, :H, :W])
 
 
 def make_prefill(name: str, *, seed: int, B: int, T: int, H: int, W: int,
                  cube: Tuple[int, int, int], n_text: int, Hq: int, Hkv: int, D: int,
                  top_p: float, offset_std: float, with_q: bool = True,
-                 device: str = "cpu", q_offset_std: float = 0.0, q_noise_std: float = 1.0) -> Workload:
+                 device: str = "cpu", q_offset_std: float = 0.0, q_noise_std: float = 1.0,
+                 n_prefix: int = 0) -> Workload:
     """i.i.d. N(0,1) Q/K/V; video K gets a per-cube shared offset of std ``offset_std``.
 
     ``q_offset_std`` > 0 additionally gives the video queries of one cube a shared offset (per query
@@ -118,9 +125,15 @@ def make_prefill(name: str, *, seed: int, B: int, T: int, H: int, W: int,
             if q_noise_std != 1.0:
                 q[:, :S_v].mul_(q_noise_std)
             _add_cube_offsets(q[:, :S_v], g, T, H, W, cube, q_offset_std)
+    if n_prefix > 0:   # drawn last, so that the video and text part equals the workload without a prefix
+        k = torch.cat([_randn(g, B, n_prefix, Hkv, D), k], dim=1)
+        v = torch.cat([_randn(g, B, n_prefix, Hkv, D), v], dim=1)
+        if with_q:
+            q = torch.cat([_randn(g, B, n_prefix, Hq, D), q], dim=1)
+    if with_q:
         q = q.to(torch.bfloat16)
     return Workload(name=name, B=B, T=T, H=H, W=W, cube=cube, n_text=n_text, Hq=Hq, Hkv=Hkv,
-                    D=D, top_p=top_p, q=q, k=k.to(torch.bfloat16), v=v.to(torch.bfloat16),
+                    D=D, top_p=top_p, n_prefix=n_prefix, q=q, k=k.to(torch.bfloat16), v=v.to(torch.bfloat16),
                     meta={"seed": seed, "offset_std": offset_std, "q_offset_std": q_offset_std})
 
 
@@ -230,10 +243,10 @@ def config5(variant: int = 0, B: int = 16, device: str = "cpu") -> Workload:
 def small_prefill(seed: int = 7, *, B: int = 1, T: int = 8, H: int = 8, W: int = 8,
                   cube: Tuple[int, int, int] = (4, 4, 4), n_text: int = 40, Hq: int = 4,
                   Hkv: int = 2, D: int = 128, top_p: float = 0.9,
-                  offset_std: float = 1.5) -> Workload:
+                  offset_std: float = 1.5, n_prefix: int = 0) -> Workload:
     """A scaled-down prefill problem for element-by-element parity (several tiles, ragged text)."""
     return make_prefill("small_prefill", seed=seed, B=B, T=T, H=H, W=W, cube=cube, n_text=n_text,
-                        Hq=Hq, Hkv=Hkv, D=D, top_p=top_p, offset_std=offset_std)
+                        Hq=Hq, Hkv=Hkv, D=D, top_p=top_p, offset_std=offset_std, n_prefix=n_prefix)
 
 
 def small_decode(seed: int = 11, *, B: int = 2, T: int = 16, H: int = 8, W: int = 8,
