@@ -21,7 +21,8 @@
  *     device memory in _forward / _decode and never synchronises the host with the device.
  *     Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = default stream).
  *   - Tensors are bf16, row-major, raster order: q/out [B,S,Hq,D], k/v [B,S,Hkv,D] with
- *     S = T*H*W + n_text and video token (t,y,x) at s = (t*H + y)*W + x.  Q and K are post-RoPE.
+ *     S = T*H*W + n_text and video token (t,y,x) at s = (t*H + y)*W + x (after the n_prefix prefix
+ *     tokens of adaspark_attn_forward_prefix).  Q and K are post-RoPE.
  *   - Query head h uses KV head h / (Hq/Hkv).  Mean keys are per KV head, selection per query head.
  *   - Errors are return codes; argument errors are found on the host before any launch.
  *     adaspark_attn_last_error() returns a message for the most recent failure on a handle.
@@ -68,7 +69,7 @@ typedef struct {
 typedef struct {
     int64_t n_cubes;         /* N                                                              */
     int64_t cube_tokens;     /* C = cube_t*cube_h*cube_w                                       */
-    int64_t s_video;         /* T*H*W                                                          */
+    int64_t s_video;         /* video slots N*C (= T*H*W when the cube window divides the grid) */
     int64_t s_cap;           /* cache rows per (batch, kv head): s_video + n_text_max + 1
                                 rounded up to a multiple of 128                                */
     int64_t bitmap_words;    /* ceil(N/32): uint32 words per selection bitmap row              */
@@ -106,8 +107,11 @@ adaspark_status_t adaspark_attn_create(const adaspark_attn_config_t *config,
  * buffer size.  `batch`, `frames`, `grid_h`, `grid_w` describe the video token grid;
  * `n_text_max` is the largest number of text tokens any later _forward/_decode will hold.
  * `*workspace_bytes` (nullable) receives max(forward, decode) workspace size.  Host only.
- * ERR_UNSUPPORTED if the grid is not divisible by the cube window, N > 4096, or the cache would
- * hold more than 2097152 rows per sequence (s_video + n_text_max + 1).
+ * A grid the cube window does not divide (the paper is silent) is covered by ceil(T/cube_t) x
+ * ceil(H/cube_h) x ceil(W/cube_w) cubes: the cubes at the far faces hold fewer tokens, their mean key is
+ * the mean over the tokens they hold, their other slots stay empty in the caches and are never attended.
+ * ERR_UNSUPPORTED if N > 4096 or the cache would hold more than 2097152 rows per sequence
+ * (s_video + n_text_max + 1).
  * The forward workspace holds two buffers of fp64 cube scores for a chunk of query tiles each
  * (512 MB each by default, less when the whole problem is smaller); the environment variable
  * ADASPARK_SCORE_BUFFER_MB, read here, overrides the size of one buffer (1 .. 65536). */
@@ -142,6 +146,21 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t *handle, const void *q, 
                                         int32_t *sel_count, void *workspace,
                                         size_t workspace_bytes, void *cuda_stream);
 
+/* Prefill of a sequence whose text partly PRECEDES the video: [n_prefix text tokens][video][n_text
+ * text tokens] (the paper places the text after the video and is silent on a prompt before it).
+ * Reading taken: the prefix is attended by every video and text token always and in full, like a
+ * token's own cube: it is no candidate of Eq. 1, its mass does not count toward top_p, and prefix
+ * tokens attend causally among themselves.  q/k/v/out hold the n_prefix + T*H*W + n_text tokens in
+ * that order; n_prefix + n_text <= n_text_max.  In the caches the prefix occupies the first n_prefix
+ * text slots (positions s_video ..), the later text follows it; a decode step after it passes
+ * text_len = n_prefix + n_text.  Everything else as adaspark_attn_forward (= n_prefix 0). */
+adaspark_status_t adaspark_attn_forward_prefix(adaspark_attn_t *handle, const void *q, const void *k,
+                                               const void *v, int32_t n_prefix, int32_t n_text,
+                                               void *out, void *k_cube, void *v_cube,
+                                               float *cube_keys, uint32_t *sel_bitmap,
+                                               int32_t *sel_count, void *workspace,
+                                               size_t workspace_bytes, void *cuda_stream);
+
 /* Chunked prefill: the same computation as adaspark_attn_forward, fed one run of frames at a time
  * (the long-video setting of the paper: a later frame never changes an earlier row, because a video
  * query of Eq. 1 only sees the cubes that precede its own and the text comes after the video).
@@ -149,7 +168,8 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t *handle, const void *q, 
  * their cubes to k_cube / v_cube / cube_keys and computes `out` for these tokens only, attending the
  * cubes of earlier calls through the caches.
  *   frame_begin, frame_count  multiples of cube_t (whole time blocks of cubes); frame_begin * H * W
- *                must be a multiple of 256 (ERR_UNSUPPORTED otherwise).  Chunks must be fed in
+ *                must be a multiple of 256 (ERR_UNSUPPORTED otherwise; so is a grid that the cube
+ *                window does not divide, except through the single chunk (0, T)).  Chunks must be fed in
  *                order, without gaps, to the same caches; the library keeps no record of them.
  *   n_text       < 0: more video follows (no text in this call).  >= 0: this is the last call of the
  *                sequence: it must end the video (frame_begin + frame_count = T; frame_count may be 0

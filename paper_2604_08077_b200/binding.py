@@ -43,7 +43,7 @@ class AdasparkError(RuntimeError):
 _lib: Optional[ctypes.CDLL] = None
 
 EXPORTS = ["adaspark_attn_create", "adaspark_attn_partition", "adaspark_attn_get_layout",
-           "adaspark_attn_forward", "adaspark_attn_forward_chunk", "adaspark_attn_decode", "adaspark_attn_destroy",
+           "adaspark_attn_forward", "adaspark_attn_forward_prefix", "adaspark_attn_forward_chunk", "adaspark_attn_decode", "adaspark_attn_destroy",
            "adaspark_attn_last_error", "adaspark_attn_last_launch_count",
            "adaspark_attn_set_prefill_kernel", "adaspark_attn_enable_stage_timing",
            "adaspark_attn_get_stage_times", "adaspark_attn_decode_static",
@@ -65,6 +65,7 @@ def load() -> ctypes.CDLL:
     lib.adaspark_attn_partition.argtypes = [vp, i32, i32, i32, i32, i32, ctypes.POINTER(sz)]
     lib.adaspark_attn_get_layout.argtypes = [vp, ctypes.POINTER(Layout)]
     lib.adaspark_attn_forward.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.adaspark_attn_forward_prefix.argtypes = [vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.adaspark_attn_forward_chunk.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.adaspark_attn_decode.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.adaspark_attn_decode_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
@@ -138,6 +139,14 @@ def adaspark_attn_forward(handle: int, q, k, v, n_text: int, out, k_cube, v_cube
                           sel_bitmap, sel_count, workspace, workspace_bytes: int, stream=None):
     _check(handle, load().adaspark_attn_forward(
         handle, _ptr(q), _ptr(k), _ptr(v), n_text, _ptr(out), _ptr(k_cube), _ptr(v_cube),
+        _ptr(cube_keys), _ptr(sel_bitmap), _ptr(sel_count), _ptr(workspace), workspace_bytes,
+        _stream_ptr(stream)))
+
+
+def adaspark_attn_forward_prefix(handle: int, q, k, v, n_prefix: int, n_text: int, out, k_cube, v_cube, cube_keys,
+                                 sel_bitmap, sel_count, workspace, workspace_bytes: int, stream=None):
+    _check(handle, load().adaspark_attn_forward_prefix(
+        handle, _ptr(q), _ptr(k), _ptr(v), n_prefix, n_text, _ptr(out), _ptr(k_cube), _ptr(v_cube),
         _ptr(cube_keys), _ptr(sel_bitmap), _ptr(sel_count), _ptr(workspace), workspace_bytes,
         _stream_ptr(stream)))
 
@@ -251,8 +260,9 @@ class AdaSAttn:
         self.workspace = torch.empty(self.ws_bytes, dtype=torch.uint8, device=dev)
         return self
 
-    def forward(self, q, k, v, n_text, *, out=None, want_selection=False, stream=None):
-        """q may be None: builds only the caches.  Returns (out, sel_bitmap, sel_count)."""
+    def forward(self, q, k, v, n_text, *, out=None, want_selection=False, stream=None, n_prefix=0):
+        """q may be None: builds only the caches.  Returns (out, sel_bitmap, sel_count).
+        n_prefix > 0: the first n_prefix tokens of the tensors are text that precedes the video."""
         lay = self.layout
         bitmap = count = None
         if q is not None:
@@ -262,8 +272,12 @@ class AdaSAttn:
                 B, S, Hq, _ = q.shape
                 bitmap = torch.empty(B, Hq, S, lay.bitmap_words, dtype=torch.int32, device=q.device)
                 count = torch.empty(B, Hq, S, dtype=torch.int32, device=q.device)
-        adaspark_attn_forward(self.handle, q, k, v, n_text, out, self.k_cube, self.v_cube,
-                              self.cube_keys, bitmap, count, self.workspace, self.ws_bytes, stream)
+        if n_prefix:
+            adaspark_attn_forward_prefix(self.handle, q, k, v, n_prefix, n_text, out, self.k_cube, self.v_cube,
+                                         self.cube_keys, bitmap, count, self.workspace, self.ws_bytes, stream)
+        else:
+            adaspark_attn_forward(self.handle, q, k, v, n_text, out, self.k_cube, self.v_cube,
+                                  self.cube_keys, bitmap, count, self.workspace, self.ws_bytes, stream)
         return out, bitmap, count
 
     def forward_chunk(self, q, k, v, frame_begin, frame_count, n_text, *, out=None, want_selection=False,

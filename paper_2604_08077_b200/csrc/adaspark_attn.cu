@@ -31,7 +31,7 @@ struct adaspark_attn {
     int C, N, S_v, S_cap;
     adaspark_attn_layout_t layout;
     // workspace carving (byte offsets)
-    size_t fw_status_off, fw_headmax_off, fw_mask_off, fw_union_off, fw_fallback_off, fw_scratch_off, fw_qcube_off,
+    size_t fw_status_off, fw_headmax_off, fw_valid_off, fw_mask_off, fw_union_off, fw_fallback_off, fw_scratch_off, fw_qcube_off,
         fw_kplanes_off, fw_total;
     size_t dc_status_off, dc_bitmap_off, dc_items_off, dc_nitems_off, dc_partial_off, dc_total;
     int dc_splits;
@@ -62,12 +62,15 @@ adaspark_status_t fail(adaspark_attn* h, adaspark_status_t st, const char* fmt, 
 
 // Geometry of one call.  frame_begin / frame_end delimit the video frames this call brings (whole time
 // blocks of cubes); n_text text tokens are present after the call (0 while the video is incomplete).
-Geom make_geom(const adaspark_attn* h, int n_text, int frame_begin = 0, int frame_end = -1) {
+Geom make_geom(const adaspark_attn* h, int n_text, int frame_begin = 0, int frame_end = -1, int n_prefix = 0) {
     Geom g;
     if (frame_end < 0) frame_end = h->T;
     g.B = h->B; g.T = h->T; g.H = h->H; g.W = h->W;
     g.ct = h->cfg.cube_t; g.ch = h->cfg.cube_h; g.cw = h->cfg.cube_w;
-    g.nH = h->H / g.ch; g.nW = h->W / g.cw;
+    g.nH = (h->H + g.ch - 1) / g.ch; g.nW = (h->W + g.cw - 1) / g.cw;
+    g.ragged = (h->T % g.ct || h->H % g.ch || h->W % g.cw) ? 1 : 0;
+    g.S_tok = h->T * h->H * h->W;
+    g.n_prefix = n_prefix;
     g.C = h->C; g.N = h->N;
     g.c_shift = 0;
     while ((1 << g.c_shift) < g.C) ++g.c_shift;
@@ -75,12 +78,14 @@ Geom make_geom(const adaspark_attn* h, int n_text, int frame_begin = 0, int fram
     while ((1 << g.cw_shift) < g.cw) ++g.cw_shift;
     g.ch_shift = 0;
     while ((1 << g.ch_shift) < g.ch) ++g.ch_shift;
-    g.S_v = h->S_v; g.n_text = n_text;
-    g.S = frame_end * h->H * h->W + n_text;                  // n_text > 0 only once the video is complete
+    g.S_v = h->S_v; g.n_text = n_text + n_prefix;
+    // slots present after the call (text only once the video is complete; chunks need H and W divisible,
+    // so that frames count the same in tokens and in slots)
+    g.S = (frame_end == h->T ? h->S_v : frame_end * h->H * h->W) + n_prefix + n_text;
     g.pos_begin = frame_begin * h->H * h->W;
-    g.S_io = g.S - g.pos_begin;
+    g.S_io = (frame_end - frame_begin) * h->H * h->W + n_prefix + n_text;
     g.tile_begin = g.pos_begin / kTileRows;
-    g.N_live = (frame_end / h->cfg.cube_t) * (h->H / g.ch) * (h->W / g.cw);
+    g.N_live = ((frame_end + g.ct - 1) / g.ct) * g.nH * g.nW;
     g.S_cap = h->S_cap;
     g.n_words = (h->N + 31) / 32;
     g.n_tiles = (g.S + kTileRows - 1) / kTileRows;
@@ -165,12 +170,11 @@ adaspark_status_t adaspark_attn_partition(adaspark_attn_t* h, int32_t batch, int
     if (batch <= 0 || frames <= 0 || grid_h <= 0 || grid_w <= 0 || n_text_max < 0)
         return fail(h, ADASPARK_ERR_INVALID_ARG, "partition: non-positive size");
     const adaspark_attn_config_t& c = h->cfg;
-    if (frames % c.cube_t || grid_h % c.cube_h || grid_w % c.cube_w)
-        return fail(h, ADASPARK_ERR_UNSUPPORTED, "partition: grid %dx%dx%d not divisible by cube %dx%dx%d",
-                    frames, grid_h, grid_w, c.cube_t, c.cube_h, c.cube_w);
-    long long N = (long long)(frames / c.cube_t) * (grid_h / c.cube_h) * (grid_w / c.cube_w);
+    // a grid the window does not divide is covered by ceil() cubes per axis; the far cubes hold fewer tokens
+    long long N = (long long)((frames + c.cube_t - 1) / c.cube_t) * ((grid_h + c.cube_h - 1) / c.cube_h) *
+                  ((grid_w + c.cube_w - 1) / c.cube_w);
     if (N > 4096) return fail(h, ADASPARK_ERR_UNSUPPORTED, "partition: %lld cubes > 4096", N);
-    long long S_v = (long long)frames * grid_h * grid_w;
+    long long S_v = N * h->C;                                // cache slots of the video (= tokens unless ragged)
     long long S_cap = (S_v + n_text_max + 1 + 127) / 128 * 128;
     if ((long long)batch * S_cap * c.n_q_heads * c.head_dim >= (1ll << 40) || S_cap >= (1ll << 30))
         return fail(h, ADASPARK_ERR_UNSUPPORTED, "partition: problem too large");
@@ -197,6 +201,7 @@ adaspark_status_t adaspark_attn_partition(adaspark_attn_t* h, int32_t batch, int
     size_t off = 0;
     h->fw_status_off = off; off = align_up(off + 256);
     h->fw_headmax_off = off; off = align_up(off + (size_t)batch * Hkv * 4);
+    h->fw_valid_off = off; off = align_up(off + (size_t)(S_cap / kBlockTok) * 2 * 4);   // which slots of a block hold a token
     h->fw_mask_off = off; off = align_up(off + (size_t)batch * Hq * n_tiles_cap * n_words * kTileRows * 4);
     h->fw_union_off = off; off = align_up(off + (size_t)batch * Hq * n_tiles_cap * n_words * 4);
     h->fw_fallback_off = off; off = align_up(off + (size_t)batch * Hq * n_tiles_cap * kTileRows * 4);
@@ -253,7 +258,7 @@ namespace {
 // sequence), n_text text tokens; n_text < 0: more video follows.  The one-shot forward is the window
 // [0, T) with its text.
 adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* q, const void* k, const void* v,
-                               int32_t frame_begin, int32_t frame_count, int32_t n_text_arg, void* out, void* k_cube,
+                               int32_t frame_begin, int32_t frame_count, int32_t n_text_arg, int32_t n_prefix, void* out, void* k_cube,
                                void* v_cube, float* cube_keys, uint32_t* sel_bitmap, int32_t* sel_count, void* workspace,
                                size_t workspace_bytes, void* cuda_stream) {
     if (!h) return ADASPARK_ERR_INVALID_ARG;
@@ -262,11 +267,16 @@ adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* 
     if ((q == nullptr) != (out == nullptr)) return fail(h, ADASPARK_ERR_INVALID_ARG, "%s: q and out must both be given or both be NULL", who);
     const bool last_call = n_text_arg >= 0;
     const int n_text = last_call ? n_text_arg : 0;
-    if (n_text > h->n_text_max) return fail(h, ADASPARK_ERR_INVALID_ARG, "%s: n_text %d outside [0, %d]", who, n_text, h->n_text_max);
+    if (n_prefix < 0 || (long long)n_text + n_prefix > h->n_text_max)
+        return fail(h, ADASPARK_ERR_INVALID_ARG, "%s: %d prefix + %d text tokens outside [0, %d]", who, n_prefix, n_text, h->n_text_max);
     const int ct = h->cfg.cube_t;
-    if (frame_begin < 0 || frame_count < 0 || frame_begin % ct || frame_count % ct || frame_begin + frame_count > h->T)
+    const bool whole = frame_begin == 0 && frame_count == h->T;
+    if (frame_begin < 0 || frame_count < 0 || frame_begin + frame_count > h->T || frame_begin % ct ||
+        ((frame_begin + frame_count) % ct && frame_begin + frame_count != h->T))
         return fail(h, ADASPARK_ERR_INVALID_ARG, "%s: frames [%d, %d) are not whole time blocks of %d frames inside [0, %d)", who,
                     frame_begin, frame_begin + frame_count, ct, h->T);
+    if (!whole && (n_prefix > 0 || h->T % ct || h->H % h->cfg.cube_h || h->W % h->cfg.cube_w))
+        return fail(h, ADASPARK_ERR_UNSUPPORTED, "%s: a chunked prefill takes no text prefix and needs a grid the cube window divides", who);
     if (last_call && frame_begin + frame_count != h->T)
         return fail(h, ADASPARK_ERR_INVALID_ARG, "%s: the call that brings the text must end the video (frame %d of %d)", who,
                     frame_begin + frame_count, h->T);
@@ -284,7 +294,7 @@ adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* 
     if (ce != cudaSuccess) return fail(h, ADASPARK_ERR_CUDA, "%s: cudaSetDevice(%d): %s", who, h->cfg.device, cudaGetErrorString(ce));
     cudaStream_t st = (cudaStream_t)cuda_stream;
     h->launches = 0;
-    const Geom g = make_geom(h, n_text, frame_begin, frame_begin + frame_count);
+    const Geom g = make_geom(h, n_text, frame_begin, frame_begin + frame_count, n_prefix);
     const int D = g.D;
     auto* kb = (const __nv_bfloat16*)k;
     auto* vb = (const __nv_bfloat16*)v;
@@ -300,8 +310,9 @@ adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* 
         const int blk_begin = g.pos_begin / kBlockTok;
         const int blk_end = last_call ? g.n_kv_blocks_cap : (g.S + kBlockTok - 1) / kBlockTok;
         dim3 grid(blk_end - blk_begin, g.Hkv, g.B);
-        if (D == 128) relayout_pool_kernel<128><<<grid, 256, 0, st>>>(g, kb, vb, kc, vc, cube_keys);
-        else relayout_pool_kernel<64><<<grid, 256, 0, st>>>(g, kb, vb, kc, vc, cube_keys);
+        uint32_t* slot_valid = (!cache_only && g.ragged) ? (uint32_t*)((char*)workspace + h->fw_valid_off) : nullptr;
+        if (D == 128) relayout_pool_kernel<128><<<grid, 256, 0, st>>>(g, kb, vb, kc, vc, cube_keys, slot_valid);
+        else relayout_pool_kernel<64><<<grid, 256, 0, st>>>(g, kb, vb, kc, vc, cube_keys, slot_valid);
         if (!launch_ok(h, "relayout_pool_kernel")) return ADASPARK_ERR_CUDA;
         const int cube_begin = g.pos_begin >> g.c_shift;
         if (g.C > kBlockTok && g.N_live > cube_begin) {
@@ -311,7 +322,7 @@ adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* 
     }
 #ifdef ADASPARK_WITH_TCGEN05
     if (!cache_only && h->prefill_kernel != 0) {   // cube-major staging of Q for the TMA loads of K3 / K4
-        dim3 rgrid((g.S_io + 3) / 4, g.B);
+        dim3 rgrid((g.S - g.pos_begin + 3) / 4, g.B);     // slots of the call's row window
         __nv_bfloat16* q_cube = (__nv_bfloat16*)((char*)workspace + h->fw_qcube_off);
         if (D == 128) relayout_q_kernel<128><<<rgrid, 256, 0, st>>>(g, (const __nv_bfloat16*)q, q_cube);
         else relayout_q_kernel<64><<<rgrid, 256, 0, st>>>(g, (const __nv_bfloat16*)q, q_cube);
@@ -399,15 +410,16 @@ adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* 
             !encode_bf16_2d(&tmV, vc, (uint64_t)g.B * g.Hkv * g.n_kv_blocks_cap * D, 64, 64, D))
             return fail(h, ADASPARK_ERR_CUDA, "%s: cuTensorMapEncodeTiled failed", who);
         dim3 grid(((g.S + kPairRows - 1) / kPairRows - g.pos_begin / kPairRows) * g.Hq * g.B);
+        const uint32_t* slot_valid_c = (const uint32_t*)(ws + h->fw_valid_off);
         if (D == 128) {
             size_t smem = sizeof(TcAttnSmem<128>) + 1024;
             if (!set_smem(h, attn_prefill_tc_kernel<128>, smem, "attn_prefill_tc_kernel")) return ADASPARK_ERR_CUDA;
-            attn_prefill_tc_kernel<128><<<grid, kTcThreads, smem, st>>>(g, tmQ, tmK, tmV, tile_mask, tile_union, (__nv_bfloat16*)out,
+            attn_prefill_tc_kernel<128><<<grid, kTcThreads, smem, st>>>(g, tmQ, tmK, tmV, tile_mask, tile_union, slot_valid_c, (__nv_bfloat16*)out,
                                                                         (unsigned long long*)&hdr->executed_kv_blocks, &hdr->max_tile_kv_blocks, &hdr->status);
         } else {
             size_t smem = sizeof(TcAttnSmem<64>) + 1024;
             if (!set_smem(h, attn_prefill_tc_kernel<64>, smem, "attn_prefill_tc_kernel")) return ADASPARK_ERR_CUDA;
-            attn_prefill_tc_kernel<64><<<grid, kTcThreads, smem, st>>>(g, tmQ, tmK, tmV, tile_mask, tile_union, (__nv_bfloat16*)out,
+            attn_prefill_tc_kernel<64><<<grid, kTcThreads, smem, st>>>(g, tmQ, tmK, tmV, tile_mask, tile_union, slot_valid_c, (__nv_bfloat16*)out,
                                                                        (unsigned long long*)&hdr->executed_kv_blocks, &hdr->max_tile_kv_blocks, &hdr->status);
         }
         if (!launch_ok(h, "attn_prefill_tc_kernel")) return ADASPARK_ERR_CUDA;
@@ -441,8 +453,18 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
                                         size_t workspace_bytes, void* cuda_stream) {
     if (!h) return ADASPARK_ERR_INVALID_ARG;
     if (n_text < 0) return fail(h, ADASPARK_ERR_INVALID_ARG, "forward: n_text %d outside [0, %d]", n_text, h->n_text_max);
-    return forward_impl(h, "forward", q, k, v, 0, h->partitioned ? h->T : 0, n_text, out, k_cube, v_cube, cube_keys, sel_bitmap,
+    return forward_impl(h, "forward", q, k, v, 0, h->partitioned ? h->T : 0, n_text, 0, out, k_cube, v_cube, cube_keys, sel_bitmap,
                         sel_count, workspace, workspace_bytes, cuda_stream);
+}
+
+adaspark_status_t adaspark_attn_forward_prefix(adaspark_attn_t* h, const void* q, const void* k, const void* v,
+                                               int32_t n_prefix, int32_t n_text, void* out, void* k_cube, void* v_cube,
+                                               float* cube_keys, uint32_t* sel_bitmap, int32_t* sel_count,
+                                               void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!h) return ADASPARK_ERR_INVALID_ARG;
+    if (n_text < 0 || n_prefix < 0) return fail(h, ADASPARK_ERR_INVALID_ARG, "forward_prefix: negative token count");
+    return forward_impl(h, "forward_prefix", q, k, v, 0, h->partitioned ? h->T : 0, n_text, n_prefix, out, k_cube, v_cube, cube_keys,
+                        sel_bitmap, sel_count, workspace, workspace_bytes, cuda_stream);
 }
 
 adaspark_status_t adaspark_attn_forward_chunk(adaspark_attn_t* h, const void* q, const void* k, const void* v,
@@ -450,7 +472,7 @@ adaspark_status_t adaspark_attn_forward_chunk(adaspark_attn_t* h, const void* q,
                                               void* k_cube, void* v_cube, float* cube_keys, uint32_t* sel_bitmap,
                                               int32_t* sel_count, void* workspace, size_t workspace_bytes,
                                               void* cuda_stream) {
-    return forward_impl(h, "forward_chunk", q, k, v, frame_begin, frame_count, n_text < 0 ? -1 : n_text, out, k_cube, v_cube,
+    return forward_impl(h, "forward_chunk", q, k, v, frame_begin, frame_count, n_text < 0 ? -1 : n_text, 0, out, k_cube, v_cube,
                         cube_keys, sel_bitmap, sel_count, workspace, workspace_bytes, cuda_stream);
 }
 

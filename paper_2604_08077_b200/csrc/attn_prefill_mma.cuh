@@ -47,7 +47,7 @@ __global__ void __launch_bounds__(256) attn_prefill_mma_kernel(Geom g, const __n
         int row = idx / kQChunks, c = idx - row * kQChunks;
         int pos = tile_pos0 + row;
         uint4 val = make_uint4(0, 0, 0, 0);
-        if (pos < g.S)
+        if (slot_live(g, pos))
             val = *reinterpret_cast<const uint4*>(q + (io_row(g, b, pos) * g.Hq + h) * D + c * 8);
         *reinterpret_cast<uint4*>(&sm.q[row][swz(row, c) * 8]) = val;
     }
@@ -63,9 +63,14 @@ __global__ void __launch_bounds__(256) attn_prefill_mma_kernel(Geom g, const __n
     // local range of the tile: from the first row's own cube (video) or the text start
     const int local_start = tile_pos0 < g.S_v ? (tile_pos0 / g.C) * g.C : g.S_v;
     const int first_local_blk = local_start / kBlockTok;
-    const int n_blk = (tile_end + kBlockTok - 1) / kBlockTok;
+    // blocks up to the tile's own end, and for a tile with video rows also those of the text prefix
+    const int n_blk_own = (tile_end + kBlockTok - 1) / kBlockTok;
+    const bool sees_prefix = g.n_prefix > 0 && tile_pos0 < g.S_v;
+    const int prefix_blk0 = g.S_v / kBlockTok;
+    const int n_blk = sees_prefix ? max(n_blk_own, (g.S_v + g.n_prefix + kBlockTok - 1) / kBlockTok) : n_blk_own;
 
     auto block_needed = [&](int kb) -> bool {
+        if (kb >= n_blk_own) return kb >= prefix_blk0;
         if (kb >= first_local_blk) return true;
         // cubes overlapping block kb: [kb*64 / C, (kb*64 + 63) / C]
         int c_lo = (kb * kBlockTok) / g.C, c_hi = (kb * kBlockTok + kBlockTok - 1) / g.C;
@@ -220,13 +225,13 @@ __global__ void __launch_bounds__(256) attn_prefill_mma_kernel(Geom g, const __n
     lB += __shfl_xor_sync(0xffffffffu, lB, 1);
     lB += __shfl_xor_sync(0xffffffffu, lB, 2);
     float invA = lA > 0.f ? 1.f / lA : 0.f, invB = lB > 0.f ? 1.f / lB : 0.f;
-    if (posA < g.S) {
+    if (slot_live(g, posA)) {
         __nv_bfloat16* dst = out + (io_row(g, b, posA) * g.Hq + h) * D + 2 * (lane & 3);
 #pragma unroll
         for (int dt = 0; dt < kDTiles; ++dt)
             *reinterpret_cast<uint32_t*>(dst + dt * 8) = pack_bf16x2(o[dt][0] * invA, o[dt][1] * invA);
     }
-    if (posB < g.S) {
+    if (slot_live(g, posB)) {
         __nv_bfloat16* dst = out + (io_row(g, b, posB) * g.Hq + h) * D + 2 * (lane & 3);
 #pragma unroll
         for (int dt = 0; dt < kDTiles; ++dt)

@@ -61,7 +61,7 @@ template <int D>
 __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     Geom g, const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
     const __grid_constant__ CUtensorMap tmV, const uint32_t* __restrict__ tile_mask,
-    const uint32_t* __restrict__ tile_union, __nv_bfloat16* __restrict__ out,
+    const uint32_t* __restrict__ tile_union, const uint32_t* __restrict__ slot_valid, __nv_bfloat16* __restrict__ out,
     unsigned long long* __restrict__ executed_blocks, uint32_t* __restrict__ max_tile_blocks, int32_t* __restrict__ status) {
     extern __shared__ unsigned char tc_smem_raw[];
     TcAttnSmem<D>& sm = *reinterpret_cast<TcAttnSmem<D>*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -80,7 +80,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int pair_pos0 = pair * kPairRows;
     const int pair_end = min(pair_pos0 + kPairRows, g.S);       // exclusive
-    const int n_blk = (pair_end + kBlockTok - 1) / kBlockTok;   // key blocks that can matter
+    // key blocks that can matter: up to the pair's own end, and for a pair with video rows also the blocks
+    // of the text prefix (attended by every video row)
+    const int prefix_blk0 = g.S_v / kBlockTok, prefix_blk1 = (g.S_v + g.n_prefix + kBlockTok - 1) / kBlockTok;
+    const bool sees_prefix = g.n_prefix > 0 && pair_pos0 < g.S_v;
+    const int n_blk_own = (pair_end + kBlockTok - 1) / kBlockTok;
+    const int n_blk = sees_prefix ? max(n_blk_own, prefix_blk1) : n_blk_own;
     const int local_start = pair_pos0 < g.S_v ? ((pair_pos0 >> g.c_shift) << g.c_shift) : g.S_v;
     const int first_local_blk = local_start / kBlockTok;
 
@@ -134,13 +139,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     const int n_blk_words = (n_blk + 31) / 32;
     for (int wi = tid; wi < n_blk_words; wi += kTcThreads) {
         uint32_t bits = 0;
-        if (g.c_shift == 6 && wi * 32 + 31 < first_local_blk) {
+        if (g.c_shift == 6 && wi * 32 + 31 < first_local_blk) {   // (first_local_blk <= prefix_blk0)
             bits = sm.union_words[wi];             // 64-token cubes: key block = cube, the word is the union word
         } else {
             for (int i = 0; i < 32; ++i) {
                 int kb = wi * 32 + i;
                 if (kb >= n_blk) break;
-                bool need = kb >= first_local_blk;
+                bool need = (kb >= first_local_blk && kb < n_blk_own) || (sees_prefix && kb >= prefix_blk0);
                 if (!need) {
                     int c_lo = (kb * kBlockTok) >> g.c_shift, c_hi = (kb * kBlockTok + kBlockTok - 1) >> g.c_shift;
                     uint32_t span = c_hi - c_lo + 1;   // <= 4 cubes, aligned: never crosses a word
@@ -318,7 +323,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
 #pragma unroll
                     for (int q4 = 0; q4 < 4; ++q4) {
                         const int pg = pk0 + q4 * 16;
-                        const int n_causal = min(max(pr - pg + 1, 0), 16);           // keys pg..pr
+                        // keys pg..pr; a video row sees the text prefix (slots S_v .. S_v + n_prefix) in full
+                        const int n_causal = (pg >= g.S_v && pr < g.S_v) ? min(max(g.S_v + g.n_prefix - pg, 0), 16)
+                                                                         : min(max(pr - pg + 1, 0), 16);
                         const uint32_t causal = (1u << n_causal) - 1u;
                         const int ck = pg >> g.c_shift;
                         const bool own = pg >= g.S_v || (pr < g.S_v && ck == (pr >> g.c_shift));
@@ -327,6 +334,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
                     }
                     m0 = gm[0] | (gm[1] << 16);
                     m1 = gm[2] | (gm[3] << 16);
+                }
+                if (g.ragged && pk0 < g.S_v && !(hf == 1 && !has_b)) {   // empty slots of boundary cubes are never attended
+                    m0 &= __ldg(slot_valid + 2 * kb);
+                    m1 &= __ldg(slot_valid + 2 * kb + 1);
                 }
                 amask[hf * 2] = m0;
                 amask[hf * 2 + 1] = m1;
@@ -456,7 +467,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
         if (ok) {
             tc::tc_fence_after_sync();
             const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
-            const bool live = pr < g.S;
+            const bool live = slot_live(g, pr);
             __nv_bfloat16* dst = out + ((live ? io_row(g, b, pr) : 0) * g.Hq + h) * D;
             uint32_t o[D / 32][32];                                // the whole output row in one round of loads
 #pragma unroll
@@ -513,7 +524,8 @@ __global__ void __launch_bounds__(256) relayout_q_kernel(Geom g, const __nv_bflo
         int h = rem / kChunks, c = rem - h * kChunks;
         int pos = pos0 + p;
         if (pos >= g.S) break;
-        uint4 val = *reinterpret_cast<const uint4*>(q + (io_row(g, b, pos) * g.Hq + h) * D + c * 8);
+        uint4 val = make_uint4(0u, 0u, 0u, 0u);              // an empty slot of a boundary cube stays zero
+        if (slot_live(g, pos)) val = *reinterpret_cast<const uint4*>(q + (io_row(g, b, pos) * g.Hq + h) * D + c * 8);
         *reinterpret_cast<uint4*>(q_cube + ((size_t)(b * g.Hq + h) * g.S_cap + pos) * D + c * 8) = val;
     }
 }

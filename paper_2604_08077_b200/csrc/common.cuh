@@ -33,8 +33,12 @@ struct FastDiv {
     }
 };
 
-// Geometry of one partitioned problem (Sec. 3.1).  "pos" is the cube-major position of a token:
-// video token of cube c with intra-cube rank r sits at pos = c*C + r, text token u at S_v + u.
+// Geometry of one partitioned problem (Sec. 3.1).  "pos" is the cube-major position of a token in
+// the caches: the video token of cube c with in-window rank r sits at pos = c*C + r (a cube at the far
+// face of a grid that the window does not divide holds fewer tokens than its C slots: the other slots
+// stay empty), text token u at S_v + u.  Text that precedes the video in the sequence (a prompt prefix,
+// n_prefix tokens) occupies the first n_prefix text slots: it is attended by every video and text row in
+// full and is no candidate of Eq. 1; the text after the video follows it.
 struct Geom {
     int B, T, H, W;      // batch, frames, patch rows, patch columns
     int ct, ch, cw;      // cube window
@@ -43,7 +47,10 @@ struct Geom {
     int c_shift;         // log2(C)
     int cw_shift, ch_shift;   // log2(cw), log2(ch): C is a power of two, so every window side is one
     FastDiv div_nW, div_nH, div_n_tiles, div_Hq;
-    int S_v, n_text, S;  // video tokens of the partition, text tokens so far, positions present after this call
+    int S_v, n_text, S;  // video slots N*C of the partition, text tokens so far (prefix included), slots present after this call
+    int S_tok;           // video tokens T*H*W (= S_v unless the grid is ragged)
+    int n_prefix;        // text tokens of the sequence that precede the video
+    int ragged;          // 1: the window does not divide the grid (some slots of boundary cubes are empty)
     // Row window of this call (chunked prefill): the q/k/v/out tensors hold the S_io tokens whose
     // cube-major positions are [pos_begin, S) -- whole time blocks of cubes, so they are also the raster
     // tokens pos_begin .. -- and only those rows are computed.  One-shot prefill: pos_begin = 0, S_io = S.
@@ -64,9 +71,13 @@ struct Geom {
     int top_k;           // > 0: Top-K rule instead of Top-p
 };
 
-// O1 inverse: cube-major position -> raster token index.
-__device__ __forceinline__ int pos_to_raster(const Geom& g, int pos) {
-    if (pos >= g.S_v) return pos;
+// O1 inverse: cube-major position -> index of the token in the sequence [prefix][video, raster][text],
+// or -1 for a slot that holds no token.
+__device__ __forceinline__ int pos_to_io(const Geom& g, int pos) {
+    if (pos >= g.S_v) {
+        const int u = pos - g.S_v;
+        return u < g.n_prefix ? u : u + g.S_tok;        // text after the video: n_prefix + S_tok + (u - n_prefix)
+    }
     const int c = pos >> g.c_shift, r = pos & (g.C - 1);
     int cx, cy, cb, t;
     g.div_nW.divmod(c, t, cx);
@@ -74,17 +85,34 @@ __device__ __forceinline__ int pos_to_raster(const Geom& g, int pos) {
     const int rx = r & (g.cw - 1);
     const int ry = (r >> g.cw_shift) & (g.ch - 1);
     const int rt = r >> (g.cw_shift + g.ch_shift);
-    return ((cb * g.ct + rt) * g.H + (cy * g.ch + ry)) * g.W + (cx * g.cw + rx);
+    const int tt = cb * g.ct + rt, yy = cy * g.ch + ry, xx = cx * g.cw + rx;
+    if (g.ragged && (tt >= g.T || yy >= g.H || xx >= g.W)) return -1;
+    return g.n_prefix + (tt * g.H + yy) * g.W + xx;
 }
 
-// Row of the call's q/k/v/out tensors (batch b) that holds the token at cube-major position pos.
+// Does the slot at pos hold a token of the sequence so far?
+__device__ __forceinline__ bool slot_live(const Geom& g, int pos) {
+    return pos < g.S && (!g.ragged || pos >= g.S_v || pos_to_io(g, pos) >= 0);
+}
+
+// Row of the call's q/k/v/out tensors (batch b) that holds the token at cube-major position pos (a live slot).
 __device__ __forceinline__ size_t io_row(const Geom& g, int b, int pos) {
-    return (size_t)b * g.S_io + (pos_to_raster(g, pos) - g.pos_begin);
+    return (size_t)b * g.S_io + (pos_to_io(g, pos) - g.pos_begin);
 }
 
-// Number of candidate cubes of the row at `pos`: preceding cubes for video, all cubes for text.
+// Number of candidate cubes of the row at `pos`: preceding cubes for video, none for the prefix, all cubes
+// for the text after the video.
 __device__ __forceinline__ int n_candidates(const Geom& g, int pos) {
-    return pos < g.S_v ? (pos >> g.c_shift) : g.N;
+    return pos < g.S_v ? (pos >> g.c_shift) : (pos < g.S_v + g.n_prefix ? 0 : g.N);
+}
+
+// Largest candidate count among the rows of query tile `tile` (candidate counts grow along the video, drop
+// to zero on the text prefix and are N on the text after it).
+__device__ __forceinline__ int tile_max_candidates(const Geom& g, int tile) {
+    const int first = tile * kTileRows, last = min(first + kTileRows, g.S) - 1;
+    int m = n_candidates(g, last);
+    if (first < g.S_v && last >= g.S_v) m = max(m, n_candidates(g, g.S_v - 1));
+    return m;
 }
 
 // Per-tile selection mask matrix: word w of row r of global tile gt at
@@ -97,9 +125,10 @@ __device__ __forceinline__ size_t mask_index(const Geom& g, int b, int h, int ti
 // `word` is the row's selection word that covers cube pk/C (bits of cubes that are not
 // candidates of the row are never set by the selection kernel).
 __device__ __forceinline__ bool key_allowed(const Geom& g, int pr, int pk, uint32_t word) {
-    if (pk <= pr && (pk >= g.S_v || (pk >> g.c_shift) == (pr >> g.c_shift))) return true;  // own cube / text prefix
-    if (pk < g.S_v) return (word >> ((pk >> g.c_shift) & 31)) & 1u;                        // selected cube
-    return false;
+    if (pk >= g.S_v) return pk <= pr || (pr < g.S_v && pk < g.S_v + g.n_prefix);   // text causally; the prefix for every video row
+    if (g.ragged && pos_to_io(g, pk) < 0) return false;                            // an empty slot of a boundary cube
+    if (pk <= pr && (pk >> g.c_shift) == (pr >> g.c_shift)) return true;           // own cube up to the query
+    return (word >> ((pk >> g.c_shift) & 31)) & 1u;                                // selected cube
 }
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {

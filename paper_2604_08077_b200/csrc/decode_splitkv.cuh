@@ -136,8 +136,9 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_splitkv_kernel(
                     int pk = pk0 + nt * 8 + 2 * (lane & 3) + e;
                     bool text_ok = pk >= g.S_v && pk <= pos_new;
                     int cb = (pk >> g.c_shift) & 31;
-                    bool okA = text_ok || (pk < g.S_v && ((wordA >> cb) & 1u));
-                    bool okB = text_ok || (pk < g.S_v && ((wordB >> cb) & 1u));
+                    bool held = pk < g.S_v && (!g.ragged || pos_to_io(g, pk) >= 0);   // not an empty slot of a boundary cube
+                    bool okA = text_ok || (held && ((wordA >> cb) & 1u));
+                    bool okB = text_ok || (held && ((wordB >> cb) & 1u));
                     float va = okA ? sc[nt][e] * g.scale_log2 : -INFINITY;
                     float vb = okB ? sc[nt][2 + e] * g.scale_log2 : -INFINITY;
                     sc[nt][e] = va;

@@ -13,12 +13,22 @@
 
 namespace adaspark {
 
+// Tokens a cube holds: C, fewer at the far faces of a grid the window does not divide.
+__device__ __forceinline__ int cube_tokens_held(const Geom& g, int cube) {
+    if (!g.ragged) return g.C;
+    int cx, cy, cb, t;
+    g.div_nW.divmod(cube, t, cx);
+    g.div_nH.divmod(t, cb, cy);
+    return min(g.ct, g.T - cb * g.ct) * min(g.ch, g.H - cy * g.ch) * min(g.cw, g.W - cx * g.cw);
+}
+
 template <int D>
 __global__ void __launch_bounds__(256) relayout_pool_kernel(Geom g, const __nv_bfloat16* __restrict__ k,
                                                             const __nv_bfloat16* __restrict__ v,
                                                             __nv_bfloat16* __restrict__ k_cube,
                                                             __nv_bfloat16* __restrict__ v_cube,
-                                                            float* __restrict__ cube_keys) {
+                                                            float* __restrict__ cube_keys,
+                                                            uint32_t* __restrict__ slot_valid) {
     constexpr int kChunks = D / 8;    // 16-byte chunks per row
     constexpr int kVPitch = D + 2;    // padded pitch (elements) of the V staging tile
     __shared__ __align__(16) __nv_bfloat16 Ks[kBlockTok][D];
@@ -32,7 +42,7 @@ __global__ void __launch_bounds__(256) relayout_pool_kernel(Geom g, const __nv_b
         int row = idx / kChunks, c = idx - row * kChunks;
         int pos = pos0 + row;
         uint4 kv4 = make_uint4(0, 0, 0, 0), vv4 = make_uint4(0, 0, 0, 0);
-        if (pos < g.S) {
+        if (slot_live(g, pos)) {
             size_t src = (io_row(g, b, pos) * g.Hkv + gk) * D + c * 8;
             kv4 = *reinterpret_cast<const uint4*>(k + src);
             vv4 = *reinterpret_cast<const uint4*>(v + src);
@@ -43,6 +53,13 @@ __global__ void __launch_bounds__(256) relayout_pool_kernel(Geom g, const __nv_b
         vdst[0] = vv4.x; vdst[1] = vv4.y; vdst[2] = vv4.z; vdst[3] = vv4.w;
     }
     __syncthreads();
+
+    // Which of the block's 64 slots hold a token (two words per block; read by the attention kernels of a
+    // ragged grid, whose boundary cubes have empty slots)
+    if (slot_valid != nullptr && gk == 0 && b == 0 && tid < 64) {
+        const uint32_t bits = __ballot_sync(0xffffffffu, slot_live(g, pos0 + tid));
+        if ((tid & 31) == 0) slot_valid[2 * blk + (tid >> 5)] = bits;
+    }
 
     // V^T: 8 consecutive threads write one 128-byte row (64 tokens of one d).
     __nv_bfloat16* vt = v_cube + ((size_t)(b * g.Hkv + gk) * g.n_kv_blocks_cap + blk) * D * kBlockTok;
@@ -61,9 +78,9 @@ __global__ void __launch_bounds__(256) relayout_pool_kernel(Geom g, const __nv_b
             int cb = idx / D, d = idx - cb * D;
             int cube = pos0 / g.C + cb;
             if (cube < g.N_live) {
-                double acc = 0.0;
+                double acc = 0.0;                                   // empty slots hold zeros
                 for (int r = 0; r < g.C; ++r) acc += (double)__bfloat162float(Ks[cb * g.C + r][d]);
-                cube_keys[((size_t)(b * g.Hkv + gk) * g.N + cube) * D + d] = (float)(acc / (double)g.C);
+                cube_keys[((size_t)(b * g.Hkv + gk) * g.N + cube) * D + d] = (float)(acc / (double)cube_tokens_held(g, cube));
             }
         }
     }
@@ -78,7 +95,7 @@ __global__ void pool_large_cubes_kernel(Geom g, const __nv_bfloat16* __restrict_
     const __nv_bfloat16* src = k_cube + ((size_t)(b * g.Hkv + gk) * g.S_cap + (size_t)cube * g.C) * g.D + d;
     double acc = 0.0;
     for (int r = 0; r < g.C; ++r) acc += (double)__bfloat162float(src[(size_t)r * g.D]);
-    cube_keys[((size_t)(b * g.Hkv + gk) * g.N + cube) * g.D + d] = (float)(acc / (double)g.C);
+    cube_keys[((size_t)(b * g.Hkv + gk) * g.N + cube) * g.D + d] = (float)(acc / (double)cube_tokens_held(g, cube));
 }
 
 }  // namespace adaspark

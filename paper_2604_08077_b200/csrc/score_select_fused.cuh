@@ -188,8 +188,7 @@ __device__ __forceinline__ FusedItem fused_item(const Geom& g, int it) {
     w.tile = g.n_tiles - 1 - lvl;
     g.div_Hq.divmod(hb, w.b, w.h);
     w.gk = w.h / g.G;
-    const int last_pos = min(w.tile * kTileRows + kTileRows, g.S) - 1;
-    w.n_ct = (n_candidates(g, last_pos) + kScoreTcCols - 1) / kScoreTcCols;
+    w.n_ct = (tile_max_candidates(g, w.tile) + kScoreTcCols - 1) / kScoreTcCols;
     return w;
 }
 
@@ -358,7 +357,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
             const FusedItem w = fused_item(g, it);
             if (w.n_ct == 0) continue;
             const int pos = w.tile * kTileRows + r;
-            const bool live = pos < g.S;
+            const bool live = slot_live(g, pos);
             const uint4* src = reinterpret_cast<const uint4*>(q_cube + ((size_t)(w.b * g.Hq + w.h) * g.S_cap + pos) * D);
             // first sweep over the row (before the planes are free): its largest exponent
             uint32_t mxbits = 0;
@@ -449,13 +448,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
         for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x, t_par ^= 1) {
             const FusedItem w = fused_item(g, it);
             const int pos = w.tile * kTileRows + r;
-            const bool live = pos < g.S;
+            const bool live = slot_live(g, pos);
             const int n = live ? n_candidates(g, pos) : 0;
             const int n_warp = __reduce_max_sync(0xffffffffu, n);
             const size_t gt_cap = (size_t)(w.b * g.Hq + w.h) * g.n_tiles_cap + w.tile;
             uint32_t* mask_row = tile_mask + gt_cap * g.n_words * kTileRows + r;        // word w at mask_row[w * 128]
             const bool extra = live && (sel_bitmap != nullptr || sel_count != nullptr);
-            const size_t raster_row = extra ? (size_t)(w.b * g.Hq + w.h) * g.S_io + (pos_to_raster(g, pos) - g.pos_begin) : 0;
+            const size_t raster_row = extra ? (size_t)(w.b * g.Hq + w.h) * g.S_io + (pos_to_io(g, pos) - g.pos_begin) : 0;
             uint32_t* bm_row = (extra && sel_bitmap) ? sel_bitmap + raster_row * g.n_words : nullptr;
             // every word starts at zero: the collect pass ORs the selected cubes' bits into them
             for (int wd = part; wd < g.n_words; wd += 4) {
@@ -730,11 +729,11 @@ __global__ void __launch_bounds__(128) select_all_kernel(Geom g, uint32_t* __res
                                                          int32_t* __restrict__ sel_count) {
     const int tile = blockIdx.x + g.tile_begin, h = blockIdx.y, b = blockIdx.z, r = threadIdx.x;
     const int pos = tile * kTileRows + r;
-    const bool live = pos < g.S;
+    const bool live = slot_live(g, pos);
     const int n = live ? n_candidates(g, pos) : 0;
     const size_t gt_cap = (size_t)(b * g.Hq + h) * g.n_tiles_cap + tile;
-    const size_t raster_row = live ? (size_t)(b * g.Hq + h) * g.S_io + (pos_to_raster(g, pos) - g.pos_begin) : 0;
-    const int n_max = n_candidates(g, min(tile * kTileRows + kTileRows, g.S) - 1);
+    const size_t raster_row = live ? (size_t)(b * g.Hq + h) * g.S_io + (pos_to_io(g, pos) - g.pos_begin) : 0;
+    const int n_max = tile_max_candidates(g, tile);
     for (int w = 0; w < g.n_words; ++w) {
         const int rem = n - w * 32;
         const uint32_t word = rem >= 32 ? 0xffffffffu : (rem > 0 ? (1u << rem) - 1u : 0u);

@@ -46,9 +46,9 @@ __global__ void __launch_bounds__(kExactWarps * 32) select_exact_kernel(
         g.div_Hq.divmod(bh, b, h);
         const int gk = h / g.G;
         const int pos = tile * kTileRows + r;
-        const bool live = pos < g.S;
+        const bool live = slot_live(g, pos);
         const int n = live ? n_candidates(g, pos) : 0;
-        const int raster = live ? pos_to_raster(g, pos) - g.pos_begin : 0;   // row of the call's tensors
+        const int raster = live ? pos_to_io(g, pos) - g.pos_begin : 0;   // row of the call's tensors
         unsigned long long bd = 0ull;                    // 0: every candidate is selected
         if (!all && n > 0) {
             // ---- scores: s[j] = scale * <q, kbar_j> in fp64

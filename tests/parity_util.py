@@ -16,7 +16,7 @@ TIE_MARGIN = 1e-6        # rows whose cumulative-probability margin is below thi
 def make_engine(wl, n_text_max=None, top_p=None, prefill_kernel=None):
     eng = binding.AdaSAttn(cube=wl.cube, n_q_heads=wl.Hq, n_kv_heads=wl.Hkv, head_dim=wl.D,
                            top_p=wl.top_p if top_p is None else top_p, top_k=getattr(wl, "top_k", 0))
-    eng.partition(wl.B, wl.T, wl.H, wl.W, wl.n_text if n_text_max is None else n_text_max)
+    eng.partition(wl.B, wl.T, wl.H, wl.W, (wl.n_text + getattr(wl, "n_prefix", 0)) if n_text_max is None else n_text_max)
     if prefill_kernel is not None:
         binding.adaspark_attn_set_prefill_kernel(eng.handle, prefill_kernel)
     return eng
@@ -38,7 +38,8 @@ def unpack_bitmap(words: torch.Tensor, n_cubes: int) -> np.ndarray:
 def run_forward(wl, *, top_p=None, prefill_kernel=None, want_selection=True):
     eng = make_engine(wl, top_p=top_p, prefill_kernel=prefill_kernel)
     q, k, v = wl.q.cuda(), wl.k.cuda(), wl.v.cuda()
-    out, bitmap, count = eng.forward(q, k, v, wl.n_text, want_selection=want_selection)
+    out, bitmap, count = eng.forward(q, k, v, wl.n_text, want_selection=want_selection,
+                                     n_prefix=getattr(wl, "n_prefix", 0))
     torch.cuda.synchronize()
     return eng, out, bitmap, count
 
@@ -102,7 +103,8 @@ def check_selection(sh, wl, rows, got_sel, res, *, label=""):
         for i in differing:
             b, h, n = (int(x) for x in rows[i])
             pos = int(pos_of[n])
-            n_cand = pos // sh.C if pos < sh.S_v else sh.N
+            P0 = sh.n_prefix
+            n_cand = 0 if pos < P0 else ((pos - P0) // sh.C if pos < P0 + sh.N * sh.C else sh.N)
             _, probs, _ = oracle.select_row(qf[b, n, h], kbar[b, h // G], n_cand, sh.scale, sh.top_p, sh.top_k)
             why = check_nucleus_legal(probs, res["sel"][i], got_sel[i], sh.top_p, sh.top_k)
             assert why is None, f"{label}: row {rows[i].tolist()} differs from the oracle illegally: {why}"

@@ -81,14 +81,23 @@ def test_partition_layout(lib, T, H, W, cube, n_text, N, C):
 
 def test_partition_rejections(lib):
     hd = binding.adaspark_attn_create(cfg())
-    for args, code in [((1, 6, 16, 16, 0), binding.ERR_UNSUPPORTED),      # frames % 4
-                       ((1, 8, 18, 16, 0), binding.ERR_UNSUPPORTED),      # rows % 4
-                       ((1, 1024, 32, 32, 0), binding.ERR_UNSUPPORTED),   # 16384 cubes > 4096
+    for args, code in [((1, 1024, 32, 32, 0), binding.ERR_UNSUPPORTED),   # 16384 cubes > 4096
+                       ((1, 1021, 30, 31, 0), binding.ERR_UNSUPPORTED),   # the same count with cut boundary cubes
                        ((0, 8, 16, 16, 0), binding.ERR_INVALID_ARG),
                        ((1, 8, 16, 16, -1), binding.ERR_INVALID_ARG)]:
         with pytest.raises(binding.AdasparkError) as e:
             binding.adaspark_attn_partition(hd, *args)
         assert e.value.status == code, args
+    binding.adaspark_attn_destroy(hd)
+
+
+def test_partition_of_a_grid_the_window_does_not_divide(lib):
+    """ceil() cubes per axis; the cache holds C slots per cube, so s_video counts slots, not tokens."""
+    hd = binding.adaspark_attn_create(cfg())
+    binding.adaspark_attn_partition(hd, 1, 6, 18, 15, 5)
+    lay = binding.adaspark_attn_get_layout(hd)
+    assert lay.n_cubes == 2 * 5 * 4 and lay.s_video == 40 * 64 > 6 * 18 * 15
+    assert lay.s_cap % 128 == 0 and lay.s_cap >= lay.s_video + 5 + 1
     binding.adaspark_attn_destroy(hd)
 
 
