@@ -13,7 +13,7 @@
 // key exponent is shared by the whole head, all scores of a row are the SAME positive factor
 // f = 2^(e_q + E_K - 34) * scale times an integer: order and distances between the scores of a row
 // are integer arithmetic.  Rows whose exponents are so large that the fixed-point error could reach
-// the margin (e_q + E_K > kMaxExponentSum) are not decided here: they go to the fp64 kernel of
+// the margin (f > kMaxScorePerUnit) are not decided here: they go to the fp64 kernel of
 // select_exact.cuh through a list in the workspace, and so does any row this kernel gives up on.
 //
 // Selection (query row = TMEM lane).  The scores of a
@@ -61,7 +61,10 @@ constexpr int kScoreTcCols = 64;         // cubes per column tile
 constexpr int kDigitRowBytes = 128;      // bytes per row of a digit plane
 constexpr int kCandCap = 24;             // cubes a row may collect from its boundary interval
 constexpr int kMaxHistPasses = 10;       // histogram passes a row may take before it is handed to the fp64 kernel
-constexpr int kMaxExponentSum = 6;       // largest e_q + E_K this kernel decides itself
+// Largest score per unit of V (f) this kernel decides itself: 2^(6 - 34) / sqrt(64), i.e. exponents up to
+// e_q + E_K = 6 at the default scale of head_dim 64 (the fixed-point error grows with f; the benchmark
+// inputs reach e_q + E_K = 5 at head_dim 128)
+constexpr double kMaxScorePerUnit = 0.125 / 268435456.0;
 // Per-thread registers after setmaxnreg.  The re-allocation only moves registers inside the CTA's launch
 // allocation (768 threads x 80): 4 * 88 + 88 + 40 = 6 * 80.  (A sum above it would block forever.)
 constexpr int kSelRegs = 88, kSlicerRegs = 88, kIssueRegs = 40;
@@ -501,7 +504,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
                 unsigned long long lo = 0ull, span = kOpen, base = 0ull, target = 0ull;
                 int state = n > 0 ? kHist : kDone;
                 bool first_level = true;
-                if (n > 0 && e_sum > kMaxExponentSum) { state = kDone; give_up = true; }
+                if (n > 0 && !(f <= kMaxScorePerUnit)) { state = kDone; give_up = true; }   // also a non-finite f
                 int hist_passes = 0;
                 // ---------------- passes
                 int fpass = 0;

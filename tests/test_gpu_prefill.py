@@ -5,7 +5,7 @@ import pytest
 import torch
 
 import oracle
-from paper_2604_08077_b200 import inputs
+from paper_2604_08077_b200 import binding, inputs
 
 import parity_util as pu
 
@@ -149,3 +149,35 @@ def test_two_handles_on_two_streams_do_not_interfere():
     for xa, xb in outs:
         assert torch.equal(xa, oa) and torch.equal(xb, ob)
     assert ea.header().status == 0 and eb.header().status == 0
+
+
+@pytest.mark.parametrize("scale_q,scale_k", [(16.0, 1.0), (4.0, 8.0), (1.0 / 64, 1.0 / 32)])
+def test_inputs_far_from_unit_scale(scale_q, scale_k):
+    """Queries and keys scaled by powers of two far from the N(0,1) scale of the benchmark inputs.  The
+    tensor-core selection kernel works in fixed point relative to the largest exponents of a query row and
+    of a head's mean keys; rows whose exponents leave the range it was validated for are handed to the fp64
+    kernel (header counter fallback_rows), so the selection stays exact at any scale.  The logit scale is
+    set so that the softmax stays comparable."""
+    import dataclasses
+    base = inputs.small_prefill(seed=33, T=16, H=8, W=8, n_text=19)
+    wl = dataclasses.replace(base, q=(base.q.float() * scale_q).to(torch.bfloat16),
+                             k=(base.k.float() * scale_k).to(torch.bfloat16))
+    softmax_scale = 1.0 / (np.sqrt(wl.D) * scale_q * scale_k)
+    eng = binding.AdaSAttn(cube=wl.cube, n_q_heads=wl.Hq, n_kv_heads=wl.Hkv, head_dim=wl.D, top_p=wl.top_p,
+                           softmax_scale=softmax_scale)
+    eng.partition(wl.B, wl.T, wl.H, wl.W, wl.n_text)
+    out, bitmap, count = eng.forward(wl.q.cuda(), wl.k.cuda(), wl.v.cuda(), wl.n_text, want_selection=True)
+    torch.cuda.synchronize()
+    hdr = eng.header()
+    assert hdr.status == 0
+    sh = oracle.make_shape(B=wl.B, T=wl.T, H=wl.H, W=wl.W, cube=wl.cube, n_text=wl.n_text, Hq=wl.Hq, Hkv=wl.Hkv,
+                           D=wl.D, top_p=float(np.float32(wl.top_p)), scale=float(np.float32(softmax_scale)))
+    rows = oracle.all_rows(sh)
+    res = oracle.rows(sh, wl.q, wl.k, wl.v, rows)
+    got_sel = pu.unpack_bitmap(bitmap, sh.N).reshape(-1, sh.N)
+    same, rep = pu.check_selection(sh, wl, rows, got_sel, res, label=f"scale {scale_q} x {scale_k}")
+    got = out.float().cpu().numpy().transpose(0, 2, 1, 3).reshape(-1, wl.D)
+    assert np.abs(got[same] - res["out"][same]).max() <= pu.MAX_ABS_TOL
+    if scale_q * scale_k >= 16:
+        assert hdr.fallback_rows > 0, "rows with large exponents should have gone to the fp64 kernel"
+    print(scale_q, scale_k, rep, "fallback rows", hdr.fallback_rows)
