@@ -151,18 +151,20 @@ def test_two_handles_on_two_streams_do_not_interfere():
     assert ea.header().status == 0 and eb.header().status == 0
 
 
-@pytest.mark.parametrize("scale_q,scale_k", [(16.0, 1.0), (4.0, 8.0), (1.0 / 64, 1.0 / 32)])
-def test_inputs_far_from_unit_scale(scale_q, scale_k):
+@pytest.mark.parametrize("scale_q,scale_k,compensate", [(16.0, 1.0, True), (1.0 / 64, 1.0 / 32, True),
+                                                        (4.0, 4.0, False), (2.0, 16.0, False)])
+def test_inputs_far_from_unit_scale(scale_q, scale_k, compensate):
     """Queries and keys scaled by powers of two far from the N(0,1) scale of the benchmark inputs.  The
     tensor-core selection kernel works in fixed point relative to the largest exponents of a query row and
-    of a head's mean keys; rows whose exponents leave the range it was validated for are handed to the fp64
-    kernel (header counter fallback_rows), so the selection stays exact at any scale.  The logit scale is
-    set so that the softmax stays comparable."""
+    of a head's mean keys, so a common factor that the logit scale compensates changes nothing; without
+    the compensation the logits grow, the fixed-point error in logit units grows with them, and the rows
+    leave the range the kernel was validated for: they are handed to the fp64 kernel (header counter
+    fallback_rows), so the selection stays exact."""
     import dataclasses
     base = inputs.small_prefill(seed=33, T=16, H=8, W=8, n_text=19)
     wl = dataclasses.replace(base, q=(base.q.float() * scale_q).to(torch.bfloat16),
                              k=(base.k.float() * scale_k).to(torch.bfloat16))
-    softmax_scale = 1.0 / (np.sqrt(wl.D) * scale_q * scale_k)
+    softmax_scale = 1.0 / (np.sqrt(wl.D) * (scale_q * scale_k if compensate else 1.0))
     eng = binding.AdaSAttn(cube=wl.cube, n_q_heads=wl.Hq, n_kv_heads=wl.Hkv, head_dim=wl.D, top_p=wl.top_p,
                            softmax_scale=softmax_scale)
     eng.partition(wl.B, wl.T, wl.H, wl.W, wl.n_text)
@@ -178,6 +180,8 @@ def test_inputs_far_from_unit_scale(scale_q, scale_k):
     same, rep = pu.check_selection(sh, wl, rows, got_sel, res, label=f"scale {scale_q} x {scale_k}")
     got = out.float().cpu().numpy().transpose(0, 2, 1, 3).reshape(-1, wl.D)
     assert np.abs(got[same] - res["out"][same]).max() <= pu.MAX_ABS_TOL
-    if scale_q * scale_k >= 16:
-        assert hdr.fallback_rows > 0, "rows with large exponents should have gone to the fp64 kernel"
-    print(scale_q, scale_k, rep, "fallback rows", hdr.fallback_rows)
+    if compensate:
+        assert hdr.fallback_rows == 0
+    else:
+        assert hdr.fallback_rows > 0, "rows with large logits should have gone to the fp64 kernel"
+    print(scale_q, scale_k, compensate, rep, "fallback rows", hdr.fallback_rows)
