@@ -350,52 +350,45 @@ def main():
     peak_tflops = peaks["bf16_tflops"]
 
     # ------------------------------------------------------------------ end to end (host buffers)
-    # Every step copies its q, k, v from pinned host memory and copies its output back.  The copies
-    # run on their own streams with two device buffer sets, so the upload of step i+1 and the download
-    # of step i-1 overlap the kernels of step i (the library takes the caller's stream; its own side
-    # stream is joined inside every call).  Time = first upload to last download, per step.
-    bufs = [(q, k, v, out), tuple(torch.empty_like(t) for t in (q, k, v, out))]
-    s_in, s_comp, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
+    # Every step goes through adaspark_attn_forward_host: the library copies q, k, v from pinned host
+    # memory, runs the prefill and copies the output back, all on the stream it is given.  Three streams with
+    # a device buffer set, caches and a workspace each take turns, so that the upload, the kernels and the
+    # download of neighbouring steps overlap (a handle's buffers belong to one step at a time).
+    # Time = first upload to last download, per step.
+    lanes = [(eng, (q, k, v, out), torch.cuda.Stream(), out_h)]
+    for _ in range(2):                                        # three lanes: upload, kernels and download of different steps overlap
+        e_x = binding.AdaSAttn(cube=wl.cube, n_q_heads=wl.Hq, n_kv_heads=wl.Hkv, head_dim=wl.D,
+                               top_p=wl.top_p, device=local_rank)
+        e_x.partition(wl.B, wl.T, wl.H, wl.W, wl.n_text)
+        if args.prefill_kernel is not None:
+            binding.adaspark_attn_set_prefill_kernel(e_x.handle, args.prefill_kernel)
+        lanes.append((e_x, tuple(torch.empty_like(t) for t in (q, k, v, out)), torch.cuda.Stream(),
+                      torch.empty_like(out_h).pin_memory()))
 
     def e2e_pipelined(n_steps):
-        uploaded = [torch.cuda.Event() for _ in range(n_steps)]
-        computed = [torch.cuda.Event() for _ in range(n_steps)]
-        downloaded = [torch.cuda.Event() for _ in range(n_steps)]
         t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
         barrier()
         t0.record()
-        for s_ in (s_in, s_comp, s_out):
+        for _, _, s_, _ in lanes:
             s_.wait_event(t0)
         for i in range(n_steps):
-            qb, kb, vb, ob = bufs[i % 2]
-            with torch.cuda.stream(s_in):
-                if i >= 2:
-                    s_in.wait_event(computed[i - 2])          # the kernels of step i-2 have read this buffer set
-                qb.copy_(q_h, non_blocking=True)
-                kb.copy_(k_h, non_blocking=True)
-                vb.copy_(v_h, non_blocking=True)
-                uploaded[i].record(s_in)
-            with torch.cuda.stream(s_comp):
-                s_comp.wait_event(uploaded[i])
-                if i >= 2:
-                    s_comp.wait_event(downloaded[i - 2])      # the output buffer of step i-2 has been read back
-                eng.forward(qb, kb, vb, wl.n_text, out=ob)
-                computed[i].record(s_comp)
-            with torch.cuda.stream(s_out):
-                s_out.wait_event(computed[i])
-                out_h.copy_(ob, non_blocking=True)
-                downloaded[i].record(s_out)
-        torch.cuda.current_stream().wait_event(downloaded[-1])
+            e_, staging, s_, oh = lanes[i % len(lanes)]
+            e_.forward_host(q_h, k_h, v_h, wl.n_text, oh, staging, stream=s_)
+        for _, _, s_, _ in lanes:
+            torch.cuda.current_stream().wait_stream(s_)
         t1.record()
         torch.cuda.synchronize()
         barrier()
         return t0.elapsed_time(t1) / n_steps
 
-    e2e_pipelined(3)                                          # warm-up
-    e2e_ms = e2e_pipelined(max(6, args.steps))
+    e2e_pipelined(6)                                          # warm-up
+    e2e_ms = e2e_pipelined(max(9, args.steps))
     e2e_value = job_throughput(tokens, world, max_over_ranks(e2e_ms, dist, "cuda"))
-    del bufs
+    assert torch.equal(lanes[1][3], out_h) and torch.equal(lanes[2][3], out_h), "the end-to-end lanes disagree"
+    for e_x, _, _, _ in lanes[1:]:
+        e_x.close()
+    del lanes
     h2d = q_h.numel() * 2 + k_h.numel() * 2 + v_h.numel() * 2
     d2h = out_h.numel() * 2
 

@@ -161,6 +161,23 @@ adaspark_status_t adaspark_attn_forward_prefix(adaspark_attn_t *handle, const vo
                                                int32_t *sel_count, void *workspace,
                                                size_t workspace_bytes, void *cuda_stream);
 
+/* adaspark_attn_forward with HOST input and output buffers: the call copies q, k, v from host memory
+ * into the caller's device buffers, runs the prefill there and copies `out` back, all enqueued on
+ * `cuda_stream` (no host synchronisation: the output is in out_host once the stream has reached
+ * this point; use pinned host memory for the copies to be asynchronous).
+ *   q_host, k_host, v_host  in : host bf16 [B, S, H*, D] as in adaspark_attn_forward (q_host and
+ *                                out_host may both be NULL: caches only).
+ *   out_host                out: host bf16 [B, S, Hq, D].
+ *   q_dev, k_dev, v_dev, out_dev  caller-owned DEVICE staging buffers of the same shapes (the
+ *                                library allocates nothing); their contents are overwritten.
+ * Everything else as adaspark_attn_forward. */
+adaspark_status_t adaspark_attn_forward_host(adaspark_attn_t *handle, const void *q_host,
+                                             const void *k_host, const void *v_host, int32_t n_text,
+                                             void *out_host, void *q_dev, void *k_dev, void *v_dev,
+                                             void *out_dev, void *k_cube, void *v_cube,
+                                             float *cube_keys, void *workspace,
+                                             size_t workspace_bytes, void *cuda_stream);
+
 /* Chunked prefill: the same computation as adaspark_attn_forward, fed one run of frames at a time
  * (the long-video setting of the paper: a later frame never changes an earlier row, because a video
  * query of Eq. 1 only sees the cubes that precede its own and the text comes after the video).

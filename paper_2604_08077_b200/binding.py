@@ -43,7 +43,7 @@ class AdasparkError(RuntimeError):
 _lib: Optional[ctypes.CDLL] = None
 
 EXPORTS = ["adaspark_attn_create", "adaspark_attn_partition", "adaspark_attn_get_layout",
-           "adaspark_attn_forward", "adaspark_attn_forward_prefix", "adaspark_attn_forward_chunk", "adaspark_attn_decode", "adaspark_attn_destroy",
+           "adaspark_attn_forward", "adaspark_attn_forward_host", "adaspark_attn_forward_prefix", "adaspark_attn_forward_chunk", "adaspark_attn_decode", "adaspark_attn_destroy",
            "adaspark_attn_last_error", "adaspark_attn_last_launch_count",
            "adaspark_attn_set_prefill_kernel", "adaspark_attn_enable_stage_timing",
            "adaspark_attn_get_stage_times", "adaspark_attn_decode_static",
@@ -65,6 +65,7 @@ def load() -> ctypes.CDLL:
     lib.adaspark_attn_partition.argtypes = [vp, i32, i32, i32, i32, i32, ctypes.POINTER(sz)]
     lib.adaspark_attn_get_layout.argtypes = [vp, ctypes.POINTER(Layout)]
     lib.adaspark_attn_forward.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.adaspark_attn_forward_host.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.adaspark_attn_forward_prefix.argtypes = [vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.adaspark_attn_forward_chunk.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.adaspark_attn_decode.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -141,6 +142,15 @@ def adaspark_attn_forward(handle: int, q, k, v, n_text: int, out, k_cube, v_cube
         handle, _ptr(q), _ptr(k), _ptr(v), n_text, _ptr(out), _ptr(k_cube), _ptr(v_cube),
         _ptr(cube_keys), _ptr(sel_bitmap), _ptr(sel_count), _ptr(workspace), workspace_bytes,
         _stream_ptr(stream)))
+
+
+def adaspark_attn_forward_host(handle: int, q_host, k_host, v_host, n_text: int, out_host, q_dev, k_dev, v_dev,
+                               out_dev, k_cube, v_cube, cube_keys, workspace, workspace_bytes: int, stream=None):
+    """Prefill from and to host (pinned) tensors: the library issues the copies on the stream."""
+    _check(handle, load().adaspark_attn_forward_host(
+        handle, _ptr(q_host), _ptr(k_host), _ptr(v_host), n_text, _ptr(out_host), _ptr(q_dev), _ptr(k_dev),
+        _ptr(v_dev), _ptr(out_dev), _ptr(k_cube), _ptr(v_cube), _ptr(cube_keys), _ptr(workspace),
+        workspace_bytes, _stream_ptr(stream)))
 
 
 def adaspark_attn_forward_prefix(handle: int, q, k, v, n_prefix: int, n_text: int, out, k_cube, v_cube, cube_keys,
@@ -279,6 +289,13 @@ class AdaSAttn:
             adaspark_attn_forward(self.handle, q, k, v, n_text, out, self.k_cube, self.v_cube,
                                   self.cube_keys, bitmap, count, self.workspace, self.ws_bytes, stream)
         return out, bitmap, count
+
+    def forward_host(self, q_host, k_host, v_host, n_text, out_host, staging, stream=None):
+        """Prefill with host tensors; `staging` = (q, k, v, out) device tensors of the same shapes."""
+        qd, kd, vd, od = staging
+        adaspark_attn_forward_host(self.handle, q_host, k_host, v_host, n_text, out_host, qd, kd, vd, od,
+                                   self.k_cube, self.v_cube, self.cube_keys, self.workspace, self.ws_bytes, stream)
+        return out_host
 
     def forward_chunk(self, q, k, v, frame_begin, frame_count, n_text, *, out=None, want_selection=False,
                       stream=None):

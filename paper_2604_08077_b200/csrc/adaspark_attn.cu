@@ -457,6 +457,36 @@ adaspark_status_t adaspark_attn_forward(adaspark_attn_t* h, const void* q, const
                         sel_count, workspace, workspace_bytes, cuda_stream);
 }
 
+adaspark_status_t adaspark_attn_forward_host(adaspark_attn_t* h, const void* q_host, const void* k_host, const void* v_host,
+                                             int32_t n_text, void* out_host, void* q_dev, void* k_dev, void* v_dev,
+                                             void* out_dev, void* k_cube, void* v_cube, float* cube_keys, void* workspace,
+                                             size_t workspace_bytes, void* cuda_stream) {
+    if (!h) return ADASPARK_ERR_INVALID_ARG;
+    if (!h->partitioned) return fail(h, ADASPARK_ERR_NOT_PARTITIONED, "forward_host: call adaspark_attn_partition first");
+    if (!k_host || !v_host || !k_dev || !v_dev) return fail(h, ADASPARK_ERR_INVALID_ARG, "forward_host: NULL k/v buffer");
+    if ((q_host == nullptr) != (out_host == nullptr) || (q_host != nullptr && (!q_dev || !out_dev)))
+        return fail(h, ADASPARK_ERR_INVALID_ARG, "forward_host: q/out host and device buffers must be given together");
+    if (n_text < 0 || n_text > h->n_text_max) return fail(h, ADASPARK_ERR_INVALID_ARG, "forward_host: n_text %d outside [0, %d]", n_text, h->n_text_max);
+    cudaError_t ce = cudaSetDevice(h->cfg.device);
+    if (ce != cudaSuccess) return fail(h, ADASPARK_ERR_CUDA, "forward_host: cudaSetDevice(%d): %s", h->cfg.device, cudaGetErrorString(ce));
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const size_t S = (size_t)h->T * h->H * h->W + n_text, D = h->cfg.head_dim;
+    const size_t q_bytes = (size_t)h->B * S * h->cfg.n_q_heads * D * 2, kv_bytes = (size_t)h->B * S * h->cfg.n_kv_heads * D * 2;
+    if (q_host) ce = cudaMemcpyAsync(q_dev, q_host, q_bytes, cudaMemcpyHostToDevice, st);
+    if (ce == cudaSuccess) ce = cudaMemcpyAsync(k_dev, k_host, kv_bytes, cudaMemcpyHostToDevice, st);
+    if (ce == cudaSuccess) ce = cudaMemcpyAsync(v_dev, v_host, kv_bytes, cudaMemcpyHostToDevice, st);
+    if (ce != cudaSuccess) return fail(h, ADASPARK_ERR_CUDA, "forward_host: host-to-device copy: %s", cudaGetErrorString(ce));
+    adaspark_status_t rc = forward_impl(h, "forward_host", q_host ? q_dev : nullptr, k_dev, v_dev, 0, h->T, n_text, 0,
+                                        q_host ? out_dev : nullptr, k_cube, v_cube, cube_keys, nullptr, nullptr, workspace,
+                                        workspace_bytes, cuda_stream);
+    if (rc != ADASPARK_OK) return rc;
+    if (q_host) {
+        ce = cudaMemcpyAsync(out_host, out_dev, q_bytes, cudaMemcpyDeviceToHost, st);
+        if (ce != cudaSuccess) return fail(h, ADASPARK_ERR_CUDA, "forward_host: device-to-host copy: %s", cudaGetErrorString(ce));
+    }
+    return ADASPARK_OK;
+}
+
 adaspark_status_t adaspark_attn_forward_prefix(adaspark_attn_t* h, const void* q, const void* k, const void* v,
                                                int32_t n_prefix, int32_t n_text, void* out, void* k_cube, void* v_cube,
                                                float* cube_keys, uint32_t* sel_bitmap, int32_t* sel_count,

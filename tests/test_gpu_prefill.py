@@ -185,3 +185,18 @@ def test_inputs_far_from_unit_scale(scale_q, scale_k, compensate):
     else:
         assert hdr.fallback_rows > 0, "rows with large logits should have gone to the fp64 kernel"
     print(scale_q, scale_k, compensate, rep, "fallback rows", hdr.fallback_rows)
+
+
+def test_forward_from_host_buffers_equals_forward():
+    """adaspark_attn_forward_host copies q, k, v from pinned host memory, runs the prefill and copies the
+    output back on the caller's stream: same bytes as the device-buffer call."""
+    wl = inputs.small_prefill(seed=34, T=16, H=8, W=8, n_text=27)
+    eng, out_ref, _, _ = pu.run_forward(wl, want_selection=False)
+    q_h, k_h, v_h = wl.q.pin_memory(), wl.k.pin_memory(), wl.v.pin_memory()
+    out_h = torch.empty_like(q_h).pin_memory()
+    staging = tuple(torch.empty_like(t, device="cuda") for t in (wl.q, wl.k, wl.v, wl.q))
+    s = torch.cuda.Stream()
+    eng.forward_host(q_h, k_h, v_h, wl.n_text, out_h, staging, stream=s)
+    s.synchronize()
+    assert torch.equal(out_h, out_ref.cpu())
+    assert eng.header().status == 0
