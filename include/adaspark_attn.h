@@ -86,14 +86,20 @@ typedef struct {
     int32_t status;               /* 0 = ok; 1 = text_len out of range (decode); 6 = a bounded
                                      device wait expired (ADASPARK_ERR_TIMEOUT)               */
     int32_t reserved;
-    uint64_t executed_kv_blocks;  /* prefill: (query tile, 64-key block) pairs the attention
-                                     kernel computed; executed FLOPs = this * 128*64*D*4    */
+    uint64_t executed_kv_blocks;  /* prefill: (128 query rows, 64-key block) products the attention
+                                     kernels computed (union path: per tile and visited block;
+                                     gather path: per item); executed FLOPs = this * 128*64*D*4 */
     uint64_t decode_kv_blocks;    /* decode: 64-key blocks gathered, summed over (b, kv head) */
     uint32_t fallback_rows;       /* prefill: query rows whose selection the tensor-core kernel
                                      left to the fp64 selection kernel (normally 0)           */
     uint32_t max_tile_kv_blocks;  /* prefill: largest number of 64-key blocks one 256-row pair of
                                      query tiles visited (load imbalance: compare with the mean
                                      executed_kv_blocks / 2 / number of pair tiles)           */
+    uint32_t gather_entries;      /* prefill: (query row, 64-key block) entries computed by the
+                                     query-gather path (0: every pair took the union path)     */
+    uint32_t gather_items;        /* ... in this many items of up to 128 gathered rows          */
+    uint32_t gather_pair_tiles;   /* ... for this many 256-row pairs of query tiles             */
+    uint32_t reserved2;
 } adaspark_attn_workspace_header_t;
 
 /* Create a handle for one configuration.  Host only.  Fails with ERR_UNSUPPORTED for a
@@ -112,9 +118,8 @@ adaspark_status_t adaspark_attn_create(const adaspark_attn_config_t *config,
  * the mean over the tokens they hold, their other slots stay empty in the caches and are never attended.
  * ERR_UNSUPPORTED if N > 4096 or the cache would hold more than 2097152 rows per sequence
  * (s_video + n_text_max + 1).
- * The forward workspace holds two buffers of fp64 cube scores for a chunk of query tiles each
- * (512 MB each by default, less when the whole problem is smaller); the environment variable
- * ADASPARK_SCORE_BUFFER_MB, read here, overrides the size of one buffer (1 .. 65536). */
+ * The forward workspace holds the selection masks, the cube-major copy of Q and the digit planes of the
+ * mean keys; cube scores are never stored. */
 adaspark_status_t adaspark_attn_partition(adaspark_attn_t *handle, int32_t batch, int32_t frames,
                                           int32_t grid_h, int32_t grid_w, int32_t n_text_max,
                                           size_t *workspace_bytes);
@@ -285,6 +290,23 @@ adaspark_status_t adaspark_attn_get_stage_times(adaspark_attn_t *handle, float *
  * scoring from error-free digit slices (default when built in); 2 = tcgen05 attention + fp64
  * scoring.  ERR_UNSUPPORTED for an unknown value. */
 adaspark_status_t adaspark_attn_set_prefill_kernel(adaspark_attn_t *handle, int32_t which);
+
+/* Query-gather path of the prefill (kernels 1 only; Eq. 3 over the selected cubes alone).  The attention
+ * kernel visits, per pair of 128-row query tiles, the union of the key blocks its 256 rows selected; when
+ * the rows pick different cubes that union is nearly every block.  For such pairs the library instead
+ * gathers, per 64-key block, the query rows (of all tiles and all heads of the GQA group) that selected a
+ * cube in it, computes their attention over that block on the tensor cores, and merges each row's partial
+ * results with the result of its local range (own cube, text) by the softmax identity.  The choice is made
+ * on the device, per pair: gathered iff (row, key block) entries of the pair's rows <= pairs_per_block *
+ * key blocks in the pair's union.  pairs_per_block = 0 switches the path off (every pair takes the union
+ * path); a huge value forces it for every pair with a selected cube.  budget_bytes bounds the workspace
+ * the path may use for its partial results (2*head_dim + 24 bytes per entry, at most 32 entries per query
+ * row); if the pairs that qualify need more, all pairs take the union path in that call.  The budget
+ * sizes the forward workspace: set it before _partition (ERR_INVALID_ARG afterwards); the threshold may
+ * change at any time.  Defaults: 20 entries per block, 8 GiB.  Outputs agree with the union path within
+ * bf16 rounding of the partial results; the selection is the same. */
+adaspark_status_t adaspark_attn_set_gather(adaspark_attn_t *handle, float pairs_per_block,
+                                           uint64_t budget_bytes);
 
 #ifdef __cplusplus
 }

@@ -45,7 +45,7 @@ _lib: Optional[ctypes.CDLL] = None
 EXPORTS = ["adaspark_attn_create", "adaspark_attn_partition", "adaspark_attn_get_layout",
            "adaspark_attn_forward", "adaspark_attn_forward_host", "adaspark_attn_forward_prefix", "adaspark_attn_forward_chunk", "adaspark_attn_decode", "adaspark_attn_destroy",
            "adaspark_attn_last_error", "adaspark_attn_last_launch_count",
-           "adaspark_attn_set_prefill_kernel", "adaspark_attn_enable_stage_timing",
+           "adaspark_attn_set_prefill_kernel", "adaspark_attn_set_gather", "adaspark_attn_enable_stage_timing",
            "adaspark_attn_get_stage_times", "adaspark_attn_decode_static",
            "adaspark_attn_debug_umma_selftest", "adaspark_attn_debug_imma_selftest",
            "adaspark_attn_debug_fastdiv", "adaspark_attn_debug_wait_timeout"]
@@ -81,6 +81,7 @@ def load() -> ctypes.CDLL:
     lib.adaspark_attn_last_launch_count.argtypes = [vp]
     lib.adaspark_attn_last_launch_count.restype = ctypes.c_int64
     lib.adaspark_attn_set_prefill_kernel.argtypes = [vp, i32]
+    lib.adaspark_attn_set_gather.argtypes = [vp, ctypes.c_float, ctypes.c_uint64]
     lib.adaspark_attn_enable_stage_timing.argtypes = [vp, i32]
     lib.adaspark_attn_get_stage_times.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     for name in EXPORTS:
@@ -226,6 +227,10 @@ def adaspark_attn_set_prefill_kernel(handle: int, which: int):
     _check(handle, load().adaspark_attn_set_prefill_kernel(handle, which))
 
 
+def adaspark_attn_set_gather(handle: int, pairs_per_block: float, budget_bytes: int):
+    _check(handle, load().adaspark_attn_set_gather(handle, float(pairs_per_block), int(budget_bytes)))
+
+
 def adaspark_attn_enable_stage_timing(handle: int, enable: bool):
     _check(handle, load().adaspark_attn_enable_stage_timing(handle, int(enable)))
 
@@ -240,7 +245,9 @@ def adaspark_attn_get_stage_times(handle: int):
 class WorkspaceHeader(ctypes.Structure):
     _fields_ = [("status", ctypes.c_int32), ("reserved", ctypes.c_int32),
                 ("executed_kv_blocks", ctypes.c_uint64), ("decode_kv_blocks", ctypes.c_uint64),
-                ("fallback_rows", ctypes.c_uint32), ("max_tile_kv_blocks", ctypes.c_uint32)]
+                ("fallback_rows", ctypes.c_uint32), ("max_tile_kv_blocks", ctypes.c_uint32),
+                ("gather_entries", ctypes.c_uint32), ("gather_items", ctypes.c_uint32),
+                ("gather_pair_tiles", ctypes.c_uint32), ("reserved2", ctypes.c_uint32)]
 
 
 # ---- a small convenience owner of the handle and of the caller-side buffers --------------------
@@ -255,6 +262,10 @@ class AdaSAttn:
         self.handle = adaspark_attn_create(self.cfg)
         self.device = torch.device("cuda", device)
         self.layout: Optional[Layout] = None
+
+    def set_gather(self, pairs_per_block: float, budget_bytes: int = 8 << 30):
+        """Threshold and workspace budget of the query-gather path (budget: before partition())."""
+        adaspark_attn_set_gather(self.handle, pairs_per_block, budget_bytes)
 
     def partition(self, batch, frames, grid_h, grid_w, n_text_max):
         self.ws_bytes = adaspark_attn_partition(self.handle, batch, frames, grid_h, grid_w, n_text_max)

@@ -20,6 +20,7 @@
 #ifdef ADASPARK_WITH_TCGEN05
 #include "attn_prefill_tc.cuh"
 #include "score_select_fused.cuh"
+#include "attn_gather.cuh"
 #endif
 
 using namespace adaspark;
@@ -31,8 +32,13 @@ struct adaspark_attn {
     int C, N, S_v, S_cap;
     adaspark_attn_layout_t layout;
     // workspace carving (byte offsets)
-    size_t fw_status_off, fw_headmax_off, fw_valid_off, fw_mask_off, fw_union_off, fw_fallback_off, fw_scratch_off, fw_qcube_off,
-        fw_kplanes_off, fw_total;
+    size_t fw_status_off, fw_headmax_off, fw_valid_off, fw_gcol_off, fw_mask_off, fw_union_off, fw_fallback_off, fw_scratch_off,
+        fw_qcube_off, fw_kplanes_off, fw_gpair_off, fw_grow_off, fw_gml_off, fw_gitems_off, fw_gentries_off, fw_gparto_off,
+        fw_gpartml_off, fw_total;
+    // query-gather path of the prefill: capacity in (row, key block) entries, decision threshold, byte budget
+    uint32_t gather_cap;
+    float gather_pairs_per_block;
+    uint64_t gather_budget;
     size_t dc_status_off, dc_bitmap_off, dc_items_off, dc_nitems_off, dc_partial_off, dc_total;
     int dc_splits;
     int prefill_kernel;
@@ -48,6 +54,12 @@ namespace {
 
 constexpr size_t kAlign = 256;
 constexpr int kExactCtas = 296;   // CTAs of the fp64 selection kernel (its scratch rows are sized for them)
+// query-gather path: pairs of query tiles take it when their rows' (row, key block) entries are at most this
+// many per key block of the pair's union (measured break-even on a B200, see the attention profile), and the
+// partial results of all such pairs must fit this many bytes of workspace
+constexpr float kGatherDefaultPairsPerBlock = 20.f;
+constexpr uint64_t kGatherDefaultBudget = 8ull << 30;
+constexpr uint64_t kGatherEntriesPerRow = 32;
 size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 
 adaspark_status_t fail(adaspark_attn* h, adaspark_status_t st, const char* fmt, ...) {
@@ -157,6 +169,8 @@ adaspark_status_t adaspark_attn_create(const adaspark_attn_config_t* config, ada
     h->C = (int)C;
 #ifdef ADASPARK_WITH_TCGEN05
     h->prefill_kernel = 1;
+    h->gather_pairs_per_block = kGatherDefaultPairsPerBlock;
+    h->gather_budget = kGatherDefaultBudget;
 #else
     h->prefill_kernel = 0;
 #endif
@@ -202,6 +216,8 @@ adaspark_status_t adaspark_attn_partition(adaspark_attn_t* h, int32_t batch, int
     h->fw_status_off = off; off = align_up(off + 256);
     h->fw_headmax_off = off; off = align_up(off + (size_t)batch * Hkv * 4);
     h->fw_valid_off = off; off = align_up(off + (size_t)(S_cap / kBlockTok) * 2 * 4);   // which slots of a block hold a token
+    const size_t n_cols = (size_t)(S_v + kBlockTok - 1) / kBlockTok;                     // key blocks that hold video
+    h->fw_gcol_off = off; off = align_up(off + (size_t)batch * Hkv * n_cols * 2 * 4);   // entry counts and fill cursors (zeroed per call)
     h->fw_mask_off = off; off = align_up(off + (size_t)batch * Hq * n_tiles_cap * n_words * kTileRows * 4);
     h->fw_union_off = off; off = align_up(off + (size_t)batch * Hq * n_tiles_cap * n_words * 4);
     h->fw_fallback_off = off; off = align_up(off + (size_t)batch * Hq * n_tiles_cap * kTileRows * 4);
@@ -210,6 +226,23 @@ adaspark_status_t adaspark_attn_partition(adaspark_attn_t* h, int32_t batch, int
     // digit planes (4 x int8 [B*Hkv*N_ld, 128]) of the mean keys; 128 rows of slack so that the last TMA box
     // stays inside the allocation
     h->fw_kplanes_off = off; off = align_up(off + ((size_t)4 * batch * Hkv * N_ld + 128) * 128);
+    // query-gather path: per pair (mode, entries, offset) | per row (entries, first partial) | per row (m, l) of the
+    // local range | per key block offsets + work items | entries | partial outputs | partial (m, l)
+    {
+        const size_t rows_cap = (size_t)batch * Hq * S_cap, n_pairs_cap = ((size_t)S_cap + 255) / 256;
+        const uint64_t per_entry = 2ull * D + 16ull + 8ull;      // partial output + (m, l) + entry
+        uint64_t cap = h->gather_budget / per_entry;
+        if (cap > rows_cap * kGatherEntriesPerRow) cap = rows_cap * kGatherEntriesPerRow;
+        if (cap > 0xfffffff0ull) cap = 0xfffffff0ull;
+        h->gather_cap = (uint32_t)cap;
+        h->fw_gpair_off = off; off = align_up(off + (size_t)batch * Hq * n_pairs_cap * 3 * 4);
+        h->fw_grow_off = off; off = align_up(off + (cap ? rows_cap * 2 * 4 : 0));
+        h->fw_gml_off = off; off = align_up(off + (cap ? rows_cap * 8 : 0));
+        h->fw_gitems_off = off; off = align_up(off + (cap ? ((size_t)batch * Hkv * n_cols * 2 + cap / 128 + 1) * 8 : 0));
+        h->fw_gentries_off = off; off = align_up(off + (size_t)cap * 8);
+        h->fw_gparto_off = off; off = align_up(off + (size_t)cap * D * 2);
+        h->fw_gpartml_off = off; off = align_up(off + (size_t)cap * 8);
+    }
     h->fw_total = off;
     L.forward_workspace_bytes = (int64_t)off;
 
@@ -411,18 +444,79 @@ adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* 
             return fail(h, ADASPARK_ERR_CUDA, "%s: cuTensorMapEncodeTiled failed", who);
         dim3 grid(((g.S + kPairRows - 1) / kPairRows - g.pos_begin / kPairRows) * g.Hq * g.B);
         const uint32_t* slot_valid_c = (const uint32_t*)(ws + h->fw_valid_off);
+        // query-gather path for pairs of query tiles with sparse selections (off for p >= 1: nothing is skipped)
+        const bool all_sel = g.top_k <= 0 && !(g.top_p < 1.0);
+        const bool gather = h->prefill_kernel == 1 && !all_sel && h->gather_cap > 0 && h->gather_pairs_per_block > 0.f;
+        GatherWs gw;
+        std::memset(&gw, 0, sizeof(gw));
+        if (gather) {
+            const size_t n_cols = (size_t)(g.S_v + kBlockTok - 1) / kBlockTok, n_col_all = (size_t)g.B * g.Hkv * n_cols;
+            const size_t rows_cap = (size_t)g.B * g.Hq * g.S_cap, n_pairs_cap = ((size_t)g.S_cap + 255) / 256;
+            const size_t n_pair_all = (size_t)g.B * g.Hq * n_pairs_cap;
+            gw.ctrl = &hdr->gather_entries;
+            gw.pair_mode = (uint32_t*)(ws + h->fw_gpair_off);
+            gw.pair_cnt = gw.pair_mode + n_pair_all;
+            gw.pair_off = gw.pair_cnt + n_pair_all;
+            gw.row_cnt = (uint32_t*)(ws + h->fw_grow_off);
+            gw.row_ptr = gw.row_cnt + rows_cap;
+            gw.col_cnt = (uint32_t*)(ws + h->fw_gcol_off);
+            gw.col_cur = gw.col_cnt + n_col_all;
+            gw.col_off = (uint32_t*)(ws + h->fw_gitems_off);
+            gw.items = (uint2*)(ws + h->fw_gitems_off + n_col_all * 8);
+            gw.entries = (uint2*)(ws + h->fw_gentries_off);
+            gw.part_o = (__nv_bfloat16*)(ws + h->fw_gparto_off);
+            gw.part_ml = (float2*)(ws + h->fw_gpartml_off);
+            gw.ml_local = (float2*)(ws + h->fw_gml_off);
+            gw.cap_entries = h->gather_cap;
+            gw.n_cols = (int)n_cols;
+            gw.n_pairs_cap = (int)n_pairs_cap;
+            gw.pairs_per_block = h->gather_pairs_per_block;
+            gather_count_kernel<<<grid, 256, 0, st>>>(g, gw, tile_mask, tile_union);
+            if (!launch_ok(h, "gather_count_kernel")) return ADASPARK_ERR_CUDA;
+            gather_scan_kernel<<<1, 1024, 0, st>>>(g, gw);
+            if (!launch_ok(h, "gather_scan_kernel")) return ADASPARK_ERR_CUDA;
+        }
+        const uint32_t* pair_mode_c = gather ? gw.pair_mode : nullptr;
         if (D == 128) {
             size_t smem = sizeof(TcAttnSmem<128>) + 1024;
             if (!set_smem(h, attn_prefill_tc_kernel<128>, smem, "attn_prefill_tc_kernel")) return ADASPARK_ERR_CUDA;
-            attn_prefill_tc_kernel<128><<<grid, kTcThreads, smem, st>>>(g, tmQ, tmK, tmV, tile_mask, tile_union, slot_valid_c, (__nv_bfloat16*)out,
+            attn_prefill_tc_kernel<128><<<grid, kTcThreads, smem, st>>>(g, tmQ, tmK, tmV, tile_mask, tile_union, slot_valid_c, pair_mode_c,
+                                                                        gw.n_pairs_cap, gw.ml_local, (__nv_bfloat16*)out,
                                                                         (unsigned long long*)&hdr->executed_kv_blocks, &hdr->max_tile_kv_blocks, &hdr->status);
         } else {
             size_t smem = sizeof(TcAttnSmem<64>) + 1024;
             if (!set_smem(h, attn_prefill_tc_kernel<64>, smem, "attn_prefill_tc_kernel")) return ADASPARK_ERR_CUDA;
-            attn_prefill_tc_kernel<64><<<grid, kTcThreads, smem, st>>>(g, tmQ, tmK, tmV, tile_mask, tile_union, slot_valid_c, (__nv_bfloat16*)out,
+            attn_prefill_tc_kernel<64><<<grid, kTcThreads, smem, st>>>(g, tmQ, tmK, tmV, tile_mask, tile_union, slot_valid_c, pair_mode_c,
+                                                                       gw.n_pairs_cap, gw.ml_local, (__nv_bfloat16*)out,
                                                                        (unsigned long long*)&hdr->executed_kv_blocks, &hdr->max_tile_kv_blocks, &hdr->status);
         }
         if (!launch_ok(h, "attn_prefill_tc_kernel")) return ADASPARK_ERR_CUDA;
+        if (gather) {
+            gather_fill_kernel<<<grid, 256, 0, st>>>(g, gw, tile_mask);
+            if (!launch_ok(h, "gather_fill_kernel")) return ADASPARK_ERR_CUDA;
+            CUtensorMap tmKg;      // one key block per load: box of 64 d x 64 keys (tmK's) serves as it is
+            tmKg = tmK;
+            const int ggrid = 2 * h->sm_count;
+            const long long n_rows = (long long)g.B * g.Hq * (g.S - g.pos_begin);
+            if (D == 128) {
+                const size_t smem = sizeof(GatherSmem<128>) + 1024;
+                if (!set_smem(h, attn_gather_kernel<128>, smem, "attn_gather_kernel")) return ADASPARK_ERR_CUDA;
+                attn_gather_kernel<128><<<ggrid, kGatherThreads, smem, st>>>(g, gw, tmKg, tmV, q_cube, slot_valid_c,
+                                                                            (unsigned long long*)&hdr->executed_kv_blocks, &hdr->status);
+                if (!launch_ok(h, "attn_gather_kernel")) return ADASPARK_ERR_CUDA;
+                const long long ctas = (n_rows + 15) / 16;
+                gather_merge_kernel<128><<<(unsigned)(ctas < 8ll * h->sm_count ? ctas : 8ll * h->sm_count), 256, 0, st>>>(g, gw, (__nv_bfloat16*)out);
+            } else {
+                const size_t smem = sizeof(GatherSmem<64>) + 1024;
+                if (!set_smem(h, attn_gather_kernel<64>, smem, "attn_gather_kernel")) return ADASPARK_ERR_CUDA;
+                attn_gather_kernel<64><<<ggrid, kGatherThreads, smem, st>>>(g, gw, tmKg, tmV, q_cube, slot_valid_c,
+                                                                           (unsigned long long*)&hdr->executed_kv_blocks, &hdr->status);
+                if (!launch_ok(h, "attn_gather_kernel")) return ADASPARK_ERR_CUDA;
+                const long long ctas = (n_rows + 31) / 32;
+                gather_merge_kernel<64><<<(unsigned)(ctas < 8ll * h->sm_count ? ctas : 8ll * h->sm_count), 256, 0, st>>>(g, gw, (__nv_bfloat16*)out);
+            }
+            if (!launch_ok(h, "gather_merge_kernel")) return ADASPARK_ERR_CUDA;
+        }
     } else
 #endif
     {
@@ -617,6 +711,16 @@ adaspark_status_t adaspark_attn_set_prefill_kernel(adaspark_attn_t* h, int32_t w
     if (which != 0) return fail(h, ADASPARK_ERR_UNSUPPORTED, "set_prefill_kernel: kernel %d not built", which);
 #endif
     h->prefill_kernel = which;
+    return ADASPARK_OK;
+}
+
+adaspark_status_t adaspark_attn_set_gather(adaspark_attn_t* h, float pairs_per_block, uint64_t budget_bytes) {
+    if (!h) return ADASPARK_ERR_INVALID_ARG;
+    if (!(pairs_per_block >= 0.f)) return fail(h, ADASPARK_ERR_INVALID_ARG, "set_gather: threshold %g is not >= 0", (double)pairs_per_block);
+    if (h->partitioned && budget_bytes != h->gather_budget)
+        return fail(h, ADASPARK_ERR_INVALID_ARG, "set_gather: the byte budget sizes the workspace; set it before adaspark_attn_partition");
+    h->gather_pairs_per_block = pairs_per_block;
+    h->gather_budget = budget_bytes;
     return ADASPARK_OK;
 }
 

@@ -61,7 +61,8 @@ template <int D>
 __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     Geom g, const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
     const __grid_constant__ CUtensorMap tmV, const uint32_t* __restrict__ tile_mask,
-    const uint32_t* __restrict__ tile_union, const uint32_t* __restrict__ slot_valid, __nv_bfloat16* __restrict__ out,
+    const uint32_t* __restrict__ tile_union, const uint32_t* __restrict__ slot_valid, const uint32_t* __restrict__ pair_mode,
+    int n_pairs_cap, float2* __restrict__ ml_local, __nv_bfloat16* __restrict__ out,
     unsigned long long* __restrict__ executed_blocks, uint32_t* __restrict__ max_tile_blocks, int32_t* __restrict__ status) {
     extern __shared__ unsigned char tc_smem_raw[];
     TcAttnSmem<D>& sm = *reinterpret_cast<TcAttnSmem<D>*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -86,8 +87,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     const bool sees_prefix = g.n_prefix > 0 && pair_pos0 < g.S_v;
     const int n_blk_own = (pair_end + kBlockTok - 1) / kBlockTok;
     const int n_blk = sees_prefix ? max(n_blk_own, prefix_blk1) : n_blk_own;
-    const int local_start = pair_pos0 < g.S_v ? ((pair_pos0 >> g.c_shift) << g.c_shift) : g.S_v;
-    const int first_local_blk = local_start / kBlockTok;
+    const int first_local_blk = pair_first_local_blk(g, pair_pos0);
+    // A pair whose selected cubes go through the query-gather kernels (attn_gather.cuh) visits only its local
+    // range and the text prefix here and leaves (reference exponent, sum) of every row for the merge.
+    const bool gathered = pair_mode != nullptr && __ldg(pair_mode + (size_t)(b * g.Hq + h) * n_pairs_cap + pair) != 0u;
 
     // ---------------------------------------------------------------- set-up
     if (tid == 0) {
@@ -140,13 +143,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     for (int wi = tid; wi < n_blk_words; wi += kTcThreads) {
         uint32_t bits = 0;
         if (g.c_shift == 6 && wi * 32 + 31 < first_local_blk) {   // (first_local_blk <= prefix_blk0)
-            bits = sm.union_words[wi];             // 64-token cubes: key block = cube, the word is the union word
+            bits = gathered ? 0u : sm.union_words[wi];   // 64-token cubes: key block = cube, the word is the union word
         } else {
             for (int i = 0; i < 32; ++i) {
                 int kb = wi * 32 + i;
                 if (kb >= n_blk) break;
                 bool need = (kb >= first_local_blk && kb < n_blk_own) || (sees_prefix && kb >= prefix_blk0);
-                if (!need) {
+                if (!need && !gathered) {
                     int c_lo = (kb * kBlockTok) >> g.c_shift, c_hi = (kb * kBlockTok + kBlockTok - 1) >> g.c_shift;
                     uint32_t span = c_hi - c_lo + 1;   // <= 4 cubes, aligned: never crosses a word
                     uint32_t m = (span >= 32 ? 0xffffffffu : ((1u << span) - 1u)) << (c_lo & 31);
@@ -468,6 +471,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
             tc::tc_fence_after_sync();
             const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
             const bool live = slot_live(g, pr);
+            if (gathered && live) ml_local[(size_t)(b * g.Hq + h) * g.S_cap + pr] = make_float2(m_ref, l_sum);
             __nv_bfloat16* dst = out + ((live ? io_row(g, b, pr) : 0) * g.Hq + h) * D;
             uint32_t o[D / 32][32];                                // the whole output row in one round of loads
 #pragma unroll

@@ -115,6 +115,14 @@ __device__ __forceinline__ int tile_max_candidates(const Geom& g, int tile) {
     return m;
 }
 
+// First 64-key block of the local range of the 256-row pair of query tiles that starts at pair_pos0: the block
+// that holds the first slot of the own cube of the pair's first row (video) or the first text slot.  Cubes
+// that end before this block are attended only if selected; from this block on the per-key rule applies.
+__device__ __forceinline__ int pair_first_local_blk(const Geom& g, int pair_pos0) {
+    const int local_start = pair_pos0 < g.S_v ? ((pair_pos0 >> g.c_shift) << g.c_shift) : g.S_v;
+    return local_start / kBlockTok;
+}
+
 // Per-tile selection mask matrix: word w of row r of global tile gt at
 // mask[(gt * n_words + w) * 128 + r]; gt = (b*Hq + h) * n_tiles_cap + tile.
 __device__ __forceinline__ size_t mask_index(const Geom& g, int b, int h, int tile, int w, int r) {

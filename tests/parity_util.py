@@ -13,9 +13,16 @@ MEAN_REL_TOL = 1e-2      # mean|o - o_ref| / mean|o_ref|
 TIE_MARGIN = 1e-6        # rows whose cumulative-probability margin is below this may differ
 
 
-def make_engine(wl, n_text_max=None, top_p=None, prefill_kernel=None):
+FORCE_GATHER = 1e30   # threshold of the query-gather path that sends every pair with a selected cube through it
+
+
+def make_engine(wl, n_text_max=None, top_p=None, prefill_kernel=None, gather=None, gather_budget=8 << 30):
+    """gather: None = the library's default decision; 0 = union path only; FORCE_GATHER = gather path
+    wherever a row selected a cube before its local range."""
     eng = binding.AdaSAttn(cube=wl.cube, n_q_heads=wl.Hq, n_kv_heads=wl.Hkv, head_dim=wl.D,
                            top_p=wl.top_p if top_p is None else top_p, top_k=getattr(wl, "top_k", 0))
+    if gather is not None:
+        eng.set_gather(gather, gather_budget)
     eng.partition(wl.B, wl.T, wl.H, wl.W, (wl.n_text + getattr(wl, "n_prefix", 0)) if n_text_max is None else n_text_max)
     if prefill_kernel is not None:
         binding.adaspark_attn_set_prefill_kernel(eng.handle, prefill_kernel)
@@ -35,8 +42,8 @@ def unpack_bitmap(words: torch.Tensor, n_cubes: int) -> np.ndarray:
     return bits.reshape(*w.shape[:-1], -1)[..., :n_cubes].astype(np.uint8)
 
 
-def run_forward(wl, *, top_p=None, prefill_kernel=None, want_selection=True):
-    eng = make_engine(wl, top_p=top_p, prefill_kernel=prefill_kernel)
+def run_forward(wl, *, top_p=None, prefill_kernel=None, want_selection=True, gather=None, gather_budget=8 << 30):
+    eng = make_engine(wl, top_p=top_p, prefill_kernel=prefill_kernel, gather=gather, gather_budget=gather_budget)
     q, k, v = wl.q.cuda(), wl.k.cuda(), wl.v.cuda()
     out, bitmap, count = eng.forward(q, k, v, wl.n_text, want_selection=want_selection,
                                      n_prefix=getattr(wl, "n_prefix", 0))

@@ -1,0 +1,150 @@
+"""GPU parity of the query-gather path of the prefill (Eq. 3 over the selected cubes alone: per key block the
+rows that selected it are gathered, partial results are merged with the result of the row's local range).
+The path is forced for every pair of query tiles, then every row is compared with the CPU oracle exactly as
+for the union path; the decision rule, the capacity fallback and the agreement of the two paths are tested
+apart."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2604_08077_b200 import binding, inputs
+
+import parity_util as pu
+from test_gpu_prefill import SMALL_CASES
+from test_gpu_prefix_ragged import CASES as OPEN_CASES
+
+pytestmark = pytest.mark.gpu
+
+
+def expected_entries(wl, bitmap):
+    """(row, 64-key block) entries the path must produce when forced: for every row the key blocks before
+    the local range of its 256-row pair that hold a cube it selected.  Pure index arithmetic on the
+    selection the library reported (which the caller compares with the oracle)."""
+    sh = oracle.shape_of(wl)
+    pos_of, _ = oracle.positions(sh)                        # oracle position of every token
+    C, N, P0 = sh.C, sh.N, sh.n_prefix
+    S_v = N * C
+    sel = pu.unpack_bitmap(bitmap, N)                       # [B, Hq, S, N]
+    total = 0
+    for s in range(wl.S):
+        p = int(pos_of[s])
+        # cube-major position in the caches: video slots first, then prefix, then text
+        if P0 <= p < P0 + S_v:
+            cpos = p - P0
+        elif p < P0:
+            cpos = S_v + p
+        else:
+            cpos = p
+        pair_pos0 = cpos // 256 * 256
+        local_start = (pair_pos0 // C) * C if pair_pos0 < S_v else S_v
+        first_local_blk = local_start // 64
+        cube_lim = first_local_blk * 64 // C
+        rows = sel[:, :, s, :cube_lim]                      # [B, Hq, cube_lim]
+        if C >= 64:
+            total += int(rows.sum()) * (C // 64)
+        else:
+            per = 64 // C
+            pad = (-cube_lim) % per
+            r = np.pad(rows, ((0, 0), (0, 0), (0, pad)))
+            total += int(r.reshape(*r.shape[:2], -1, per).any(-1).sum())
+    return total
+
+
+@pytest.mark.parametrize("case", sorted(SMALL_CASES))
+def test_forced_gather_every_row(case):
+    """Every row of the small problems with all selected cubes before the local range on the gather path."""
+    wl = SMALL_CASES[case]()
+    eng, out, bitmap, count = pu.run_forward(wl, prefill_kernel=1, gather=pu.FORCE_GATHER)
+    hdr = eng.header()
+    assert hdr.status == 0
+    rep = pu.compare_rows(wl, oracle.all_rows(oracle.shape_of(wl)), out, bitmap, count, label=case)
+    assert rep["rows"] == wl.B * wl.Hq * wl.S
+    assert hdr.gather_entries == expected_entries(wl, bitmap)
+    print(case, rep, "entries", hdr.gather_entries, "items", hdr.gather_items, "pairs", hdr.gather_pair_tiles)
+
+
+@pytest.mark.parametrize("case", sorted(OPEN_CASES))
+def test_forced_gather_prefix_and_ragged(case):
+    """Text prefix (attended by the union kernel's local part) and ragged grids (empty slots masked in the
+    gathered blocks)."""
+    wl = OPEN_CASES[case]()
+    eng, out, bitmap, count = pu.run_forward(wl, prefill_kernel=1, gather=pu.FORCE_GATHER)
+    hdr = eng.header()
+    assert hdr.status == 0
+    rep = pu.compare_rows(wl, oracle.all_rows(oracle.shape_of(wl)), out, bitmap, count, label=case)
+    assert rep["rows"] == wl.B * wl.Hq * wl.S
+    assert hdr.gather_entries == expected_entries(wl, bitmap)
+    print(case, rep, "entries", hdr.gather_entries)
+
+
+def test_paths_agree_and_off_switch():
+    """Threshold 0 switches the path off (no entries); both paths select the same cubes bit for bit and their
+    outputs differ by bf16 rounding of the partial results only."""
+    wl = inputs.small_prefill(seed=31, T=24, H=8, W=8, n_text=50, Hq=4, Hkv=2, top_p=0.6, offset_std=3.0)
+    e0, out0, bm0, cnt0 = pu.run_forward(wl, prefill_kernel=1, gather=0.0)
+    e1, out1, bm1, cnt1 = pu.run_forward(wl, prefill_kernel=1, gather=pu.FORCE_GATHER)
+    assert e0.header().gather_entries == 0 and e0.header().gather_pair_tiles == 0
+    assert e1.header().gather_entries > 0
+    assert torch.equal(bm0, bm1) and torch.equal(cnt0, cnt1)
+    diff = (out0.float() - out1.float()).abs().max().item()
+    assert diff < 2e-2, diff
+    # executed work: the gather path computes one 128 x 64 product per item, the union path two per visited
+    # block of a pair; with 4-5 cubes kept per row the former must be far below the latter
+    assert e1.header().executed_kv_blocks < e0.header().executed_kv_blocks
+
+
+def test_capacity_fallback():
+    """A byte budget too small for the entries sends every pair back to the union path in that call; the
+    result is still the oracle's."""
+    wl = inputs.small_prefill(seed=32, T=16, H=8, W=8, n_text=20, top_p=0.8)
+    eng, out, bitmap, count = pu.run_forward(wl, prefill_kernel=1, gather=pu.FORCE_GATHER, gather_budget=64 * 280)
+    hdr = eng.header()
+    assert hdr.status == 0 and hdr.gather_entries == 0 and hdr.gather_pair_tiles == 0
+    rep = pu.compare_rows(wl, oracle.all_rows(oracle.shape_of(wl)), out, bitmap, count, label="capacity")
+    assert rep["rows"] == wl.B * wl.Hq * wl.S
+
+
+def test_decision_rule_per_pair():
+    """With a finite threshold only the pairs whose rows' entries are at most threshold x union blocks take the
+    path: a sharp selection (few cubes per row, different per row) qualifies, a flat one does not."""
+    sharp = inputs.small_prefill(seed=33, T=64, H=8, W=8, n_text=0, Hq=2, Hkv=1, top_p=0.3, offset_std=4.0)
+    flat = inputs.small_prefill(seed=34, T=64, H=8, W=8, n_text=0, Hq=2, Hkv=1, top_p=0.95, offset_std=0.3)
+    for wl, expect_on in ((sharp, True), (flat, False)):
+        eng, out, bitmap, count = pu.run_forward(wl, prefill_kernel=1, gather=20.0)
+        hdr = eng.header()
+        assert hdr.status == 0
+        assert (hdr.gather_pair_tiles > 0) == expect_on, (hdr.gather_pair_tiles, hdr.gather_entries)
+        rep = pu.compare_rows(wl, pu.random_rows(wl, 1500, seed=5), out, bitmap, count, label="rule")
+        print("sharp" if expect_on else "flat", rep, hdr.gather_pair_tiles, hdr.gather_entries)
+
+
+def test_set_gather_arguments():
+    wl = inputs.small_prefill(seed=35)
+    eng = pu.make_engine(wl)
+    with pytest.raises(binding.AdasparkError):
+        binding.adaspark_attn_set_gather(eng.handle, -1.0, 8 << 30)
+    with pytest.raises(binding.AdasparkError):           # the budget sizes the workspace: not after partition
+        binding.adaspark_attn_set_gather(eng.handle, 20.0, 1 << 30)
+    binding.adaspark_attn_set_gather(eng.handle, 5.0, 8 << 30)   # the threshold alone may change
+
+
+def test_forced_gather_chunked_prefill():
+    """Chunks of a chunked prefill gather from the caches the earlier chunks built."""
+    wl = inputs.small_prefill(seed=36, T=32, H=8, W=8, n_text=23, Hq=4, Hkv=2, D=128, top_p=0.7, offset_std=2.5)
+    eng = pu.make_engine(wl, prefill_kernel=1, gather=pu.FORCE_GATHER)
+    q, k, v = wl.q.cuda(), wl.k.cuda(), wl.v.cuda()
+    hw = wl.H * wl.W
+    outs, bms, cnts, entries = [], [], [], 0
+    for fb, fc, nt in [(0, 8, -1), (8, 16, -1), (24, 8, wl.n_text)]:
+        lo, hi = fb * hw, (fb + fc) * hw + max(nt, 0)
+        o, b, c = eng.forward_chunk(q[:, lo:hi].contiguous(), k[:, lo:hi].contiguous(), v[:, lo:hi].contiguous(),
+                                    fb, fc, nt, want_selection=True)
+        torch.cuda.synchronize()
+        assert eng.header().status == 0
+        entries += eng.header().gather_entries
+        outs.append(o); bms.append(b); cnts.append(c)
+    out, bm, cnt = torch.cat(outs, 1), torch.cat(bms, 2), torch.cat(cnts, 2)
+    rep = pu.compare_rows(wl, oracle.all_rows(oracle.shape_of(wl)), out, bm, cnt, label="chunked")
+    assert rep["rows"] == wl.B * wl.Hq * wl.S
+    assert entries == expected_entries(wl, bm)
