@@ -59,7 +59,7 @@ constexpr int kExactCtas = 296;   // CTAs of the fp64 selection kernel (its scra
 // partial results of all such pairs must fit this many bytes of workspace
 constexpr float kGatherDefaultPairsPerBlock = 20.f;
 constexpr uint64_t kGatherDefaultBudget = 8ull << 30;
-constexpr uint64_t kGatherEntriesPerRow = 32;
+constexpr uint64_t kGatherEntriesPerRow = 128;
 size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 
 adaspark_status_t fail(adaspark_attn* h, adaspark_status_t st, const char* fmt, ...) {
@@ -217,7 +217,7 @@ adaspark_status_t adaspark_attn_partition(adaspark_attn_t* h, int32_t batch, int
     h->fw_headmax_off = off; off = align_up(off + (size_t)batch * Hkv * 4);
     h->fw_valid_off = off; off = align_up(off + (size_t)(S_cap / kBlockTok) * 2 * 4);   // which slots of a block hold a token
     const size_t n_cols = (size_t)(S_v + kBlockTok - 1) / kBlockTok;                     // key blocks that hold video
-    h->fw_gcol_off = off; off = align_up(off + (size_t)batch * Hkv * n_cols * 2 * 4);   // entry counts and fill cursors (zeroed per call)
+    h->fw_gcol_off = off; off = align_up(off + (size_t)batch * Hkv * n_cols * 2 * kGatherReplicas * 4);   // entry counts and fill cursors (zeroed per call)
     h->fw_mask_off = off; off = align_up(off + (size_t)batch * Hq * n_tiles_cap * n_words * kTileRows * 4);
     h->fw_union_off = off; off = align_up(off + (size_t)batch * Hq * n_tiles_cap * n_words * 4);
     h->fw_fallback_off = off; off = align_up(off + (size_t)batch * Hq * n_tiles_cap * kTileRows * 4);
@@ -238,7 +238,7 @@ adaspark_status_t adaspark_attn_partition(adaspark_attn_t* h, int32_t batch, int
         h->fw_gpair_off = off; off = align_up(off + (size_t)batch * Hq * n_pairs_cap * 3 * 4);
         h->fw_grow_off = off; off = align_up(off + (cap ? rows_cap * 2 * 4 : 0));
         h->fw_gml_off = off; off = align_up(off + (cap ? rows_cap * 8 : 0));
-        h->fw_gitems_off = off; off = align_up(off + (cap ? ((size_t)batch * Hkv * n_cols * 2 + cap / 128 + 1) * 8 : 0));
+        h->fw_gitems_off = off; off = align_up(off + (cap ? align_up(((size_t)batch * Hkv * n_cols * (kGatherReplicas + 2) + 2) * 4) + ((size_t)batch * Hkv * n_cols + cap / 128 + 1) * 16 : 0));
         h->fw_gentries_off = off; off = align_up(off + (size_t)cap * 8);
         h->fw_gparto_off = off; off = align_up(off + (size_t)cap * D * 2);
         h->fw_gpartml_off = off; off = align_up(off + (size_t)cap * 8);
@@ -460,10 +460,13 @@ adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* 
             gw.row_cnt = (uint32_t*)(ws + h->fw_grow_off);
             gw.row_ptr = gw.row_cnt + rows_cap;
             gw.col_cnt = (uint32_t*)(ws + h->fw_gcol_off);
-            gw.col_cur = gw.col_cnt + n_col_all;
-            gw.col_off = (uint32_t*)(ws + h->fw_gitems_off);
-            gw.items = (uint2*)(ws + h->fw_gitems_off + n_col_all * 8);
-            gw.entries = (uint2*)(ws + h->fw_gentries_off);
+            gw.col_cur = gw.col_cnt + n_col_all * kGatherReplicas;
+            gw.col_roff = (uint32_t*)(ws + h->fw_gitems_off);
+            gw.col_off = gw.col_roff + n_col_all * kGatherReplicas;
+            gw.col_item = gw.col_off + n_col_all + 1;
+            gw.items = (uint4*)(ws + h->fw_gitems_off + align_up((n_col_all * (kGatherReplicas + 2) + 2) * 4));
+            gw.entries = (uint32_t*)(ws + h->fw_gentries_off);
+            gw.row_slots = gw.entries + h->gather_cap;
             gw.part_o = (__nv_bfloat16*)(ws + h->fw_gparto_off);
             gw.part_ml = (float2*)(ws + h->fw_gpartml_off);
             gw.ml_local = (float2*)(ws + h->fw_gml_off);
@@ -475,6 +478,9 @@ adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* 
             if (!launch_ok(h, "gather_count_kernel")) return ADASPARK_ERR_CUDA;
             gather_scan_kernel<<<1, 1024, 0, st>>>(g, gw);
             if (!launch_ok(h, "gather_scan_kernel")) return ADASPARK_ERR_CUDA;
+            const int icta = (int)((n_col_all + 7) / 8);
+            gather_items_kernel<<<icta < 4 * h->sm_count ? icta : 4 * h->sm_count, 256, 0, st>>>(g, gw);
+            if (!launch_ok(h, "gather_items_kernel")) return ADASPARK_ERR_CUDA;
         }
         const uint32_t* pair_mode_c = gather ? gw.pair_mode : nullptr;
         if (D == 128) {
@@ -496,7 +502,7 @@ adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* 
             if (!launch_ok(h, "gather_fill_kernel")) return ADASPARK_ERR_CUDA;
             CUtensorMap tmKg;      // one key block per load: box of 64 d x 64 keys (tmK's) serves as it is
             tmKg = tmK;
-            const int ggrid = 2 * h->sm_count;
+            const int ggrid = h->sm_count;                      // persistent: one CTA per SM
             const long long n_rows = (long long)g.B * g.Hq * (g.S - g.pos_begin);
             if (D == 128) {
                 const size_t smem = sizeof(GatherSmem<128>) + 1024;

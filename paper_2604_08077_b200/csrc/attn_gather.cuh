@@ -10,7 +10,8 @@
 // and the result of its local range (own cube, text, text prefix: still the tile kernel, which then skips
 // the union) are merged by the softmax identity
 //     out = sum_i w_i O_i / sum_i w_i,   w_i = l_i 2^(m_i - M),  M = max_i m_i.
-// Executed work = selected work, at the price of 2 D + 8 bytes written and read per entry.
+// Executed work = selected work, at the price of 2 D + 8 bytes written and read per entry (plus the gathered
+// Q row).
 //
 // Which pairs of query tiles take this path is decided on the device, per pair, from the counts the selection
 // left: entries of the pair's rows (P) against key blocks in the pair's union (U), gathered iff
@@ -30,8 +31,8 @@
 
 namespace adaspark {
 
-constexpr int kGatherThreads = 160;     // 4 softmax / gather warps + 1 TMA / MMA warp
 constexpr int kGatherItemRows = 128;
+constexpr int kGatherReplicas = 8;
 constexpr uint32_t kEntryPosMask = 0x1fffffu;   // 21 bits of cube-major position (caches hold at most 2^21 rows)
 
 // Pointers into the forward workspace and sizes (all filled by the host).
@@ -41,13 +42,20 @@ struct GatherWs {
     uint32_t* pair_cnt;    // entries of the pair's rows (0 when the pair stays on the tile kernel)
     uint32_t* pair_off;    // exclusive prefix sum of pair_cnt
     uint32_t* row_cnt;     // [B*Hq*S_cap] entries of a row
-    uint32_t* row_ptr;     // index of the row's first partial
-    uint32_t* col_cnt;     // [B*Hkv*n_cols] entries of a key block; zero at the start of a forward
-    uint32_t* col_off;     // exclusive prefix sum of col_cnt
-    uint32_t* col_cur;     // fill cursors; zero at the start of a forward
-    uint2* items;          // (key block column, chunk of 128 entries)
-    uint2* entries;        // x: pos | head in group << 21 | cube bits << 25;  y: index of the partial
-    __nv_bfloat16* part_o; // [cap_entries][D] normalised partial outputs
+    uint32_t* row_ptr;     // index of the row's first slot in row_slots
+    uint32_t* col_cnt;     // [kGatherReplicas][B*Hkv*n_cols] entries of a key block, counted in kGatherReplicas
+                           // separate sets of counters (a CTA uses set blockIdx.x % kGatherReplicas: the atomics of
+                           // all CTAs on one set of a few thousand counters were the slowest part of the count);
+                           // zero at the start of a forward
+    uint32_t* col_cur;     // [kGatherReplicas][...] fill cursors; zero at the start of a forward
+    uint32_t* col_roff;    // [kGatherReplicas][...] first entry of the set's share of the block's list
+    uint32_t* col_off;     // [B*Hkv*n_cols + 1] first entry of the block's list (exclusive prefix sum)
+    uint32_t* col_item;    // [B*Hkv*n_cols + 1] first work item of the block
+    uint4* items;          // (key block column, first entry, entries (<= 128), 0)
+    uint32_t* entries;     // per key block, its entries: pos | head in group << 21 | cube bits << 25
+    uint32_t* row_slots;   // per row (from row_ptr on), the indices of its entries in ascending block order
+    __nv_bfloat16* part_o; // [cap_entries][D] normalised partial output of every entry (in entry order: an item
+                           // of the attention kernel writes one contiguous piece)
     float2* part_ml;       // [cap_entries] (reference exponent in log2 units, sum)
     float2* ml_local;      // [B*Hq*S_cap] the same for the local range, written by the tile kernel
     uint32_t cap_entries;
@@ -62,6 +70,24 @@ __device__ __forceinline__ uint32_t fold_to_blocks(uint32_t word, int c_shift) {
     if (c_shift == 5) return (word | (word >> 1)) & 0x55555555u;
     if (c_shift == 4) return (word | (word >> 1) | (word >> 2) | (word >> 3)) & 0x11111111u;
     return word;
+}
+
+// Transposes the 32 x 32 bit matrix whose row i is the word of lane i: afterwards bit i of lane j's word is the
+// former bit j of lane i (five exchange steps on ever smaller blocks).  With rows = query rows and bits =
+// cubes, lane j ends up with the set of rows that selected cube j: one step instead of one ballot per cube.
+__device__ __forceinline__ uint32_t transpose_32x32(uint32_t x, int lane) {
+    uint32_t y;
+    y = __shfl_xor_sync(0xffffffffu, x, 16);
+    x = (lane & 16) ? ((x & 0xffff0000u) | (y >> 16)) : ((x & 0x0000ffffu) | (y << 16));
+    y = __shfl_xor_sync(0xffffffffu, x, 8);
+    x = (lane & 8) ? ((x & 0xff00ff00u) | ((y >> 8) & 0x00ff00ffu)) : ((x & 0x00ff00ffu) | ((y << 8) & 0xff00ff00u));
+    y = __shfl_xor_sync(0xffffffffu, x, 4);
+    x = (lane & 4) ? ((x & 0xf0f0f0f0u) | ((y >> 4) & 0x0f0f0f0fu)) : ((x & 0x0f0f0f0fu) | ((y << 4) & 0xf0f0f0f0u));
+    y = __shfl_xor_sync(0xffffffffu, x, 2);
+    x = (lane & 2) ? ((x & 0xccccccccu) | ((y >> 2) & 0x33333333u)) : ((x & 0x33333333u) | ((y << 2) & 0xccccccccu));
+    y = __shfl_xor_sync(0xffffffffu, x, 1);
+    x = (lane & 1) ? ((x & 0xaaaaaaaau) | ((y >> 1) & 0x55555555u)) : ((x & 0x55555555u) | ((y << 1) & 0xaaaaaaaau));
+    return x;
 }
 
 struct PairItem {
@@ -85,7 +111,21 @@ __device__ __forceinline__ PairItem pair_item(const Geom& g, int bid) {
     return it;
 }
 
+// entries of the lane's row before the pair's local range, in key blocks
+__device__ __forceinline__ uint32_t row_entries(const Geom& g, const PairItem& it, const uint32_t* my) {
+    const int bshift = max(g.c_shift - 6, 0);
+    uint32_t cnt = 0;
+#pragma unroll 4
+    for (int w = 0; w < it.n_w; ++w) {
+        uint32_t word = __ldg(my + (size_t)w * kTileRows);
+        if (w == it.n_w - 1) word &= it.last_keep;
+        cnt += (uint32_t)__popc(fold_to_blocks(word, g.c_shift)) << bshift;
+    }
+    return cnt;
+}
+
 // ------------------------------------------------------------------------------------------------ count
+// One CTA per pair of query tiles and head.
 __global__ void __launch_bounds__(256) gather_count_kernel(Geom g, GatherWs ws, const uint32_t* __restrict__ tile_mask,
                                                            const uint32_t* __restrict__ tile_union) {
     __shared__ uint32_t red[2][8];
@@ -97,14 +137,8 @@ __global__ void __launch_bounds__(256) gather_count_kernel(Geom g, GatherWs ws, 
     const bool tile_ok = tile < g.n_tiles;
     const uint32_t* my = tile_mask + mask_index(g, it.b, it.h, tile_ok ? tile : 0, 0, r);
     const size_t bh = (size_t)(it.b * g.Hq + it.h);
-    uint32_t cnt = 0;
-    if (tile_ok)
-        for (int w = 0; w < it.n_w; ++w) {
-            uint32_t word = __ldg(my + (size_t)w * kTileRows);
-            if (w == it.n_w - 1) word &= it.last_keep;
-            cnt += (uint32_t)__popc(fold_to_blocks(word, g.c_shift)) << bshift;
-        }
-    if (pos < g.S_cap) ws.row_cnt[bh * g.S_cap + pos] = cnt;
+    const uint32_t my_cnt = tile_ok ? row_entries(g, it, my) : 0u;
+    uint32_t cnt = my_cnt;
     uint32_t ub = 0;
     for (int w = tid; w < it.n_w; w += 256) {
         uint32_t u = 0;
@@ -127,24 +161,27 @@ __global__ void __launch_bounds__(256) gather_count_kernel(Geom g, GatherWs ws, 
         s_mode = mode;
     }
     __syncthreads();
+    // rows of a pair that stays on the union path have no entries (the merge kernel reads only this)
+    if (pos < g.S_cap) ws.row_cnt[bh * g.S_cap + pos] = s_mode ? my_cnt : 0u;
     if (!s_mode || !tile_ok) return;
-    // entries per key block: one atomic per (32 rows, block)
-    uint32_t* col_cnt = ws.col_cnt + (size_t)(it.b * g.Hkv + it.gk) * ws.n_cols;
-    for (int w = 0; w < it.n_w; ++w) {
-        uint32_t word = __ldg(my + (size_t)w * kTileRows);
-        if (w == it.n_w - 1) word &= it.last_keep;
-        const uint32_t fw = fold_to_blocks(word, g.c_shift);
-        uint32_t orw = __reduce_or_sync(0xffffffffu, fw);
-        while (orw) {
-            const int beta = __ffs(orw) - 1;
-            orw &= orw - 1;
-            const int n = __popc(__ballot_sync(0xffffffffu, (fw >> beta) & 1u));
-            if (lane == 0) {
-                const int cube = w * 32 + beta;
+    // entries per key block: the warp's 32 x 32 bits of a word are transposed, lane j then counts the rows that
+    // selected cube 32 w + j and adds them to the cube's block(s)
+    uint32_t* col_cnt = ws.col_cnt + ((size_t)(blockIdx.x % kGatherReplicas) * g.B * g.Hkv + (it.b * g.Hkv + it.gk)) * ws.n_cols;
+    for (int w0 = 0; w0 < it.n_w; w0 += 4) {
+        uint32_t wd[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) wd[k] = w0 + k < it.n_w ? __ldg(my + (size_t)(w0 + k) * kTileRows) : 0u;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            if (w0 + k >= it.n_w) break;
+            if (w0 + k == it.n_w - 1) wd[k] &= it.last_keep;
+            const uint32_t n = (uint32_t)__popc(transpose_32x32(fold_to_blocks(wd[k], g.c_shift), lane));
+            if (n) {
+                const int cube = (w0 + k) * 32 + lane;
                 if (g.c_shift >= 6) {
-                    for (int i = 0; i < (1 << bshift); ++i) atomicAdd(col_cnt + ((size_t)cube << bshift) + i, (uint32_t)n);
+                    for (int i = 0; i < (1 << bshift); ++i) atomicAdd(col_cnt + ((size_t)cube << bshift) + i, n);
                 } else {
-                    atomicAdd(col_cnt + (cube >> (6 - g.c_shift)), (uint32_t)n);
+                    atomicAdd(col_cnt + (cube >> (6 - g.c_shift)), n);
                 }
             }
         }
@@ -181,8 +218,6 @@ __device__ __forceinline__ uint32_t cta_exclusive_scan_1024(uint32_t v, uint32_t
 __global__ void __launch_bounds__(1024) gather_scan_kernel(Geom g, GatherWs ws) {
     __shared__ uint32_t warp_sums[32];
     __shared__ uint32_t total_s;
-    __shared__ uint32_t big_col[1024], big_base[1024], big_n[1024];
-    __shared__ uint32_t big_count;
     const int tid = threadIdx.x;
     const int pair0 = g.pos_begin / kPairRows, n_pairs = (g.S + kPairRows - 1) / kPairRows - pair0;
     const int n_hb = g.Hq * g.B;
@@ -223,38 +258,53 @@ __global__ void __launch_bounds__(1024) gather_scan_kernel(Geom g, GatherWs ws) 
         ws.ctrl[0] = (uint32_t)carry;
         ws.ctrl[2] = s;
     }
-    // ---- key blocks: offsets of their entry lists and the work items (chunks of 128 entries)
+    // ---- key blocks: offsets of their entry lists (and of every counter set's share) and of their work items
     const int n_cols_all = g.B * g.Hkv * ws.n_cols;
     uint32_t ent_carry = 0, item_carry = 0;
     for (int base = 0; base < n_cols_all; base += 1024) {
         const int col = base + tid;
-        const uint32_t v = col < n_cols_all ? ws.col_cnt[col] : 0u;
+        uint32_t part[kGatherReplicas];
+        uint32_t v = 0;
+#pragma unroll
+        for (int r = 0; r < kGatherReplicas; ++r) {
+            part[r] = col < n_cols_all ? ws.col_cnt[(size_t)r * n_cols_all + col] : 0u;
+            v += part[r];
+        }
         const uint32_t chunks = (v + kGatherItemRows - 1) / kGatherItemRows;
         const uint32_t ex = cta_exclusive_scan_1024(v, warp_sums, &total_s);
         const uint32_t tot_e = total_s;
         const uint32_t exi = cta_exclusive_scan_1024(chunks, warp_sums, &total_s);
         const uint32_t tot_i = total_s;
-        if (tid == 0) big_count = 0u;
-        __syncthreads();
         if (col < n_cols_all) {
-            ws.col_off[col] = ent_carry + ex;
-            const uint32_t ib = item_carry + exi;
-            if (chunks <= 32u) {
-                for (uint32_t c = 0; c < chunks; ++c) ws.items[ib + c] = make_uint2((uint32_t)col, c);
-            } else {
-                const uint32_t k = atomicAdd(&big_count, 1u);
-                big_col[k] = (uint32_t)col; big_base[k] = ib; big_n[k] = chunks;
+            uint32_t o = ent_carry + ex;
+            ws.col_off[col] = o;
+            ws.col_item[col] = item_carry + exi;
+#pragma unroll
+            for (int r = 0; r < kGatherReplicas; ++r) {
+                ws.col_roff[(size_t)r * n_cols_all + col] = o;
+                o += part[r];
             }
         }
-        __syncthreads();
-        const uint32_t nb = big_count;
-        for (uint32_t k = 0; k < nb; ++k)
-            for (uint32_t c = tid; c < big_n[k]; c += 1024) ws.items[big_base[k] + c] = make_uint2(big_col[k], c);
         ent_carry += tot_e;
         item_carry += tot_i;
-        __syncthreads();
     }
-    if (tid == 0) ws.ctrl[1] = item_carry;
+    if (tid == 0) {
+        ws.col_off[n_cols_all] = ent_carry;
+        ws.col_item[n_cols_all] = item_carry;
+        ws.ctrl[1] = item_carry;
+    }
+}
+
+// Work items of every key block: chunks of up to 128 entries of its list.  One warp per block.
+__global__ void __launch_bounds__(256) gather_items_kernel(Geom g, GatherWs ws) {
+    if (ws.ctrl[0] == 0u) return;
+    const int n_cols_all = g.B * g.Hkv * ws.n_cols;
+    const int lane = threadIdx.x & 31;
+    for (int col = blockIdx.x * 8 + (threadIdx.x >> 5); col < n_cols_all; col += gridDim.x * 8) {
+        const uint32_t first = ws.col_off[col], n = ws.col_off[col + 1] - first, ib = ws.col_item[col];
+        for (uint32_t c = lane; c * kGatherItemRows < n; c += 32)
+            ws.items[ib + c] = make_uint4((uint32_t)col, first + c * kGatherItemRows, min(n - c * kGatherItemRows, (uint32_t)kGatherItemRows), 0u);
+    }
 }
 
 // ------------------------------------------------------------------------------------------------ fill
@@ -284,79 +334,127 @@ __global__ void __launch_bounds__(256) gather_fill_kernel(Geom g, GatherWs ws, c
     if (pos < g.S_cap) ws.row_ptr[bh * g.S_cap + pos] = ptr;
     if (!tile_ok) return;
     const uint32_t* my = tile_mask + mask_index(g, it.b, it.h, tile, 0, r);
-    const size_t colbase = (size_t)(it.b * g.Hkv + it.gk) * ws.n_cols;
+    const size_t colbase = ((size_t)(blockIdx.x % kGatherReplicas) * g.B * g.Hkv + (it.b * g.Hkv + it.gk)) * ws.n_cols;
     const uint32_t ent_x = (uint32_t)pos | ((uint32_t)(it.h - it.gk * g.G) << 21);
     const uint32_t lt_mask = (1u << lane) - 1u;
+    // Four words per step.  After the transposition lane j holds the rows of the warp that selected cube 32 w + j;
+    // ONE round of atomics reserves the slots of all (word, cube) pairs of the step in their blocks' lists (the
+    // return value of an atomic takes about a microsecond: one round per selected cube was the whole run time);
+    // then every row walks its own cubes, fetching start and row set from the lane that owns the cube.
     const int group = g.c_shift >= 6 ? 1 : (kBlockTok >> g.c_shift);    // cubes per key block (small cubes)
-    for (int w = 0; w < it.n_w; ++w) {
-        uint32_t word = __ldg(my + (size_t)w * kTileRows);
-        if (w == it.n_w - 1) word &= it.last_keep;
-        const uint32_t fw = fold_to_blocks(word, g.c_shift);
-        uint32_t orw = __reduce_or_sync(0xffffffffu, fw);
-        while (orw) {
-            const int beta = __ffs(orw) - 1;
-            orw &= orw - 1;
-            const bool has = (fw >> beta) & 1u;
-            const uint32_t m = __ballot_sync(0xffffffffu, has);
-            const uint32_t n = (uint32_t)__popc(m), rank = (uint32_t)__popc(m & lt_mask);
-            const int cube = w * 32 + beta;
-            const int nblk = 1 << bshift;
-            const size_t col0 = colbase + (g.c_shift >= 6 ? ((size_t)cube << bshift) : (size_t)(cube >> (6 - g.c_shift)));
-            const uint32_t sub = g.c_shift >= 6 ? 0xfu : ((word >> beta) & ((1u << group) - 1u));
-            for (int i = 0; i < nblk; ++i) {
-                uint32_t start = 0;
-                if (lane == 0) start = ws.col_off[col0 + i] + atomicAdd(ws.col_cur + col0 + i, n);
-                start = __shfl_sync(0xffffffffu, start, 0);
-                if (has) ws.entries[start + rank] = make_uint2(ent_x | (sub << 25), ptr + (uint32_t)i);
+    const int nblk = 1 << bshift;                                       // key blocks per cube (large cubes)
+    for (int w0 = 0; w0 < it.n_w; w0 += 4) {
+        uint32_t wd[4], fw[4], tw[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) wd[k] = w0 + k < it.n_w ? __ldg(my + (size_t)(w0 + k) * kTileRows) : 0u;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            if (w0 + k == it.n_w - 1) wd[k] &= it.last_keep;
+            fw[k] = fold_to_blocks(wd[k], g.c_shift);
+            tw[k] = transpose_32x32(fw[k], lane);
+        }
+        uint32_t slot0[4];                                              // first slot of the row for the cubes of word k
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            slot0[k] = ptr;
+            ptr += (uint32_t)(__popc(fw[k]) * nblk);
+        }
+        for (int i = 0; i < nblk; ++i) {
+            uint32_t st[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                st[k] = 0u;
+                if (tw[k]) {
+                    const int cube = (w0 + k) * 32 + lane;
+                    const size_t col = colbase + (g.c_shift >= 6 ? ((size_t)cube << bshift) + i : (size_t)(cube >> (6 - g.c_shift)));
+                    st[k] = ws.col_roff[col] + atomicAdd(ws.col_cur + col, (uint32_t)__popc(tw[k]));
+                }
             }
-            if (has) ptr += (uint32_t)nblk;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                uint32_t t = fw[k];
+                const int trips = __reduce_max_sync(0xffffffffu, __popc(t));
+                for (int j = 0; j < trips; ++j) {
+                    const int beta = t ? __ffs(t) - 1 : 0;
+                    const uint32_t m = __shfl_sync(0xffffffffu, tw[k], beta), start = __shfl_sync(0xffffffffu, st[k], beta);
+                    if (t) {
+                        const uint32_t e = start + (uint32_t)__popc(m & lt_mask);
+                        ws.entries[e] = ent_x | (((wd[k] >> beta) & ((1u << group) - 1u)) << 25);
+                        ws.row_slots[slot0[k] + (uint32_t)(j * nblk + i)] = e;
+                        t &= t - 1;
+                    }
+                }
+            }
         }
     }
 }
 
 // ------------------------------------------------------------------------------------------------ attention
+// One persistent CTA per SM, 512 threads in four warpgroups:
+//   warps 0-3 / 4-7   consumers of the even / odd items: softmax of S (thread = gathered row = TMEM lane),
+//                     P into TMEM, normalised partial output and (reference, sum) to global memory
+//   warps 8-11        gather producers: the Q rows of an item into a ring of three shared-memory tiles with
+//                     cp.async (16 rows x 32 bytes per warp instruction), up to two items in flight
+//   warp 12           MMA issuer: S_i = Q_i K^T (operands in shared memory), O_i = P_i V (P in TMEM); the S of
+//                     item i+1 is issued before the P of item i is waited for, so the tensor pipe, the two
+//                     softmax warpgroups and the gathers overlap
+//   warp 13           TMA producer of the K / V^T blocks (ring of three)
+//   warps 14-15       idle
+// TMEM: consumer c owns columns [256 c, 256 c + 64) for S (P overwrites the first 32) and
+// [256 c + 64, 256 c + 64 + D) for O.
+constexpr int kGatherThreads = 512;
+constexpr int kGatherStages = 3;
+
 template <int D>
 struct GatherSmem {
-    __nv_bfloat16 q[D / 64][128][64];        // [d panel][gathered row][64 d], 128-byte swizzle
-    __nv_bfloat16 k[2][D / 64][64][64];      // [stage][d panel][key][64 d]
-    __nv_bfloat16 v[2][D][64];               // [stage][d][64 keys]  (V^T)
-    uint2 ent[2][kGatherItemRows];
-    uint64_t q_full, kv_full[2], s_full, p_full, o_full, ent_full;
+    __nv_bfloat16 q[kGatherStages][D / 64][128][64];   // [stage][d panel][gathered row][64 d], 128-byte swizzle
+    __nv_bfloat16 k[kGatherStages][D / 64][64][64];    // [stage][d panel][key][64 d]
+    __nv_bfloat16 v[kGatherStages][D][64];             // [stage][d][64 keys]  (V^T)
+    uint64_t q_full[kGatherStages], q_empty[kGatherStages], kv_full[kGatherStages], kv_empty[kGatherStages];
+    uint64_t s_full[2], p_full[2], o_full[2];
     uint32_t tmem_base;
     int abort_flag;
 };
 
 template <int D>
-__global__ void __launch_bounds__(kGatherThreads, 2) attn_gather_kernel(
+__global__ void __launch_bounds__(kGatherThreads, 1) attn_gather_kernel(
     Geom g, GatherWs ws, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
     const __nv_bfloat16* __restrict__ q_cube, const uint32_t* __restrict__ slot_valid,
     unsigned long long* __restrict__ executed_blocks, int32_t* __restrict__ status) {
     extern __shared__ unsigned char gather_smem_raw[];
     GatherSmem<D>& sm = *reinterpret_cast<GatherSmem<D>*>((reinterpret_cast<uintptr_t>(gather_smem_raw) + 1023) & ~(uintptr_t)1023);
-    constexpr int kPanels = D / 64, kQKSteps = D / 16, kChunks = D / 8;
+    constexpr int kPanels = D / 64, kQKSteps = D / 16;
+    constexpr int kPairsPerRow = D / 16;                         // 32-byte pieces of a Q row
     constexpr uint32_t kIdescS = tc::make_idesc_bf16(128, 64);   // S: 128 gathered rows x 64 keys
     constexpr uint32_t kIdescO = tc::make_idesc_bf16(128, D);    // O: 128 rows x D
     constexpr uint32_t kKVBytes = 64 * D * 2 * 2;
-    constexpr int kTmemCols = 256;                               // S / P at [0, 64), O at [64, 64 + D)
 
     const uint32_t n_items = ws.ctrl[1];
     if (ws.ctrl[0] == 0u || blockIdx.x >= n_items) return;       // the path is off, or fewer items than CTAs
-    const int my_items = (int)((n_items - blockIdx.x + gridDim.x - 1) / gridDim.x);
+    // a contiguous run of items per CTA: consecutive items mostly share their key block, whose K / V^T tiles
+    // then stay in shared memory
+    const uint32_t per = n_items / gridDim.x, rem = n_items - per * gridDim.x;
+    const uint32_t item0 = blockIdx.x * per + min((uint32_t)blockIdx.x, rem);
+    const int my_items = (int)(per + (blockIdx.x < rem ? 1u : 0u));
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     if (tid == 0) {
-        tc::mbar_init(&sm.q_full, kGatherItemRows);
-        tc::mbar_init(&sm.kv_full[0], 1);
-        tc::mbar_init(&sm.kv_full[1], 1);
-        tc::mbar_init(&sm.s_full, 1);
-        tc::mbar_init(&sm.p_full, kGatherItemRows);
-        tc::mbar_init(&sm.o_full, 1);
-        tc::mbar_init(&sm.ent_full, kGatherItemRows);
+        for (int i = 0; i < kGatherStages; ++i) {
+            tc::mbar_init(&sm.q_full[i], 128);
+            tc::mbar_init(&sm.q_empty[i], 1);
+            tc::mbar_init(&sm.kv_full[i], 1);
+            tc::mbar_init(&sm.kv_empty[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            tc::mbar_init(&sm.s_full[i], 1);
+            tc::mbar_init(&sm.p_full[i], 128);
+            tc::mbar_init(&sm.o_full[i], 1);
+        }
         sm.abort_flag = 0;
         tc::fence_barrier_init();
     }
-    if (warp == 4) {
-        tc::tmem_alloc<kTmemCols>(&sm.tmem_base);
+    if (warp == 12) {
+        tc::tmem_alloc<512>(&sm.tmem_base);
         if (lane == 0) {
             tc::prefetch_tensormap(&tmK);
             tc::prefetch_tensormap(&tmV);
@@ -367,98 +465,26 @@ __global__ void __launch_bounds__(kGatherThreads, 2) attn_gather_kernel(
     tc::tc_fence_after_sync();
     const uint32_t tbase = sm.tmem_base;
     volatile int* abort_flag = &sm.abort_flag;
+    // item i of this CTA: (column = (batch x kv head) * n_cols + key block, first entry, entries, -)
+    auto item_at = [&](int i) -> uint4 { return __ldg(ws.items + item0 + i); };
 
-    // column of an item -> (batch x kv head, key block)
-    auto item_col = [&](int i, int& bg, int& blk, uint32_t& first, int& n) {
-        const uint2 iv = ws.items[blockIdx.x + (size_t)i * gridDim.x];
-        bg = (int)(iv.x / (uint32_t)ws.n_cols);
-        blk = (int)(iv.x - (uint32_t)bg * (uint32_t)ws.n_cols);
-        first = ws.col_off[iv.x] + iv.y * kGatherItemRows;
-        n = min(kGatherItemRows, (int)(ws.col_cnt[iv.x] - iv.y * kGatherItemRows));
-    };
-
-    if (warp == 4) {
-        // ------------------------------------------------------------ TMA producer + MMA issuer (one thread)
-        if (lane == 0) {
-            auto load_kv = [&](int i) {
-                int bg, blk, n;
-                uint32_t first;
-                item_col(i, bg, blk, first, n);
-                const int st = i & 1;
-                tc::mbar_arrive_expect_tx(&sm.kv_full[st], kKVBytes);
-                for (int p = 0; p < kPanels; ++p)
-                    tc::tma_load_2d(&sm.k[st][p][0][0], &tmK, p * 64, bg * g.S_cap + blk * kBlockTok, &sm.kv_full[st]);
-                tc::tma_load_2d(&sm.v[st][0][0], &tmV, 0, (bg * g.n_kv_blocks_cap + blk) * D, &sm.kv_full[st]);
-            };
-            constexpr uint32_t kQPanelStep = (128 * 64 * 2) >> 4, kKPanelStep = (64 * 64 * 2) >> 4, kKStep = 32 >> 4;
-            const uint32_t q_lo = tc::smem_desc_lo_sw128(smem_u32(&sm.q[0][0][0]));
-            load_kv(0);
-            for (int i = 0; i < my_items; ++i) {
-                const int st = i & 1;
-                const uint32_t k_lo = tc::smem_desc_lo_sw128(smem_u32(&sm.k[st][0][0][0]));
-                const uint32_t v_lo = tc::smem_desc_lo_sw128(smem_u32(&sm.v[st][0][0]));
-                if (!tc::mbar_wait(&sm.q_full, i & 1, abort_flag)) break;
-                if (!tc::mbar_wait(&sm.kv_full[st], (i >> 1) & 1, abort_flag)) break;
-                tc::tc_fence_after_sync();
-#pragma unroll
-                for (int ks = 0; ks < kQKSteps; ++ks) {
-                    const uint32_t qo = (ks >> 2) * kQPanelStep + (ks & 3) * kKStep, ko = (ks >> 2) * kKPanelStep + (ks & 3) * kKStep;
-                    tc::umma_ss(tbase, tc::smem_desc_from_halves(q_lo + qo, tc::kSmemDescHiSw128),
-                                tc::smem_desc_from_halves(k_lo + ko, tc::kSmemDescHiSw128), kIdescS, ks > 0);
-                }
-                tc::umma_commit(&sm.s_full);
-                if (!tc::mbar_wait(&sm.p_full, i & 1, abort_flag)) break;
-                tc::tc_fence_after_sync();
-                // every worker has passed the epilogue of item i-1, so that item's MMAs have completed and its
-                // K / V stage can take the next block
-                if (i + 1 < my_items) load_kv(i + 1);
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    tc::umma_ts(tbase + 64, tbase + ks * 8, tc::smem_desc_from_halves(v_lo + ks * kKStep, tc::kSmemDescHiSw128), kIdescO, ks > 0);
-                tc::umma_commit(&sm.o_full);
-            }
-        }
-    } else {
-        // ------------------------------------------------------------ workers: gather, softmax, epilogue
-        const uint32_t lane_addr = tbase + ((uint32_t)(warp * 32) << 16);
+    if (warp < 8) {
+        // ------------------------------------------------------------ consumers
+        const int c = warp >> 2, row = tid & 127;
+        const uint32_t lane_addr = tbase + ((uint32_t)((warp & 3) * 32) << 16) + c * 256;
         const float scale_log2 = g.scale_log2;
-        int bg = 0, blk = 0, n = 0, bg_n = 0, blk_n = 0, n_n = 0;
-        uint32_t first = 0, first_n = 0;
-        auto gather_issue = [&](int buf, int bgi, int ni) {
-            const int b = bgi / g.Hkv, gk = bgi - b * g.Hkv;
-            const size_t head0 = (size_t)(b * g.Hq + gk * g.G);
-            for (int idx = tid; idx < ni * kChunks; idx += kGatherItemRows) {
-                const int row = idx / kChunks, c = idx - row * kChunks;
-                const uint32_t e = sm.ent[buf][row].x;
-                const __nv_bfloat16* src = q_cube + ((head0 + ((e >> 21) & 15u)) * g.S_cap + (e & kEntryPosMask)) * D + c * 8;
-                unsigned char* dst = reinterpret_cast<unsigned char*>(&sm.q[0][0][0]) + (c >> 3) * (128 * 128) + sw128(row, c & 7);
-                cp_async_16(dst, src);
-            }
-            cp_async_commit();
-        };
-        item_col(0, bg, blk, first, n);
-        if (tid < n) sm.ent[0][tid] = ws.entries[first + tid];
-        // the workers meet on an mbarrier (bounded wait) once the entries of an item are in shared memory
-        tc::mbar_arrive(&sm.ent_full);
-        bool ok = tc::mbar_wait(&sm.ent_full, 0, abort_flag);
-        if (ok) gather_issue(0, bg, n);
-        for (int i = 0; ok && i < my_items; ++i) {
-            const int cur = i & 1;
-            cp_async_wait<0>();
-            asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
-            tc::mbar_arrive(&sm.q_full);
-            const bool more = i + 1 < my_items;
-            if (more) {
-                item_col(i + 1, bg_n, blk_n, first_n, n_n);
-                if (tid < n_n) sm.ent[cur ^ 1][tid] = ws.entries[first_n + tid];
-                tc::mbar_arrive(&sm.ent_full);
-            }
-            const bool valid = tid < n;
-            const uint2 ent = valid ? sm.ent[cur][tid] : make_uint2(0u, 0u);
+        uint4 d_cur = c < my_items ? item_at(c) : make_uint4(0u, 0u, 0u, 0u);
+        uint32_t ent = 0u;
+        if (c < my_items && row < (int)d_cur.z) ent = __ldg(ws.entries + d_cur.y + row);
+        for (int i = c, j = 0; i < my_items; i += 2, ++j) {
+            // the next item of this warpgroup: descriptor and entry are requested now, used after the epilogue
+            uint4 d_nxt = make_uint4(0u, 0u, 0u, 0u);
+            if (i + 2 < my_items) d_nxt = item_at(i + 2);
+            const bool valid = row < (int)d_cur.z;
             // ---- which of the 64 keys of the block this row attends: the cubes it selected, minus empty slots
             uint32_t m0 = 0u, m1 = 0u;
             if (valid) {
-                const uint32_t sub = ent.x >> 25;
+                const uint32_t sub = ent >> 25;
                 if (g.c_shift >= 6) {
                     m0 = m1 = 0xffffffffu;
                 } else if (g.c_shift == 5) {
@@ -469,81 +495,223 @@ __global__ void __launch_bounds__(kGatherThreads, 2) attn_gather_kernel(
                     m1 = ((sub & 4u) ? 0x0000ffffu : 0u) | ((sub & 8u) ? 0xffff0000u : 0u);
                 }
                 if (g.ragged) {
+                    const int blk = (int)(d_cur.x % (uint32_t)ws.n_cols);
                     m0 &= __ldg(slot_valid + 2 * blk);
                     m1 &= __ldg(slot_valid + 2 * blk + 1);
                 }
             }
-            if (!(ok = tc::mbar_wait(&sm.s_full, i & 1, abort_flag))) break;
+            if (!tc::mbar_wait(&sm.s_full[c], j & 1, abort_flag)) break;
             tc::tc_fence_after_sync();
             uint32_t s[2][32];
             tc::tmem_ld_32x32(lane_addr, s[0]);
             tc::tmem_ld_32x32(lane_addr + 32, s[1]);
             tc::tmem_wait_ld();
+            const bool full = (m0 & m1) == 0xffffffffu;
             float mx = -INFINITY;
+            if (full) {
+                float a[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                const uint32_t am = c ? m1 : m0;
-                float a0 = -INFINITY, a1 = -INFINITY;
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    a0 = fmaxf(a0, ((am >> (2 * j)) & 1u) ? __uint_as_float(s[c][2 * j]) : -INFINITY);
-                    a1 = fmaxf(a1, ((am >> (2 * j + 1)) & 1u) ? __uint_as_float(s[c][2 * j + 1]) : -INFINITY);
+                for (int t = 0; t < 8; ++t) {
+                    a[0] = fmax3(a[0], __uint_as_float(s[0][4 * t]), __uint_as_float(s[0][4 * t + 1]));
+                    a[1] = fmax3(a[1], __uint_as_float(s[0][4 * t + 2]), __uint_as_float(s[0][4 * t + 3]));
+                    a[2] = fmax3(a[2], __uint_as_float(s[1][4 * t]), __uint_as_float(s[1][4 * t + 1]));
+                    a[3] = fmax3(a[3], __uint_as_float(s[1][4 * t + 2]), __uint_as_float(s[1][4 * t + 3]));
                 }
-                mx = fmax3(mx, a0, a1);
+                mx = fmaxf(fmaxf(a[0], a[1]), fmaxf(a[2], a[3]));
+            } else {
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    const uint32_t am = hf ? m1 : m0;
+                    float a0 = -INFINITY, a1 = -INFINITY;
+#pragma unroll
+                    for (int t = 0; t < 16; ++t) {
+                        a0 = fmaxf(a0, ((am >> (2 * t)) & 1u) ? __uint_as_float(s[hf][2 * t]) : -INFINITY);
+                        a1 = fmaxf(a1, ((am >> (2 * t + 1)) & 1u) ? __uint_as_float(s[hf][2 * t + 1]) : -INFINITY);
+                    }
+                    mx = fmax3(mx, a0, a1);
+                }
             }
             const float m_ref = mx * scale_log2;                   // -inf: no key of the block is visible to this row
             const float neg_ref = mx == -INFINITY ? 0.f : -m_ref;
             float l0 = 0.f, l1 = 0.f;
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                const uint32_t am = c ? m1 : m0;
+            for (int hf = 0; hf < 2; ++hf) {
+                const uint32_t am = hf ? m1 : m0;
                 uint32_t pk[16];
+                if (full) {
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const float p0 = fast_exp2(fmaf(__uint_as_float(s[c][2 * j]), scale_log2, ((am >> (2 * j)) & 1u) ? neg_ref : -INFINITY));
-                    const float p1 = fast_exp2(fmaf(__uint_as_float(s[c][2 * j + 1]), scale_log2, ((am >> (2 * j + 1)) & 1u) ? neg_ref : -INFINITY));
-                    l0 += p0;
-                    l1 += p1;
-                    pk[j] = pack_bf16x2(p0, p1);
+                    for (int t = 0; t < 16; ++t) {
+                        const float p0 = fast_exp2(fmaf(__uint_as_float(s[hf][2 * t]), scale_log2, neg_ref));
+                        const float p1 = fast_exp2(fmaf(__uint_as_float(s[hf][2 * t + 1]), scale_log2, neg_ref));
+                        l0 += p0;
+                        l1 += p1;
+                        pk[t] = pack_bf16x2(p0, p1);
+                    }
+                } else {
+#pragma unroll
+                    for (int t = 0; t < 16; ++t) {
+                        const float p0 = fast_exp2(fmaf(__uint_as_float(s[hf][2 * t]), scale_log2, ((am >> (2 * t)) & 1u) ? neg_ref : -INFINITY));
+                        const float p1 = fast_exp2(fmaf(__uint_as_float(s[hf][2 * t + 1]), scale_log2, ((am >> (2 * t + 1)) & 1u) ? neg_ref : -INFINITY));
+                        l0 += p0;
+                        l1 += p1;
+                        pk[t] = pack_bf16x2(p0, p1);
+                    }
                 }
-                tc::tmem_st_32x16(lane_addr + c * 16, pk);
+                tc::tmem_st_32x16(lane_addr + hf * 16, pk);
             }
             const float l_sum = l0 + l1;
             tc::tmem_wait_st();
             tc::tc_fence_before_sync();
-            tc::mbar_arrive(&sm.p_full);
-            // ---- the S MMAs have completed: the Q tile can take the rows of the next item
-            if (more) {
-                if (!(ok = tc::mbar_wait(&sm.ent_full, (i + 1) & 1, abort_flag))) break;   // its entries are in shared memory
-                gather_issue(cur ^ 1, bg_n, n_n);
-            }
+            tc::mbar_arrive(&sm.p_full[c]);
+            uint32_t e_nxt = 0u;
+            if (i + 2 < my_items && row < (int)d_nxt.z) e_nxt = __ldg(ws.entries + d_nxt.y + row);
             // ---- epilogue: normalised partial output, (reference, sum)
-            if (!(ok = tc::mbar_wait(&sm.o_full, i & 1, abort_flag))) break;
+            if (!tc::mbar_wait(&sm.o_full[c], j & 1, abort_flag)) break;
             tc::tc_fence_after_sync();
             const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
-            uint4* dst = reinterpret_cast<uint4*>(ws.part_o + (size_t)ent.y * D);
+            uint4* dst = reinterpret_cast<uint4*>(ws.part_o + (size_t)(d_cur.y + row) * D);
+            // the output row in rounds of 64 columns (the whole row at once does not fit the register budget of
+            // a 512-thread CTA)
 #pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
-                uint32_t o[32];
-                tc::tmem_ld_32x32(lane_addr + 64 + c * 32, o);
+            for (int hf = 0; hf < D / 64; ++hf) {
+                uint32_t o[2][32];
+                tc::tmem_ld_32x32(lane_addr + 64 + hf * 64, o[0]);
+                tc::tmem_ld_32x32(lane_addr + 64 + hf * 64 + 32, o[1]);
                 tc::tmem_wait_ld();
                 if (valid) {
 #pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                        uint4 val;
-                        val.x = pack_bf16x2(__uint_as_float(o[8 * q4 + 0]) * inv, __uint_as_float(o[8 * q4 + 1]) * inv);
-                        val.y = pack_bf16x2(__uint_as_float(o[8 * q4 + 2]) * inv, __uint_as_float(o[8 * q4 + 3]) * inv);
-                        val.z = pack_bf16x2(__uint_as_float(o[8 * q4 + 4]) * inv, __uint_as_float(o[8 * q4 + 5]) * inv);
-                        val.w = pack_bf16x2(__uint_as_float(o[8 * q4 + 6]) * inv, __uint_as_float(o[8 * q4 + 7]) * inv);
-                        dst[c * 4 + q4] = val;
+                    for (int cc = 0; cc < 2; ++cc) {
+#pragma unroll
+                        for (int q4 = 0; q4 < 4; ++q4) {
+                            uint4 val;
+                            val.x = pack_bf16x2(__uint_as_float(o[cc][8 * q4 + 0]) * inv, __uint_as_float(o[cc][8 * q4 + 1]) * inv);
+                            val.y = pack_bf16x2(__uint_as_float(o[cc][8 * q4 + 2]) * inv, __uint_as_float(o[cc][8 * q4 + 3]) * inv);
+                            val.z = pack_bf16x2(__uint_as_float(o[cc][8 * q4 + 4]) * inv, __uint_as_float(o[cc][8 * q4 + 5]) * inv);
+                            val.w = pack_bf16x2(__uint_as_float(o[cc][8 * q4 + 6]) * inv, __uint_as_float(o[cc][8 * q4 + 7]) * inv);
+                            dst[(hf * 2 + cc) * 4 + q4] = val;
+                        }
                     }
                 }
             }
-            if (valid) ws.part_ml[ent.y] = make_float2(m_ref, l_sum);
             tc::tc_fence_before_sync();
-            bg = bg_n; blk = blk_n; n = n_n; first = first_n;
+            if (valid) {
+                ws.part_ml[d_cur.y + row] = make_float2(m_ref, l_sum);
+            }
+            d_cur = d_nxt;
+            ent = e_nxt;
+        }
+    } else if (warp < 12) {
+        // ------------------------------------------------------------ gather producers
+        // lanes (2k, 2k+1) copy the two 16-byte halves of a 32-byte piece; a warp instruction covers 16 rows,
+        // the warpgroup 64 rows per pass: two passes of D/16 pieces per item
+        const int pt = tid - 256;                                  // 0..127
+        const int half = pt & 1, rsub = pt >> 1;                   // row inside the pass: 0..63
+        uint4 d_cur = item_at(0);
+        bool ok = true;
+        for (int i = 0; i < my_items; ++i) {
+            const int st = i % kGatherStages;
+            uint4 d_nxt = make_uint4(0u, 0u, 0u, 0u);
+            if (i + 1 < my_items) d_nxt = item_at(i + 1);
+            const int n = (int)d_cur.z;
+            uint32_t e[2];
+#pragma unroll
+            for (int ps = 0; ps < 2; ++ps) e[ps] = (ps * 64 + rsub < n) ? __ldg(ws.entries + d_cur.y + ps * 64 + rsub) : 0u;
+            if (!(ok = tc::mbar_wait(&sm.q_empty[st], ((i / kGatherStages) & 1) ^ 1, abort_flag))) break;
+            const int bg = (int)(d_cur.x / (uint32_t)ws.n_cols);
+            const int b = bg / g.Hkv, gk = bg - b * g.Hkv;
+            const size_t head0 = (size_t)(b * g.Hq + gk * g.G);
+            unsigned char* qbase = reinterpret_cast<unsigned char*>(&sm.q[st][0][0][0]);
+#pragma unroll
+            for (int ps = 0; ps < 2; ++ps) {
+                const int row = ps * 64 + rsub;
+                if (row < n) {
+                    const __nv_bfloat16* src = q_cube + ((head0 + ((e[ps] >> 21) & 15u)) * g.S_cap + (e[ps] & kEntryPosMask)) * D;
+#pragma unroll
+                    for (int pc = 0; pc < kPairsPerRow; ++pc) {
+                        const int ch = pc * 2 + half;                  // 16-byte chunk of the row
+                        cp_async_16(qbase + (ch >> 3) * (128 * 128) + sw128(row, ch & 7), src + ch * 8);
+                    }
+                }
+            }
+            cp_async_commit();
+            if (i > 0) {                                             // the previous item has landed
+                cp_async_wait<1>();
+                asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+                tc::mbar_arrive(&sm.q_full[(i - 1) % kGatherStages]);
+            }
+            d_cur = d_nxt;
         }
         cp_async_wait<0>();
+        if (ok) {
+            asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+            tc::mbar_arrive(&sm.q_full[(my_items - 1) % kGatherStages]);
+        }
+    } else if (warp == 12) {
+        // ------------------------------------------------------------ MMA issuer (one thread)
+        if (lane == 0) {
+            constexpr uint32_t kQPanelStep = (128 * 64 * 2) >> 4, kKPanelStep = (64 * 64 * 2) >> 4, kKStep = 32 >> 4;
+            // K / V^T stage of an item: a new one only when the key block changes (kvn counts the loads so far)
+            int kvn_s = -1, kvn_pv = -1;
+            uint32_t col_s = 0xffffffffu, col_pv = 0xffffffffu;
+            auto issue_s = [&](int i) -> bool {
+                const int st = i % kGatherStages, ph = (i / kGatherStages) & 1;
+                const uint32_t col = item_at(i).x;
+                if (col != col_s) { col_s = col; ++kvn_s; }
+                const int kst = kvn_s % kGatherStages;
+                if (!tc::mbar_wait(&sm.q_full[st], ph, abort_flag)) return false;
+                if (!tc::mbar_wait(&sm.kv_full[kst], (kvn_s / kGatherStages) & 1, abort_flag)) return false;
+                tc::tc_fence_after_sync();
+                const uint32_t q_lo = tc::smem_desc_lo_sw128(smem_u32(&sm.q[st][0][0][0]));
+                const uint32_t k_lo = tc::smem_desc_lo_sw128(smem_u32(&sm.k[kst][0][0][0]));
+                const uint32_t dst = tbase + (i & 1) * 256;
+#pragma unroll
+                for (int ks = 0; ks < kQKSteps; ++ks) {
+                    const uint32_t qo = (ks >> 2) * kQPanelStep + (ks & 3) * kKStep, ko = (ks >> 2) * kKPanelStep + (ks & 3) * kKStep;
+                    tc::umma_ss(dst, tc::smem_desc_from_halves(q_lo + qo, tc::kSmemDescHiSw128),
+                                tc::smem_desc_from_halves(k_lo + ko, tc::kSmemDescHiSw128), kIdescS, ks > 0);
+                }
+                tc::umma_commit(&sm.s_full[i & 1]);
+                tc::umma_commit(&sm.q_empty[st]);                      // the Q tile is free once these MMAs have run
+                return true;
+            };
+            bool ok = issue_s(0);
+            for (int i = 0; ok && i < my_items; ++i) {
+                // S of the next item (other TMEM set; its P of two items ago was consumed by an earlier MMA of this thread)
+                if (i + 1 < my_items && !(ok = issue_s(i + 1))) break;
+                if (!(ok = tc::mbar_wait(&sm.p_full[i & 1], (i >> 1) & 1, abort_flag))) break;
+                tc::tc_fence_after_sync();
+                const uint32_t col = item_at(i).x;
+                if (col != col_pv) { col_pv = col; ++kvn_pv; }
+                const int kst = kvn_pv % kGatherStages;
+                const uint32_t v_lo = tc::smem_desc_lo_sw128(smem_u32(&sm.v[kst][0][0]));
+                const uint32_t set = tbase + (i & 1) * 256;
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
+                    tc::umma_ts(set + 64, set + ks * 8, tc::smem_desc_from_halves(v_lo + ks * kKStep, tc::kSmemDescHiSw128), kIdescO, ks > 0);
+                tc::umma_commit(&sm.o_full[i & 1]);
+                // the stage is free after the last item of its key block
+                if (i + 1 == my_items || item_at(i + 1).x != col) tc::umma_commit(&sm.kv_empty[kst]);
+            }
+        }
+    } else if (warp == 13) {
+        // ------------------------------------------------------------ TMA producer of K / V^T blocks
+        if (lane == 0) {
+            int kvn = -1;
+            uint32_t col_prev = 0xffffffffu;
+            for (int i = 0; i < my_items; ++i) {
+                const uint32_t col = item_at(i).x;
+                if (col == col_prev) continue;                         // same key block as the item before: tiles stay
+                col_prev = col;
+                ++kvn;
+                const int st = kvn % kGatherStages;
+                const int bg = (int)(col / (uint32_t)ws.n_cols), blk = (int)(col - (uint32_t)bg * (uint32_t)ws.n_cols);
+                if (!tc::mbar_wait(&sm.kv_empty[st], ((kvn / kGatherStages) & 1) ^ 1, abort_flag)) break;
+                tc::mbar_arrive_expect_tx(&sm.kv_full[st], kKVBytes);
+                for (int p = 0; p < kPanels; ++p)
+                    tc::tma_load_2d(&sm.k[st][p][0][0], &tmK, p * 64, bg * g.S_cap + blk * kBlockTok, &sm.kv_full[st]);
+                tc::tma_load_2d(&sm.v[st][0][0], &tmV, 0, (bg * g.n_kv_blocks_cap + blk) * D, &sm.kv_full[st]);
+            }
+        }
     }
     // ---------------------------------------------------------------- teardown
     tc::tc_fence_before_sync();
@@ -552,11 +720,12 @@ __global__ void __launch_bounds__(kGatherThreads, 2) attn_gather_kernel(
         if (sm.abort_flag) atomicExch(status, 6);   // a bounded wait expired
         else atomicAdd(executed_blocks, (unsigned long long)my_items);
     }
-    if (warp == 4) tc::tmem_dealloc<kTmemCols>(tbase);
+    if (warp == 12) tc::tmem_dealloc<512>(tbase);
 }
 
 // ------------------------------------------------------------------------------------------------ merge
-// D/8 threads per row, 16 bytes (8 elements) of the row each.
+// D/8 threads per row, 16 bytes (8 elements) of the row each.  The partials are folded in one pass with a
+// running reference exponent (their loads do not depend on it, so several are in flight per thread).
 template <int D>
 __global__ void __launch_bounds__(256) gather_merge_kernel(Geom g, GatherWs ws, __nv_bfloat16* __restrict__ out) {
     if (ws.ctrl[0] == 0u) return;
@@ -564,44 +733,58 @@ __global__ void __launch_bounds__(256) gather_merge_kernel(Geom g, GatherWs ws, 
     const int sub = threadIdx.x % kLanes;
     const int win = g.S - g.pos_begin;
     const long long n_rows = (long long)g.B * g.Hq * win;
-    const unsigned gmask = kLanes == 32 ? 0xffffffffu : (((1u << kLanes) - 1u) << ((threadIdx.x & 31) / kLanes * kLanes));
     for (long long idx = (long long)blockIdx.x * kRowsPerCta + threadIdx.x / kLanes; idx < n_rows; idx += (long long)gridDim.x * kRowsPerCta) {
         const int bh = (int)(idx / win), pos = g.pos_begin + (int)(idx - (long long)bh * win);
-        if (ws.pair_mode[(size_t)bh * ws.n_pairs_cap + pos / kPairRows] == 0u) continue;
         const size_t row = (size_t)bh * g.S_cap + pos;
-        const uint32_t cnt = ws.row_cnt[row];
-        if (cnt == 0u) continue;                                   // also every slot that holds no token
-        const uint32_t ptr = ws.row_ptr[row];
-        const float2 loc = ws.ml_local[row];
-        float M = loc.x;
-        for (uint32_t i = sub; i < cnt; i += kLanes) M = fmaxf(M, ws.part_ml[ptr + i].x);
-#pragma unroll
-        for (int d = 1; d < kLanes; d <<= 1) M = fmaxf(M, __shfl_xor_sync(gmask, M, d));
+        // everything that does not depend on the row's count is requested first (one round of memory latency)
+        const uint32_t cnt = __ldg(ws.row_cnt + row);              // 0: a pair on the union path, or a slot without token
+        const uint32_t ptr = __ldg(ws.row_ptr + row);
+        const float2 loc = __ldg(ws.ml_local + row);
+        if (cnt == 0u) continue;
         const int b = bh / g.Hq, h = bh - b * g.Hq;
         uint4* dst = reinterpret_cast<uint4*>(out + (io_row(g, b, pos) * g.Hq + h) * D) + sub;
+        const uint4 own = *dst;
+        const uint4* src = reinterpret_cast<const uint4*>(ws.part_o) + sub;
         float acc[8];
-        float W = loc.y * exp2f(loc.x - M);
+        float M = loc.x, W = loc.y;                                // the local range always has a visible key
         {
-            const uint4 v = *dst;
-            const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+            const uint32_t u[4] = {own.x, own.y, own.z, own.w};
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 acc[2 * k] = W * __uint_as_float(u[k] << 16);
                 acc[2 * k + 1] = W * __uint_as_float(u[k] & 0xffff0000u);
             }
         }
-        const uint4* src = reinterpret_cast<const uint4*>(ws.part_o + (size_t)ptr * D) + sub;
-#pragma unroll 4
-        for (uint32_t i = 0; i < cnt; ++i) {
-            const float2 ml = ws.part_ml[ptr + i];
-            const float w = ml.y * exp2f(ml.x - M);               // 0 for a partial without a visible key
-            const uint4 v = __ldg(src + (size_t)i * kLanes);
-            const uint32_t u[4] = {v.x, v.y, v.z, v.w};
-            W += w;
+        for (uint32_t i0 = 0; i0 < cnt; i0 += 4) {
+            // four partials at a time: indices, then (m, l) and data of all four, then the arithmetic
+            uint32_t e[4];
+            float2 ml[4];
+            uint4 v[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) e[k] = i0 + k < cnt ? __ldg(ws.row_slots + ptr + i0 + k) : 0xffffffffu;
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                acc[2 * k] = fmaf(w, __uint_as_float(u[k] << 16), acc[2 * k]);
-                acc[2 * k + 1] = fmaf(w, __uint_as_float(u[k] & 0xffff0000u), acc[2 * k + 1]);
+                ml[k] = make_float2(0.f, 0.f);
+                v[k] = make_uint4(0u, 0u, 0u, 0u);
+                if (e[k] != 0xffffffffu) {
+                    ml[k] = __ldg(ws.part_ml + e[k]);
+                    v[k] = __ldg(src + (size_t)e[k] * kLanes);
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                if (ml[k].y > 0.f) {                               // a partial without a visible key has sum 0
+                    const uint32_t u[4] = {v[k].x, v[k].y, v[k].z, v[k].w};
+                    const float Mn = fmaxf(M, ml[k].x);
+                    const float so = exp2f(M - Mn), w = ml[k].y * exp2f(ml[k].x - Mn);
+                    M = Mn;
+                    W = fmaf(W, so, w);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        acc[2 * q] = fmaf(w, __uint_as_float(u[q] << 16), acc[2 * q] * so);
+                        acc[2 * q + 1] = fmaf(w, __uint_as_float(u[q] & 0xffff0000u), acc[2 * q + 1] * so);
+                    }
+                }
             }
         }
         const float inv = 1.f / W;
