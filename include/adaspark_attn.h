@@ -300,10 +300,12 @@ adaspark_status_t adaspark_attn_set_prefill_kernel(adaspark_attn_t *handle, int3
  * on the device, per pair: gathered iff (row, key block) entries of the pair's rows <= pairs_per_block *
  * key blocks in the pair's union.  pairs_per_block = 0 switches the path off (every pair takes the union
  * path); a huge value forces it for every pair with a selected cube.  budget_bytes bounds the workspace
- * the path may use for its partial results (2*head_dim + 24 bytes per entry, at most 32 entries per query
- * row); if the pairs that qualify need more, all pairs take the union path in that call.  The budget
- * sizes the forward workspace: set it before _partition (ERR_INVALID_ARG afterwards); the threshold may
- * change at any time.  Defaults: 20 entries per block, 8 GiB.  Outputs agree with the union path within
+ * the path may use for its partial results (2*head_dim + 24 bytes per entry; _partition reserves
+ * min(budget, what pairs_per_block lets the pairs of the partition produce, 128 entries per query row));
+ * if the pairs that qualify in a call need more, all pairs take the union path in that call.  Budget and
+ * threshold size the forward workspace: set them before _partition (a different budget afterwards is
+ * ERR_INVALID_ARG; the threshold may still change, the reserved capacity does not).  Defaults: 30 entries
+ * per block (gathering pays up to about 44 on a B200), 16 GiB.  Outputs agree with the union path within
  * bf16 rounding of the partial results; the selection is the same. */
 adaspark_status_t adaspark_attn_set_gather(adaspark_attn_t *handle, float pairs_per_block,
                                            uint64_t budget_bytes);

@@ -37,6 +37,7 @@ struct adaspark_attn {
         fw_gpartml_off, fw_total;
     // query-gather path of the prefill: capacity in (row, key block) entries, decision threshold, byte budget
     uint32_t gather_cap;
+    int gather_windows;
     float gather_pairs_per_block;
     uint64_t gather_budget;
     size_t dc_status_off, dc_bitmap_off, dc_items_off, dc_nitems_off, dc_partial_off, dc_total;
@@ -57,9 +58,10 @@ constexpr int kExactCtas = 296;   // CTAs of the fp64 selection kernel (its scra
 // query-gather path: pairs of query tiles take it when their rows' (row, key block) entries are at most this
 // many per key block of the pair's union (measured break-even on a B200, see the attention profile), and the
 // partial results of all such pairs must fit this many bytes of workspace
-constexpr float kGatherDefaultPairsPerBlock = 20.f;
-constexpr uint64_t kGatherDefaultBudget = 8ull << 30;
+constexpr float kGatherDefaultPairsPerBlock = 30.f;
+constexpr uint64_t kGatherDefaultBudget = 16ull << 30;
 constexpr uint64_t kGatherEntriesPerRow = 128;
+constexpr size_t kGatherWindowBytes = 40u << 20;
 size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 
 adaspark_status_t fail(adaspark_attn* h, adaspark_status_t st, const char* fmt, ...) {
@@ -217,7 +219,14 @@ adaspark_status_t adaspark_attn_partition(adaspark_attn_t* h, int32_t batch, int
     h->fw_headmax_off = off; off = align_up(off + (size_t)batch * Hkv * 4);
     h->fw_valid_off = off; off = align_up(off + (size_t)(S_cap / kBlockTok) * 2 * 4);   // which slots of a block hold a token
     const size_t n_cols = (size_t)(S_v + kBlockTok - 1) / kBlockTok;                     // key blocks that hold video
-    h->fw_gcol_off = off; off = align_up(off + (size_t)batch * Hkv * n_cols * 2 * kGatherReplicas * 4);   // entry counts and fill cursors (zeroed per call)
+    // query-gather path: the rows are cut into windows whose slice of Q (all heads) is about a third of the L2
+    {
+        const size_t q_bytes = (size_t)batch * Hq * S_cap * D * 2;
+        size_t w = (q_bytes + kGatherWindowBytes - 1) / kGatherWindowBytes;
+        h->gather_windows = (int)(w < 1 ? 1 : (w > 16 ? 16 : w));
+    }
+    const size_t n_lists = (size_t)h->gather_windows * batch * Hkv;
+    h->fw_gcol_off = off; off = align_up(off + n_lists * n_cols * 2 * kGatherReplicas * 4);   // entry counts and fill cursors (zeroed per call)
     h->fw_mask_off = off; off = align_up(off + (size_t)batch * Hq * n_tiles_cap * n_words * kTileRows * 4);
     h->fw_union_off = off; off = align_up(off + (size_t)batch * Hq * n_tiles_cap * n_words * 4);
     h->fw_fallback_off = off; off = align_up(off + (size_t)batch * Hq * n_tiles_cap * kTileRows * 4);
@@ -232,13 +241,16 @@ adaspark_status_t adaspark_attn_partition(adaspark_attn_t* h, int32_t batch, int
         const size_t rows_cap = (size_t)batch * Hq * S_cap, n_pairs_cap = ((size_t)S_cap + 255) / 256;
         const uint64_t per_entry = 2ull * D + 16ull + 8ull;      // partial output + (m, l) + entry
         uint64_t cap = h->gather_budget / per_entry;
-        if (cap > rows_cap * kGatherEntriesPerRow) cap = rows_cap * kGatherEntriesPerRow;
+        // a pair qualifies with at most threshold x (key blocks of the video) entries, i.e. threshold x n_cols / 256 per row
+        double per_row = std::ceil((double)h->gather_pairs_per_block * (double)n_cols / 256.0);
+        if (!(per_row < (double)kGatherEntriesPerRow)) per_row = (double)kGatherEntriesPerRow;
+        if ((double)cap > (double)rows_cap * per_row) cap = (uint64_t)((double)rows_cap * per_row);
         if (cap > 0xfffffff0ull) cap = 0xfffffff0ull;
         h->gather_cap = (uint32_t)cap;
         h->fw_gpair_off = off; off = align_up(off + (size_t)batch * Hq * n_pairs_cap * 3 * 4);
         h->fw_grow_off = off; off = align_up(off + (cap ? rows_cap * 2 * 4 : 0));
         h->fw_gml_off = off; off = align_up(off + (cap ? rows_cap * 8 : 0));
-        h->fw_gitems_off = off; off = align_up(off + (cap ? align_up(((size_t)batch * Hkv * n_cols * (kGatherReplicas + 2) + 2) * 4) + ((size_t)batch * Hkv * n_cols + cap / 128 + 1) * 16 : 0));
+        h->fw_gitems_off = off; off = align_up(off + (cap ? align_up((n_lists * n_cols * (kGatherReplicas + 2) + 2) * 4) + (n_lists * n_cols + cap / 128 + 1) * 16 : 0));
         h->fw_gentries_off = off; off = align_up(off + (size_t)cap * 8);
         h->fw_gparto_off = off; off = align_up(off + (size_t)cap * D * 2);
         h->fw_gpartml_off = off; off = align_up(off + (size_t)cap * 8);
@@ -450,7 +462,9 @@ adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* 
         GatherWs gw;
         std::memset(&gw, 0, sizeof(gw));
         if (gather) {
-            const size_t n_cols = (size_t)(g.S_v + kBlockTok - 1) / kBlockTok, n_col_all = (size_t)g.B * g.Hkv * n_cols;
+            const size_t n_cols = (size_t)(g.S_v + kBlockTok - 1) / kBlockTok;
+            const size_t n_lists = (size_t)h->gather_windows * g.B * g.Hkv, n_col_all = n_lists * n_cols;
+            const int n_pairs_win = (g.S + kPairRows - 1) / kPairRows - g.pos_begin / kPairRows;
             const size_t rows_cap = (size_t)g.B * g.Hq * g.S_cap, n_pairs_cap = ((size_t)g.S_cap + 255) / 256;
             const size_t n_pair_all = (size_t)g.B * g.Hq * n_pairs_cap;
             gw.ctrl = &hdr->gather_entries;
@@ -472,6 +486,8 @@ adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* 
             gw.ml_local = (float2*)(ws + h->fw_gml_off);
             gw.cap_entries = h->gather_cap;
             gw.n_cols = (int)n_cols;
+            gw.n_lists = (int)n_lists;
+            gw.pairs_per_window = (n_pairs_win + h->gather_windows - 1) / h->gather_windows;
             gw.n_pairs_cap = (int)n_pairs_cap;
             gw.pairs_per_block = h->gather_pairs_per_block;
             gather_count_kernel<<<grid, 256, 0, st>>>(g, gw, tile_mask, tile_union);

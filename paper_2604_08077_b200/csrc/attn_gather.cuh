@@ -32,7 +32,7 @@
 namespace adaspark {
 
 constexpr int kGatherItemRows = 128;
-constexpr int kGatherReplicas = 8;
+constexpr int kGatherReplicas = 1;
 constexpr uint32_t kEntryPosMask = 0x1fffffu;   // 21 bits of cube-major position (caches hold at most 2^21 rows)
 
 // Pointers into the forward workspace and sizes (all filled by the host).
@@ -60,6 +60,10 @@ struct GatherWs {
     float2* ml_local;      // [B*Hq*S_cap] the same for the local range, written by the tile kernel
     uint32_t cap_entries;
     int n_cols;            // key blocks that hold video slots: ceil(S_v / 64)
+    int n_lists;           // entry lists per key block column set: windows x B x Hkv (each of n_cols lists)
+    int pairs_per_window;  // The query rows are cut into windows of this many pairs of tiles and every (window,
+                           // batch, kv head, key block) has its own entry list: the items of a window gather from a
+                           // slice of Q that stays in L2, and a row's partial results lie close together.
     int n_pairs_cap;       // pairs of query tiles per (b, head): ceil(S_cap / 256)
     float pairs_per_block; // decision threshold (entries per union block)
 };
@@ -166,7 +170,8 @@ __global__ void __launch_bounds__(256) gather_count_kernel(Geom g, GatherWs ws, 
     if (!s_mode || !tile_ok) return;
     // entries per key block: the warp's 32 x 32 bits of a word are transposed, lane j then counts the rows that
     // selected cube 32 w + j and adds them to the cube's block(s)
-    uint32_t* col_cnt = ws.col_cnt + ((size_t)(blockIdx.x % kGatherReplicas) * g.B * g.Hkv + (it.b * g.Hkv + it.gk)) * ws.n_cols;
+    const int win = (it.pair - g.pos_begin / kPairRows) / ws.pairs_per_window;
+    uint32_t* col_cnt = ws.col_cnt + ((size_t)(blockIdx.x % kGatherReplicas) * ws.n_lists + ((size_t)win * g.B + it.b) * g.Hkv + it.gk) * ws.n_cols;
     for (int w0 = 0; w0 < it.n_w; w0 += 4) {
         uint32_t wd[4];
 #pragma unroll
@@ -259,7 +264,7 @@ __global__ void __launch_bounds__(1024) gather_scan_kernel(Geom g, GatherWs ws) 
         ws.ctrl[2] = s;
     }
     // ---- key blocks: offsets of their entry lists (and of every counter set's share) and of their work items
-    const int n_cols_all = g.B * g.Hkv * ws.n_cols;
+    const int n_cols_all = ws.n_lists * ws.n_cols;
     uint32_t ent_carry = 0, item_carry = 0;
     for (int base = 0; base < n_cols_all; base += 1024) {
         const int col = base + tid;
@@ -298,7 +303,7 @@ __global__ void __launch_bounds__(1024) gather_scan_kernel(Geom g, GatherWs ws) 
 // Work items of every key block: chunks of up to 128 entries of its list.  One warp per block.
 __global__ void __launch_bounds__(256) gather_items_kernel(Geom g, GatherWs ws) {
     if (ws.ctrl[0] == 0u) return;
-    const int n_cols_all = g.B * g.Hkv * ws.n_cols;
+    const int n_cols_all = ws.n_lists * ws.n_cols;
     const int lane = threadIdx.x & 31;
     for (int col = blockIdx.x * 8 + (threadIdx.x >> 5); col < n_cols_all; col += gridDim.x * 8) {
         const uint32_t first = ws.col_off[col], n = ws.col_off[col + 1] - first, ib = ws.col_item[col];
@@ -334,7 +339,8 @@ __global__ void __launch_bounds__(256) gather_fill_kernel(Geom g, GatherWs ws, c
     if (pos < g.S_cap) ws.row_ptr[bh * g.S_cap + pos] = ptr;
     if (!tile_ok) return;
     const uint32_t* my = tile_mask + mask_index(g, it.b, it.h, tile, 0, r);
-    const size_t colbase = ((size_t)(blockIdx.x % kGatherReplicas) * g.B * g.Hkv + (it.b * g.Hkv + it.gk)) * ws.n_cols;
+    const int win = (it.pair - g.pos_begin / kPairRows) / ws.pairs_per_window;
+    const size_t colbase = ((size_t)(blockIdx.x % kGatherReplicas) * ws.n_lists + ((size_t)win * g.B + it.b) * g.Hkv + it.gk) * ws.n_cols;
     const uint32_t ent_x = (uint32_t)pos | ((uint32_t)(it.h - it.gk * g.G) << 21);
     const uint32_t lt_mask = (1u << lane) - 1u;
     // Four words per step.  After the transposition lane j holds the rows of the warp that selected cube 32 w + j;
@@ -403,14 +409,18 @@ __global__ void __launch_bounds__(256) gather_fill_kernel(Geom g, GatherWs ws, c
 // TMEM: consumer c owns columns [256 c, 256 c + 64) for S (P overwrites the first 32) and
 // [256 c + 64, 256 c + 64 + D) for O.
 constexpr int kGatherThreads = 512;
-constexpr int kGatherStages = 3;
+constexpr int kGatherRun = 16;          // consecutive items per CTA turn
+constexpr int kGatherStages = 3;        // Q tiles in flight
+constexpr int kGatherKvStages = 2;      // K / V^T tiles in flight
+constexpr int kGatherOutPitch = 144;    // bytes per row of the output staging (128 + 16: conflict-free 16-byte accesses)
 
 template <int D>
 struct GatherSmem {
     __nv_bfloat16 q[kGatherStages][D / 64][128][64];   // [stage][d panel][gathered row][64 d], 128-byte swizzle
-    __nv_bfloat16 k[kGatherStages][D / 64][64][64];    // [stage][d panel][key][64 d]
-    __nv_bfloat16 v[kGatherStages][D][64];             // [stage][d][64 keys]  (V^T)
-    uint64_t q_full[kGatherStages], q_empty[kGatherStages], kv_full[kGatherStages], kv_empty[kGatherStages];
+    __nv_bfloat16 k[kGatherKvStages][D / 64][64][64];  // [stage][d panel][key][64 d]
+    __nv_bfloat16 v[kGatherKvStages][D][64];           // [stage][d][64 keys]  (V^T)
+    unsigned char out_stage[8][32 * kGatherOutPitch];  // per consumer warp: 32 rows x 64 output columns (bf16)
+    uint64_t q_full[kGatherStages], q_empty[kGatherStages], kv_full[kGatherKvStages], kv_empty[kGatherKvStages];
     uint64_t s_full[2], p_full[2], o_full[2];
     uint32_t tmem_base;
     int abort_flag;
@@ -430,18 +440,22 @@ __global__ void __launch_bounds__(kGatherThreads, 1) attn_gather_kernel(
     constexpr uint32_t kKVBytes = 64 * D * 2 * 2;
 
     const uint32_t n_items = ws.ctrl[1];
-    if (ws.ctrl[0] == 0u || blockIdx.x >= n_items) return;       // the path is off, or fewer items than CTAs
-    // a contiguous run of items per CTA: consecutive items mostly share their key block, whose K / V^T tiles
-    // then stay in shared memory
-    const uint32_t per = n_items / gridDim.x, rem = n_items - per * gridDim.x;
-    const uint32_t item0 = blockIdx.x * per + min((uint32_t)blockIdx.x, rem);
-    const int my_items = (int)(per + (blockIdx.x < rem ? 1u : 0u));
+    if (ws.ctrl[0] == 0u || (size_t)blockIdx.x * kGatherRun >= n_items) return;   // the path is off, or fewer runs than CTAs
+    // Items are dealt to the CTAs in runs of kGatherRun: inside a run consecutive items mostly share their key
+    // block, whose K / V^T tiles then stay in shared memory; across the grid all CTAs work on neighbouring runs,
+    // i.e. on the same window of query rows, whose slice of Q stays in L2.
+    const uint32_t n_runs = (n_items + kGatherRun - 1) / kGatherRun;
+    const uint32_t my_runs = (n_runs - blockIdx.x + gridDim.x - 1) / gridDim.x;
+    const bool has_tail = ((my_runs - 1) * gridDim.x + blockIdx.x) == n_runs - 1;   // the last (possibly short) run is this CTA's
+    const int my_items = (int)(my_runs * kGatherRun - (has_tail ? n_runs * kGatherRun - n_items : 0u));
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     if (tid == 0) {
         for (int i = 0; i < kGatherStages; ++i) {
             tc::mbar_init(&sm.q_full[i], 128);
             tc::mbar_init(&sm.q_empty[i], 1);
+        }
+        for (int i = 0; i < kGatherKvStages; ++i) {
             tc::mbar_init(&sm.kv_full[i], 1);
             tc::mbar_init(&sm.kv_empty[i], 1);
         }
@@ -465,8 +479,10 @@ __global__ void __launch_bounds__(kGatherThreads, 1) attn_gather_kernel(
     tc::tc_fence_after_sync();
     const uint32_t tbase = sm.tmem_base;
     volatile int* abort_flag = &sm.abort_flag;
-    // item i of this CTA: (column = (batch x kv head) * n_cols + key block, first entry, entries, -)
-    auto item_at = [&](int i) -> uint4 { return __ldg(ws.items + item0 + i); };
+    // item i of this CTA: (column = ((window x batch) x kv head) * n_cols + key block, first entry, entries, -)
+    auto item_at = [&](int i) -> uint4 {
+        return __ldg(ws.items + ((size_t)(i / kGatherRun) * gridDim.x + blockIdx.x) * kGatherRun + (i % kGatherRun));
+    };
 
     if (warp < 8) {
         // ------------------------------------------------------------ consumers
@@ -569,70 +585,87 @@ __global__ void __launch_bounds__(kGatherThreads, 1) attn_gather_kernel(
             if (!tc::mbar_wait(&sm.o_full[c], j & 1, abort_flag)) break;
             tc::tc_fence_after_sync();
             const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
-            uint4* dst = reinterpret_cast<uint4*>(ws.part_o + (size_t)(d_cur.y + row) * D);
-            // the output row in rounds of 64 columns (the whole row at once does not fit the register budget of
-            // a 512-thread CTA)
+            // The output rows in rounds of 64 columns.  A thread holds one row, but 32 threads storing 16 bytes to 32
+            // different rows cost the L1 one step per row; so the warp transposes through shared memory and writes its
+            // 32 rows (contiguous in the partial buffer: entry order) as whole 128-byte lines, four rows per
+            // instruction.
+            unsigned char* stage = sm.out_stage[warp];
+            unsigned char* gdst = reinterpret_cast<unsigned char*>(ws.part_o + (size_t)(d_cur.y + (row & ~31)) * D);
+            const int n_warp_rows = min(32, (int)d_cur.z - (row & ~31));          // rows of this warp that hold an entry
 #pragma unroll
             for (int hf = 0; hf < D / 64; ++hf) {
                 uint32_t o[2][32];
                 tc::tmem_ld_32x32(lane_addr + 64 + hf * 64, o[0]);
                 tc::tmem_ld_32x32(lane_addr + 64 + hf * 64 + 32, o[1]);
                 tc::tmem_wait_ld();
-                if (valid) {
 #pragma unroll
-                    for (int cc = 0; cc < 2; ++cc) {
+                for (int cc = 0; cc < 2; ++cc) {
 #pragma unroll
-                        for (int q4 = 0; q4 < 4; ++q4) {
-                            uint4 val;
-                            val.x = pack_bf16x2(__uint_as_float(o[cc][8 * q4 + 0]) * inv, __uint_as_float(o[cc][8 * q4 + 1]) * inv);
-                            val.y = pack_bf16x2(__uint_as_float(o[cc][8 * q4 + 2]) * inv, __uint_as_float(o[cc][8 * q4 + 3]) * inv);
-                            val.z = pack_bf16x2(__uint_as_float(o[cc][8 * q4 + 4]) * inv, __uint_as_float(o[cc][8 * q4 + 5]) * inv);
-                            val.w = pack_bf16x2(__uint_as_float(o[cc][8 * q4 + 6]) * inv, __uint_as_float(o[cc][8 * q4 + 7]) * inv);
-                            dst[(hf * 2 + cc) * 4 + q4] = val;
-                        }
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        uint4 val;
+                        val.x = pack_bf16x2(__uint_as_float(o[cc][8 * q4 + 0]) * inv, __uint_as_float(o[cc][8 * q4 + 1]) * inv);
+                        val.y = pack_bf16x2(__uint_as_float(o[cc][8 * q4 + 2]) * inv, __uint_as_float(o[cc][8 * q4 + 3]) * inv);
+                        val.z = pack_bf16x2(__uint_as_float(o[cc][8 * q4 + 4]) * inv, __uint_as_float(o[cc][8 * q4 + 5]) * inv);
+                        val.w = pack_bf16x2(__uint_as_float(o[cc][8 * q4 + 6]) * inv, __uint_as_float(o[cc][8 * q4 + 7]) * inv);
+                        *reinterpret_cast<uint4*>(stage + lane * kGatherOutPitch + (cc * 4 + q4) * 16) = val;
                     }
                 }
+                __syncwarp();
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int r = j * 4 + (lane >> 3), ch = lane & 7;
+                    const uint4 val = *reinterpret_cast<const uint4*>(stage + r * kGatherOutPitch + ch * 16);
+                    if (r < n_warp_rows) __stcs(reinterpret_cast<uint4*>(gdst + (size_t)r * (2 * D) + hf * 128 + ch * 16), val);   // written once, read once: keep it from displacing Q in L2
+                }
+                __syncwarp();
             }
             tc::tc_fence_before_sync();
             if (valid) {
-                ws.part_ml[d_cur.y + row] = make_float2(m_ref, l_sum);
+                __stcs(ws.part_ml + d_cur.y + row, make_float2(m_ref, l_sum));
             }
             d_cur = d_nxt;
             ent = e_nxt;
         }
     } else if (warp < 12) {
         // ------------------------------------------------------------ gather producers
-        // lanes (2k, 2k+1) copy the two 16-byte halves of a 32-byte piece; a warp instruction covers 16 rows,
-        // the warpgroup 64 rows per pass: two passes of D/16 pieces per item
+        // A row of Q is 2 D bytes = 2 D / 16 pieces of 16 bytes; consecutive lanes copy consecutive pieces, so a warp
+        // instruction covers whole 128-byte lines of one or two rows (16 rows x 32 bytes per instruction cost the L1 one
+        // step per row and made this kernel L1-bound).  The warpgroup copies 128 / kRowsPerPass rows per pass.
+        constexpr int kPieces = D / 8;                               // 16-byte pieces per row
+        constexpr int kRowsPerPass = 128 / kPieces;                  // rows the 128 producer threads cover per pass
         const int pt = tid - 256;                                  // 0..127
-        const int half = pt & 1, rsub = pt >> 1;                   // row inside the pass: 0..63
+        const int piece = pt % kPieces, rsub = pt / kPieces;
+        constexpr int kPasses = 128 / kRowsPerPass;
         uint4 d_cur = item_at(0);
+        // the entries of the next item are requested while the rows of this one are copied: a load of the entry
+        // right before its copy left this warpgroup waiting on L2 latency once per pass
+        uint32_t e_cur[kPasses], e_nxt[kPasses];
+#pragma unroll
+        for (int ps = 0; ps < kPasses; ++ps) e_cur[ps] = (ps * kRowsPerPass + rsub < (int)d_cur.z) ? __ldg(ws.entries + d_cur.y + ps * kRowsPerPass + rsub) : 0u;
         bool ok = true;
         for (int i = 0; i < my_items; ++i) {
             const int st = i % kGatherStages;
             uint4 d_nxt = make_uint4(0u, 0u, 0u, 0u);
             if (i + 1 < my_items) d_nxt = item_at(i + 1);
             const int n = (int)d_cur.z;
-            uint32_t e[2];
 #pragma unroll
-            for (int ps = 0; ps < 2; ++ps) e[ps] = (ps * 64 + rsub < n) ? __ldg(ws.entries + d_cur.y + ps * 64 + rsub) : 0u;
+            for (int ps = 0; ps < kPasses; ++ps) e_nxt[ps] = (ps * kRowsPerPass + rsub < (int)d_nxt.z) ? __ldg(ws.entries + d_nxt.y + ps * kRowsPerPass + rsub) : 0u;
             if (!(ok = tc::mbar_wait(&sm.q_empty[st], ((i / kGatherStages) & 1) ^ 1, abort_flag))) break;
-            const int bg = (int)(d_cur.x / (uint32_t)ws.n_cols);
+            const int bg = (int)(d_cur.x / (uint32_t)ws.n_cols) % (g.B * g.Hkv);
             const int b = bg / g.Hkv, gk = bg - b * g.Hkv;
             const size_t head0 = (size_t)(b * g.Hq + gk * g.G);
-            unsigned char* qbase = reinterpret_cast<unsigned char*>(&sm.q[st][0][0][0]);
+            unsigned char* qbase = reinterpret_cast<unsigned char*>(&sm.q[st][0][0][0]) + (piece >> 3) * (128 * 128);
 #pragma unroll
-            for (int ps = 0; ps < 2; ++ps) {
-                const int row = ps * 64 + rsub;
+            for (int ps = 0; ps < kPasses; ++ps) {
+                const int row = ps * kRowsPerPass + rsub;
                 if (row < n) {
-                    const __nv_bfloat16* src = q_cube + ((head0 + ((e[ps] >> 21) & 15u)) * g.S_cap + (e[ps] & kEntryPosMask)) * D;
-#pragma unroll
-                    for (int pc = 0; pc < kPairsPerRow; ++pc) {
-                        const int ch = pc * 2 + half;                  // 16-byte chunk of the row
-                        cp_async_16(qbase + (ch >> 3) * (128 * 128) + sw128(row, ch & 7), src + ch * 8);
-                    }
+                    const uint32_t e = e_cur[ps];
+                    const __nv_bfloat16* src = q_cube + ((head0 + ((e >> 21) & 15u)) * g.S_cap + (e & kEntryPosMask)) * D;
+                    cp_async_16(qbase + sw128(row, piece & 7), src + piece * 8);
                 }
             }
+#pragma unroll
+            for (int ps = 0; ps < kPasses; ++ps) e_cur[ps] = e_nxt[ps];
             cp_async_commit();
             if (i > 0) {                                             // the previous item has landed
                 cp_async_wait<1>();
@@ -657,9 +690,9 @@ __global__ void __launch_bounds__(kGatherThreads, 1) attn_gather_kernel(
                 const int st = i % kGatherStages, ph = (i / kGatherStages) & 1;
                 const uint32_t col = item_at(i).x;
                 if (col != col_s) { col_s = col; ++kvn_s; }
-                const int kst = kvn_s % kGatherStages;
+                const int kst = kvn_s % kGatherKvStages;
                 if (!tc::mbar_wait(&sm.q_full[st], ph, abort_flag)) return false;
-                if (!tc::mbar_wait(&sm.kv_full[kst], (kvn_s / kGatherStages) & 1, abort_flag)) return false;
+                if (!tc::mbar_wait(&sm.kv_full[kst], (kvn_s / kGatherKvStages) & 1, abort_flag)) return false;
                 tc::tc_fence_after_sync();
                 const uint32_t q_lo = tc::smem_desc_lo_sw128(smem_u32(&sm.q[st][0][0][0]));
                 const uint32_t k_lo = tc::smem_desc_lo_sw128(smem_u32(&sm.k[kst][0][0][0]));
@@ -682,7 +715,7 @@ __global__ void __launch_bounds__(kGatherThreads, 1) attn_gather_kernel(
                 tc::tc_fence_after_sync();
                 const uint32_t col = item_at(i).x;
                 if (col != col_pv) { col_pv = col; ++kvn_pv; }
-                const int kst = kvn_pv % kGatherStages;
+                const int kst = kvn_pv % kGatherKvStages;
                 const uint32_t v_lo = tc::smem_desc_lo_sw128(smem_u32(&sm.v[kst][0][0]));
                 const uint32_t set = tbase + (i & 1) * 256;
 #pragma unroll
@@ -703,9 +736,10 @@ __global__ void __launch_bounds__(kGatherThreads, 1) attn_gather_kernel(
                 if (col == col_prev) continue;                         // same key block as the item before: tiles stay
                 col_prev = col;
                 ++kvn;
-                const int st = kvn % kGatherStages;
-                const int bg = (int)(col / (uint32_t)ws.n_cols), blk = (int)(col - (uint32_t)bg * (uint32_t)ws.n_cols);
-                if (!tc::mbar_wait(&sm.kv_empty[st], ((kvn / kGatherStages) & 1) ^ 1, abort_flag)) break;
+                const int st = kvn % kGatherKvStages;
+                const int list = (int)(col / (uint32_t)ws.n_cols), blk = (int)(col - (uint32_t)list * (uint32_t)ws.n_cols);
+                const int bg = list % (g.B * g.Hkv);
+                if (!tc::mbar_wait(&sm.kv_empty[st], ((kvn / kGatherKvStages) & 1) ^ 1, abort_flag)) break;
                 tc::mbar_arrive_expect_tx(&sm.kv_full[st], kKVBytes);
                 for (int p = 0; p < kPanels; ++p)
                     tc::tma_load_2d(&sm.k[st][p][0][0], &tmK, p * 64, bg * g.S_cap + blk * kBlockTok, &sm.kv_full[st]);
@@ -767,8 +801,8 @@ __global__ void __launch_bounds__(256) gather_merge_kernel(Geom g, GatherWs ws, 
                 ml[k] = make_float2(0.f, 0.f);
                 v[k] = make_uint4(0u, 0u, 0u, 0u);
                 if (e[k] != 0xffffffffu) {
-                    ml[k] = __ldg(ws.part_ml + e[k]);
-                    v[k] = __ldg(src + (size_t)e[k] * kLanes);
+                    ml[k] = __ldcs(ws.part_ml + e[k]);
+                    v[k] = __ldcs(src + (size_t)e[k] * kLanes);
                 }
             }
 #pragma unroll
