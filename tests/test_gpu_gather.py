@@ -121,12 +121,12 @@ def test_decision_rule_per_pair():
 
 def test_set_gather_arguments():
     wl = inputs.small_prefill(seed=35)
-    eng = pu.make_engine(wl)
+    eng = pu.make_engine(wl, gather=20.0, gather_budget=1 << 30)
     with pytest.raises(binding.AdasparkError):
-        binding.adaspark_attn_set_gather(eng.handle, -1.0, 8 << 30)
+        binding.adaspark_attn_set_gather(eng.handle, -1.0, 1 << 30)
     with pytest.raises(binding.AdasparkError):           # the budget sizes the workspace: not after partition
-        binding.adaspark_attn_set_gather(eng.handle, 20.0, 1 << 30)
-    binding.adaspark_attn_set_gather(eng.handle, 5.0, 8 << 30)   # the threshold alone may change
+        binding.adaspark_attn_set_gather(eng.handle, 20.0, 2 << 30)
+    binding.adaspark_attn_set_gather(eng.handle, 5.0, 1 << 30)   # the threshold alone may change
 
 
 def test_forced_gather_chunked_prefill():
