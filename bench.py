@@ -76,7 +76,21 @@ class ClockSampler:
     def __init__(self, index: int):
         self.index = index
         self.proc = None
-        self.lines = []
+        self.lines = []          # (host time of arrival, line)
+        self.t_begin = self.t_end = None
+
+    def wait_first(self, timeout_s: float = 5.0):
+        """nvidia-smi needs a fraction of a second before its first line: wait for it, so that the
+        timed region (tens of milliseconds) is sampled from its start."""
+        t0 = time.time()
+        while self.proc is not None and not self.lines and time.time() - t0 < timeout_s:
+            time.sleep(0.01)
+
+    def begin(self):
+        self.t_begin = time.time()
+
+    def end(self):
+        self.t_end = time.time()
 
     def start(self):
         try:
@@ -91,7 +105,7 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.time(), line.strip()))
 
     def stop(self) -> dict:
         if self.proc is None:
@@ -103,7 +117,15 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in self.lines:
+        lines = self.lines
+        if self.t_begin is not None and self.t_end is not None:
+            # samples taken during the timed region; a region shorter than the sampling period may hold none:
+            # then the samples within a quarter of a second around it
+            inside = [ln for t, ln in lines if self.t_begin <= t <= self.t_end + 0.02]
+            if len(inside) < 2:
+                inside = [ln for t, ln in lines if self.t_begin - 0.25 <= t <= self.t_end + 0.25]
+            lines = [(0.0, ln) for ln in inside]
+        for _, line in lines:
             parts = [x.strip() for x in line.split(",")]
             if len(parts) < 7:
                 continue
@@ -137,7 +159,7 @@ def job_throughput(units_per_rank: float, world: int, ms_max: float) -> float:
     return world * units_per_rank / (ms_max * 1e-3)
 
 
-def timed_steps(step_fn, steps, warmup, flush, dist_barrier):
+def timed_steps(step_fn, steps, warmup, flush, dist_barrier, on_begin=None, on_end=None):
     """W warm-ups, then K steps each bracketed by CUDA events on the current stream, with an L2
     flush (not timed) before every step.  Returns per-step milliseconds."""
     for _ in range(warmup):
@@ -149,6 +171,8 @@ def timed_steps(step_fn, steps, warmup, flush, dist_barrier):
     starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
     ends = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
     extra = []
+    if on_begin:
+        on_begin()
     for i in range(steps):
         flush()
         starts[i].record()
@@ -157,6 +181,8 @@ def timed_steps(step_fn, steps, warmup, flush, dist_barrier):
         if r is not None:
             extra.append(r())
     torch.cuda.synchronize()
+    if on_end:
+        on_end()
     dist_barrier()
     return [s.elapsed_time(e) for s, e in zip(starts, ends)], extra
 
@@ -253,6 +279,50 @@ def cpu_baseline(wl, n_rows=32768):
                       f"{sec:.1f} s; tokens/s = rows / n_q_heads / seconds"}
 
 
+GATHER_DEFAULT_THRESHOLD = 30.0    # the library's default decision threshold of the query-gather path
+SWEEP_GATHER_BUDGET = 32 << 30     # workspace the query-gather path may use on the long-video workloads
+
+def one_config(wx, p, flush, local_rank, n_steps=3, gather=None, budget=SWEEP_GATHER_BUDGET, warmup=3):
+    """One forward configuration timed with stage times: gather None = the library's own per-pair decision
+    (default threshold), 0.0 = union path only."""
+    from paper_2604_08077_b200 import binding
+    e = binding.AdaSAttn(cube=wx.cube, n_q_heads=wx.Hq, n_kv_heads=wx.Hkv, head_dim=wx.D, top_p=p,
+                         device=local_rank)
+    e.set_gather(GATHER_DEFAULT_THRESHOLD if gather is None else gather, budget)
+    e.partition(wx.B, wx.T, wx.H, wx.W, wx.n_text)
+    binding.adaspark_attn_enable_stage_timing(e.handle, True)
+    ox = torch.empty_like(wx.q)
+
+    def stp():
+        e.forward(wx.q, wx.k, wx.v, wx.n_text, out=ox)
+        return lambda: binding.adaspark_attn_get_stage_times(e.handle)
+
+    t, stg = timed_steps(stp, n_steps, warmup, flush, lambda: None)
+    stg = np.asarray(stg).mean(axis=0)
+    hx = e.header()
+    _, _, cnt = e.forward(wx.q, wx.k, wx.v, wx.n_text, out=ox, want_selection=True)
+    torch.cuda.synchronize()
+    sel = int(cnt.sum().item())
+    Cx = wx.C
+    local_x = wx.S_v // Cx * (Cx * (Cx + 1) // 2) + wx.n_text * (wx.n_text + 1) // 2
+    useful = 4.0 * wx.D * (sel * Cx + wx.B * wx.Hq * local_x)
+    executed = float(hx.executed_kv_blocks) * 128 * 64 * wx.D * 4
+    n_pairs = wx.B * wx.Hq * ((wx.S + 255) // 256)
+    rec = {"p": p, "forward_ms": sum(t) / len(t),
+           "stages_ms": {"relayout_pool": float(stg[0]), "score_select": float(stg[1]), "attention": float(stg[2])},
+           "mean_selected_cubes_per_row": sel / (wx.B * wx.Hq * wx.S),
+           "useful_over_executed": useful / max(executed, 1.0),
+           "executed_tflops": executed / (float(stg[2]) * 1e-3) / 1e12,
+           "kv_blocks_per_pair_tile": {"mean": float(hx.executed_kv_blocks) / 2 / n_pairs, "max": int(hx.max_tile_kv_blocks)},
+           "gather": {"pair_tiles": int(hx.gather_pair_tiles), "of_pair_tiles": n_pairs,
+                      "entries": int(hx.gather_entries), "items": int(hx.gather_items)},
+           "fallback_rows": int(hx.fallback_rows), "status": int(hx.status)}
+    e.close()
+    del e, ox, cnt
+    return rec
+
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -268,6 +338,8 @@ def main():
     ap.add_argument("--no-sweep", action="store_true", help="skip the config-3 sweep and config 4")
     ap.add_argument("--decode-batch", type=int, default=16)
     ap.add_argument("--prefill-kernel", type=int, default=None)
+    ap.add_argument("--point", default=None, metavar="SIGMA,P[,BUDGET_GIB[,THRESHOLD]]",
+                    help="time only this point of the config-3 sweep (profiling runs) and print its record")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -296,6 +368,15 @@ def main():
     barrier()
     binding.load()
     peaks = load_peaks()
+    if args.point is not None:
+        f = [float(x) for x in args.point.split(",")]
+        wp = inputs.config3(sigma=f[0], device="cuda")
+        fb = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+        rec = one_config(wp, f[1], lambda: fb.fill_(1), local_rank, n_steps=args.steps, warmup=args.warmup,
+                         budget=int(f[2] * 2**30) if len(f) > 2 else SWEEP_GATHER_BUDGET, gather=f[3] if len(f) > 3 else None)
+        rec["sigma"] = f[0]
+        print(json.dumps({"config3_point": rec}))
+        return
 
     # ------------------------------------------------------------------ prefill (the metric)
     wl = inputs.config2(variant=rank)
@@ -314,17 +395,18 @@ def main():
     def flush():
         flush_buf.fill_(1)
 
+    sampler = ClockSampler(local_rank)
+    sampler.start()                    # early: the first line of nvidia-smi takes a while
     parity = None
     if rank == 0 and not args.no_parity:
         parity = parity_check(wl, eng, q, k, v)
 
     def step():
         eng.forward(q, k, v, wl.n_text, out=out)
-        return lambda: binding.adaspark_attn_get_stage_times(eng.handle)
+        return lambda: binding.adaspark_attn_get_stage_times(eng.handle) + [binding.adaspark_attn_get_attention_kernel_ms(eng.handle)]
 
-    sampler = ClockSampler(local_rank)
-    sampler.start()
-    times, stages = timed_steps(step, args.steps, args.warmup, flush, barrier)
+    sampler.wait_first()
+    times, stages = timed_steps(step, args.steps, args.warmup, flush, barrier, on_begin=sampler.begin, on_end=sampler.end)
     clocks = sampler.stop()
     launches_per_step = eng.launches()
     hdr = eng.header()
@@ -343,10 +425,11 @@ def main():
     useful_flops = 4.0 * wl.D * (sel_total * C + wl.B * wl.Hq * local)
     executed_flops = float(hdr.executed_kv_blocks) * 128 * 64 * wl.D * 4
     dense_flops = 4.0 * wl.D * wl.B * wl.Hq * (wl.S * (wl.S + 1) / 2)
-    st = np.asarray(stages)          # [steps, 4]: relayout, score+select, attention
+    st = np.asarray(stages)          # [steps, 5]: relayout, score+select, attention stage, -, the attention kernel alone
     st_mean = st.mean(axis=0)
     attn_ms = float(st_mean[2])
-    achieved_tflops = executed_flops / (attn_ms * 1e-3) / 1e12
+    attn_kernel_ms = float(st_mean[4])   # the stage also holds the six small kernels of the query-gather decision
+    achieved_tflops = executed_flops / (attn_kernel_ms * 1e-3) / 1e12
     peak_tflops = peaks["bf16_tflops"]
 
     # ------------------------------------------------------------------ end to end (host buffers)
@@ -404,7 +487,7 @@ def main():
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h},
         "gpu_launches": launches_per_step * args.steps,
-        "roofline": {"kernel": "prefill attention", "bound": "tensor", "achieved": achieved_tflops,
+        "roofline": {"kernel": "attn_prefill_tc_kernel (prefill attention)", "kernel_ms": attn_kernel_ms, "bound": "tensor", "achieved": achieved_tflops,
                      "peak": peak_tflops, "unit": "TFLOP/s", "frac": achieved_tflops / peak_tflops,
                      "traffic": profiled_traffic("attn_prefill_tc.cuh", "attn_prefill_tc_kernel_config2.md"),
                      "traffic_unit": "bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum)",
@@ -464,39 +547,6 @@ def main():
     }
 
     # ------------------------------------------------------------------ config 3 sweep and config 4
-    def one_config(wx, p, n_steps=3):
-        e = binding.AdaSAttn(cube=wx.cube, n_q_heads=wx.Hq, n_kv_heads=wx.Hkv, head_dim=wx.D, top_p=p,
-                             device=local_rank)
-        e.partition(wx.B, wx.T, wx.H, wx.W, wx.n_text)
-        binding.adaspark_attn_enable_stage_timing(e.handle, True)
-        ox = torch.empty_like(wx.q)
-
-        def stp():
-            e.forward(wx.q, wx.k, wx.v, wx.n_text, out=ox)
-            return lambda: binding.adaspark_attn_get_stage_times(e.handle)
-
-        t, stg = timed_steps(stp, n_steps, 3, flush, lambda: None)
-        stg = np.asarray(stg).mean(axis=0)
-        hx = e.header()
-        _, _, cnt = e.forward(wx.q, wx.k, wx.v, wx.n_text, out=ox, want_selection=True)
-        torch.cuda.synchronize()
-        sel = int(cnt.sum().item())
-        Cx = wx.C
-        local_x = wx.S_v // Cx * (Cx * (Cx + 1) // 2) + wx.n_text * (wx.n_text + 1) // 2
-        useful = 4.0 * wx.D * (sel * Cx + wx.B * wx.Hq * local_x)
-        executed = float(hx.executed_kv_blocks) * 128 * 64 * wx.D * 4
-        n_pairs = wx.B * wx.Hq * ((wx.S + 255) // 256)
-        rec = {"p": p, "forward_ms": sum(t) / len(t),
-               "stages_ms": {"relayout_pool": float(stg[0]), "score_select": float(stg[1]), "attention": float(stg[2])},
-               "mean_selected_cubes_per_row": sel / (wx.B * wx.Hq * wx.S),
-               "useful_over_executed": useful / max(executed, 1.0),
-               "executed_tflops": executed / (float(stg[2]) * 1e-3) / 1e12,
-               "kv_blocks_per_pair_tile": {"mean": float(hx.executed_kv_blocks) / 2 / n_pairs, "max": int(hx.max_tile_kv_blocks)},
-               "fallback_rows": int(hx.fallback_rows), "status": int(hx.status)}
-        e.close()
-        del e, ox, cnt
-        return rec
-
     if not args.no_sweep and rank == 0:
         try:
             del bitmap, count
@@ -514,9 +564,13 @@ def main():
                     sd3, _ = timed_steps(sdpa3, 3, 3, flush, lambda: None)
                     del q3, k3, v3
                     sdpa_ms = sum(sd3) / len(sd3)
-                recs = {p: one_config(w3, p) for p in (1.0, 0.95, 0.9, 0.7, 0.5)}
+                recs = {p: one_config(w3, p, flush, local_rank) for p in (1.0, 0.95, 0.9, 0.7, 0.5)}
                 for p in (0.5, 0.7, 0.9, 0.95, 1.0):
                     r3 = recs[p]
+                    if r3["gather"]["pair_tiles"] > 0:     # the same point with every pair on the union path
+                        ru = one_config(w3, p, flush, local_rank, n_steps=2, gather=0.0)
+                        r3["union_path_only"] = {"forward_ms": ru["forward_ms"], "attention_ms": ru["stages_ms"]["attention"],
+                                                 "useful_over_executed": ru["useful_over_executed"]}
                     r3["sigma"] = sigma
                     r3["speedup_vs_own_p1"] = recs[1.0]["forward_ms"] / r3["forward_ms"]
                     r3["speedup_vs_torch_sdpa"] = sdpa_ms / r3["forward_ms"] if sdpa_ms else None
@@ -525,9 +579,10 @@ def main():
                 torch.cuda.empty_cache()
             result["config3_sweep"] = {"workload": "config3: 256x16x16 video tokens (1024 cubes) + 256 text, 28/4 heads, "
                                                    "head_dim 128; p=1.0 is the dense reference of the same kernels",
+                                       "gather": {"pairs_per_block": GATHER_DEFAULT_THRESHOLD, "budget_gib": SWEEP_GATHER_BUDGET >> 30},
                                        "torch_sdpa_causal_ms": sdpa_ms, "points": sweep}
             w4 = inputs.config4(device="cuda")
-            r4 = one_config(w4, w4.top_p, n_steps=2)
+            r4 = one_config(w4, w4.top_p, flush, local_rank, n_steps=2)
             r4["workload"] = "config4: 512x16x16 video tokens (2048 cubes), first half of the frames static, p=0.9"
             r4["tokens_per_s"] = w4.B * w4.S / (r4["forward_ms"] * 1e-3)
             result["config4"] = r4

@@ -284,6 +284,10 @@ int64_t adaspark_attn_last_launch_count(const adaspark_attn_t *handle);
  * token is fused into the selection kernel). */
 adaspark_status_t adaspark_attn_enable_stage_timing(adaspark_attn_t *handle, int32_t enable);
 adaspark_status_t adaspark_attn_get_stage_times(adaspark_attn_t *handle, float *ms_out /* host [4] */);
+/* With stage timing on, the last prefill's union attention kernel alone (Eq. 3 on the tensor cores, kernels
+ * 1 and 2), in milliseconds: the attention stage also holds the small kernels of the query-gather decision.
+ * Waits for that kernel's end event.  ERR_INVALID_ARG if no timed tcgen05 prefill was recorded. */
+adaspark_status_t adaspark_attn_get_attention_kernel_ms(adaspark_attn_t *handle, float *ms_out /* host [1] */);
 
 /* Selects the prefill kernels: 0 = mma.sync attention + fp64 (mma.m8n8k4.f64) scoring, the legacy
  * tensor path kept as a cross-check; 1 = tcgen05/TMEM attention with TMA-staged tiles + tcgen05
@@ -298,8 +302,10 @@ adaspark_status_t adaspark_attn_set_prefill_kernel(adaspark_attn_t *handle, int3
  * cube in it, computes their attention over that block on the tensor cores, and merges each row's partial
  * results with the result of its local range (own cube, text) by the softmax identity.  The choice is made
  * on the device, per pair: gathered iff (row, key block) entries of the pair's rows <= pairs_per_block *
- * key blocks in the pair's union.  pairs_per_block = 0 switches the path off (every pair takes the union
- * path); a huge value forces it for every pair with a selected cube.  budget_bytes bounds the workspace
+ * key blocks in the pair's union -- and only if all qualifying pairs together save more than the fixed
+ * cost of the path (about 50 us by the library's estimate, in which a union block costs as much as 44
+ * entries).  pairs_per_block = 0 switches the path off (every pair takes the union path); a value above 44
+ * forces it for every pair that meets the threshold, a huge value for every pair with a selected cube.  budget_bytes bounds the workspace
  * the path may use for its partial results (2*head_dim + 24 bytes per entry; _partition reserves
  * min(budget, what pairs_per_block lets the pairs of the partition produce, 128 entries per query row));
  * if the pairs that qualify in a call need more, all pairs take the union path in that call.  Budget and

@@ -46,7 +46,7 @@ EXPORTS = ["adaspark_attn_create", "adaspark_attn_partition", "adaspark_attn_get
            "adaspark_attn_forward", "adaspark_attn_forward_host", "adaspark_attn_forward_prefix", "adaspark_attn_forward_chunk", "adaspark_attn_decode", "adaspark_attn_destroy",
            "adaspark_attn_last_error", "adaspark_attn_last_launch_count",
            "adaspark_attn_set_prefill_kernel", "adaspark_attn_set_gather", "adaspark_attn_enable_stage_timing",
-           "adaspark_attn_get_stage_times", "adaspark_attn_decode_static",
+           "adaspark_attn_get_stage_times", "adaspark_attn_get_attention_kernel_ms", "adaspark_attn_decode_static",
            "adaspark_attn_debug_umma_selftest", "adaspark_attn_debug_imma_selftest",
            "adaspark_attn_debug_fastdiv", "adaspark_attn_debug_wait_timeout"]
 
@@ -84,6 +84,7 @@ def load() -> ctypes.CDLL:
     lib.adaspark_attn_set_gather.argtypes = [vp, ctypes.c_float, ctypes.c_uint64]
     lib.adaspark_attn_enable_stage_timing.argtypes = [vp, i32]
     lib.adaspark_attn_get_stage_times.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
+    lib.adaspark_attn_get_attention_kernel_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     for name in EXPORTS:
         if name not in ("adaspark_attn_last_error", "adaspark_attn_last_launch_count"):
             getattr(lib, name).restype = ctypes.c_int
@@ -240,6 +241,13 @@ def adaspark_attn_get_stage_times(handle: int):
     ms = (ctypes.c_float * 4)()
     _check(handle, load().adaspark_attn_get_stage_times(handle, ms))
     return [float(x) for x in ms]
+
+
+def adaspark_attn_get_attention_kernel_ms(handle: int) -> float:
+    """Milliseconds of the union attention kernel of the last timed prefill."""
+    ms = (ctypes.c_float * 1)()
+    _check(handle, load().adaspark_attn_get_attention_kernel_ms(handle, ms))
+    return float(ms[0])
 
 
 class WorkspaceHeader(ctypes.Structure):

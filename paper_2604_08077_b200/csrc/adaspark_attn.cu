@@ -46,7 +46,7 @@ struct adaspark_attn {
     int sm_count;
     int64_t launches;
     bool timing;
-    cudaEvent_t ev[5];
+    cudaEvent_t ev[7];          // stage boundaries [0..4], around the union attention kernel of the prefill [5, 6]
     bool ev_recorded;
     char err[256];
 };
@@ -247,7 +247,7 @@ adaspark_status_t adaspark_attn_partition(adaspark_attn_t* h, int32_t batch, int
         if ((double)cap > (double)rows_cap * per_row) cap = (uint64_t)((double)rows_cap * per_row);
         if (cap > 0xfffffff0ull) cap = 0xfffffff0ull;
         h->gather_cap = (uint32_t)cap;
-        h->fw_gpair_off = off; off = align_up(off + (size_t)batch * Hq * n_pairs_cap * 3 * 4);
+        h->fw_gpair_off = off; off = align_up(off + (size_t)batch * Hq * n_pairs_cap * 5 * 4);
         h->fw_grow_off = off; off = align_up(off + (cap ? rows_cap * 2 * 4 : 0));
         h->fw_gml_off = off; off = align_up(off + (cap ? rows_cap * 8 : 0));
         h->fw_gitems_off = off; off = align_up(off + (cap ? align_up((n_lists * n_cols * (kGatherReplicas + 2) + 2) * 4) + (n_lists * n_cols + cap / 128 + 1) * 16 : 0));
@@ -471,6 +471,8 @@ adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* 
             gw.pair_mode = (uint32_t*)(ws + h->fw_gpair_off);
             gw.pair_cnt = gw.pair_mode + n_pair_all;
             gw.pair_off = gw.pair_cnt + n_pair_all;
+            gw.pair_u = gw.pair_off + n_pair_all;
+            gw.pair_list = gw.pair_u + n_pair_all;
             gw.row_cnt = (uint32_t*)(ws + h->fw_grow_off);
             gw.row_ptr = gw.row_cnt + rows_cap;
             gw.col_cnt = (uint32_t*)(ws + h->fw_gcol_off);
@@ -499,6 +501,7 @@ adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* 
             if (!launch_ok(h, "gather_items_kernel")) return ADASPARK_ERR_CUDA;
         }
         const uint32_t* pair_mode_c = gather ? gw.pair_mode : nullptr;
+        mark(h, 5, st);
         if (D == 128) {
             size_t smem = sizeof(TcAttnSmem<128>) + 1024;
             if (!set_smem(h, attn_prefill_tc_kernel<128>, smem, "attn_prefill_tc_kernel")) return ADASPARK_ERR_CUDA;
@@ -513,13 +516,14 @@ adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* 
                                                                        (unsigned long long*)&hdr->executed_kv_blocks, &hdr->max_tile_kv_blocks, &hdr->status);
         }
         if (!launch_ok(h, "attn_prefill_tc_kernel")) return ADASPARK_ERR_CUDA;
+        mark(h, 6, st);
         if (gather) {
             gather_fill_kernel<<<grid, 256, 0, st>>>(g, gw, tile_mask);
             if (!launch_ok(h, "gather_fill_kernel")) return ADASPARK_ERR_CUDA;
             CUtensorMap tmKg;      // one key block per load: box of 64 d x 64 keys (tmK's) serves as it is
             tmKg = tmK;
             const int ggrid = h->sm_count;                      // persistent: one CTA per SM
-            const long long n_rows = (long long)g.B * g.Hq * (g.S - g.pos_begin);
+            const long long n_rows = (long long)g.B * g.Hq * (g.S - g.pos_begin);    // at most: the rows of all pairs
             if (D == 128) {
                 const size_t smem = sizeof(GatherSmem<128>) + 1024;
                 if (!set_smem(h, attn_gather_kernel<128>, smem, "attn_gather_kernel")) return ADASPARK_ERR_CUDA;
@@ -692,7 +696,7 @@ adaspark_status_t adaspark_attn_decode(adaspark_attn_t* h, const void* q_new, co
 
 adaspark_status_t adaspark_attn_destroy(adaspark_attn_t* h) {
     if (h && h->timing)
-        for (int i = 0; i < 5; ++i) cudaEventDestroy(h->ev[i]);
+        for (int i = 0; i < 7; ++i) cudaEventDestroy(h->ev[i]);
     delete h;
     return ADASPARK_OK;
 }
@@ -701,12 +705,12 @@ adaspark_status_t adaspark_attn_enable_stage_timing(adaspark_attn_t* h, int32_t 
     if (!h) return ADASPARK_ERR_INVALID_ARG;
     if (enable && !h->timing) {
         cudaError_t ce = cudaSetDevice(h->cfg.device);
-        for (int i = 0; i < 5 && ce == cudaSuccess; ++i) ce = cudaEventCreate(&h->ev[i]);
+        for (int i = 0; i < 7 && ce == cudaSuccess; ++i) ce = cudaEventCreate(&h->ev[i]);
         if (ce != cudaSuccess) return fail(h, ADASPARK_ERR_CUDA, "enable_stage_timing: %s", cudaGetErrorString(ce));
         h->timing = true;
         h->ev_recorded = false;
     } else if (!enable && h->timing) {
-        for (int i = 0; i < 5; ++i) cudaEventDestroy(h->ev[i]);
+        for (int i = 0; i < 7; ++i) cudaEventDestroy(h->ev[i]);
         h->timing = false;
     }
     return ADASPARK_OK;
@@ -718,6 +722,15 @@ adaspark_status_t adaspark_attn_get_stage_times(adaspark_attn_t* h, float* ms_ou
     cudaError_t ce = cudaEventSynchronize(h->ev[4]);
     for (int i = 0; i < 4 && ce == cudaSuccess; ++i) ce = cudaEventElapsedTime(&ms_out[i], h->ev[i], h->ev[i + 1]);
     if (ce != cudaSuccess) return fail(h, ADASPARK_ERR_CUDA, "get_stage_times: %s", cudaGetErrorString(ce));
+    return ADASPARK_OK;
+}
+
+adaspark_status_t adaspark_attn_get_attention_kernel_ms(adaspark_attn_t* h, float* ms_out) {
+    if (!h || !ms_out) return ADASPARK_ERR_INVALID_ARG;
+    if (!h->timing || !h->ev_recorded || h->prefill_kernel == 0) return fail(h, ADASPARK_ERR_INVALID_ARG, "get_attention_kernel_ms: no timed tcgen05 prefill recorded");
+    cudaError_t ce = cudaEventSynchronize(h->ev[6]);
+    if (ce == cudaSuccess) ce = cudaEventElapsedTime(ms_out, h->ev[5], h->ev[6]);
+    if (ce != cudaSuccess) return fail(h, ADASPARK_ERR_CUDA, "get_attention_kernel_ms: %s", cudaGetErrorString(ce));
     return ADASPARK_OK;
 }
 

@@ -33,6 +33,12 @@ namespace adaspark {
 
 constexpr int kGatherItemRows = 128;
 constexpr int kGatherReplicas = 1;
+// Measured on a B200 (65536-token video, 1024 cubes): a (pair of tiles, key block) visit of the union kernel costs
+// as much as about 44 entries of this path.  The path is taken only when the pairs that qualify save, by that
+// estimate, at least kGatherMinGain entries' worth of time (~50 us): below that its fixed costs (six small
+// launches, the scan) eat the gain.
+constexpr long long kGatherBreakEven = 44;
+constexpr long long kGatherMinGain = 300000;
 constexpr uint32_t kEntryPosMask = 0x1fffffu;   // 21 bits of cube-major position (caches hold at most 2^21 rows)
 
 // Pointers into the forward workspace and sizes (all filled by the host).
@@ -41,6 +47,8 @@ struct GatherWs {
     uint32_t* pair_mode;   // [B*Hq*n_pairs_cap] 1: the pair's selected cubes go through this path
     uint32_t* pair_cnt;    // entries of the pair's rows (0 when the pair stays on the tile kernel)
     uint32_t* pair_off;    // exclusive prefix sum of pair_cnt
+    uint32_t* pair_u;      // key blocks in the pair's union (before its local range)
+    uint32_t* pair_list;   // the pairs on this path, compacted (ctrl[2] of them)
     uint32_t* row_cnt;     // [B*Hq*S_cap] entries of a row
     uint32_t* row_ptr;     // index of the row's first slot in row_slots
     uint32_t* col_cnt;     // [kGatherReplicas][B*Hkv*n_cols] entries of a key block, counted in kGatherReplicas
@@ -162,6 +170,7 @@ __global__ void __launch_bounds__(256) gather_count_kernel(Geom g, GatherWs ws, 
         const size_t slot = bh * ws.n_pairs_cap + it.pair;
         ws.pair_mode[slot] = mode;
         ws.pair_cnt[slot] = mode ? P : 0u;
+        ws.pair_u[slot] = U;
         s_mode = mode;
     }
     __syncthreads();
@@ -222,7 +231,7 @@ __device__ __forceinline__ uint32_t cta_exclusive_scan_1024(uint32_t v, uint32_t
 
 __global__ void __launch_bounds__(1024) gather_scan_kernel(Geom g, GatherWs ws) {
     __shared__ uint32_t warp_sums[32];
-    __shared__ uint32_t total_s;
+    __shared__ uint32_t total_s, total_s2;
     const int tid = threadIdx.x;
     const int pair0 = g.pos_begin / kPairRows, n_pairs = (g.S + kPairRows - 1) / kPairRows - pair0;
     const int n_hb = g.Hq * g.B;
@@ -230,6 +239,7 @@ __global__ void __launch_bounds__(1024) gather_scan_kernel(Geom g, GatherWs ws) 
     // ---- pairs: offsets of their rows' partials
     unsigned long long carry = 0ull;
     uint32_t n_on = 0;
+    long long gain = 0;
     for (int base = 0; base < n_slots; base += 1024) {
         const int idx = base + tid;
         size_t slot = 0;
@@ -238,14 +248,28 @@ __global__ void __launch_bounds__(1024) gather_scan_kernel(Geom g, GatherWs ws) 
             const int hb = idx / n_pairs, pr = idx - hb * n_pairs;
             slot = (size_t)hb * ws.n_pairs_cap + pair0 + pr;
             v = ws.pair_cnt[slot];
+            if (v) gain += kGatherBreakEven * (long long)ws.pair_u[slot] - (long long)v;
         }
         const uint32_t ex = cta_exclusive_scan_1024(v, warp_sums, &total_s);
-        if (idx < n_slots) ws.pair_off[slot] = (uint32_t)(carry + ex);   // meaningless when the capacity check below fails
-        n_on += (v != 0u);
+        if (idx < n_slots) ws.pair_off[slot] = (uint32_t)(carry + ex);   // meaningless when the checks below fail
+        const uint32_t exl = cta_exclusive_scan_1024(v != 0u ? 1u : 0u, warp_sums, &total_s2);
+        if (idx < n_slots && v != 0u) ws.pair_list[n_on + exl] = (uint32_t)slot;
+        n_on += total_s2;
         carry += total_s;
     }
-    if (carry == 0ull || carry > (unsigned long long)ws.cap_entries) {
-        // nothing to do, or more entries than the workspace holds: every pair stays on the tile kernel
+    // estimated gain of all qualifying pairs together (block sum of a signed 64-bit value)
+    __shared__ long long gain_s[32];
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) gain += __shfl_xor_sync(0xffffffffu, gain, d);
+    if ((tid & 31) == 0) gain_s[tid >> 5] = gain;
+    __syncthreads();
+    gain = 0;
+    for (int i = 0; i < 32; ++i) gain += gain_s[i];
+    // (a threshold above the break-even estimate is a request to force the path: the estimate is not consulted)
+    const bool too_little = ws.pairs_per_block <= (float)kGatherBreakEven && gain < kGatherMinGain;
+    if (carry == 0ull || carry > (unsigned long long)ws.cap_entries || too_little) {
+        // nothing to do, more entries than the workspace holds, or too little to gain: every pair stays on the
+        // tile kernel
         for (int idx = tid; idx < n_slots; idx += 1024) {
             const int hb = idx / n_pairs, pr = idx - hb * n_pairs;
             ws.pair_mode[(size_t)hb * ws.n_pairs_cap + pair0 + pr] = 0u;
@@ -253,15 +277,9 @@ __global__ void __launch_bounds__(1024) gather_scan_kernel(Geom g, GatherWs ws) 
         if (tid == 0) { ws.ctrl[0] = 0u; ws.ctrl[1] = 0u; ws.ctrl[2] = 0u; }
         return;
     }
-    n_on = __reduce_add_sync(0xffffffffu, n_on);
-    __syncthreads();
-    if ((tid & 31) == 0) warp_sums[tid >> 5] = n_on;
-    __syncthreads();
     if (tid == 0) {
-        uint32_t s = 0;
-        for (int i = 0; i < 32; ++i) s += warp_sums[i];
         ws.ctrl[0] = (uint32_t)carry;
-        ws.ctrl[2] = s;
+        ws.ctrl[2] = n_on;
     }
     // ---- key blocks: offsets of their entry lists (and of every counter set's share) and of their work items
     const int n_cols_all = ws.n_lists * ws.n_cols;
@@ -765,10 +783,12 @@ __global__ void __launch_bounds__(256) gather_merge_kernel(Geom g, GatherWs ws, 
     if (ws.ctrl[0] == 0u) return;
     constexpr int kLanes = D / 8, kRowsPerCta = 256 / kLanes;
     const int sub = threadIdx.x % kLanes;
-    const int win = g.S - g.pos_begin;
-    const long long n_rows = (long long)g.B * g.Hq * win;
+    const long long n_rows = (long long)ws.ctrl[2] * kPairRows;    // the rows of the pairs on this path
     for (long long idx = (long long)blockIdx.x * kRowsPerCta + threadIdx.x / kLanes; idx < n_rows; idx += (long long)gridDim.x * kRowsPerCta) {
-        const int bh = (int)(idx / win), pos = g.pos_begin + (int)(idx - (long long)bh * win);
+        const uint32_t slot = __ldg(ws.pair_list + (idx >> 8));
+        const int bh = (int)(slot / (uint32_t)ws.n_pairs_cap);
+        const int pos = (int)(slot - (uint32_t)bh * (uint32_t)ws.n_pairs_cap) * kPairRows + (int)(idx & 255);
+        if (pos >= g.S) continue;
         const size_t row = (size_t)bh * g.S_cap + pos;
         // everything that does not depend on the row's count is requested first (one round of memory latency)
         const uint32_t cnt = __ldg(ws.row_cnt + row);              // 0: a pair on the union path, or a slot without token

@@ -38,7 +38,11 @@ def _config3(sigma):
     return _CFG3[sigma]
 
 
-CFG3_OUTPUT_POINTS = {(0.5, 0.5), (0.5, 1.0), (3.0, 0.5), (3.0, 1.0), (1.5, 0.9), (0.5, 0.95)}
+CFG3_OUTPUT_POINTS = {(0.5, 0.5), (0.5, 1.0), (3.0, 0.5), (3.0, 1.0), (1.5, 0.9), (0.5, 0.95), (3.0, 0.9), (1.5, 0.5)}
+# points whose selections are sparse enough for the library's own decision to send (nearly) every pair of
+# query tiles through the query-gather path, and points that must stay on the union path
+CFG3_GATHERED = {(3.0, 0.5), (3.0, 0.7), (3.0, 0.9), (1.5, 0.5)}
+CFG3_UNION = {(0.5, 0.5), (0.5, 0.7), (0.5, 0.9), (0.5, 0.95), (1.5, 0.9), (1.5, 0.95)}
 
 
 @pytest.mark.parametrize("p", [0.5, 0.7, 0.9, 0.95, 1.0])
@@ -47,7 +51,7 @@ def test_config3_full_size_sweep(sigma, p):
     """Config 3 (65536 video tokens in 1024 cubes + 256 text) at all 15 points of its (sigma, p)
     sweep: selection on 20000 sampled rows everywhere; outputs on sampled rows plus whole query tiles
     (first, middle, last) at the corners of the sweep, at the sharpest point (sigma 3, p 0.5) and at
-    two interior points."""
+    interior points, among them points that run through the query-gather path by the library's default rule."""
     wl = _config3(sigma)
     eng, out, bitmap, count = pu.run_forward(wl, top_p=p)
     label = f"cfg3 s={sigma} p={p}"
@@ -62,6 +66,12 @@ def test_config3_full_size_sweep(sigma, p):
         print(label, rep)
     hdr = eng.header()
     assert hdr.status == 0
+    n_pairs = ((wl.S + 255) // 256) * wl.Hq
+    print(label, "gathered pairs", hdr.gather_pair_tiles, "of", n_pairs, "entries", hdr.gather_entries)
+    if (sigma, p) in CFG3_GATHERED:
+        assert hdr.gather_pair_tiles > 0.9 * n_pairs
+    if (sigma, p) in CFG3_UNION or p >= 1.0:
+        assert hdr.gather_pair_tiles == 0 and hdr.gather_entries == 0
     del eng, out, bitmap, count
     _free()
 

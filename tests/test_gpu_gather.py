@@ -108,8 +108,8 @@ def test_capacity_fallback():
 def test_decision_rule_per_pair():
     """With a finite threshold only the pairs whose rows' entries are at most threshold x union blocks take the
     path: a sharp selection (few cubes per row, different per row) qualifies, a flat one does not."""
-    sharp = inputs.small_prefill(seed=33, T=64, H=8, W=8, n_text=0, Hq=2, Hkv=1, top_p=0.3, offset_std=4.0)
-    flat = inputs.small_prefill(seed=34, T=64, H=8, W=8, n_text=0, Hq=2, Hkv=1, top_p=0.95, offset_std=0.3)
+    sharp = inputs.small_prefill(seed=33, T=256, H=8, W=8, n_text=0, Hq=4, Hkv=2, top_p=0.3, offset_std=4.0)
+    flat = inputs.small_prefill(seed=34, T=256, H=8, W=8, n_text=0, Hq=4, Hkv=2, top_p=0.95, offset_std=0.3)
     for wl, expect_on in ((sharp, True), (flat, False)):
         eng, out, bitmap, count = pu.run_forward(wl, prefill_kernel=1, gather=20.0)
         hdr = eng.header()
@@ -117,6 +117,17 @@ def test_decision_rule_per_pair():
         assert (hdr.gather_pair_tiles > 0) == expect_on, (hdr.gather_pair_tiles, hdr.gather_entries)
         rep = pu.compare_rows(wl, pu.random_rows(wl, 1500, seed=5), out, bitmap, count, label="rule")
         print("sharp" if expect_on else "flat", rep, hdr.gather_pair_tiles, hdr.gather_entries)
+
+
+def test_small_gains_stay_on_the_union_path():
+    """The same sharp selection on a problem so small that gathering cannot repay its fixed cost: with a threshold
+    inside the library's break-even estimate nothing is gathered; forcing (a threshold above it) still gathers."""
+    wl = inputs.small_prefill(seed=33, T=32, H=8, W=8, n_text=0, Hq=2, Hkv=1, top_p=0.3, offset_std=4.0)
+    eng, out, bitmap, count = pu.run_forward(wl, prefill_kernel=1, gather=20.0)
+    assert eng.header().status == 0 and eng.header().gather_entries == 0
+    pu.compare_rows(wl, pu.random_rows(wl, 500, seed=6), out, bitmap, count, label="small gain")
+    eng, out, bitmap, count = pu.run_forward(wl, prefill_kernel=1, gather=pu.FORCE_GATHER)
+    assert eng.header().status == 0 and eng.header().gather_entries > 0
 
 
 def test_set_gather_arguments():
