@@ -280,7 +280,7 @@ def cpu_baseline(wl, n_rows=32768):
 
 
 GATHER_DEFAULT_THRESHOLD = 30.0    # the library's default decision threshold of the query-gather path
-SWEEP_GATHER_BUDGET = 32 << 30     # workspace the query-gather path may use on the long-video workloads
+SWEEP_GATHER_BUDGET = 32 << 30     # workspace the query-gather path may use on the long-video workloads (library default: 24 GiB)
 
 def one_config(wx, p, flush, local_rank, n_steps=3, gather=None, budget=SWEEP_GATHER_BUDGET, warmup=3):
     """One forward configuration timed with stage times: gather None = the library's own per-pair decision

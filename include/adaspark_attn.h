@@ -311,7 +311,7 @@ adaspark_status_t adaspark_attn_set_prefill_kernel(adaspark_attn_t *handle, int3
  * if the pairs that qualify in a call need more, all pairs take the union path in that call.  Budget and
  * threshold size the forward workspace: set them before _partition (a different budget afterwards is
  * ERR_INVALID_ARG; the threshold may still change, the reserved capacity does not).  Defaults: 30 entries
- * per block (gathering pays up to about 44 on a B200), 16 GiB.  Outputs agree with the union path within
+ * per block (gathering pays up to about 44 on a B200), 24 GiB.  Outputs agree with the union path within
  * bf16 rounding of the partial results; the selection is the same. */
 adaspark_status_t adaspark_attn_set_gather(adaspark_attn_t *handle, float pairs_per_block,
                                            uint64_t budget_bytes);

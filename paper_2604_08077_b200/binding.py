@@ -271,7 +271,7 @@ class AdaSAttn:
         self.device = torch.device("cuda", device)
         self.layout: Optional[Layout] = None
 
-    def set_gather(self, pairs_per_block: float, budget_bytes: int = 16 << 30):
+    def set_gather(self, pairs_per_block: float, budget_bytes: int = 24 << 30):
         """Threshold and workspace budget of the query-gather path (budget: before partition())."""
         adaspark_attn_set_gather(self.handle, pairs_per_block, budget_bytes)
 

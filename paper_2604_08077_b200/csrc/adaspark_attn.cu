@@ -59,7 +59,7 @@ constexpr int kExactCtas = 296;   // CTAs of the fp64 selection kernel (its scra
 // many per key block of the pair's union (measured break-even on a B200, see the attention profile), and the
 // partial results of all such pairs must fit this many bytes of workspace
 constexpr float kGatherDefaultPairsPerBlock = 30.f;
-constexpr uint64_t kGatherDefaultBudget = 16ull << 30;
+constexpr uint64_t kGatherDefaultBudget = 24ull << 30;
 constexpr uint64_t kGatherEntriesPerRow = 128;
 constexpr size_t kGatherWindowBytes = 40u << 20;
 size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }

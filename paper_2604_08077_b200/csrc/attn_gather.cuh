@@ -281,40 +281,43 @@ __global__ void __launch_bounds__(1024) gather_scan_kernel(Geom g, GatherWs ws) 
         ws.ctrl[0] = (uint32_t)carry;
         ws.ctrl[2] = n_on;
     }
-    // ---- key blocks: offsets of their entry lists (and of every counter set's share) and of their work items
+    // ---- key blocks: offsets of their entry lists (and of every counter set's share) and of their work items.
+    // Every thread owns a contiguous run of blocks: it sums them, one scan over the 1024 sums gives its start,
+    // and it walks the run again (two scans in all instead of two per 1024 blocks).
     const int n_cols_all = ws.n_lists * ws.n_cols;
-    uint32_t ent_carry = 0, item_carry = 0;
-    for (int base = 0; base < n_cols_all; base += 1024) {
-        const int col = base + tid;
-        uint32_t part[kGatherReplicas];
+    const int per = (n_cols_all + 1023) / 1024;
+    const int c0 = min(tid * per, n_cols_all), c1 = min(c0 + per, n_cols_all);
+    uint32_t my_e = 0, my_i = 0;
+    for (int col = c0; col < c1; ++col) {
+        uint32_t v = 0;
+#pragma unroll
+        for (int r = 0; r < kGatherReplicas; ++r) v += ws.col_cnt[(size_t)r * n_cols_all + col];
+        my_e += v;
+        my_i += (v + kGatherItemRows - 1) / kGatherItemRows;
+    }
+    uint32_t e_off = cta_exclusive_scan_1024(my_e, warp_sums, &total_s);
+    const uint32_t tot_e = total_s;
+    uint32_t i_off = cta_exclusive_scan_1024(my_i, warp_sums, &total_s);
+    const uint32_t tot_i = total_s;
+    for (int col = c0; col < c1; ++col) {
+        uint32_t o = e_off;
+        ws.col_off[col] = o;
+        ws.col_item[col] = i_off;
         uint32_t v = 0;
 #pragma unroll
         for (int r = 0; r < kGatherReplicas; ++r) {
-            part[r] = col < n_cols_all ? ws.col_cnt[(size_t)r * n_cols_all + col] : 0u;
-            v += part[r];
+            const uint32_t part = ws.col_cnt[(size_t)r * n_cols_all + col];
+            ws.col_roff[(size_t)r * n_cols_all + col] = o;
+            o += part;
+            v += part;
         }
-        const uint32_t chunks = (v + kGatherItemRows - 1) / kGatherItemRows;
-        const uint32_t ex = cta_exclusive_scan_1024(v, warp_sums, &total_s);
-        const uint32_t tot_e = total_s;
-        const uint32_t exi = cta_exclusive_scan_1024(chunks, warp_sums, &total_s);
-        const uint32_t tot_i = total_s;
-        if (col < n_cols_all) {
-            uint32_t o = ent_carry + ex;
-            ws.col_off[col] = o;
-            ws.col_item[col] = item_carry + exi;
-#pragma unroll
-            for (int r = 0; r < kGatherReplicas; ++r) {
-                ws.col_roff[(size_t)r * n_cols_all + col] = o;
-                o += part[r];
-            }
-        }
-        ent_carry += tot_e;
-        item_carry += tot_i;
+        e_off += v;
+        i_off += (v + kGatherItemRows - 1) / kGatherItemRows;
     }
     if (tid == 0) {
-        ws.col_off[n_cols_all] = ent_carry;
-        ws.col_item[n_cols_all] = item_carry;
-        ws.ctrl[1] = item_carry;
+        ws.col_off[n_cols_all] = tot_e;
+        ws.col_item[n_cols_all] = tot_i;
+        ws.ctrl[1] = tot_i;
     }
 }
 

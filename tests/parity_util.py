@@ -16,7 +16,7 @@ TIE_MARGIN = 1e-6        # rows whose cumulative-probability margin is below thi
 FORCE_GATHER = 1e30   # threshold of the query-gather path that sends every pair with a selected cube through it
 
 
-def make_engine(wl, n_text_max=None, top_p=None, prefill_kernel=None, gather=None, gather_budget=16 << 30):
+def make_engine(wl, n_text_max=None, top_p=None, prefill_kernel=None, gather=None, gather_budget=24 << 30):
     """gather: None = the library's default decision; 0 = union path only; FORCE_GATHER = gather path
     wherever a row selected a cube before its local range."""
     eng = binding.AdaSAttn(cube=wl.cube, n_q_heads=wl.Hq, n_kv_heads=wl.Hkv, head_dim=wl.D,
@@ -42,7 +42,7 @@ def unpack_bitmap(words: torch.Tensor, n_cubes: int) -> np.ndarray:
     return bits.reshape(*w.shape[:-1], -1)[..., :n_cubes].astype(np.uint8)
 
 
-def run_forward(wl, *, top_p=None, prefill_kernel=None, want_selection=True, gather=None, gather_budget=16 << 30):
+def run_forward(wl, *, top_p=None, prefill_kernel=None, want_selection=True, gather=None, gather_budget=24 << 30):
     eng = make_engine(wl, top_p=top_p, prefill_kernel=prefill_kernel, gather=gather, gather_budget=gather_budget)
     q, k, v = wl.q.cuda(), wl.k.cuda(), wl.v.cuda()
     out, bitmap, count = eng.forward(q, k, v, wl.n_text, want_selection=want_selection,
