@@ -308,7 +308,10 @@ adaspark_status_t adaspark_attn_set_prefill_kernel(adaspark_attn_t *handle, int3
  * forces it for every pair that meets the threshold, a huge value for every pair with a selected cube.  budget_bytes bounds the workspace
  * the path may use for its partial results (2*head_dim + 24 bytes per entry; _partition reserves
  * min(budget, what pairs_per_block lets the pairs of the partition produce, 128 entries per query row));
- * if the pairs that qualify in a call need more, all pairs take the union path in that call.  Budget and
+ * if the pairs that qualify in a call need more, only part of them is gathered in that call: the pairs fall
+ * into four classes by entries per union block (up to 1/8, 1/4, 1/2 of the threshold, up to the threshold)
+ * and into row windows; (class, window) units are kept while they fit, sparsest class first and inside a
+ * class the latest rows first.  Budget and
  * threshold size the forward workspace: set them before _partition (a different budget afterwards is
  * ERR_INVALID_ARG; the threshold may still change, the reserved capacity does not).  Defaults: 30 entries
  * per block (gathering pays up to about 44 on a B200), 24 GiB.  Outputs agree with the union path within

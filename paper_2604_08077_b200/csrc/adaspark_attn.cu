@@ -226,7 +226,7 @@ adaspark_status_t adaspark_attn_partition(adaspark_attn_t* h, int32_t batch, int
         h->gather_windows = (int)(w < 1 ? 1 : (w > 16 ? 16 : w));
     }
     const size_t n_lists = (size_t)h->gather_windows * batch * Hkv;
-    h->fw_gcol_off = off; off = align_up(off + n_lists * n_cols * 2 * kGatherReplicas * 4);   // entry counts and fill cursors (zeroed per call)
+    h->fw_gcol_off = off; off = align_up(off + n_lists * n_cols * 2 * kGatherClasses * 4);   // entry counts and fill cursors (zeroed per call)
     h->fw_mask_off = off; off = align_up(off + (size_t)batch * Hq * n_tiles_cap * n_words * kTileRows * 4);
     h->fw_union_off = off; off = align_up(off + (size_t)batch * Hq * n_tiles_cap * n_words * 4);
     h->fw_fallback_off = off; off = align_up(off + (size_t)batch * Hq * n_tiles_cap * kTileRows * 4);
@@ -250,7 +250,7 @@ adaspark_status_t adaspark_attn_partition(adaspark_attn_t* h, int32_t batch, int
         h->fw_gpair_off = off; off = align_up(off + (size_t)batch * Hq * n_pairs_cap * 5 * 4);
         h->fw_grow_off = off; off = align_up(off + (cap ? rows_cap * 2 * 4 : 0));
         h->fw_gml_off = off; off = align_up(off + (cap ? rows_cap * 8 : 0));
-        h->fw_gitems_off = off; off = align_up(off + (cap ? align_up((n_lists * n_cols * (kGatherReplicas + 2) + 2) * 4) + (n_lists * n_cols + cap / 128 + 1) * 16 : 0));
+        h->fw_gitems_off = off; off = align_up(off + (cap ? align_up((n_lists * n_cols * (kGatherClasses + 2) + 2) * 4) + (n_lists * n_cols + cap / 128 + 1) * 16 : 0));
         h->fw_gentries_off = off; off = align_up(off + (size_t)cap * 8);
         h->fw_gparto_off = off; off = align_up(off + (size_t)cap * D * 2);
         h->fw_gpartml_off = off; off = align_up(off + (size_t)cap * 8);
@@ -476,11 +476,11 @@ adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* 
             gw.row_cnt = (uint32_t*)(ws + h->fw_grow_off);
             gw.row_ptr = gw.row_cnt + rows_cap;
             gw.col_cnt = (uint32_t*)(ws + h->fw_gcol_off);
-            gw.col_cur = gw.col_cnt + n_col_all * kGatherReplicas;
+            gw.col_cur = gw.col_cnt + n_col_all * kGatherClasses;
             gw.col_roff = (uint32_t*)(ws + h->fw_gitems_off);
-            gw.col_off = gw.col_roff + n_col_all * kGatherReplicas;
+            gw.col_off = gw.col_roff + n_col_all * kGatherClasses;
             gw.col_item = gw.col_off + n_col_all + 1;
-            gw.items = (uint4*)(ws + h->fw_gitems_off + align_up((n_col_all * (kGatherReplicas + 2) + 2) * 4));
+            gw.items = (uint4*)(ws + h->fw_gitems_off + align_up((n_col_all * (kGatherClasses + 2) + 2) * 4));
             gw.entries = (uint32_t*)(ws + h->fw_gentries_off);
             gw.row_slots = gw.entries + h->gather_cap;
             gw.part_o = (__nv_bfloat16*)(ws + h->fw_gparto_off);
@@ -489,6 +489,7 @@ adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* 
             gw.cap_entries = h->gather_cap;
             gw.n_cols = (int)n_cols;
             gw.n_lists = (int)n_lists;
+            gw.n_windows = h->gather_windows;
             gw.pairs_per_window = (n_pairs_win + h->gather_windows - 1) / h->gather_windows;
             gw.n_pairs_cap = (int)n_pairs_cap;
             gw.pairs_per_block = h->gather_pairs_per_block;

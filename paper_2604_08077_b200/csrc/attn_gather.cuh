@@ -32,7 +32,14 @@
 namespace adaspark {
 
 constexpr int kGatherItemRows = 128;
-constexpr int kGatherReplicas = 1;
+constexpr int kGatherMaxWindows = 16;
+constexpr int kGatherClasses = 4;       // a qualifying pair falls into a class by its ratio entries / union blocks:
+                                        // <= 1/8, 1/4, 1/2 of the threshold, or up to the threshold.  When the
+                                        // entries of all qualifying pairs exceed the workspace, (class, row window)
+                                        // units are kept while they fit -- sparsest class first (its pairs gain most
+                                        // per byte), inside a class the latest window first (longest unions) -- and
+                                        // the other pairs stay on the union path; every unit counts its key blocks
+                                        // in its own counters, so nothing is recounted
 // Measured on a B200 (65536-token video, 1024 cubes): a (pair of tiles, key block) visit of the union kernel costs
 // as much as about 44 entries of this path.  The path is taken only when the pairs that qualify save, by that
 // estimate, at least kGatherMinGain entries' worth of time (~50 us): below that its fixed costs (six small
@@ -44,19 +51,17 @@ constexpr uint32_t kEntryPosMask = 0x1fffffu;   // 21 bits of cube-major positio
 // Pointers into the forward workspace and sizes (all filled by the host).
 struct GatherWs {
     uint32_t* ctrl;        // [0] entries, [1] items, [2] pairs on this path (0 entries: the path is off)
-    uint32_t* pair_mode;   // [B*Hq*n_pairs_cap] 1: the pair's selected cubes go through this path
+    uint32_t* pair_mode;   // [B*Hq*n_pairs_cap] 0: union path; c + 1: this path, ratio class c
     uint32_t* pair_cnt;    // entries of the pair's rows (0 when the pair stays on the tile kernel)
     uint32_t* pair_off;    // exclusive prefix sum of pair_cnt
     uint32_t* pair_u;      // key blocks in the pair's union (before its local range)
     uint32_t* pair_list;   // the pairs on this path, compacted (ctrl[2] of them)
     uint32_t* row_cnt;     // [B*Hq*S_cap] entries of a row
     uint32_t* row_ptr;     // index of the row's first slot in row_slots
-    uint32_t* col_cnt;     // [kGatherReplicas][B*Hkv*n_cols] entries of a key block, counted in kGatherReplicas
-                           // separate sets of counters (a CTA uses set blockIdx.x % kGatherReplicas: the atomics of
-                           // all CTAs on one set of a few thousand counters were the slowest part of the count);
-                           // zero at the start of a forward
-    uint32_t* col_cur;     // [kGatherReplicas][...] fill cursors; zero at the start of a forward
-    uint32_t* col_roff;    // [kGatherReplicas][...] first entry of the set's share of the block's list
+    uint32_t* col_cnt;     // [kGatherClasses][lists * n_cols] entries of a key block list, per ratio class of the
+                           // pairs they come from; zero at the start of a forward
+    uint32_t* col_cur;     // [kGatherClasses][...] fill cursors; zero at the start of a forward
+    uint32_t* col_roff;    // [kGatherClasses][...] first entry of the set's share of the block's list
     uint32_t* col_off;     // [B*Hkv*n_cols + 1] first entry of the block's list (exclusive prefix sum)
     uint32_t* col_item;    // [B*Hkv*n_cols + 1] first work item of the block
     uint4* items;          // (key block column, first entry, entries (<= 128), 0)
@@ -69,6 +74,7 @@ struct GatherWs {
     uint32_t cap_entries;
     int n_cols;            // key blocks that hold video slots: ceil(S_v / 64)
     int n_lists;           // entry lists per key block column set: windows x B x Hkv (each of n_cols lists)
+    int n_windows;         // row windows (<= kGatherMaxWindows)
     int pairs_per_window;  // The query rows are cut into windows of this many pairs of tiles and every (window,
                            // batch, kv head, key block) has its own entry list: the items of a window gather from a
                            // slice of Q that stays in L2, and a row's partial results lie close together.
@@ -166,7 +172,9 @@ __global__ void __launch_bounds__(256) gather_count_kernel(Geom g, GatherWs ws, 
     if (tid == 0) {
         uint32_t P = 0, U = 0;
         for (int i = 0; i < 8; ++i) { P += red[0][i]; U += red[1][i]; }
-        const uint32_t mode = (P > 0 && (float)P <= ws.pairs_per_block * (float)U) ? 1u : 0u;
+        uint32_t mode = 0u;
+        const float lim = ws.pairs_per_block * (float)U;
+        if (P > 0 && (float)P <= lim) mode = (float)P <= 0.125f * lim ? 1u : ((float)P <= 0.25f * lim ? 2u : ((float)P <= 0.5f * lim ? 3u : 4u));
         const size_t slot = bh * ws.n_pairs_cap + it.pair;
         ws.pair_mode[slot] = mode;
         ws.pair_cnt[slot] = mode ? P : 0u;
@@ -180,7 +188,7 @@ __global__ void __launch_bounds__(256) gather_count_kernel(Geom g, GatherWs ws, 
     // entries per key block: the warp's 32 x 32 bits of a word are transposed, lane j then counts the rows that
     // selected cube 32 w + j and adds them to the cube's block(s)
     const int win = (it.pair - g.pos_begin / kPairRows) / ws.pairs_per_window;
-    uint32_t* col_cnt = ws.col_cnt + ((size_t)(blockIdx.x % kGatherReplicas) * ws.n_lists + ((size_t)win * g.B + it.b) * g.Hkv + it.gk) * ws.n_cols;
+    uint32_t* col_cnt = ws.col_cnt + ((size_t)(s_mode - 1u) * ws.n_lists + ((size_t)win * g.B + it.b) * g.Hkv + it.gk) * ws.n_cols;
     for (int w0 = 0; w0 < it.n_w; w0 += 4) {
         uint32_t wd[4];
 #pragma unroll
@@ -236,10 +244,55 @@ __global__ void __launch_bounds__(1024) gather_scan_kernel(Geom g, GatherWs ws) 
     const int pair0 = g.pos_begin / kPairRows, n_pairs = (g.S + kPairRows - 1) / kPairRows - pair0;
     const int n_hb = g.Hq * g.B;
     const int n_slots = n_pairs * n_hb;
-    // ---- pairs: offsets of their rows' partials
+    // ---- which (ratio class, row window) units fit the workspace, and whether they are worth the fixed cost
+    __shared__ unsigned long long unit_entries[kGatherClasses][kGatherMaxWindows];
+    __shared__ long long unit_gain[kGatherClasses][kGatherMaxWindows];
+    __shared__ uint32_t unit_keep[kGatherClasses];          // bit w: window w of the class takes the path
+    __shared__ int any_keep_s;
+    for (int i = tid; i < kGatherClasses * kGatherMaxWindows; i += 1024) {
+        (&unit_entries[0][0])[i] = 0ull;
+        (&unit_gain[0][0])[i] = 0ll;
+    }
+    __syncthreads();
+    for (int idx = tid; idx < n_slots; idx += 1024) {
+        const int hb = idx / n_pairs, pr = idx - hb * n_pairs;
+        const size_t slot = (size_t)hb * ws.n_pairs_cap + pair0 + pr;
+        const uint32_t mode = ws.pair_mode[slot];
+        if (mode) {
+            const uint32_t v = ws.pair_cnt[slot];
+            const int win = pr / ws.pairs_per_window;
+            atomicAdd(&unit_entries[mode - 1][win], (unsigned long long)v);
+            atomicAdd(reinterpret_cast<unsigned long long*>(&unit_gain[mode - 1][win]),
+                      (unsigned long long)(kGatherBreakEven * (long long)ws.pair_u[slot] - (long long)v));
+        }
+    }
+    __syncthreads();
+    if (tid == 0) {
+        unsigned long long tot = 0ull;
+        long long gain = 0ll;
+        for (int c = 0; c < kGatherClasses; ++c) {
+            uint32_t keep = 0u;
+            for (int w = ws.n_windows - 1; w >= 0; --w) {
+                const unsigned long long e = unit_entries[c][w];
+                if (e == 0ull || tot + e > (unsigned long long)ws.cap_entries) continue;
+                tot += e;
+                gain += unit_gain[c][w];
+                keep |= 1u << w;
+            }
+            unit_keep[c] = keep;
+        }
+        // (a threshold above the break-even estimate is a request to force the path: the estimate is not consulted)
+        if (tot == 0ull || (ws.pairs_per_block <= (float)kGatherBreakEven && gain < kGatherMinGain)) {
+            for (int c = 0; c < kGatherClasses; ++c) unit_keep[c] = 0u;
+            tot = 0ull;
+        }
+        any_keep_s = tot != 0ull;
+    }
+    __syncthreads();
+    const bool any_keep = any_keep_s != 0;
+    // ---- pairs: offsets of their rows' partials, compact list; pairs of the other units go back to the union path
     unsigned long long carry = 0ull;
     uint32_t n_on = 0;
-    long long gain = 0;
     for (int base = 0; base < n_slots; base += 1024) {
         const int idx = base + tid;
         size_t slot = 0;
@@ -247,33 +300,20 @@ __global__ void __launch_bounds__(1024) gather_scan_kernel(Geom g, GatherWs ws) 
         if (idx < n_slots) {
             const int hb = idx / n_pairs, pr = idx - hb * n_pairs;
             slot = (size_t)hb * ws.n_pairs_cap + pair0 + pr;
-            v = ws.pair_cnt[slot];
-            if (v) gain += kGatherBreakEven * (long long)ws.pair_u[slot] - (long long)v;
+            const uint32_t mode = ws.pair_mode[slot];
+            if (mode != 0u && ((unit_keep[mode - 1] >> (pr / ws.pairs_per_window)) & 1u)) v = ws.pair_cnt[slot];
+            else if (mode != 0u) { ws.pair_mode[slot] = 0u; ws.pair_cnt[slot] = 0u; }
         }
+        if (!any_keep) continue;
         const uint32_t ex = cta_exclusive_scan_1024(v, warp_sums, &total_s);
-        if (idx < n_slots) ws.pair_off[slot] = (uint32_t)(carry + ex);   // meaningless when the checks below fail
+        if (idx < n_slots) ws.pair_off[slot] = (uint32_t)(carry + ex);
         const uint32_t exl = cta_exclusive_scan_1024(v != 0u ? 1u : 0u, warp_sums, &total_s2);
         if (idx < n_slots && v != 0u) ws.pair_list[n_on + exl] = (uint32_t)slot;
         n_on += total_s2;
         carry += total_s;
     }
-    // estimated gain of all qualifying pairs together (block sum of a signed 64-bit value)
-    __shared__ long long gain_s[32];
-#pragma unroll
-    for (int d = 16; d >= 1; d >>= 1) gain += __shfl_xor_sync(0xffffffffu, gain, d);
-    if ((tid & 31) == 0) gain_s[tid >> 5] = gain;
-    __syncthreads();
-    gain = 0;
-    for (int i = 0; i < 32; ++i) gain += gain_s[i];
-    // (a threshold above the break-even estimate is a request to force the path: the estimate is not consulted)
-    const bool too_little = ws.pairs_per_block <= (float)kGatherBreakEven && gain < kGatherMinGain;
-    if (carry == 0ull || carry > (unsigned long long)ws.cap_entries || too_little) {
-        // nothing to do, more entries than the workspace holds, or too little to gain: every pair stays on the
-        // tile kernel
-        for (int idx = tid; idx < n_slots; idx += 1024) {
-            const int hb = idx / n_pairs, pr = idx - hb * n_pairs;
-            ws.pair_mode[(size_t)hb * ws.n_pairs_cap + pair0 + pr] = 0u;
-        }
+    if (!any_keep) {
+        // nothing to do, nothing fits, or too little to gain: every pair stays on the union path
         if (tid == 0) { ws.ctrl[0] = 0u; ws.ctrl[1] = 0u; ws.ctrl[2] = 0u; }
         return;
     }
@@ -285,13 +325,16 @@ __global__ void __launch_bounds__(1024) gather_scan_kernel(Geom g, GatherWs ws) 
     // Every thread owns a contiguous run of blocks: it sums them, one scan over the 1024 sums gives its start,
     // and it walks the run again (two scans in all instead of two per 1024 blocks).
     const int n_cols_all = ws.n_lists * ws.n_cols;
+    const int cols_per_window = n_cols_all / ws.n_windows;       // lists are window-major
     const int per = (n_cols_all + 1023) / 1024;
     const int c0 = min(tid * per, n_cols_all), c1 = min(c0 + per, n_cols_all);
     uint32_t my_e = 0, my_i = 0;
     for (int col = c0; col < c1; ++col) {
         uint32_t v = 0;
 #pragma unroll
-        for (int r = 0; r < kGatherReplicas; ++r) v += ws.col_cnt[(size_t)r * n_cols_all + col];
+        const int win = col / cols_per_window;
+        for (int r = 0; r < kGatherClasses; ++r)
+            if ((unit_keep[r] >> win) & 1u) v += ws.col_cnt[(size_t)r * n_cols_all + col];
         my_e += v;
         my_i += (v + kGatherItemRows - 1) / kGatherItemRows;
     }
@@ -305,11 +348,14 @@ __global__ void __launch_bounds__(1024) gather_scan_kernel(Geom g, GatherWs ws) 
         ws.col_item[col] = i_off;
         uint32_t v = 0;
 #pragma unroll
-        for (int r = 0; r < kGatherReplicas; ++r) {
-            const uint32_t part = ws.col_cnt[(size_t)r * n_cols_all + col];
-            ws.col_roff[(size_t)r * n_cols_all + col] = o;
-            o += part;
-            v += part;
+        const int win = col / cols_per_window;
+        for (int r = 0; r < kGatherClasses; ++r) {
+            if ((unit_keep[r] >> win) & 1u) {
+                const uint32_t part = ws.col_cnt[(size_t)r * n_cols_all + col];
+                ws.col_roff[(size_t)r * n_cols_all + col] = o;
+                o += part;
+                v += part;
+            }
         }
         e_off += v;
         i_off += (v + kGatherItemRows - 1) / kGatherItemRows;
@@ -339,7 +385,8 @@ __global__ void __launch_bounds__(256) gather_fill_kernel(Geom g, GatherWs ws, c
     const PairItem it = pair_item(g, blockIdx.x);
     const size_t bh = (size_t)(it.b * g.Hq + it.h);
     const size_t slot = bh * ws.n_pairs_cap + it.pair;
-    if (ws.ctrl[0] == 0u || ws.pair_mode[slot] == 0u) return;
+    const uint32_t mode = ws.pair_mode[slot];
+    if (ws.ctrl[0] == 0u || mode == 0u) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int bshift = max(g.c_shift - 6, 0);
     const int tile = it.pair * 2 + (warp >> 2), r = (warp & 3) * 32 + lane, pos = it.pair_pos0 + tid;
@@ -361,7 +408,7 @@ __global__ void __launch_bounds__(256) gather_fill_kernel(Geom g, GatherWs ws, c
     if (!tile_ok) return;
     const uint32_t* my = tile_mask + mask_index(g, it.b, it.h, tile, 0, r);
     const int win = (it.pair - g.pos_begin / kPairRows) / ws.pairs_per_window;
-    const size_t colbase = ((size_t)(blockIdx.x % kGatherReplicas) * ws.n_lists + ((size_t)win * g.B + it.b) * g.Hkv + it.gk) * ws.n_cols;
+    const size_t colbase = ((size_t)(mode - 1u) * ws.n_lists + ((size_t)win * g.B + it.b) * g.Hkv + it.gk) * ws.n_cols;
     const uint32_t ent_x = (uint32_t)pos | ((uint32_t)(it.h - it.gk * g.G) << 21);
     const uint32_t lt_mask = (1u << lane) - 1u;
     // Four words per step.  After the transposition lane j holds the rows of the warp that selected cube 32 w + j;

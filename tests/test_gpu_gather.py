@@ -105,6 +105,35 @@ def test_capacity_fallback():
     assert rep["rows"] == wl.B * wl.Hq * wl.S
 
 
+def test_partial_capacity_keeps_the_sparsest_pairs():
+    """When the qualifying pairs need more workspace than the budget gives, part of them is gathered -- units of
+    (ratio class, row window), sparsest class first -- and the rest take the union path; the result is the
+    oracle's either way."""
+    wl = inputs.small_prefill(seed=37, T=64, H=8, W=8, n_text=40, Hq=4, Hkv=2, top_p=0.8, offset_std=2.5)
+    full, out_f, bm_f, cnt_f = pu.run_forward(wl, prefill_kernel=1, gather=pu.FORCE_GATHER)
+    n_all, pairs_all = full.header().gather_entries, full.header().gather_pair_tiles
+    assert n_all > 0
+    # FORCE puts every pair into one class; a finite threshold above the break-even estimate still forces the
+    # path and spreads the pairs over the ratio classes.  Which threshold splits this workload is found by trying.
+    found = None
+    for thr in (50.0, 70.0, 100.0, 140.0, 200.0, 280.0, 400.0):
+        ref, _, _, _ = pu.run_forward(wl, prefill_kernel=1, gather=thr)
+        n_thr, pairs_thr = ref.header().gather_entries, ref.header().gather_pair_tiles
+        if n_thr == 0:
+            continue
+        part, out_p, bm_p, cnt_p = pu.run_forward(wl, prefill_kernel=1, gather=thr,
+                                                  gather_budget=(n_thr * 3 // 4) * (2 * wl.D + 24))
+        hp = part.header()
+        assert hp.status == 0 and hp.gather_entries <= n_thr * 3 // 4
+        if 0 < hp.gather_entries and 0 < hp.gather_pair_tiles < pairs_thr:
+            found = (thr, n_thr, pairs_thr, hp.gather_entries, hp.gather_pair_tiles)
+            rep = pu.compare_rows(wl, oracle.all_rows(oracle.shape_of(wl)), out_p, bm_p, cnt_p, label="partial capacity")
+            assert rep["rows"] == wl.B * wl.Hq * wl.S
+            break
+    assert found is not None, "no threshold split the pairs of this workload over several classes"
+    print("partial capacity (threshold, entries, pairs, kept entries, kept pairs)", found)
+
+
 def test_decision_rule_per_pair():
     """With a finite threshold only the pairs whose rows' entries are at most threshold x union blocks take the
     path: a sharp selection (few cubes per row, different per row) qualifies, a flat one does not."""
