@@ -27,6 +27,9 @@ namespace adaspark {
 constexpr int kTcThreads = 384;
 constexpr int kSoftmaxRegs = 216;   // per-thread registers of the softmax warpgroups after setmaxnreg
 constexpr int kHelperRegs = 72;     // ... of the producer / MMA warpgroup
+// setmaxnreg only moves registers inside what the CTA got at launch: 384 threads x 168 registers (the
+// compile-time bound of __launch_bounds__(384, 1)).  A request beyond that blocks forever.
+static_assert(8 * 32 * kSoftmaxRegs + 4 * 32 * kHelperRegs <= kTcThreads * 168, "setmaxnreg must stay inside the CTA's launch allocation");
 constexpr int kPairRows = 256;
 constexpr int kMaxBlockWords = 1024;   // up to 32768 key blocks (2M positions) per sequence
 
