@@ -80,10 +80,10 @@ __global__ void __launch_bounds__(256) decode_select_plan_kernel(
                 for (int s = 0; s < 4; ++s)
                     a[4 * S + s] = live ? (double)__bfloat162float(qsrc[16 * S + 4 * kq + s]) : 0.0;
         }
-        // two groups of 8 cubes per iteration, all 16-byte loads of both issued before the tensor ops
-        // (the mean keys stream from HBM: bytes in flight decide the speed of this loop)
-        for (int c0 = warp * 8; c0 < g.N_ld; c0 += 128) {
-            float4 kv[2][D / 16];
+        // Two groups of 8 cubes per iteration.  The mean keys stream from HBM and nothing else hides their latency
+        // (one CTA per SM, eight warps): the loads of the next iteration are issued before the tensor ops of this
+        // one, so that two iterations' worth of bytes are in flight per warp.
+        auto load_keys = [&](int c0, float4 (&kv)[2][D / 16]) {
 #pragma unroll
             for (int u = 0; u < 2; ++u) {
                 const int cube = c0 + u * 64 + rq;
@@ -92,6 +92,8 @@ __global__ void __launch_bounds__(256) decode_select_plan_kernel(
                 for (int S = 0; S < D / 16; ++S)
                     kv[u][S] = cube < g.N ? *reinterpret_cast<const float4*>(ksrc + 16 * S) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
+        };
+        auto score_keys = [&](int c0, const float4 (&kv)[2][D / 16]) {
 #pragma unroll
             for (int u = 0; u < 2; ++u) {
                 if (c0 + u * 64 >= g.N_ld) break;
@@ -106,6 +108,19 @@ __global__ void __launch_bounds__(256) decode_select_plan_kernel(
                 if (rq < rpp) {   // C fragment: row = lane/4, columns 2*(lane%4) + {0,1}
                     logit[(size_t)rq * g.N_ld + c0 + u * 64 + 2 * kq] = acc[0] * g.scale_d;
                     logit[(size_t)rq * g.N_ld + c0 + u * 64 + 2 * kq + 1] = acc[1] * g.scale_d;
+                }
+            }
+        };
+        {
+            float4 kv_a[2][D / 16], kv_b[2][D / 16];
+            int c0 = warp * 8;
+            if (c0 < g.N_ld) load_keys(c0, kv_a);
+            for (; c0 < g.N_ld; c0 += 256) {
+                if (c0 + 128 < g.N_ld) load_keys(c0 + 128, kv_b);
+                score_keys(c0, kv_a);
+                if (c0 + 128 < g.N_ld) {
+                    if (c0 + 256 < g.N_ld) load_keys(c0 + 256, kv_a);
+                    score_keys(c0 + 128, kv_b);
                 }
             }
         }
@@ -144,33 +159,46 @@ __global__ void __launch_bounds__(256) decode_select_plan_kernel(
         bm[w] = u;
     }
     __syncthreads();
-    if (warp != 0) return;
+    // every warp takes a contiguous run of blocks: count, prefix over the warps, then write
+    __shared__ int plan_cnt[8];
     const int tl = text_len[b];
     const int last_pos = g.S_v + tl;                     // position of the new token
     int n_blk = 0;
     if (tl >= 0 && tl <= g.n_text) n_blk = last_pos / kBlockTok + 1;
-    int32_t* dst = items + (size_t)(b * g.Hkv + gk) * g.n_kv_blocks_cap;
-    int count = 0;
-    for (int kb0 = 0; kb0 < n_blk; kb0 += 32) {
-        int kb = kb0 + lane;
-        bool need = false;
-        if (kb < n_blk) {
-            if (kb * kBlockTok + kBlockTok - 1 >= g.S_v) need = true;   // holds text positions
-            if (kb * kBlockTok < g.S_v) {
-                int c_lo = (kb * kBlockTok) >> g.c_shift;
-                int c_hi = min((kb * kBlockTok + kBlockTok - 1) >> g.c_shift, g.N - 1);
-                uint32_t span = c_hi - c_lo + 1;
-                uint32_t bits = (span >= 32 ? 0xffffffffu : ((1u << span) - 1u)) << (c_lo & 31);
-                if (bm[c_lo >> 5] & bits) need = true;
-            }
+    const int per_warp = ((n_blk + 7) / 8 + 31) / 32 * 32;
+    const int kb_lo = warp * per_warp, kb_hi = min(kb_lo + per_warp, n_blk);
+    auto block_needed = [&](int kb) -> bool {
+        if (kb >= kb_hi) return false;
+        bool need = kb * kBlockTok + kBlockTok - 1 >= g.S_v;   // holds text positions
+        if (kb * kBlockTok < g.S_v) {
+            int c_lo = (kb * kBlockTok) >> g.c_shift;
+            int c_hi = min((kb * kBlockTok + kBlockTok - 1) >> g.c_shift, g.N - 1);
+            uint32_t span = c_hi - c_lo + 1;
+            uint32_t bits = (span >= 32 ? 0xffffffffu : ((1u << span) - 1u)) << (c_lo & 31);
+            if (bm[c_lo >> 5] & bits) need = true;
         }
-        uint32_t ball = __ballot_sync(0xffffffffu, need);
+        return need;
+    };
+    int mine = 0;
+    for (int kb0 = kb_lo; kb0 < kb_hi; kb0 += 32) mine += __popc(__ballot_sync(0xffffffffu, block_needed(kb0 + lane)));
+    if (lane == 0) plan_cnt[warp] = mine;
+    __syncthreads();
+    int count = 0, total = 0;
+    for (int i = 0; i < 8; ++i) {
+        if (i < warp) count += plan_cnt[i];
+        total += plan_cnt[i];
+    }
+    int32_t* dst = items + (size_t)(b * g.Hkv + gk) * g.n_kv_blocks_cap;
+    for (int kb0 = kb_lo; kb0 < kb_hi; kb0 += 32) {
+        const int kb = kb0 + lane;
+        const bool need = block_needed(kb);
+        const uint32_t ball = __ballot_sync(0xffffffffu, need);
         if (need) dst[count + __popc(ball & ((1u << lane) - 1u))] = kb;
         count += __popc(ball);
     }
-    if (lane == 0) {
-        n_items[b * g.Hkv + gk] = count;
-        atomicAdd(total_blocks, (unsigned long long)count);
+    if (threadIdx.x == 0) {
+        n_items[b * g.Hkv + gk] = total;
+        atomicAdd(total_blocks, (unsigned long long)total);
     }
 }
 
