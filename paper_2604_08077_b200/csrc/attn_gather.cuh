@@ -15,15 +15,19 @@
 //
 // Which pairs of query tiles take this path is decided on the device, per pair, from the counts the selection
 // left: entries of the pair's rows (P) against key blocks in the pair's union (U), gathered iff
-// P <= pairs_per_block * U.  If the entries of all such pairs exceed the capacity of the workspace, every
-// pair stays on the tile kernel.  Kernels, in launch order:
-//   gather_count_kernel   per pair: row counts, P, U, the decision, entries per key block (atomics)
-//   gather_scan_kernel    one CTA: prefix sums over pairs and key blocks, work items of 128 entries
+// P <= pairs_per_block * U -- provided the qualifying pairs fit the workspace (else part of them, see
+// kGatherClasses) and together save more than the path costs (kGatherMinGain).  The query rows are cut into a
+// few row windows, and every (window, batch, kv head, key block) has its own entry list: the items of a window
+// gather from a slice of Q that stays in L2.  Kernels, in launch order:
+//   gather_count_kernel   per pair: row counts, P, U, the decision, entries per key block list (the warp's
+//                         32 x 32 mask bits are transposed so that lane j holds the rows that selected cube j)
+//   gather_scan_kernel    one CTA: which pairs are kept, prefix sums over pairs and key block lists
+//   gather_items_kernel   work items of up to 128 entries of one list
 //   (attn_prefill_tc_kernel, which reads the decisions)
-//   gather_fill_kernel    per pair: row -> first partial, entries into the lists of their key blocks
-//   attn_gather_kernel    per item: gathered Q rows x one key block -> partials
-//   gather_merge_kernel   per row: merge into `out`
-// The order of a block's entries depends on the order of atomics, but an entry's arithmetic does not depend
+//   gather_fill_kernel    per pair: row -> its slots, entries into the lists of their key blocks
+//   attn_gather_kernel    per item: gathered Q rows x one key block -> partial results, in entry order
+//   gather_merge_kernel   per row of the gathered pairs: merge into `out`
+// The order of a list's entries depends on the order of atomics, but an entry's arithmetic does not depend
 // on its neighbours in the item, and a row merges its partials in ascending block order: results are
 // deterministic.
 #pragma once
@@ -62,8 +66,8 @@ struct GatherWs {
                            // pairs they come from; zero at the start of a forward
     uint32_t* col_cur;     // [kGatherClasses][...] fill cursors; zero at the start of a forward
     uint32_t* col_roff;    // [kGatherClasses][...] first entry of the set's share of the block's list
-    uint32_t* col_off;     // [B*Hkv*n_cols + 1] first entry of the block's list (exclusive prefix sum)
-    uint32_t* col_item;    // [B*Hkv*n_cols + 1] first work item of the block
+    uint32_t* col_off;     // [lists * n_cols + 1] first entry of the block's list (exclusive prefix sum)
+    uint32_t* col_item;    // [lists * n_cols + 1] first work item of the list
     uint4* items;          // (key block column, first entry, entries (<= 128), 0)
     uint32_t* entries;     // per key block, its entries: pos | head in group << 21 | cube bits << 25
     uint32_t* row_slots;   // per row (from row_ptr on), the indices of its entries in ascending block order
