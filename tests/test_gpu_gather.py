@@ -188,3 +188,19 @@ def test_forced_gather_chunked_prefill():
     rep = pu.compare_rows(wl, oracle.all_rows(oracle.shape_of(wl)), out, bm, cnt, label="chunked")
     assert rep["rows"] == wl.B * wl.Hq * wl.S
     assert entries == expected_entries(wl, bm)
+
+
+def test_default_rule_head_dim_64_two_row_windows():
+    """A 32768-token video with head_dim 64, batch 2 and a sharp selection: the library's own rule sends it
+    through the path (several row windows, 16-token cubes: four cubes per key block), sampled rows and two
+    whole query tiles against the oracle."""
+    wl = inputs.make_prefill("gather_d64", seed=41, B=2, T=128, H=16, W=16, cube=(1, 4, 4), n_text=70, Hq=8,
+                             Hkv=2, D=64, top_p=0.4, offset_std=3.0)
+    eng, out, bitmap, count = pu.run_forward(wl, prefill_kernel=1)
+    hdr = eng.header()
+    n_pairs = wl.B * wl.Hq * ((wl.S + 255) // 256)
+    assert hdr.status == 0 and hdr.gather_pair_tiles > 0.5 * n_pairs, (hdr.gather_pair_tiles, n_pairs)
+    n_tiles = (wl.S + 127) // 128
+    rows = pu.sample_rows(wl, 1200, seed=9, whole_tiles=[(1, 5, n_tiles // 2), (0, 2, n_tiles - 1)])
+    rep = pu.compare_rows(wl, rows, out, bitmap, count, label="gather d64")
+    print("gather d64", rep, hdr.gather_pair_tiles, "of", n_pairs, "pairs,", hdr.gather_entries, "entries")
