@@ -366,7 +366,10 @@ adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* 
         }
     }
 #ifdef ADASPARK_WITH_TCGEN05
-    if (!cache_only && h->prefill_kernel != 0) {   // cube-major staging of Q for the TMA loads of K3 / K4
+    // cube-major staging of Q for the TMA loads of K4: the tensor-core selection kernel writes it while it reads
+    // the rows; without that kernel (p >= 1, fp64 selection) this pass does
+    const bool q_staged_by_selection = h->prefill_kernel == 1 && (h->cfg.top_k > 0 || h->cfg.top_p < 1.0f);
+    if (!cache_only && h->prefill_kernel != 0 && !q_staged_by_selection) {
         dim3 rgrid((g.S - g.pos_begin + 3) / 4, g.B);     // slots of the call's row window
         __nv_bfloat16* q_cube = (__nv_bfloat16*)((char*)workspace + h->fw_qcube_off);
         if (D == 128) relayout_q_kernel<128><<<rgrid, 256, 0, st>>>(g, (const __nv_bfloat16*)q, q_cube);
@@ -420,14 +423,14 @@ adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* 
                 return fail(h, ADASPARK_ERR_CUDA, "%s: cuTensorMapEncodeTiled failed", who);
             const int n_items = g.B * g.Hq * (g.n_tiles - g.tile_begin);
             const int grid = n_items < h->sm_count ? n_items : h->sm_count;
-            const __nv_bfloat16* q_cube_c = (const __nv_bfloat16*)(ws + h->fw_qcube_off);
+            __nv_bfloat16* q_cube_w = (__nv_bfloat16*)(ws + h->fw_qcube_off);
             const bool by_count = g.top_k > 0;
 #define ADASPARK_LAUNCH_FUSED(DD, BC)                                                                                  \
     do {                                                                                                               \
         const size_t smem = sizeof(FusedSmem<DD>) + 1024;                                                              \
         if (!set_smem(h, score_select_fused_kernel<DD, BC>, smem, "score_select_fused_kernel")) return ADASPARK_ERR_CUDA; \
         score_select_fused_kernel<DD, BC><<<grid, kFusedThreads, smem, st>>>(                                           \
-            g, n_items, q_cube_c, tmKs, head_max, tile_mask, tile_union, sel_bitmap, sel_count, fallback_rows,         \
+            g, n_items, qb, q_cube_w, tmKs, head_max, tile_mask, tile_union, sel_bitmap, sel_count, fallback_rows,         \
             &hdr->fallback_rows, &hdr->status);                                                                        \
     } while (0)
             if (D == 128) { if (by_count) ADASPARK_LAUNCH_FUSED(128, true); else ADASPARK_LAUNCH_FUSED(128, false); }
