@@ -307,7 +307,8 @@ adaspark_status_t adaspark_attn_set_prefill_kernel(adaspark_attn_t *handle, int3
  * entries).  pairs_per_block = 0 switches the path off (every pair takes the union path); a value above 44
  * forces it for every pair that meets the threshold, a huge value for every pair with a selected cube.  budget_bytes bounds the workspace
  * the path may use for its partial results (2*head_dim + 24 bytes per entry; _partition reserves
- * min(budget, what pairs_per_block lets the pairs of the partition produce, 128 entries per query row));
+ * min(budget, pairs_per_block * video key blocks / 512 entries per query row -- what the pairs of a causal
+ * sequence can produce on average --, 128 entries per query row));
  * if the pairs that qualify in a call need more, only part of them is gathered in that call: the pairs fall
  * into four classes by entries per union block (up to 1/8, 1/4, 1/2 of the threshold, up to the threshold)
  * and into row windows; (class, window) units are kept while they fit, sparsest class first and inside a

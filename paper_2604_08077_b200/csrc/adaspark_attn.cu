@@ -241,8 +241,9 @@ adaspark_status_t adaspark_attn_partition(adaspark_attn_t* h, int32_t batch, int
         const size_t rows_cap = (size_t)batch * Hq * S_cap, n_pairs_cap = ((size_t)S_cap + 255) / 256;
         const uint64_t per_entry = 2ull * D + 16ull + 8ull;      // partial output + (m, l) + entry
         uint64_t cap = h->gather_budget / per_entry;
-        // a pair qualifies with at most threshold x (key blocks of the video) entries, i.e. threshold x n_cols / 256 per row
-        double per_row = std::ceil((double)h->gather_pairs_per_block * (double)n_cols / 256.0);
+        // a pair qualifies with at most threshold x (blocks of its union) entries for its 256 rows, and over a causal
+        // sequence a pair's union averages half the video's key blocks: threshold x n_cols / 512 entries per row
+        double per_row = std::ceil((double)h->gather_pairs_per_block * (double)n_cols / 512.0);
         if (!(per_row < (double)kGatherEntriesPerRow)) per_row = (double)kGatherEntriesPerRow;
         if ((double)cap > (double)rows_cap * per_row) cap = (uint64_t)((double)rows_cap * per_row);
         if (cap > 0xfffffff0ull) cap = 0xfffffff0ull;
