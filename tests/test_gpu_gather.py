@@ -204,3 +204,25 @@ def test_default_rule_head_dim_64_two_row_windows():
     rows = pu.sample_rows(wl, 1200, seed=9, whole_tiles=[(1, 5, n_tiles // 2), (0, 2, n_tiles - 1)])
     rep = pu.compare_rows(wl, rows, out, bitmap, count, label="gather d64")
     print("gather d64", rep, hdr.gather_pair_tiles, "of", n_pairs, "pairs,", hdr.gather_entries, "entries")
+
+
+def test_forced_gather_top_k_tiny_p_and_wide_gqa_group():
+    """The path only consumes the selection masks: the Top-K rule, p -> 0 (the argmax cube alone) and a GQA
+    group of 16 query heads (the widest the library takes: 4 bits of head index in an entry) go through it
+    unchanged."""
+    wl = inputs.small_prefill(seed=42, T=16, H=8, W=8, n_text=19, Hq=4, Hkv=2, top_p=0.9, offset_std=2.0)
+    wl.top_k = 3
+    eng, out, bitmap, count = pu.run_forward(wl, prefill_kernel=1, gather=pu.FORCE_GATHER)
+    assert eng.header().status == 0 and eng.header().gather_entries == expected_entries(wl, bitmap)
+    rep = pu.compare_rows(wl, oracle.all_rows(oracle.shape_of(wl)), out, bitmap, count, label="top-k gather")
+    assert rep["rows"] == wl.B * wl.Hq * wl.S
+    wl = inputs.small_prefill(seed=43, T=16, H=8, W=8, n_text=19, Hq=4, Hkv=2, top_p=1e-6)
+    eng, out, bitmap, count = pu.run_forward(wl, prefill_kernel=1, gather=pu.FORCE_GATHER)
+    assert eng.header().status == 0 and eng.header().gather_entries == expected_entries(wl, bitmap)
+    rep = pu.compare_rows(wl, oracle.all_rows(oracle.shape_of(wl)), out, bitmap, count, label="argmax gather")
+    assert rep["rows"] == wl.B * wl.Hq * wl.S
+    wl = inputs.small_prefill(seed=44, T=16, H=8, W=8, n_text=9, Hq=16, Hkv=1, D=64, top_p=0.7, offset_std=2.5)
+    eng, out, bitmap, count = pu.run_forward(wl, prefill_kernel=1, gather=pu.FORCE_GATHER)
+    assert eng.header().status == 0 and eng.header().gather_entries == expected_entries(wl, bitmap)
+    rep = pu.compare_rows(wl, oracle.all_rows(oracle.shape_of(wl)), out, bitmap, count, label="gqa16 gather")
+    assert rep["rows"] == wl.B * wl.Hq * wl.S
