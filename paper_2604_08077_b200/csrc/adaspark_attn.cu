@@ -33,7 +33,7 @@ struct adaspark_attn {
     adaspark_attn_layout_t layout;
     // workspace carving (byte offsets)
     size_t fw_status_off, fw_headmax_off, fw_valid_off, fw_gcol_off, fw_mask_off, fw_union_off, fw_fallback_off, fw_scratch_off,
-        fw_qcube_off, fw_kplanes_off, fw_gpair_off, fw_grow_off, fw_gml_off, fw_gitems_off, fw_gentries_off, fw_gparto_off,
+        fw_kplanes_off, fw_gpair_off, fw_grow_off, fw_gml_off, fw_gitems_off, fw_gentries_off, fw_gparto_off,
         fw_gpartml_off, fw_total;
     // query-gather path of the prefill: capacity in (row, key block) entries, decision threshold, byte budget
     uint32_t gather_cap;
@@ -97,6 +97,7 @@ Geom make_geom(const adaspark_attn* h, int n_text, int frame_begin = 0, int fram
     // so that frames count the same in tokens and in slots)
     g.S = (frame_end == h->T ? h->S_v : frame_end * h->H * h->W) + n_prefix + n_text;
     g.pos_begin = frame_begin * h->H * h->W;
+    g.frame_begin = frame_begin;
     g.S_io = (frame_end - frame_begin) * h->H * h->W + n_prefix + n_text;
     g.tile_begin = g.pos_begin / kTileRows;
     g.N_live = ((frame_end + g.ct - 1) / g.ct) * g.nH * g.nW;
@@ -231,7 +232,6 @@ adaspark_status_t adaspark_attn_partition(adaspark_attn_t* h, int32_t batch, int
     h->fw_union_off = off; off = align_up(off + (size_t)batch * Hq * n_tiles_cap * n_words * 4);
     h->fw_fallback_off = off; off = align_up(off + (size_t)batch * Hq * n_tiles_cap * kTileRows * 4);
     h->fw_scratch_off = off; off = align_up(off + (size_t)kExactCtas * kExactWarps * N_ld * 8);
-    h->fw_qcube_off = off; off = align_up(off + (size_t)batch * Hq * S_cap * D * 2);
     // digit planes (4 x int8 [B*Hkv*N_ld, 128]) of the mean keys; 128 rows of slack so that the last TMA box
     // stays inside the allocation
     h->fw_kplanes_off = off; off = align_up(off + ((size_t)4 * batch * Hkv * N_ld + 128) * 128);
@@ -366,18 +366,6 @@ adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* 
             if (!launch_ok(h, "pool_large_cubes_kernel")) return ADASPARK_ERR_CUDA;
         }
     }
-#ifdef ADASPARK_WITH_TCGEN05
-    // cube-major staging of Q for the TMA loads of K4: the tensor-core selection kernel writes it while it reads
-    // the rows; without that kernel (p >= 1, fp64 selection) this pass does
-    const bool q_staged_by_selection = h->prefill_kernel == 1 && (h->cfg.top_k > 0 || h->cfg.top_p < 1.0f);
-    if (!cache_only && h->prefill_kernel != 0 && !q_staged_by_selection) {
-        dim3 rgrid((g.S - g.pos_begin + 3) / 4, g.B);     // slots of the call's row window
-        __nv_bfloat16* q_cube = (__nv_bfloat16*)((char*)workspace + h->fw_qcube_off);
-        if (D == 128) relayout_q_kernel<128><<<rgrid, 256, 0, st>>>(g, (const __nv_bfloat16*)q, q_cube);
-        else relayout_q_kernel<64><<<rgrid, 256, 0, st>>>(g, (const __nv_bfloat16*)q, q_cube);
-        if (!launch_ok(h, "relayout_q_kernel")) return ADASPARK_ERR_CUDA;
-    }
-#endif
     mark(h, 1, st);
     if (cache_only) return ADASPARK_OK;
 
@@ -424,14 +412,13 @@ adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* 
                 return fail(h, ADASPARK_ERR_CUDA, "%s: cuTensorMapEncodeTiled failed", who);
             const int n_items = g.B * g.Hq * (g.n_tiles - g.tile_begin);
             const int grid = n_items < h->sm_count ? n_items : h->sm_count;
-            __nv_bfloat16* q_cube_w = (__nv_bfloat16*)(ws + h->fw_qcube_off);
             const bool by_count = g.top_k > 0;
 #define ADASPARK_LAUNCH_FUSED(DD, BC)                                                                                  \
     do {                                                                                                               \
         const size_t smem = sizeof(FusedSmem<DD>) + 1024;                                                              \
         if (!set_smem(h, score_select_fused_kernel<DD, BC>, smem, "score_select_fused_kernel")) return ADASPARK_ERR_CUDA; \
         score_select_fused_kernel<DD, BC><<<grid, kFusedThreads, smem, st>>>(                                           \
-            g, n_items, qb, q_cube_w, tmKs, head_max, tile_mask, tile_union, sel_bitmap, sel_count, fallback_rows,         \
+            g, n_items, qb, tmKs, head_max, tile_mask, tile_union, sel_bitmap, sel_count, fallback_rows,         \
             &hdr->fallback_rows, &hdr->status);                                                                        \
     } while (0)
             if (D == 128) { if (by_count) ADASPARK_LAUNCH_FUSED(128, true); else ADASPARK_LAUNCH_FUSED(128, false); }
@@ -452,9 +439,18 @@ adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* 
     // K4: gathered attention
 #ifdef ADASPARK_WITH_TCGEN05
     if (h->prefill_kernel != 0) {
-        __nv_bfloat16* q_cube = (__nv_bfloat16*)(ws + h->fw_qcube_off);
+        // Q tiles are boxes of the caller's tensor [B, S_io, Hq, D] seen as (head x d, x, y, frame, batch) from its first
+        // video token on: a box = min(C, 128) cube-major rows = a slab of the cube window
         CUtensorMap tmQ, tmK, tmV;
-        if (!encode_bf16_2d(&tmQ, q_cube, (uint64_t)g.B * g.Hq * g.S_cap, D, 64, 128) ||
+        uint32_t bx = (uint32_t)(g.cw < 128 ? g.cw : 128), by = (uint32_t)(g.ch < 128 / (int)bx ? g.ch : 128 / (int)bx);
+        uint32_t bt = (uint32_t)(g.ct < 128 / (int)(bx * by) ? g.ct : 128 / (int)(bx * by));
+        if (bt < 1) bt = 1;
+        const uint64_t tok = (uint64_t)g.Hq * D * 2;
+        const int frames_here = frame_count > 0 ? frame_count : 1;
+        const uint64_t qdims[5] = {(uint64_t)g.Hq * D, (uint64_t)g.W, (uint64_t)g.H, (uint64_t)frames_here, (uint64_t)g.B};
+        const uint64_t qstr[4] = {tok, (uint64_t)g.W * tok, (uint64_t)g.H * g.W * tok, (uint64_t)g.S_io * tok};
+        const uint32_t qbox[5] = {64u, bx, by, bt, 1u};
+        if (!encode_bf16_5d(&tmQ, qb + (size_t)g.n_prefix * g.Hq * D, qdims, qstr, qbox) ||
             !encode_bf16_2d(&tmK, kc, (uint64_t)g.B * g.Hkv * g.S_cap, D, 64, 64) ||
             !encode_bf16_2d(&tmV, vc, (uint64_t)g.B * g.Hkv * g.n_kv_blocks_cap * D, 64, 64, D))
             return fail(h, ADASPARK_ERR_CUDA, "%s: cuTensorMapEncodeTiled failed", who);
@@ -510,13 +506,13 @@ adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* 
         if (D == 128) {
             size_t smem = sizeof(TcAttnSmem<128>) + 1024;
             if (!set_smem(h, attn_prefill_tc_kernel<128>, smem, "attn_prefill_tc_kernel")) return ADASPARK_ERR_CUDA;
-            attn_prefill_tc_kernel<128><<<grid, kTcThreads, smem, st>>>(g, tmQ, tmK, tmV, tile_mask, tile_union, slot_valid_c, pair_mode_c,
+            attn_prefill_tc_kernel<128><<<grid, kTcThreads, smem, st>>>(g, tmQ, qb, tmK, tmV, tile_mask, tile_union, slot_valid_c, pair_mode_c,
                                                                         gw.n_pairs_cap, gw.ml_local, (__nv_bfloat16*)out,
                                                                         (unsigned long long*)&hdr->executed_kv_blocks, &hdr->max_tile_kv_blocks, &hdr->status);
         } else {
             size_t smem = sizeof(TcAttnSmem<64>) + 1024;
             if (!set_smem(h, attn_prefill_tc_kernel<64>, smem, "attn_prefill_tc_kernel")) return ADASPARK_ERR_CUDA;
-            attn_prefill_tc_kernel<64><<<grid, kTcThreads, smem, st>>>(g, tmQ, tmK, tmV, tile_mask, tile_union, slot_valid_c, pair_mode_c,
+            attn_prefill_tc_kernel<64><<<grid, kTcThreads, smem, st>>>(g, tmQ, qb, tmK, tmV, tile_mask, tile_union, slot_valid_c, pair_mode_c,
                                                                        gw.n_pairs_cap, gw.ml_local, (__nv_bfloat16*)out,
                                                                        (unsigned long long*)&hdr->executed_kv_blocks, &hdr->max_tile_kv_blocks, &hdr->status);
         }
@@ -532,7 +528,7 @@ adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* 
             if (D == 128) {
                 const size_t smem = sizeof(GatherSmem<128>) + 1024;
                 if (!set_smem(h, attn_gather_kernel<128>, smem, "attn_gather_kernel")) return ADASPARK_ERR_CUDA;
-                attn_gather_kernel<128><<<ggrid, kGatherThreads, smem, st>>>(g, gw, tmKg, tmV, q_cube, slot_valid_c,
+                attn_gather_kernel<128><<<ggrid, kGatherThreads, smem, st>>>(g, gw, tmKg, tmV, qb, slot_valid_c,
                                                                             (unsigned long long*)&hdr->executed_kv_blocks, &hdr->status);
                 if (!launch_ok(h, "attn_gather_kernel")) return ADASPARK_ERR_CUDA;
                 const long long ctas = (n_rows + 15) / 16;
@@ -540,7 +536,7 @@ adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* 
             } else {
                 const size_t smem = sizeof(GatherSmem<64>) + 1024;
                 if (!set_smem(h, attn_gather_kernel<64>, smem, "attn_gather_kernel")) return ADASPARK_ERR_CUDA;
-                attn_gather_kernel<64><<<ggrid, kGatherThreads, smem, st>>>(g, gw, tmKg, tmV, q_cube, slot_valid_c,
+                attn_gather_kernel<64><<<ggrid, kGatherThreads, smem, st>>>(g, gw, tmKg, tmV, qb, slot_valid_c,
                                                                            (unsigned long long*)&hdr->executed_kv_blocks, &hdr->status);
                 if (!launch_ok(h, "attn_gather_kernel")) return ADASPARK_ERR_CUDA;
                 const long long ctas = (n_rows + 31) / 32;

@@ -335,8 +335,8 @@ __global__ void __launch_bounds__(1024) gather_scan_kernel(Geom g, GatherWs ws) 
     uint32_t my_e = 0, my_i = 0;
     for (int col = c0; col < c1; ++col) {
         uint32_t v = 0;
-#pragma unroll
         const int win = col / cols_per_window;
+#pragma unroll
         for (int r = 0; r < kGatherClasses; ++r)
             if ((unit_keep[r] >> win) & 1u) v += ws.col_cnt[(size_t)r * n_cols_all + col];
         my_e += v;
@@ -351,8 +351,8 @@ __global__ void __launch_bounds__(1024) gather_scan_kernel(Geom g, GatherWs ws) 
         ws.col_off[col] = o;
         ws.col_item[col] = i_off;
         uint32_t v = 0;
-#pragma unroll
         const int win = col / cols_per_window;
+#pragma unroll
         for (int r = 0; r < kGatherClasses; ++r) {
             if ((unit_keep[r] >> win) & 1u) {
                 const uint32_t part = ws.col_cnt[(size_t)r * n_cols_all + col];
@@ -501,12 +501,11 @@ struct GatherSmem {
 template <int D>
 __global__ void __launch_bounds__(kGatherThreads, 1) attn_gather_kernel(
     Geom g, GatherWs ws, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-    const __nv_bfloat16* __restrict__ q_cube, const uint32_t* __restrict__ slot_valid,
+    const __nv_bfloat16* __restrict__ q, const uint32_t* __restrict__ slot_valid,
     unsigned long long* __restrict__ executed_blocks, int32_t* __restrict__ status) {
     extern __shared__ unsigned char gather_smem_raw[];
     GatherSmem<D>& sm = *reinterpret_cast<GatherSmem<D>*>((reinterpret_cast<uintptr_t>(gather_smem_raw) + 1023) & ~(uintptr_t)1023);
     constexpr int kPanels = D / 64, kQKSteps = D / 16;
-    constexpr int kPairsPerRow = D / 16;                         // 32-byte pieces of a Q row
     constexpr uint32_t kIdescS = tc::make_idesc_bf16(128, 64);   // S: 128 gathered rows x 64 keys
     constexpr uint32_t kIdescO = tc::make_idesc_bf16(128, D);    // O: 128 rows x D
     constexpr uint32_t kKVBytes = 64 * D * 2 * 2;
@@ -725,14 +724,15 @@ __global__ void __launch_bounds__(kGatherThreads, 1) attn_gather_kernel(
             if (!(ok = tc::mbar_wait(&sm.q_empty[st], ((i / kGatherStages) & 1) ^ 1, abort_flag))) break;
             const int bg = (int)(d_cur.x / (uint32_t)ws.n_cols) % (g.B * g.Hkv);
             const int b = bg / g.Hkv, gk = bg - b * g.Hkv;
-            const size_t head0 = (size_t)(b * g.Hq + gk * g.G);
+            const int head0 = gk * g.G;
             unsigned char* qbase = reinterpret_cast<unsigned char*>(&sm.q[st][0][0][0]) + (piece >> 3) * (128 * 128);
 #pragma unroll
             for (int ps = 0; ps < kPasses; ++ps) {
                 const int row = ps * kRowsPerPass + rsub;
                 if (row < n) {
                     const uint32_t e = e_cur[ps];
-                    const __nv_bfloat16* src = q_cube + ((head0 + ((e >> 21) & 15u)) * g.S_cap + (e & kEntryPosMask)) * D;
+                    // (a gathered row holds a token: its place in the caller's tensor [B, S_io, Hq, D])
+                    const __nv_bfloat16* src = q + (io_row(g, b, (int)(e & kEntryPosMask)) * g.Hq + head0 + (int)((e >> 21) & 15u)) * D;
                     cp_async_16(qbase + sw128(row, piece & 7), src + piece * 8);
                 }
             }

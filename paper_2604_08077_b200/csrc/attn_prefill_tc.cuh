@@ -62,7 +62,7 @@ struct BlockIter {
 
 template <int D>
 __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
-    Geom g, const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+    Geom g, const __grid_constant__ CUtensorMap tmQ, const __nv_bfloat16* __restrict__ q, const __grid_constant__ CUtensorMap tmK,
     const __grid_constant__ CUtensorMap tmV, const uint32_t* __restrict__ tile_mask,
     const uint32_t* __restrict__ tile_union, const uint32_t* __restrict__ slot_valid, const uint32_t* __restrict__ pair_mode,
     int n_pairs_cap, float2* __restrict__ ml_local, __nv_bfloat16* __restrict__ out,
@@ -73,7 +73,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     constexpr int kQKSteps = D / 16;                            // k-steps of S = Q K^T
     constexpr uint32_t kIdescS = tc::make_idesc_bf16(128, 128);  // S tile: 128 rows x 128 keys
     constexpr uint32_t kIdescO = tc::make_idesc_bf16(128, D);    // O tile: 128 rows x D
-    constexpr uint32_t kQBytes = 2 * 128 * D * 2, kKBytes = 128 * D * 2, kVBytes = 2 * D * 64 * 2;
+    constexpr uint32_t kKBytes = 128 * D * 2, kVBytes = 2 * D * 64 * 2;
 
     const int n_pairs = (g.S + kPairRows - 1) / kPairRows;
     // 1-D grid, pair-major: the late (long) pair tiles of every head and batch entry start first
@@ -120,12 +120,50 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
         }
     }
     __syncthreads();                                            // barriers initialised
-    if (warp == 8 && lane == 0) {
-        // the Q tiles do not depend on the block plan: their load overlaps the union computation below
-        const int q_row0 = (b * g.Hq + h) * g.S_cap + pair_pos0;
-        tc::mbar_arrive_expect_tx(&sm.q_full, kQBytes);
-        for (int t = 0; t < 2; ++t)
-            for (int p = 0; p < kPanels; ++p) tc::tma_load_2d(&sm.q[t][p][0][0], &tmQ, p * 64, q_row0 + t * 128, &sm.q_full);
+    if (warp == 8) {
+        // The Q tiles do not depend on the block plan: their load overlaps the union computation below.  They come
+        // straight from the caller's tensor [B, S_io, Hq, D]: the video rows of a tile are whole boxes of a cube's
+        // window (or the cubes themselves, below 128 tokens) in the (head x d, x, y, t, batch) view of that tensor,
+        // which one 5-D TMA load per box and 64-element panel turns into cube-major rows (a coordinate beyond the
+        // grid reads zeros: the empty slots of a boundary cube); text rows and the slots beyond the sequence,
+        // a few tiles per head, are copied by the warp's lanes.
+        const int rpb = min(g.C, 128);                            // rows per box
+        uint32_t tx_bytes = 0;
+#pragma unroll 1
+        for (int t = 0; t < 2; ++t) {
+            const int p0 = pair_pos0 + t * 128;
+            const int n_vid = max(0, min(p0 + 128, g.S_v) - p0);  // video slots of the tile (a multiple of rpb or of C)
+            for (int idx = lane; idx < (128 - n_vid) * (D / 8); idx += 32) {
+                const int row = n_vid + idx / (D / 8), c = idx % (D / 8);
+                const int pos = p0 + row;
+                uint4 val = make_uint4(0u, 0u, 0u, 0u);
+                if (pos < g.S) val = __ldg(reinterpret_cast<const uint4*>(q + (io_row(g, b, pos) * g.Hq + h) * D) + c);
+                *reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(&sm.q[t][c >> 3][0][0]) + sw128(row, c & 7)) = val;
+            }
+            tx_bytes += (uint32_t)n_vid * D * 2;
+        }
+        asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");   // the copied rows are read by the tensor core
+        __syncwarp();
+        if (lane == 0) {
+            if (tx_bytes) tc::mbar_arrive_expect_tx(&sm.q_full, tx_bytes);
+            else tc::mbar_arrive(&sm.q_full);
+            for (int t = 0; t < 2; ++t) {
+                const int p0 = pair_pos0 + t * 128;
+                const int n_vid = max(0, min(p0 + 128, g.S_v) - p0);
+                for (int r = 0; r < n_vid; r += rpb) {
+                    const int pos = p0 + r;
+                    const int c = pos >> g.c_shift, r0 = pos & (g.C - 1);
+                    int cx, cy, cb, tt;
+                    g.div_nW.divmod(c, tt, cx);
+                    g.div_nH.divmod(tt, cb, cy);
+                    const int x = cx * g.cw + (r0 & (g.cw - 1));
+                    const int y = cy * g.ch + ((r0 >> g.cw_shift) & (g.ch - 1));
+                    const int fr = cb * g.ct + (r0 >> (g.cw_shift + g.ch_shift)) - g.frame_begin;
+                    for (int p = 0; p < kPanels; ++p)
+                        tc::tma_load_5d(&sm.q[t][p][r][0], &tmQ, h * D + p * 64, x, y, fr, b, &sm.q_full);
+                }
+            }
+        }
     }
     // union of the selection words of the 256 rows = OR of the two tiles' union words (written by the
     // selection kernel)
@@ -515,26 +553,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
         }
     }
     if (warp == 8) tc::tmem_dealloc<512>(tbase);
-}
-
-// cube-major staging of Q for the TMA loads of the attention kernel:
-// q_cube[(b*Hq + h) * S_cap + pos][:] = q[b, raster(pos), h, :]
-template <int D>
-__global__ void __launch_bounds__(256) relayout_q_kernel(Geom g, const __nv_bfloat16* __restrict__ q,
-                                                         __nv_bfloat16* __restrict__ q_cube) {
-    constexpr int kChunks = D / 8;
-    const int pos0 = g.pos_begin + blockIdx.x * 4;      // 4 positions x all heads per CTA: many small CTAs
-    const int b = blockIdx.y;
-    const int per_pos = g.Hq * kChunks;
-    for (int idx = threadIdx.x; idx < 4 * per_pos; idx += 256) {
-        int p = idx / per_pos, rem = idx - p * per_pos;
-        int h = rem / kChunks, c = rem - h * kChunks;
-        int pos = pos0 + p;
-        if (pos >= g.S) break;
-        uint4 val = make_uint4(0u, 0u, 0u, 0u);              // an empty slot of a boundary cube stays zero
-        if (slot_live(g, pos)) val = *reinterpret_cast<const uint4*>(q + (io_row(g, b, pos) * g.Hq + h) * D + c * 8);
-        *reinterpret_cast<uint4*>(q_cube + ((size_t)(b * g.Hq + h) * g.S_cap + pos) * D + c * 8) = val;
-    }
 }
 
 }  // namespace adaspark

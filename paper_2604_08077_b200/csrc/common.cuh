@@ -55,6 +55,7 @@ struct Geom {
     // cube-major positions are [pos_begin, S) -- whole time blocks of cubes, so they are also the raster
     // tokens pos_begin .. -- and only those rows are computed.  One-shot prefill: pos_begin = 0, S_io = S.
     int pos_begin, S_io;
+    int frame_begin;     // first frame of this call's tensors
     int N_live;          // cubes present after this call (<= N)
     int tile_begin;      // pos_begin / 128
     int S_cap;           // cache rows per (b, kv head), multiple of 128

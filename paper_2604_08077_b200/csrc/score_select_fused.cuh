@@ -209,13 +209,13 @@ __device__ __forceinline__ void tmem_ld_32x4(uint32_t taddr, uint32_t* r) {   //
                  : "memory");
 }
 
-// q: the call's queries [B, S_io, Hq, D]; q_cube: their cube-major copy [B*Hq, S_cap, D], written here.  tile_mask as mask_index() describes;
+// q: the call's queries [B, S_io, Hq, D].  tile_mask as mask_index() describes;
 // tile_union[((b*Hq+h)*n_tiles_cap + tile)*n_words + w] = OR of word w over the tile's rows.
 // fallback_rows[0 .. *fallback_count) receives ((b*Hq+h)*n_tiles_cap + tile)*128 + r of the rows left
 // to the fp64 kernel.
 template <int D, bool kByCount>
 __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
-    Geom g, int n_items, const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ q_cube, const __grid_constant__ CUtensorMap tmK,
+    Geom g, int n_items, const __nv_bfloat16* __restrict__ q, const __grid_constant__ CUtensorMap tmK,
     const uint32_t* __restrict__ head_max_bits, uint32_t* __restrict__ tile_mask, uint32_t* __restrict__ tile_union,
     uint32_t* __restrict__ sel_bitmap, int32_t* __restrict__ sel_count, int32_t* __restrict__ fallback_rows,
     uint32_t* __restrict__ fallback_count, int32_t* __restrict__ status) {
@@ -358,17 +358,11 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
         int n_done = 0;
         for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
             const FusedItem w = fused_item(g, it);
+            if (w.n_ct == 0) continue;
             const int pos = w.tile * kTileRows + r;
             const bool live = slot_live(g, pos);
-            // The row is read from the caller's tensor (sequence order) and, on the way, written to the cube-major
-            // copy of Q that the attention kernels load with TMA: no separate re-layout pass over Q.
+            // the row is read where the caller left it (sequence order): no cube-major copy of Q exists
             const uint4* src = reinterpret_cast<const uint4*>(q + (live ? (io_row(g, w.b, pos) * g.Hq + w.h) * D : 0));
-            uint4* cube_dst = reinterpret_cast<uint4*>(q_cube + ((size_t)(w.b * g.Hq + w.h) * g.S_cap + pos) * D);
-            if (w.n_ct == 0) {                                    // a tile without candidates: only the copy
-#pragma unroll
-                for (int c = 0; c < D / 8; ++c) cube_dst[c] = live ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
-                continue;
-            }
             // first sweep over the row (before the planes are free): its largest exponent
             uint32_t mxbits = 0;
             if (live) {
@@ -391,8 +385,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
             for (int o = 0; o < D / 16; ++o) {                    // 16 elements = one 16-byte chunk of every plane
                 const uint4 va = live ? __ldg(src + 2 * o) : make_uint4(0u, 0u, 0u, 0u);
                 const uint4 vb = live ? __ldg(src + 2 * o + 1) : make_uint4(0u, 0u, 0u, 0u);
-                cube_dst[2 * o] = va;                             // an empty slot of a boundary cube stays zero
-                cube_dst[2 * o + 1] = vb;
                 uint32_t pw[4][4];                                // [plane][4 elements per word]
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4) {                  // elements 16*o + 4*q4 .. +3 = two packed bf16 words
