@@ -527,17 +527,15 @@ def main():
             result["dense"] = {"error": repr(e)[:200]}
 
     # ------------------------------------------------------------------ rooflines of the other stages
-    # re-layout + pooling (K/V once in, once out, fp32 keys): an HBM-bound copy.  (The cube-major copy of Q is
-    # written by the selection kernel while it reads the rows.)
+    # re-layout + pooling (K/V once in, once out, fp32 keys): an HBM-bound copy (Q is not re-laid out)
     relayout_bytes = 2 * (k.numel() + v.numel()) * 2 + wl.B * wl.Hkv * wl.N * wl.D * 4
     rl_gbs = relayout_bytes / (float(st_mean[0]) * 1e-3) / 1e9
-    # scoring + selection: candidate (row, cube) pairs; algorithmic bytes = Q once in, once out (cube-major copy for
-    # the attention kernels' TMA loads) + mean keys + mask words
+    # scoring + selection: candidate (row, cube) pairs; algorithmic bytes = Q once + mean keys + mask words
     n_tiles = (wl.S + 127) // 128
     pos = np.arange(wl.S)
     cand_per_row = np.where(pos < wl.S_v, pos // C, wl.N)
     pairs = float(cand_per_row.sum()) * wl.B * wl.Hq
-    ss_bytes = 2 * q.numel() * 2 + wl.B * wl.Hkv * wl.N * wl.D * 4 + wl.B * wl.Hq * n_tiles * 128 * ((wl.N + 31) // 32) * 4
+    ss_bytes = q.numel() * 2 + wl.B * wl.Hkv * wl.N * wl.D * 4 + wl.B * wl.Hq * n_tiles * 128 * ((wl.N + 31) // 32) * 4
     ss_ms = float(st_mean[1])
     result["stage_rooflines"] = {
         "relayout": {"bound": "hbm", "bytes": relayout_bytes, "ms": float(st_mean[0]), "achieved": rl_gbs,

@@ -118,8 +118,8 @@ adaspark_status_t adaspark_attn_create(const adaspark_attn_config_t *config,
  * the mean over the tokens they hold, their other slots stay empty in the caches and are never attended.
  * ERR_UNSUPPORTED if N > 4096 or the cache would hold more than 2097152 rows per sequence
  * (s_video + n_text_max + 1).
- * The forward workspace holds the selection masks, the cube-major copy of Q and the digit planes of the
- * mean keys; cube scores are never stored. */
+ * The forward workspace holds the selection masks, the digit planes of the mean keys and the buffers of the
+ * query-gather path; cube scores are never stored and Q is read where the caller left it. */
 adaspark_status_t adaspark_attn_partition(adaspark_attn_t *handle, int32_t batch, int32_t frames,
                                           int32_t grid_h, int32_t grid_w, int32_t n_text_max,
                                           size_t *workspace_bytes);

@@ -214,7 +214,7 @@ adaspark_status_t adaspark_attn_partition(adaspark_attn_t* h, int32_t batch, int
     L.cube_keys_bytes = (int64_t)((size_t)batch * Hkv * N * D * 4);
 
     // forward workspace: header | head exponents | per-tile mask matrix | per-tile union words | rows left to
-    // the fp64 selection kernel | its score scratch | cube-major Q | key digit planes (tcgen05 path)
+    // the fp64 selection kernel | its score scratch | key digit planes (tcgen05 path)
     size_t off = 0;
     h->fw_status_off = off; off = align_up(off + 256);
     h->fw_headmax_off = off; off = align_up(off + (size_t)batch * Hkv * 4);
