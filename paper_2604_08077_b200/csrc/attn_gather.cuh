@@ -50,7 +50,7 @@ constexpr int kGatherClasses = 4;       // a qualifying pair falls into a class 
 // launches, the scan) eat the gain.
 constexpr long long kGatherBreakEven = 44;
 constexpr long long kGatherMinGain = 300000;
-constexpr uint32_t kEntryPosMask = 0x1fffffu;   // 21 bits of cube-major position (caches hold at most 2^21 rows)
+constexpr uint32_t kEntryPosMask = 0x1fffffu;   // 21 bits of token index (a sequence holds at most 2^21 rows)
 
 // Pointers into the forward workspace and sizes (all filled by the host).
 struct GatherWs {
@@ -69,7 +69,7 @@ struct GatherWs {
     uint32_t* col_off;     // [lists * n_cols + 1] first entry of the block's list (exclusive prefix sum)
     uint32_t* col_item;    // [lists * n_cols + 1] first work item of the list
     uint4* items;          // (key block column, first entry, entries (<= 128), 0)
-    uint32_t* entries;     // per key block, its entries: pos | head in group << 21 | cube bits << 25
+    uint32_t* entries;     // per key block, its entries: row of the call's tensors | head in group << 21 | cube bits << 25
     uint32_t* row_slots;   // per row (from row_ptr on), the indices of its entries in ascending block order
     __nv_bfloat16* part_o; // [cap_entries][D] normalised partial output of every entry (in entry order: an item
                            // of the attention kernel writes one contiguous piece)
@@ -413,7 +413,9 @@ __global__ void __launch_bounds__(256) gather_fill_kernel(Geom g, GatherWs ws, c
     const uint32_t* my = tile_mask + mask_index(g, it.b, it.h, tile, 0, r);
     const int win = (it.pair - g.pos_begin / kPairRows) / ws.pairs_per_window;
     const size_t colbase = ((size_t)(mode - 1u) * ws.n_lists + ((size_t)win * g.B + it.b) * g.Hkv + it.gk) * ws.n_cols;
-    const uint32_t ent_x = (uint32_t)pos | ((uint32_t)(it.h - it.gk * g.G) << 21);
+    // an entry names its query row by the token's index in the call's tensors (what the gather needs), not by
+    // its cube-major position: the conversion is done once here, not per copy in the attention kernel
+    const uint32_t ent_x = (uint32_t)(slot_live(g, pos) ? pos_to_io(g, pos) - g.pos_begin : 0) | ((uint32_t)(it.h - it.gk * g.G) << 21);
     const uint32_t lt_mask = (1u << lane) - 1u;
     // Four words per step.  After the transposition lane j holds the rows of the warp that selected cube 32 w + j;
     // ONE round of atomics reserves the slots of all (word, cube) pairs of the step in their blocks' lists (the
@@ -731,8 +733,8 @@ __global__ void __launch_bounds__(kGatherThreads, 1) attn_gather_kernel(
                 const int row = ps * kRowsPerPass + rsub;
                 if (row < n) {
                     const uint32_t e = e_cur[ps];
-                    // (a gathered row holds a token: its place in the caller's tensor [B, S_io, Hq, D])
-                    const __nv_bfloat16* src = q + (io_row(g, b, (int)(e & kEntryPosMask)) * g.Hq + head0 + (int)((e >> 21) & 15u)) * D;
+                    // the row's place in the caller's tensor [B, S_io, Hq, D]
+                    const __nv_bfloat16* src = q + (((size_t)b * g.S_io + (e & kEntryPosMask)) * g.Hq + head0 + (int)((e >> 21) & 15u)) * D;
                     cp_async_16(qbase + sw128(row, piece & 7), src + piece * 8);
                 }
             }
