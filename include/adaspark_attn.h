@@ -139,12 +139,12 @@ adaspark_status_t adaspark_attn_get_layout(const adaspark_attn_t *handle,
  *                     order) is set iff cube j is in the row's nucleus S_i.
  *   sel_count    out, nullable: int32 [B, Hq, S] = |S_i|.
  *   workspace    device scratch of at least forward_workspace_bytes, 256-byte aligned.
- * Enqueues kernels and returns; no host synchronisation.  The scoring of one chunk of query tiles
- * runs concurrently with the selection of the previous chunk: the selection kernels are enqueued
- * on a stream private to the handle, ordered against `cuda_stream` with events in both directions,
- * so that everything the call enqueued is complete, from the point of view of `cuda_stream`, before
- * any later work on it.  The first _forward of a handle creates that stream and its events (make
- * that first call before any stream capture). */
+ * Enqueues its kernels on `cuda_stream` and returns; no host synchronisation, no other stream, no
+ * allocation.  The Q tiles of the attention kernel are TMA boxes of `q` itself (the tensor map is built
+ * on the host per call): `q` needs 16-byte alignment and must stay valid until the call's work is done.
+ * Which of the two attention paths a pair of query tiles takes (union of the selected key blocks, or
+ * the query-gather path of adaspark_attn_set_gather) is decided on the device; the workspace header
+ * reports it. */
 adaspark_status_t adaspark_attn_forward(adaspark_attn_t *handle, const void *q, const void *k,
                                         const void *v, int32_t n_text, void *out, void *k_cube,
                                         void *v_cube, float *cube_keys, uint32_t *sel_bitmap,
