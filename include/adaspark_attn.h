@@ -266,8 +266,9 @@ adaspark_status_t adaspark_attn_decode_static(adaspark_attn_t *handle, const voi
                                               const int32_t *text_len, void *out,
                                               uint32_t *sel_bitmap, void *cuda_stream);
 
-/* Release the handle: host memory, and the private stream / events of a handle that ran _forward
- * (waits for that stream to drain).  NULL is accepted. */
+/* Release the handle: its host memory and, if stage timing was enabled, the timing events.  It does
+ * not wait for work enqueued on the caller's streams, and the caller's buffers are not touched: destroy
+ * the handle after that work is done.  NULL is accepted. */
 adaspark_status_t adaspark_attn_destroy(adaspark_attn_t *handle);
 
 /* Message of the most recent error on this handle ("" if none). Never NULL. */
