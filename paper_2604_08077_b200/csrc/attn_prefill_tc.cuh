@@ -239,18 +239,23 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
         }
     } else if (warp == 9) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // The whole warp runs the loop and one elected lane issues: with every operand warp-uniform the
+        // thread gets a 128x128x16 MMA accepted every 85 - 90 cycles; from a branch entered by lane 0 alone
+        // it was 113 - 125 (the tensor core needs 64).
+        {
             // descriptor low halves of the tile bases; a k-step of 16 elements advances 32 bytes
             // inside a 64-element panel (128-byte rows), panels / key blocks are 128 rows apart
             constexpr uint32_t kPanelStep = (128 * 64 * 2) >> 4, kKStep = 32 >> 4;
             constexpr uint32_t kVBlockStep = (D * 64 * 2) >> 4;
             constexpr uint32_t kQTileStep = (uint32_t)sizeof(sm.q[0]) >> 4, kKStageStep = (uint32_t)sizeof(sm.k[0]) >> 4;
             constexpr uint32_t kVStageStep = (uint32_t)sizeof(sm.v[0]) >> 4;
-            const uint32_t q_lo0 = tc::smem_desc_lo_sw128(smem_u32(&sm.q[0][0][0][0]));
-            const uint32_t k_lo0 = tc::smem_desc_lo_sw128(smem_u32(&sm.k[0][0][0][0]));
-            const uint32_t v_lo0 = tc::smem_desc_lo_sw128(smem_u32(&sm.v[0][0][0][0]));
+            const uint32_t q_lo0 = __shfl_sync(0xffffffffu, tc::smem_desc_lo_sw128(smem_u32(&sm.q[0][0][0][0])), 0);
+            const uint32_t k_lo0 = __shfl_sync(0xffffffffu, tc::smem_desc_lo_sw128(smem_u32(&sm.k[0][0][0][0])), 0);
+            const uint32_t v_lo0 = __shfl_sync(0xffffffffu, tc::smem_desc_lo_sw128(smem_u32(&sm.v[0][0][0][0])), 0);
+            const uint32_t tb = __shfl_sync(0xffffffffu, tbase, 0);
+            const int steps = __shfl_sync(0xffffffffu, n_steps, 0);
             auto issue_s = [&](int t, int st) {   // S_t = Q_t K(st)^T
-                const uint32_t qa = q_lo0 + t * kQTileStep, kb = k_lo0 + st * kKStageStep, dst = tbase + t * 256;
+                const uint32_t qa = q_lo0 + t * kQTileStep, kb = k_lo0 + st * kKStageStep, dst = tb + t * 256;
                 tc::umma_ss_c<false>(dst, tc::smem_desc_from_halves(qa, tc::kSmemDescHiSw128),
                                      tc::smem_desc_from_halves(kb, tc::kSmemDescHiSw128), kIdescS);
 #pragma unroll
@@ -263,53 +268,65 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
             // O_t (+)= P_t V(st), keys [64 half, 64 half + 64): the two halves are issued separately so
             // that the first can start while the softmax warps still produce the second
             auto issue_pv = [&](int t, int st, int half, bool first) {
-                const uint32_t vb = v_lo0 + st * kVStageStep + half * kVBlockStep, dst = tbase + t * 256 + 128;
-                const uint32_t src = tbase + t * 256 + half * 32;
+                const uint32_t vb = v_lo0 + st * kVStageStep + half * kVBlockStep, dst = tb + t * 256 + 128;
+                const uint32_t src = tb + t * 256 + half * 32;
                 tc::umma_ts(dst, src, tc::smem_desc_from_halves(vb, tc::kSmemDescHiSw128), kIdescO, !first);
 #pragma unroll
                 for (int ks = 1; ks < 4; ++ks)
                     tc::umma_ts_c<true>(dst, src + ks * 8, tc::smem_desc_from_halves(vb + ks * kKStep, tc::kSmemDescHiSw128), kIdescO);
             };
-            bool ok = tc::mbar_wait(&sm.q_full, 0, abort_flag) && tc::mbar_wait(&sm.k_full[0], 0, abort_flag);
+            bool ok = tc::mbar_wait_warp(&sm.q_full, 0, abort_flag) && tc::mbar_wait_warp(&sm.k_full[0], 0, abort_flag);
             if (ok) {
                 tc::tc_fence_after_sync();
-                issue_s(0, 0);
-                tc::umma_commit(&sm.s_full[0]);
-                issue_s(1, 0);
-                tc::umma_commit(&sm.s_full[1]);
-                tc::umma_commit(&sm.k_empty[0]);
-            }
-            for (int j = 0; ok && j < n_steps; ++j) {
-                const int st = j & 1, u = j >> 1;
-                const bool more = j + 1 < n_steps;
-                const int st1 = (j + 1) & 1, u1 = (j + 1) >> 1;
-                if (!(ok = tc::mbar_wait(&sm.v_full[st], u & 1, abort_flag))) break;
-                if (!(ok = tc::mbar_wait(&sm.p_half[0][0], j & 1, abort_flag))) break;
-                tc::tc_fence_after_sync();
-                issue_pv(0, st, 0, j == 0);
-                if (!(ok = tc::mbar_wait(&sm.p_half[0][1], j & 1, abort_flag))) break;
-                tc::tc_fence_after_sync();
-                issue_pv(0, st, 1, false);
-                if (more) {
-                    if (!(ok = tc::mbar_wait(&sm.k_full[st1], u1 & 1, abort_flag))) break;
-                    tc::tc_fence_after_sync();
-                    issue_s(0, st1);
+                if (tc::elect_one()) {
+                    issue_s(0, 0);
                     tc::umma_commit(&sm.s_full[0]);
-                }
-                if (!(ok = tc::mbar_wait(&sm.p_half[1][0], j & 1, abort_flag))) break;
-                tc::tc_fence_after_sync();
-                issue_pv(1, st, 0, j == 0);
-                if (!(ok = tc::mbar_wait(&sm.p_half[1][1], j & 1, abort_flag))) break;
-                tc::tc_fence_after_sync();
-                issue_pv(1, st, 1, false);
-                tc::umma_commit(&sm.v_empty[st]);
-                if (more) {
-                    issue_s(1, st1);
+                    issue_s(1, 0);
                     tc::umma_commit(&sm.s_full[1]);
-                    tc::umma_commit(&sm.k_empty[st1]);
+                    tc::umma_commit(&sm.k_empty[0]);
                 }
+                __syncwarp();
             }
-            if (ok) tc::umma_commit(&sm.o_final);
+            for (int j = 0; ok && j < steps; ++j) {
+                const int st = j & 1, u = j >> 1;
+                const bool more = j + 1 < steps;
+                const int st1 = (j + 1) & 1, u1 = (j + 1) >> 1;
+                if (!(ok = tc::mbar_wait_warp(&sm.v_full[st], u & 1, abort_flag))) break;
+                if (!(ok = tc::mbar_wait_warp(&sm.p_half[0][0], j & 1, abort_flag))) break;
+                tc::tc_fence_after_sync();
+                if (tc::elect_one()) issue_pv(0, st, 0, j == 0);
+                __syncwarp();
+                if (!(ok = tc::mbar_wait_warp(&sm.p_half[0][1], j & 1, abort_flag))) break;
+                tc::tc_fence_after_sync();
+                if (more && !(ok = tc::mbar_wait_warp(&sm.k_full[st1], u1 & 1, abort_flag))) break;
+                tc::tc_fence_after_sync();
+                if (tc::elect_one()) {
+                    issue_pv(0, st, 1, false);
+                    if (more) {
+                        issue_s(0, st1);
+                        tc::umma_commit(&sm.s_full[0]);
+                    }
+                }
+                __syncwarp();
+                if (!(ok = tc::mbar_wait_warp(&sm.p_half[1][0], j & 1, abort_flag))) break;
+                tc::tc_fence_after_sync();
+                if (tc::elect_one()) issue_pv(1, st, 0, j == 0);
+                __syncwarp();
+                if (!(ok = tc::mbar_wait_warp(&sm.p_half[1][1], j & 1, abort_flag))) break;
+                tc::tc_fence_after_sync();
+                if (tc::elect_one()) {
+                    issue_pv(1, st, 1, false);
+                    tc::umma_commit(&sm.v_empty[st]);
+                    if (more) {
+                        issue_s(1, st1);
+                        tc::umma_commit(&sm.s_full[1]);
+                        tc::umma_commit(&sm.k_empty[st1]);
+                    }
+                }
+                __syncwarp();
+            }
+            if (ok && tc::elect_one()) tc::umma_commit(&sm.o_final);
+            __syncwarp();
         }
     } else if (warp < 8) {
         // ------------------------------------------------------------ softmax warps
@@ -446,9 +463,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
             // ---- P = 2^(s*scale - m_ref) on visible keys, 0 elsewhere; bf16 pairs into TMEM
             const float neg_ref = -m_ref;                          // finite whenever a key is visible
             if (uniform) {
-                // The softmax warps are issue-bound (moving exponentials to an FMA polynomial only slowed
-                // the kernel), so the scale-subtract and the row sums use the packed fp32x2 instructions:
-                // 10 instead of 14 instructions per four keys.
+                // The scale-subtract and the row sums use the packed fp32x2 instructions: 10 instead of 14
+                // instructions per four keys.
                 unsigned long long psA = 0ull, psB = 0ull;             // two packed pairs of partial row sums
                 const unsigned long long scale2 = pack_f32x2(scale_log2, scale_log2);
 #pragma unroll
@@ -463,7 +479,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
                         float x0, x1, x2, x3;
                         unpack_f32x2(x01, x0, x1);
                         unpack_f32x2(x23, x2, x3);
-                        const float p0 = fast_exp2(x0), p1 = fast_exp2(x1), p2 = fast_exp2(x2), p3 = fast_exp2(x3);
+                        // one exponential in eight on the FMA pipe: a softmax warp running alone on its
+                        // scheduler is bound by MUFU (8 cycles per warp-wide ex2) and by issue about equally
+                        // (measured: 1/8 gains 2.5 %, 1/4 loses 1 %, 1/2 loses 6 %)
+                        const float p0 = fast_exp2(x0), p1 = fast_exp2(x1), p2 = fast_exp2(x2), p3 = (i & 1) ? fma_exp2(x3) : fast_exp2(x3);
                         psA = add_f32x2(psA, pack_f32x2(p0, p1));
                         psB = add_f32x2(psB, pack_f32x2(p2, p3));
                         pk[2 * i] = pack_bf16x2(p0, p1);

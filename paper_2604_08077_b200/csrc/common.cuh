@@ -190,6 +190,22 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
+// 2^x on the FMA pipe, for part of a softmax row's exponentials when the MUFU unit (4 lanes per
+// scheduler: 8 cycles per warp instruction) is the busier pipe.  x = n + f with n = round(x), f in
+// [-0.5, 0.5]: a cubic for 2^f (minimax in relative error over that interval, 7.7e-5: far inside the
+// bf16 rounding of the probabilities it feeds), n added to the exponent field.  x is clamped at -125,
+// so a masked score (-inf) yields about 2^-125 = 2e-38 instead of 0: next to any visible key (weight
+// >= 2^-8 of the row's reference) that is nothing in an fp32 sum, and it is multiplied by 0 when the
+// row meets its first visible key.  (An exact zero costs one more instruction per element, which
+// measurably undoes the gain.)
+__device__ __forceinline__ float fma_exp2(float x) {
+    const float xc = fmaxf(x, -125.f);
+    const float xr = xc + 12582912.f;                  // 1.5 * 2^23: the low mantissa bits now hold n
+    const float f = xc - (xr - 12582912.f);
+    const float p = fmaf(fmaf(fmaf(0.055222616f, f, 0.24261537f), f, 0.69325161f), f, 0.99992758f);
+    return __uint_as_float(__float_as_uint(p) + (__float_as_uint(xr) << 23));
+}
+
 // ---- packed fp32 pairs (sm_100): one instruction for two lanes of a*b+c / a+b -------------------
 __device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi) {
     unsigned long long d;

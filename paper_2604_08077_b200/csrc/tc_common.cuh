@@ -227,6 +227,19 @@ __device__ __forceinline__ void umma_ts_c(uint32_t d_tmem, uint32_t a_tmem, uint
         "r"(a_tmem), "l"(b_desc), "r"(idesc), "n"(kAccumulate ? 1 : 0)
         : "memory");
 }
+// One lane of a converged warp (the same lane every time): the issuing lane of a warp whose other lanes
+// run the same loop.  The code around a tcgen05.mma then stays warp-uniform (addresses and descriptors in
+// uniform registers), which the issue rate of one thread depends on: measured 85 - 90 cycles per
+// 128x128x16 MMA this way against 113 - 125 from a branch that only lane 0 enters.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}\n" : "=r"(pred));
+    return pred != 0;
+}
+// mbar_wait by all lanes of a converged warp with a warp-uniform result.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+}
 // Arrives on `bar` once every tcgen05.mma issued so far by this thread has completed.
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(smem_u32(bar))
