@@ -217,7 +217,7 @@ adaspark_status_t adaspark_attn_partition(adaspark_attn_t* h, int32_t batch, int
     // the fp64 selection kernel | its score scratch | key digit planes (tcgen05 path)
     size_t off = 0;
     h->fw_status_off = off; off = align_up(off + 256);
-    h->fw_headmax_off = off; off = align_up(off + (size_t)batch * Hkv * 4);
+    h->fw_headmax_off = off; off = align_up(off + (size_t)batch * Hkv * 4 * 2);   // key exponents, then largest |k|^2
     h->fw_valid_off = off; off = align_up(off + (size_t)(S_cap / kBlockTok) * 2 * 4);   // which slots of a block hold a token
     const size_t n_cols = (size_t)(S_v + kBlockTok - 1) / kBlockTok;                     // key blocks that hold video
     // query-gather path: the rows are cut into windows whose slice of Q (all heads) is about a third of the L2
@@ -357,8 +357,10 @@ adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* 
         const int blk_end = last_call ? g.n_kv_blocks_cap : (g.S + kBlockTok - 1) / kBlockTok;
         dim3 grid(blk_end - blk_begin, g.Hkv, g.B);
         uint32_t* slot_valid = (!cache_only && g.ragged) ? (uint32_t*)((char*)workspace + h->fw_valid_off) : nullptr;
-        if (D == 128) relayout_pool_kernel<128><<<grid, 256, 0, st>>>(g, kb, vb, kc, vc, cube_keys, slot_valid);
-        else relayout_pool_kernel<64><<<grid, 256, 0, st>>>(g, kb, vb, kc, vc, cube_keys, slot_valid);
+        // largest |k|^2 per (batch, kv head): only a call that brings the sequence from its first frame sees every key
+        uint32_t* key_norm2 = (!cache_only && frame_begin == 0) ? (uint32_t*)((char*)workspace + h->fw_headmax_off) + g.B * g.Hkv : nullptr;
+        if (D == 128) relayout_pool_kernel<128><<<grid, 256, 0, st>>>(g, kb, vb, kc, vc, cube_keys, slot_valid, key_norm2);
+        else relayout_pool_kernel<64><<<grid, 256, 0, st>>>(g, kb, vb, kc, vc, cube_keys, slot_valid, key_norm2);
         if (!launch_ok(h, "relayout_pool_kernel")) return ADASPARK_ERR_CUDA;
         const int cube_begin = g.pos_begin >> g.c_shift;
         if (g.C > kBlockTok && g.N_live > cube_begin) {
@@ -502,18 +504,19 @@ adaspark_status_t forward_impl(adaspark_attn_t* h, const char* who, const void* 
             if (!launch_ok(h, "gather_items_kernel")) return ADASPARK_ERR_CUDA;
         }
         const uint32_t* pair_mode_c = gather ? gw.pair_mode : nullptr;
+        const uint32_t* key_norm2_c = frame_begin == 0 ? (const uint32_t*)(ws + h->fw_headmax_off) + g.B * g.Hkv : nullptr;
         mark(h, 5, st);
         if (D == 128) {
             size_t smem = sizeof(TcAttnSmem<128>) + 1024;
             if (!set_smem(h, attn_prefill_tc_kernel<128>, smem, "attn_prefill_tc_kernel")) return ADASPARK_ERR_CUDA;
             attn_prefill_tc_kernel<128><<<grid, kTcThreads, smem, st>>>(g, tmQ, qb, tmK, tmV, tile_mask, tile_union, slot_valid_c, pair_mode_c,
-                                                                        gw.n_pairs_cap, gw.ml_local, (__nv_bfloat16*)out,
+                                                                        gw.n_pairs_cap, gw.ml_local, key_norm2_c, (__nv_bfloat16*)out,
                                                                         (unsigned long long*)&hdr->executed_kv_blocks, &hdr->max_tile_kv_blocks, &hdr->status);
         } else {
             size_t smem = sizeof(TcAttnSmem<64>) + 1024;
             if (!set_smem(h, attn_prefill_tc_kernel<64>, smem, "attn_prefill_tc_kernel")) return ADASPARK_ERR_CUDA;
             attn_prefill_tc_kernel<64><<<grid, kTcThreads, smem, st>>>(g, tmQ, qb, tmK, tmV, tile_mask, tile_union, slot_valid_c, pair_mode_c,
-                                                                       gw.n_pairs_cap, gw.ml_local, (__nv_bfloat16*)out,
+                                                                       gw.n_pairs_cap, gw.ml_local, key_norm2_c, (__nv_bfloat16*)out,
                                                                        (unsigned long long*)&hdr->executed_kv_blocks, &hdr->max_tile_kv_blocks, &hdr->status);
         }
         if (!launch_ok(h, "attn_prefill_tc_kernel")) return ADASPARK_ERR_CUDA;

@@ -31,6 +31,9 @@ constexpr int kHelperRegs = 72;     // ... of the producer / MMA warpgroup
 // compile-time bound of __launch_bounds__(384, 1)).  A request beyond that blocks forever.
 static_assert(8 * 32 * kSoftmaxRegs + 4 * 32 * kHelperRegs <= kTcThreads * 168, "setmaxnreg must stay inside the CTA's launch allocation");
 constexpr int kPairRows = 256;
+// Largest score bound (log2 units) up to which a row's softmax reference is fixed in advance: the row's own
+// key has weight >= 2^-2B, which leaves 126 - 2 * 44 = 38 binades above the smallest normal fp32
+constexpr float kFixedRefMax = 44.f;
 constexpr int kMaxBlockWords = 1024;   // up to 32768 key blocks (2M positions) per sequence
 
 template <int D>
@@ -65,7 +68,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     Geom g, const __grid_constant__ CUtensorMap tmQ, const __nv_bfloat16* __restrict__ q, const __grid_constant__ CUtensorMap tmK,
     const __grid_constant__ CUtensorMap tmV, const uint32_t* __restrict__ tile_mask,
     const uint32_t* __restrict__ tile_union, const uint32_t* __restrict__ slot_valid, const uint32_t* __restrict__ pair_mode,
-    int n_pairs_cap, float2* __restrict__ ml_local, __nv_bfloat16* __restrict__ out,
+    int n_pairs_cap, float2* __restrict__ ml_local, const uint32_t* __restrict__ key_norm2_bits, __nv_bfloat16* __restrict__ out,
     unsigned long long* __restrict__ executed_blocks, uint32_t* __restrict__ max_tile_blocks, int32_t* __restrict__ status) {
     extern __shared__ unsigned char tc_smem_raw[];
     TcAttnSmem<D>& sm = *reinterpret_cast<TcAttnSmem<D>*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -349,6 +352,33 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
             return cached_word;
         };
         float m_ref = -INFINITY, l_sum = 0.f;
+        // Reference fixed in advance.  |s| <= |q| |k| for every key, so with B = |q| max|k| scale (in log2 units;
+        // the largest key norm of the head comes from the re-layout kernel) 2^(s scale - B) can never
+        // overflow: the row needs no maximum and no rescaling of O.  What it costs is range at the small end
+        // (the row's largest weight may be as low as 2^-2B), so the rows of the warp take this path only if
+        // all their bounds are small; otherwise, and when not every attended key went through this call's
+        // re-layout, the running maximum below decides as before.
+        bool fixed_ref = false;
+        if (key_norm2_bits != nullptr) {
+            float bound = INFINITY;
+            if (tc::mbar_wait(&sm.q_full, 0, abort_flag)) {
+                float q2 = 0.f;
+#pragma unroll
+                for (int c = 0; c < D / 8; ++c) {
+                    const uint4 qv = *reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned char*>(&sm.q[t][c >> 3][0][0]) + sw128(row, c & 7));
+                    const uint32_t w[4] = {qv.x, qv.y, qv.z, qv.w};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xffff0000u);
+                        q2 = fmaf(lo, lo, fmaf(hi, hi, q2));
+                    }
+                }
+                const float k2 = __uint_as_float(__ldg(key_norm2_bits + b * g.Hkv + gk));
+                bound = sqrtf(q2 * k2) * scale_log2 * 1.01f + 0.01f;     // 1 % for the rounding of the norms and of s
+            }
+            fixed_ref = __all_sync(0xffffffffu, bound <= kFixedRefMax);
+            if (fixed_ref) m_ref = bound;
+        }
         BlockIter it(sm.blk_words);
         bool ok = true;
         for (int j = 0; j < n_steps; ++j) {
@@ -412,6 +442,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
 #pragma unroll
             for (int c = 0; c < 4; ++c) tc::tmem_ld_32x32(lane_addr + c * 32, s[c]);
             tc::tmem_wait_ld();
+            if (!fixed_ref) {
             // ---- row maximum over the visible keys
             float mx = -INFINITY;
             if (uniform) {
@@ -459,6 +490,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
                 }
                 l_sum *= factor;
                 if (need) m_ref = mx_x;
+            }
             }
             // ---- P = 2^(s*scale - m_ref) on visible keys, 0 elsewhere; bf16 pairs into TMEM
             const float neg_ref = -m_ref;                          // finite whenever a key is visible

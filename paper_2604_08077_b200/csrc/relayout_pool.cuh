@@ -8,6 +8,9 @@
 //   cube_keys [B,Hkv,N,D] fp32    mean over the C keys of each cube inside the block (C <= 64);
 //                                 cubes larger than a block are pooled by pool_large_cubes_kernel.
 // Positions >= S are zero-filled so that later tensor-core reads never meet non-finite data.
+// The kernel also leaves the largest |k|^2 of every (batch, kv head) among the rows it wrote (float bits,
+// atomic maximum): with |q| it bounds every score of a query row (Cauchy-Schwarz), which lets the attention
+// kernel fix a row's softmax reference in advance.
 #pragma once
 #include "common.cuh"
 
@@ -28,7 +31,8 @@ __global__ void __launch_bounds__(256) relayout_pool_kernel(Geom g, const __nv_b
                                                             __nv_bfloat16* __restrict__ k_cube,
                                                             __nv_bfloat16* __restrict__ v_cube,
                                                             float* __restrict__ cube_keys,
-                                                            uint32_t* __restrict__ slot_valid) {
+                                                            uint32_t* __restrict__ slot_valid,
+                                                            uint32_t* __restrict__ key_norm2_bits) {
     constexpr int kChunks = D / 8;    // 16-byte chunks per row
     constexpr int kVPitch = D + 2;    // padded pitch (elements) of the V staging tile
     __shared__ __align__(16) __nv_bfloat16 Ks[kBlockTok][D];
@@ -37,6 +41,7 @@ __global__ void __launch_bounds__(256) relayout_pool_kernel(Geom g, const __nv_b
     const int blk = blockIdx.x + g.pos_begin / kBlockTok, gk = blockIdx.y, b = blockIdx.z;   // blocks of this call's row window
     const int pos0 = blk * kBlockTok;
     const int tid = threadIdx.x;
+    float row_max = 0.f;
 
     for (int idx = tid; idx < kBlockTok * kChunks; idx += 256) {
         int row = idx / kChunks, c = idx - row * kChunks;
@@ -49,8 +54,26 @@ __global__ void __launch_bounds__(256) relayout_pool_kernel(Geom g, const __nv_b
         }
         *reinterpret_cast<uint4*>(&Ks[row][c * 8]) = kv4;
         *reinterpret_cast<uint4*>(k_cube + ((size_t)(b * g.Hkv + gk) * g.S_cap + pos) * D + c * 8) = kv4;
+        if (key_norm2_bits != nullptr) {
+            // |k|^2 of the row: the kChunks consecutive lanes that hold it add their parts (64 * kChunks is a
+            // multiple of 256, so every lane of the warp is here); non-negative floats order like their bits
+            const uint32_t w[4] = {kv4.x, kv4.y, kv4.z, kv4.w};
+            float n2 = 0.f;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xffff0000u);
+                n2 = fmaf(lo, lo, fmaf(hi, hi, n2));
+            }
+#pragma unroll
+            for (int o = kChunks / 2; o > 0; o >>= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, o);
+            row_max = fmaxf(row_max, n2);
+        }
         uint32_t* vdst = reinterpret_cast<uint32_t*>(&Vs[row][c * 8]);
         vdst[0] = vv4.x; vdst[1] = vv4.y; vdst[2] = vv4.z; vdst[3] = vv4.w;
+    }
+    if (key_norm2_bits != nullptr) {
+        const uint32_t m = __reduce_max_sync(0xffffffffu, __float_as_uint(row_max));
+        if ((tid & 31) == 0 && m) atomicMax(key_norm2_bits + b * g.Hkv + gk, m);
     }
     __syncthreads();
 

@@ -61,7 +61,10 @@ def test_small_chunked_prefill_every_row(kernel):
     rep = pu.compare_rows(wl, oracle.all_rows(oracle.shape_of(wl)), out, bm, label="chunked")
     assert rep["rows"] == wl.B * wl.Hq * wl.S
     assert torch.equal(bm, bm1), "chunked and one-shot selections differ"
-    assert (out.float() - out1.float()).abs().max().item() <= 1e-2
+    # Both results are checked against the oracle above / elsewhere.  Against each other they may differ by the
+    # bf16 rounding of the probabilities: a later chunk runs its softmax against the running maximum, the
+    # one-shot call against a reference fixed in advance, so the two round different numbers.
+    assert (out.float() - out1.float()).abs().max().item() <= pu.MAX_ABS_TOL
 
 
 def test_config2_in_four_chunks_matches_one_shot():
@@ -75,7 +78,7 @@ def test_config2_in_four_chunks_matches_one_shot():
     differ = (bm != bm1).any(-1)
     assert int(differ.sum()) <= 2, f"{int(differ.sum())} rows select differently from the one-shot prefill"
     same = ~differ
-    assert (out.float() - out1.float()).abs().permute(0, 2, 1, 3)[same].max().item() <= 1e-2
+    assert (out.float() - out1.float()).abs().permute(0, 2, 1, 3)[same].max().item() <= pu.MAX_ABS_TOL
 
 
 def test_chunk_argument_errors():
