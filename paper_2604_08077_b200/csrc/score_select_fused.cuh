@@ -48,7 +48,8 @@
 //   warps 16-19  slicers (one thread per row): digit planes of the next tile's queries into shared memory
 //   warp 20      TMA producer: key digit planes of one column tile (4 x 8 KB; 2 x 8 KB in pass A), 2 slots
 //   warps 21-22  issue the tcgen05.mma stream (40 of 128x64x32 per column tile, 12 in pass A; half each)
-//                into double-buffered accumulator sets (2 x 4 levels x 64 columns = all 512 TMEM columns)
+//                into double-buffered accumulator sets (2 x 4 levels x 64 columns = all 512 TMEM columns);
+//                each warp runs converged and issues through one elected lane
 //   warp 23      idle (it completes the sixth warpgroup for the register re-allocation)
 #pragma once
 #include "tc_common.cuh"
@@ -302,51 +303,63 @@ __global__ void __launch_bounds__(kFusedThreads, 1) score_select_fused_kernel(
         }
     } else if (warp == kMmaWarp || warp == kMmaWarp + 1) {
         // ------------------------------------------------------------ MMA issuers
-        // Two threads issue the stream (one thread alone is the bottleneck: ~95 cycles per 128x64x32 MMA):
-        // issuer 0 owns the accumulators of levels 0 and 3, issuer 1 those of levels 1 and 2 (five digit
-        // pairs each, no accumulator shared); a job is ready when both have committed.
+        // Two threads issue the stream (one thread gets a 128x64x32 MMA accepted every ~90 - 110 cycles, the
+        // tensor core would take them faster): issuer 0 owns the accumulators of levels 0 and 3, issuer 1 those
+        // of levels 1 and 2 (five digit pairs each, no accumulator shared); a job is ready when both have
+        // committed.  (Three issuers, 16 / 12 / 12 MMAs per column tile, measured 0.7 % slower.)
         const int issuer = warp - kMmaWarp;
-        if (lane == 0) {
+        {
+            // The whole warp walks the jobs and one elected lane issues, with every operand warp-uniform: a thread
+            // gets its MMAs accepted faster that way than from a branch that lane 0 alone enters.
             constexpr uint32_t kQPlaneStep = (uint32_t)sizeof(sm.qd[0]) >> 4, kKPlaneStep = (uint32_t)sizeof(sm.kring[0][0]) >> 4;
             constexpr uint32_t kSlotStep = (uint32_t)sizeof(sm.kring[0]) >> 4, kKStep = 32 >> 4;
-            const uint32_t q_lo0 = tc::smem_desc_lo_sw128(smem_u32(&sm.qd[0][0][0]));
-            const uint32_t k_lo0 = tc::smem_desc_lo_sw128(smem_u32(&sm.kring[0][0][0][0]));
+            const uint32_t q_lo0 = __shfl_sync(0xffffffffu, tc::smem_desc_lo_sw128(smem_u32(&sm.qd[0][0][0])), 0);
+            const uint32_t k_lo0 = __shfl_sync(0xffffffffu, tc::smem_desc_lo_sw128(smem_u32(&sm.kring[0][0][0][0])), 0);
+            const uint32_t tb = __shfl_sync(0xffffffffu, tbase, 0);
             bool ok = true;
             int c = 0, d0 = 0, n_done = 0;
             for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
                 const FusedItem w = fused_item(g, it);
                 if (w.n_ct == 0) continue;
-                if (!(ok = tc::mbar_wait(&sm.q_sliced, n_done & 1, abort_flag))) break;
+                if (!(ok = tc::mbar_wait_warp(&sm.q_sliced, n_done & 1, abort_flag))) break;
                 int f = -1;
                 while (ok) {
                     for (int ct = 0; ok && ct < w.n_ct; ++ct, ++c) {
                         const int s = c & 1, use = c >> 1;
-                        if (use > 0 && !(ok = tc::mbar_wait(&sm.acc_free[s], (use - 1) & 1, abort_flag))) break;
-                        if (!(ok = tc::mbar_wait(&sm.k_full[s], use & 1, abort_flag))) break;
+                        if (use > 0 && !(ok = tc::mbar_wait_warp(&sm.acc_free[s], (use - 1) & 1, abort_flag))) break;
+                        if (!(ok = tc::mbar_wait_warp(&sm.k_full[s], use & 1, abort_flag))) break;
                         tc::tc_fence_after_sync();
                         const uint32_t kb0 = k_lo0 + s * kSlotStep;
                         // level L = a + blk: plane a of the queries, plane blk of the keys; the anchor pass
                         // computes levels 0 and 1 only (S_0 = Q_0 K_0, S_1 = Q_0 K_1 + Q_1 K_0)
                         const int n_levels = f < 0 ? 2 : 4;
+                        if (tc::elect_one()) {
 #pragma unroll
-                        for (int L = 0; L < 4; ++L) {
-                            if (L >= n_levels || ((L == 0 || L == 3) ? 0 : 1) != issuer) continue;
+                            for (int L = 0; L < 4; ++L) {
+                                if (L >= n_levels || ((L == 0 || L == 3) ? 0 : 1) != issuer) continue;
 #pragma unroll
-                            for (int a = 0; a <= L; ++a)
+                                for (int a = 0; a <= L; ++a)
 #pragma unroll
-                                for (int ks = 0; ks < 4; ++ks)
-                                    tc::umma_ss_i8(tbase + s * 256 + L * kScoreTcCols,
-                                                   tc::smem_desc_from_halves(q_lo0 + a * kQPlaneStep + ks * kKStep, tc::kSmemDescHiSw128),
-                                                   tc::smem_desc_from_halves(kb0 + (L - a) * kKPlaneStep + ks * kKStep, tc::kSmemDescHiSw128),
-                                                   kIdesc, !(a == 0 && ks == 0));
+                                    for (int ks = 0; ks < 4; ++ks)
+                                        tc::umma_ss_i8(tb + s * 256 + L * kScoreTcCols,
+                                                       tc::smem_desc_from_halves(q_lo0 + a * kQPlaneStep + ks * kKStep, tc::kSmemDescHiSw128),
+                                                       tc::smem_desc_from_halves(kb0 + (L - a) * kKPlaneStep + ks * kKStep, tc::kSmemDescHiSw128),
+                                                       kIdesc, !(a == 0 && ks == 0));
+                            }
+                            tc::umma_commit(&sm.acc_full[s]);         // accumulators ready; the key slot may be reloaded
                         }
-                        tc::umma_commit(&sm.acc_full[s]);         // accumulators ready; the key slot may be reloaded
+                        __syncwarp();
                     }
                     ++f;
-                    if (f >= 2 && !another_pass(d0 + f - 2, ok)) break;
+                    if (f >= 2) {
+                        const bool more = __all_sync(0xffffffffu, another_pass(d0 + f - 2, ok));
+                        ok = __all_sync(0xffffffffu, ok);
+                        if (!more) break;
+                    }
                 }
                 d0 += f;
-                if (ok) tc::umma_commit(&sm.qd_free);             // the digit planes may be overwritten (both issuers)
+                if (ok && tc::elect_one()) tc::umma_commit(&sm.qd_free);   // the digit planes may be overwritten (both issuers)
+                __syncwarp();
                 ++n_done;
             }
         }
