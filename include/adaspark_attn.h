@@ -201,7 +201,9 @@ adaspark_status_t adaspark_attn_forward_host(adaspark_attn_t *handle, const void
  *                (then its text tokens).  q and out may both be NULL (caches only).
  *   sel_bitmap / sel_count  nullable, rows of this call only: [B, Hq, tokens of the call, ...].
  * Everything else as adaspark_attn_forward; adaspark_attn_forward(n_text) is the single chunk
- * (0, T, n_text). */
+ * (0, T, n_text).  The selection is the same bit for bit however the frames are cut; outputs agree within the
+ * bf16 rounding of the attention weights (a call that starts at frame 0 may fix a row's softmax reference in
+ * advance from the norms of the keys it brought, a later call uses the running maximum). */
 adaspark_status_t adaspark_attn_forward_chunk(adaspark_attn_t *handle, const void *q, const void *k,
                                               const void *v, int32_t frame_begin, int32_t frame_count,
                                               int32_t n_text, void *out, void *k_cube, void *v_cube,
