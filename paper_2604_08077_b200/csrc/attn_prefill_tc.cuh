@@ -31,9 +31,10 @@ constexpr int kHelperRegs = 72;     // ... of the producer / MMA warpgroup
 // compile-time bound of __launch_bounds__(384, 1)).  A request beyond that blocks forever.
 static_assert(8 * 32 * kSoftmaxRegs + 4 * 32 * kHelperRegs <= kTcThreads * 168, "setmaxnreg must stay inside the CTA's launch allocation");
 constexpr int kPairRows = 256;
-// Largest score bound (log2 units) up to which a row's softmax reference is fixed in advance: the row's own
-// key has weight >= 2^-2B, which leaves 126 - 2 * 44 = 38 binades above the smallest normal fp32
-constexpr float kFixedRefMax = 44.f;
+// Largest score bound B (log2 units) up to which a row's softmax reference is fixed in advance.  Every score lies
+// in [-B, B], so every weight 2^(s - B) is at least 2^-2B = 2^-96: nothing underflows, and 30 binades remain
+// above the smallest normal fp32 for the products with V.
+constexpr float kFixedRefMax = 48.f;
 constexpr int kMaxBlockWords = 1024;   // up to 32768 key blocks (2M positions) per sequence
 
 template <int D>
@@ -355,9 +356,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
         // Reference fixed in advance.  |s| <= |q| |k| for every key, so with B = |q| max|k| scale (in log2 units;
         // the largest key norm of the head comes from the re-layout kernel) 2^(s scale - B) can never
         // overflow: the row needs no maximum and no rescaling of O.  What it costs is range at the small end
-        // (the row's largest weight may be as low as 2^-2B), so the rows of the warp take this path only if
-        // all their bounds are small; otherwise, and when not every attended key went through this call's
-        // re-layout, the running maximum below decides as before.
+        // (a weight may be as low as 2^-2B), so the rows of the warp take this path only if all their bounds
+        // are small; otherwise, and when not every attended key went through this call's re-layout, the
+        // running maximum below decides as before.
         bool fixed_ref = false;
         if (key_norm2_bits != nullptr) {
             float bound = INFINITY;

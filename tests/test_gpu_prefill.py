@@ -160,6 +160,23 @@ def test_inputs_far_from_unit_scale(scale_q, scale_k, compensate):
     the compensation the logits grow, the fixed-point error in logit units grows with them, and the rows
     leave the range the kernel was validated for: they are handed to the fp64 kernel (header counter
     fallback_rows), so the selection stays exact."""
+    hdr = _scaled_inputs_every_row(scale_q, scale_k, compensate)
+    if compensate:
+        assert hdr.fallback_rows == 0
+    else:
+        assert hdr.fallback_rows > 0, "rows with large logits should have gone to the fp64 kernel"
+
+
+@pytest.mark.parametrize("scale_q", [1.125, 1.25, 1.5, 2.0])
+def test_softmax_reference_fixed_in_advance_or_running(scale_q):
+    """The attention kernel fixes a row's softmax reference in advance when |q| max|k| scale bounds its scores
+    by 2^48, and keeps a running maximum otherwise, warp by warp.  Queries scaled so that the bound (27 to 42
+    in log2 units at unit scale for these shapes) lies below, around and above that limit: every row against
+    the oracle on both sides of the switch and in warps where the rows disagree."""
+    _scaled_inputs_every_row(scale_q, 1.0, False)
+
+
+def _scaled_inputs_every_row(scale_q, scale_k, compensate):
     import dataclasses
     base = inputs.small_prefill(seed=33, T=16, H=8, W=8, n_text=19)
     wl = dataclasses.replace(base, q=(base.q.float() * scale_q).to(torch.bfloat16),
@@ -180,11 +197,8 @@ def test_inputs_far_from_unit_scale(scale_q, scale_k, compensate):
     same, rep = pu.check_selection(sh, wl, rows, got_sel, res, label=f"scale {scale_q} x {scale_k}")
     got = out.float().cpu().numpy().transpose(0, 2, 1, 3).reshape(-1, wl.D)
     assert np.abs(got[same] - res["out"][same]).max() <= pu.MAX_ABS_TOL
-    if compensate:
-        assert hdr.fallback_rows == 0
-    else:
-        assert hdr.fallback_rows > 0, "rows with large logits should have gone to the fp64 kernel"
     print(scale_q, scale_k, compensate, rep, "fallback rows", hdr.fallback_rows)
+    return hdr
 
 
 def test_forward_from_host_buffers_equals_forward():
